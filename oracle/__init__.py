@@ -1,0 +1,229 @@
+"""ctypes front-end of the CPU oracle (``bof4_oracle.c``) and the theoretical solver.
+
+TEST INFRASTRUCTURE ONLY: the plain, slow definition of what the CUDA library must compute.
+Nothing in the product package imports this module, and this module imports nothing from
+the product package.  Inputs are CPU torch tensors or numpy arrays; bf16 inputs are widened
+to fp32 (exact) before they reach the C code.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+try:  # torch is only used to accept bf16 tensors
+    import torch
+except Exception:  # pragma: no cover
+    torch = None
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "bof4_oracle.c")
+_LIB = os.path.join(_HERE, "libbof4_oracle.so")
+_lib = None
+
+METRIC_MSE, METRIC_MAE = 0, 1
+NORM_ABS, NORM_SIGNED = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with strict IEEE flags.  Building the checker is not using it."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    cmd = ["gcc", "-O2", "-std=c11", "-fno-fast-math", "-ffp-contract=off", "-fopenmp",
+           "-shared", "-fPIC", _SRC, "-o", _LIB, "-lm"]
+    subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.orc_opq_split.restype = ctypes.c_int64
+    return _lib
+
+
+def n_threads() -> int:
+    """Threads the OpenMP loops of the oracle will use."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        return int(env.split(",")[0])
+    return len(os.sched_getaffinity(0))
+
+
+# --------------------------------------------------------------------------- marshalling
+
+
+def as_f32(w) -> np.ndarray:
+    """Flattened, contiguous fp32 numpy view/copy of a tensor (bf16 widened exactly)."""
+    if torch is not None and isinstance(w, torch.Tensor):
+        w = w.detach().cpu().reshape(-1)
+        if w.dtype != torch.float32:
+            w = w.float()
+        return np.ascontiguousarray(w.numpy())
+    a = np.ascontiguousarray(np.asarray(w).reshape(-1))
+    assert a.dtype == np.float32, a.dtype
+    return a
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _levels(xhat) -> np.ndarray:
+    a = np.ascontiguousarray(np.asarray(xhat, dtype=np.float32).reshape(-1))
+    assert a.shape == (16,)
+    return a.copy()
+
+
+def _check(n: int, I: int):
+    if I <= 0 or n % I:
+        raise ValueError("n must be a multiple of the block size")
+
+
+# --------------------------------------------------------------------------- functions
+
+
+def thresholds(xhat) -> np.ndarray:
+    lv = _levels(xhat)
+    xi = np.empty(15, np.float32)
+    _load().orc_thresholds(_p(lv), _p(xi))
+    return xi
+
+
+def block_constants(w, I: int, norm: int) -> np.ndarray:
+    a = as_f32(w)
+    _check(a.size, I)
+    m = np.empty(a.size // I, np.float32)
+    _load().orc_block_constants(_p(a), ctypes.c_int64(a.size), I, norm, _p(m))
+    return m
+
+
+def quantize(w, I: int, norm: int, xhat) -> Tuple[np.ndarray, np.ndarray]:
+    """-> (codes uint8 [n/2], scales fp32 [n/I])."""
+    a = as_f32(w)
+    _check(a.size, I)
+    lv = _levels(xhat)
+    codes = np.empty(a.size // 2, np.uint8)
+    scales = np.empty(a.size // I, np.float32)
+    _load().orc_quantize(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv), _p(codes), _p(scales))
+    return codes, scales
+
+
+def dequantize(codes: np.ndarray, scales: np.ndarray, I: int, xhat) -> np.ndarray:
+    """-> fp32 products m * xhat(code), before any rounding to the output type."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scales = np.ascontiguousarray(scales, dtype=np.float32)
+    n = codes.size * 2
+    _check(n, I)
+    assert scales.size == n // I
+    lv = _levels(xhat)
+    out = np.empty(n, np.float32)
+    _load().orc_dequantize(_p(codes), _p(scales), ctypes.c_int64(n), I, _p(lv), _p(out))
+    return out
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.size, np.uint16)
+    _load().orc_f32_to_bf16(_p(x), ctypes.c_int64(x.size), _p(out))
+    return out.reshape(x.shape)
+
+
+def bf16_bits_to_f32(h: np.ndarray) -> np.ndarray:
+    h = np.ascontiguousarray(h, dtype=np.uint16)
+    out = np.empty(h.size, np.float32)
+    _load().orc_bf16_to_f32(_p(h), ctypes.c_int64(h.size), _p(out))
+    return out.reshape(h.shape)
+
+
+def em_accumulate_mse(w, I: int, norm: int, xhat):
+    """-> dict(s1[16] f64, s0[16] f64, count[16] u64, err_sum f64, n)."""
+    a = as_f32(w)
+    _check(a.size, I)
+    lv = _levels(xhat)
+    s1 = np.zeros(16, np.float64)
+    s0 = np.zeros(16, np.float64)
+    cnt = np.zeros(16, np.uint64)
+    err = ctypes.c_double(0.0)
+    _load().orc_em_accumulate_mse(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv),
+                                  _p(s1), _p(s0), _p(cnt), ctypes.byref(err))
+    return dict(s1=s1, s0=s0, count=cnt, err_sum=err.value, n=a.size)
+
+
+def em_accumulate_mae(w, I: int, norm: int, xhat):
+    """-> dict(median[16] f32, wsum[16] f64, count[16] u64, err_sum f64, n)."""
+    a = as_f32(w)
+    _check(a.size, I)
+    lv = _levels(xhat)
+    med = np.zeros(16, np.float32)
+    ws = np.zeros(16, np.float64)
+    cnt = np.zeros(16, np.uint64)
+    err = ctypes.c_double(0.0)
+    _load().orc_em_accumulate_mae(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv),
+                                  _p(med), _p(ws), _p(cnt), ctypes.byref(err))
+    return dict(median=med, wsum=ws, count=cnt, err_sum=err.value, n=a.size)
+
+
+def fit(w, I: int, norm: int, metric: int, xhat, fixed_mask: int, iters: int):
+    """-> (levels fp32[16], err_log f64[iters])."""
+    a = as_f32(w)
+    _check(a.size, I)
+    lv = _levels(xhat)
+    log = np.zeros(max(iters, 1), np.float64)
+    _load().orc_fit(_p(a), ctypes.c_int64(a.size), I, norm, metric, _p(lv),
+                    ctypes.c_uint32(fixed_mask), iters, _p(log))
+    return lv, log[:iters]
+
+
+def quant_error(w, I: int, norm: int, xhat) -> Tuple[float, float]:
+    """-> (MSE, MAE) of the block-wise quantiser with levels xhat on w."""
+    a = as_f32(w)
+    _check(a.size, I)
+    lv = _levels(xhat)
+    mse, mae = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _load().orc_quant_error(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv),
+                            ctypes.byref(mse), ctypes.byref(mae))
+    return mse.value, mae.value
+
+
+def block_sigmas(w, I: int) -> np.ndarray:
+    a = as_f32(w)
+    _check(a.size, I)
+    s = np.empty(a.size // I, np.float32)
+    _load().orc_block_sigmas(_p(a), ctypes.c_int64(a.size), I, _p(s))
+    return s
+
+
+def opq_split(w, I: int, tau: float, capacity: Optional[int] = None):
+    """-> (w_clean fp32[n], idx int64[k], val bf16-bits uint16[k], n_out)."""
+    a = as_f32(w)
+    _check(a.size, I)
+    cap = a.size if capacity is None else int(capacity)
+    clean = np.empty(a.size, np.float32)
+    idx = np.empty(max(cap, 1), np.int64)
+    val = np.empty(max(cap, 1), np.uint16)
+    k = _load().orc_opq_split(_p(a), ctypes.c_int64(a.size), I, ctypes.c_float(tau),
+                              _p(clean), _p(idx), _p(val), ctypes.c_int64(cap))
+    kk = min(k, cap)
+    return clean, idx[:kk].copy(), val[:kk].copy(), int(k)
+
+
+def opq_restore(out: np.ndarray, idx: np.ndarray, val: np.ndarray) -> np.ndarray:
+    out = np.ascontiguousarray(out, dtype=np.float32)
+    idx = np.ascontiguousarray(idx, dtype=np.int64)
+    val = np.ascontiguousarray(val, dtype=np.uint16)
+    _load().orc_opq_restore(_p(out), _p(idx), _p(val), ctypes.c_int64(idx.size))
+    return out
+
+
+def opq_threshold(q: float, I: int) -> float:
+    """tau = F_M^{-1}(q) for unit-variance Gaussian weights: F_M(m) = (2 G(m) - 1)^I
+    (App. B.1, CDF of the absolute block maximum), hence G(tau) = (1 + q^(1/I)) / 2."""
+    from scipy.special import ndtri
+    return float(ndtri((1.0 + q ** (1.0 / I)) / 2.0))
