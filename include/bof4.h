@@ -1,0 +1,195 @@
+/*
+ * bof4.h -- C ABI of the B200 (sm_100a) library for block-wise 4-bit optimal-float
+ * quantisation: BOF4 (absolute block maximum), BOF4-S (signed block maximum), the data-driven
+ * EM/Lloyd codebook fit, and outlier-preserving quantisation (OPQ).
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ *  - Pointers named d_* are DEVICE pointers (memory of the current CUDA device); pointers
+ *    named h_* and plain value arguments live on the HOST.  The library never takes ownership:
+ *    the caller allocates and frees every buffer, including the workspace.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work is
+ *    enqueued on that stream and the call returns without synchronising; outputs are valid once
+ *    the stream has reached the end of the enqueued work.
+ *  - Weights are a flattened tensor of n elements cut into B = n / block_size contiguous blocks
+ *    (Sec. 2.1).  block_size is one of 32, 64, 128, 256 and n must be a multiple of it.
+ *  - A codebook is 16 fp32 reconstruction levels in ASCENDING order, device resident.  Code c
+ *    (0..15) is the 0-based rank of the level; decision thresholds are the fp32 midpoints
+ *    (xhat[j] + xhat[j+1]) * 0.5f and a value equal to a threshold belongs to the upper level
+ *    (Sec. 3.2: regions [xi(l-1), xi(l)), nearest-neighbour rule).
+ *  - Every function returns a status (BOF4_OK = 0, negative = error).  On error nothing has
+ *    been enqueued.  bof4_last_error() gives a message for the calling thread's last error.
+ *  - All fp32 arithmetic that decides a stored value (block constant, normalisation, threshold
+ *    comparison, dequantisation product, OPQ block statistics) is IEEE-754 round-to-nearest-even
+ *    without flush-to-zero and without fused contraction.  Inputs must be finite.
+ */
+#ifndef BOF4_H
+#define BOF4_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Exported from the shared library (the rest of it is built with hidden visibility). */
+#if defined(__GNUC__)
+#define BOF4_API __attribute__((visibility("default")))
+#else
+#define BOF4_API
+#endif
+
+/* ---- status codes ---- */
+#define BOF4_OK 0
+#define BOF4_ERR_INVALID_ARG (-1) /* NULL pointer, negative size, bad enum value            */
+#define BOF4_ERR_SHAPE (-2)       /* block size unsupported, n not a multiple, n too large  */
+#define BOF4_ERR_DTYPE (-3)       /* dtype code unknown or combination not supported        */
+#define BOF4_ERR_WORKSPACE (-4)   /* workspace NULL, misaligned or smaller than required    */
+#define BOF4_ERR_CAPACITY (-5)    /* outlier list capacity is negative or too large         */
+#define BOF4_ERR_CUDA (-6)        /* a CUDA runtime call failed (message has the reason)    */
+
+/* ---- enums (plain ints in the signatures) ---- */
+#define BOF4_F32 0  /* IEEE binary32 */
+#define BOF4_BF16 1 /* bfloat16      */
+
+#define BOF4_NORM_ABS 0    /* block constant = max_i |w_i|                    (Eq. 1) */
+#define BOF4_NORM_SIGNED 1 /* block constant = the element of largest |w_i|   (Eq. 4) */
+
+#define BOF4_METRIC_MSE 0 /* weighted-mean centroid   (Eq. 6) */
+#define BOF4_METRIC_MAE 1 /* weighted-median centroid (Eq. 8) */
+
+#define BOF4_OP_EM 0  /* bof4_em_step / bof4_fit_codebook workspace */
+#define BOF4_OP_OPQ 1 /* opq_split / bof4_quantize_opq workspace    */
+
+#define BOF4_LEVELS 16
+
+/*
+ * Result of one expectation + accumulation pass (device resident, written by bof4_em_step).
+ * Index l is the 0-based level.  MSE (Eq. 6, App. B.3):
+ *     s1[l] = sum over members of m^2 * x,   s0[l] = sum over members of m^2,
+ *     err_sum = sum over all weights of (w - m * xhat[code])^2.
+ * MAE (Eq. 8, App. B.3):
+ *     s0[l] = sum over members of |m| (total weight of the weighted median), s1[l] = 0,
+ *     median[l] = weighted median of the members (the first sample, in ascending order, whose
+ *     cumulative weight reaches half of s0[l]); the input level where s0[l] == 0,
+ *     err_sum = sum over all weights of |w - m * xhat[code]|.
+ * count[l] is the number of members of region l, n_total the number of weights seen.
+ * For MSE median[l] is the centroid s1[l]/s0[l] rounded to fp32 (input level where s0[l] == 0).
+ */
+typedef struct bof4_em_stats {
+    double s1[BOF4_LEVELS];
+    double s0[BOF4_LEVELS];
+    uint64_t count[BOF4_LEVELS];
+    double err_sum;
+    int64_t n_total;
+    float median[BOF4_LEVELS];
+} bof4_em_stats;
+
+/*
+ * Bytes of device workspace an operation needs for tensors of at most n_max elements
+ * (for the EM operations: n_max = the largest single tensor of the list).  Host function, no
+ * CUDA call.  The workspace must be 256-byte aligned.  Returns 0 for invalid arguments.
+ *   op = BOF4_OP_EM : partial records of the deterministic two-stage reduction and, for
+ *                     metric = MAE, the per-level selection histograms.
+ *   op = BOF4_OP_OPQ: per-tile outlier staging and tile offsets of the ordered compaction.
+ */
+BOF4_API size_t bof4_workspace_bytes(int op, int64_t n_max, int block_size, int metric);
+
+/*
+ * One E+M accumulation pass with the codebook held fixed (Sec. 3.2; Eq. 6 or Eq. 8 with the
+ * error of App. B.3 in the un-normalised weight domain) over the union of n_tensors tensors.
+ *   h_w       host array of n_tensors DEVICE pointers to the tensors (dtype w_dtype each)
+ *   h_n       host array of n_tensors element counts, each a multiple of block_size
+ *   d_codebook  [16] fp32 levels, read only
+ *   d_stats   out: one bof4_em_stats record
+ *   d_ws      workspace of at least bof4_workspace_bytes(BOF4_OP_EM, max_t h_n[t], ...)
+ * The sums are accumulated in a fixed order that depends only on the shapes, so two calls on
+ * the same inputs give bit-identical statistics.
+ */
+BOF4_API int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_tensors, int w_dtype,
+                 int block_size, int norm, int metric, const float* d_codebook,
+                 bof4_em_stats* d_stats, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * `iters` Lloyd iterations in place on d_codebook (Sec. 3.2): thresholds from the current
+ * levels, assignment, then every level whose bit is NOT set in fixed_mask and whose region has
+ * positive total weight is replaced by its centroid (weighted mean, Eq. 6, or weighted median,
+ * Eq. 8); levels with their bit set keep their value ("initialise and skip recomputation").
+ *   d_codebook  in: initial levels (ascending), out: fitted levels
+ *   d_err_log   [iters] fp64 or NULL: entry t = mean error (MSE or MAE over all weights,
+ *               un-normalised domain) of the levels that ENTER iteration t
+ * No host synchronisation happens inside; the whole loop is enqueued on `stream`.
+ */
+BOF4_API int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int n_tensors, int w_dtype,
+                      int block_size, int norm, int metric, float* d_codebook,
+                      uint32_t fixed_mask, int iters, double* d_err_log, void* d_ws,
+                      size_t ws_bytes, void* stream);
+
+/*
+ * Block-wise quantisation (Sec. 2.1 Eq. 1-3, Sec. 3.1 Eq. 4): per block the constant m,
+ * x = w / m (x = 0 for an all-zero block), code = region of x.
+ *   d_codes   out [n/2] bytes; byte k = (code[2k] << 4) | code[2k+1]
+ *   d_scales  out [n/block_size] block constants, dtype scale_dtype.  The constant is stored
+ *             exactly: scale_dtype must equal w_dtype, or be BOF4_F32 for bf16 weights.
+ */
+BOF4_API int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_size, int norm,
+                  const float* d_codebook, uint8_t* d_codes, void* d_scales, int scale_dtype,
+                  void* stream);
+
+/*
+ * Outlier split of OPQ alone (Sec. 3.3 Eq. 9, App. E): per block the corrected sample standard
+ * deviation sigma_b (two-pass formula in fp32, balanced binary summation tree over the block);
+ * w is an outlier iff |w| > sigma_b * tau with tau = F_M^{-1}(q) (see bof4_opq_threshold).
+ *   d_w_clean  out [n] copy of w with outliers replaced by +0 (same dtype), or NULL
+ *   d_out_idx  out [capacity] int32 flattened indices of the outliers, ASCENDING
+ *   d_out_val  out [capacity] bf16 outlier values (round-to-nearest-even from fp32 weights)
+ *   d_n_out    out: the true number of outliers, also when it exceeds `capacity` (then only
+ *              the first `capacity` entries are written)
+ * n must be below 2^31.
+ */
+BOF4_API int opq_split(const void* d_w, int w_dtype, int64_t n, int block_size, float tau,
+              void* d_w_clean, int32_t* d_out_idx, void* d_out_val, int64_t capacity,
+              int64_t* d_n_out, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * OPQ fused with quantisation in one read of the weights (Sec. 3.3): outliers are listed as in
+ * opq_split and replaced by zero BEFORE the block-constant search; the cleaned block is then
+ * quantised as in bof4_quantize.
+ */
+BOF4_API int bof4_quantize_opq(const void* d_w, int w_dtype, int64_t n, int block_size, int norm,
+                      const float* d_codebook, float tau, uint8_t* d_codes, void* d_scales,
+                      int scale_dtype, int32_t* d_out_idx, void* d_out_val, int64_t capacity,
+                      int64_t* d_n_out, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * Dequantisation (Eq. 3): out[i] = round_to_out_dtype( fp32(scale[b]) * xhat[code[i]] ), one
+ * fp32 multiplication.  With OPQ (d_out_idx != NULL) the first min(*d_n_out, capacity)
+ * outliers are then written back at their indices (Sec. 3.3, decoding side).
+ *   d_out_idx / d_out_val / d_n_out  outlier list as produced by bof4_quantize_opq, or all NULL
+ *   capacity   number of entries the outlier arrays can hold (ignored without OPQ)
+ */
+BOF4_API int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t n,
+                    int block_size, const float* d_codebook, const int32_t* d_out_idx,
+                    const void* d_out_val, const int64_t* d_n_out, int64_t capacity,
+                    void* d_out, int out_dtype, void* stream);
+
+/* ---- host helpers (no CUDA call) ---- */
+
+/* tau = F_M^{-1}(q) for unit-variance Gaussian weights, F_M(m) = (2 G(m) - 1)^I the CDF of the
+ * absolute block maximum (App. B.1): tau = G^{-1}((1 + q^(1/I)) / 2).  NaN for q outside (0,1)
+ * or block_size < 1. */
+BOF4_API double bof4_opq_threshold(double q, int block_size);
+
+/* Starting codebook with the 7 negative / zero / 8 positive split of the printed codebooks
+ * (Tab. 6): -1 + k/7 (k = 0..6), 0, k/8 (k = 1..8), and the fixed-level mask of the variant:
+ * {-1, 0, 1} for BOF4_NORM_ABS, {0, 1} for BOF4_NORM_SIGNED (Sec. 3.1, Sec. 3.2). */
+BOF4_API int bof4_default_init(int norm, float h_levels[BOF4_LEVELS], uint32_t* h_fixed_mask);
+
+/* Message of the calling thread's most recent error ("" if none). */
+BOF4_API const char* bof4_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BOF4_H */

@@ -1,0 +1,15 @@
+"""B200 (sm_100a) library for block-wise 4-bit optimal-float quantisation (BOF4 / BOF4-S / OPQ).
+
+The product is the C-ABI shared library ``libbof4.so`` (declared in ``include/bof4.h``); this
+package holds its CUDA sources (``csrc/``), the build step (``build.py``) and a thin ctypes
+binding with the same function names (``binding.py``).
+"""
+from .binding import (BF16, F32, METRIC_MAE, METRIC_MSE, NORM_ABS, NORM_SIGNED, OP_EM, OP_OPQ,
+                      Bof4Error, bof4_default_init, bof4_dequantize, bof4_em_step,
+                      bof4_fit_codebook, bof4_last_error, bof4_opq_threshold, bof4_quantize,
+                      bof4_quantize_opq, bof4_workspace_bytes, opq_split)
+
+__all__ = ["BF16", "F32", "METRIC_MAE", "METRIC_MSE", "NORM_ABS", "NORM_SIGNED", "OP_EM", "OP_OPQ",
+           "Bof4Error", "bof4_default_init", "bof4_dequantize", "bof4_em_step", "bof4_fit_codebook",
+           "bof4_last_error", "bof4_opq_threshold", "bof4_quantize", "bof4_quantize_opq",
+           "bof4_workspace_bytes", "opq_split"]

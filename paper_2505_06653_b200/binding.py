@@ -1,0 +1,290 @@
+"""ctypes binding of ``libbof4.so``: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (see ``include/bof4.h``) and
+does nothing but turn torch CUDA tensors into device pointers, allocate the outputs with torch
+(device memory and streams are the only things torch is used for) and check the status code.
+All arithmetic of the method runs in the CUDA kernels; there is no CPU fallback: if the shared
+library is missing or no CUDA device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbof4.so")
+
+F32, BF16 = 0, 1
+NORM_ABS, NORM_SIGNED = 0, 1
+METRIC_MSE, METRIC_MAE = 0, 1
+OP_EM, OP_OPQ = 0, 1
+LEVELS = 16
+
+EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
+           "opq_split", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
+           "bof4_default_init", "bof4_last_error")
+
+
+class Bof4Error(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("bof4 error %d: %s" % (code, msg))
+        self.code = code
+
+
+class EmStats(ctypes.Structure):
+    """Mirror of ``bof4_em_stats``."""
+    _fields_ = [("s1", ctypes.c_double * LEVELS), ("s0", ctypes.c_double * LEVELS),
+                ("count", ctypes.c_uint64 * LEVELS), ("err_sum", ctypes.c_double),
+                ("n_total", ctypes.c_int64), ("median", ctypes.c_float * LEVELS)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("%s not found: run `python -m paper_2505_06653_b200.build`" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+        L.bof4_workspace_bytes.restype = sz
+        L.bof4_workspace_bytes.argtypes = [i32, i64, i32, i32]
+        L.bof4_em_step.restype = i32
+        L.bof4_em_step.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.bof4_fit_codebook.restype = i32
+        L.bof4_fit_codebook.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, ctypes.c_uint32, i32,
+                                        vp, vp, sz, vp]
+        L.bof4_quantize.restype = i32
+        L.bof4_quantize.argtypes = [vp, i32, i64, i32, i32, vp, vp, vp, i32, vp]
+        L.opq_split.restype = i32
+        L.opq_split.argtypes = [vp, i32, i64, i32, ctypes.c_float, vp, vp, vp, i64, vp, vp, sz, vp]
+        L.bof4_quantize_opq.restype = i32
+        L.bof4_quantize_opq.argtypes = [vp, i32, i64, i32, i32, vp, ctypes.c_float, vp, vp, i32,
+                                        vp, vp, i64, vp, vp, sz, vp]
+        L.bof4_dequantize.restype = i32
+        L.bof4_dequantize.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp, i64, vp, i32, vp]
+        L.bof4_opq_threshold.restype = ctypes.c_double
+        L.bof4_opq_threshold.argtypes = [ctypes.c_double, i32]
+        L.bof4_default_init.restype = i32
+        L.bof4_default_init.argtypes = [i32, vp, vp]
+        L.bof4_last_error.restype = ctypes.c_char_p
+        L.bof4_last_error.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise Bof4Error(rc, lib().bof4_last_error().decode())
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("weights must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _torch_dt(code: int):
+    return torch.float32 if code == F32 else torch.bfloat16
+
+
+def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor (there is no CPU path)" % name)
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    return t
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _codebook(levels, device) -> torch.Tensor:
+    if isinstance(levels, torch.Tensor):
+        cb = levels.to(device=device, dtype=torch.float32).contiguous()
+    else:
+        cb = torch.tensor(np.asarray(levels, dtype=np.float32), device=device)
+    if cb.numel() != LEVELS:
+        raise ValueError("a codebook has 16 levels")
+    return cb
+
+
+def _workspace(op: int, n_max: int, block_size: int, metric: int, device) -> torch.Tensor:
+    nbytes = lib().bof4_workspace_bytes(op, n_max, block_size, metric)
+    if nbytes == 0:
+        raise Bof4Error(-2, "bof4_workspace_bytes rejected the arguments")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)  # torch allocations are 512-B aligned
+
+
+# --------------------------------------------------------------------------- host helpers
+
+
+def bof4_workspace_bytes(op: int, n_max: int, block_size: int, metric: int = METRIC_MSE) -> int:
+    return int(lib().bof4_workspace_bytes(op, n_max, block_size, metric))
+
+
+def bof4_opq_threshold(q: float, block_size: int) -> float:
+    return float(lib().bof4_opq_threshold(q, block_size))
+
+
+def bof4_default_init(norm: int) -> Tuple[np.ndarray, int]:
+    lv = np.zeros(LEVELS, np.float32)
+    mask = ctypes.c_uint32(0)
+    _check(lib().bof4_default_init(norm, lv.ctypes.data_as(ctypes.c_void_p), ctypes.byref(mask)))
+    return lv, int(mask.value)
+
+
+def bof4_last_error() -> str:
+    return lib().bof4_last_error().decode()
+
+
+# --------------------------------------------------------------------------- EM
+
+
+def _tensor_list(ws: Sequence[torch.Tensor]):
+    if isinstance(ws, torch.Tensor):
+        ws = [ws]
+    ws = [_dev(w, "weights").reshape(-1) for w in ws]
+    if not ws:
+        raise ValueError("empty tensor list")
+    dt = _dt(ws[0])
+    if any(_dt(w) != dt for w in ws):
+        raise TypeError("all tensors of one call must share a dtype")
+    ptrs = (ctypes.c_void_p * len(ws))(*[w.data_ptr() for w in ws])
+    sizes = (ctypes.c_int64 * len(ws))(*[w.numel() for w in ws])
+    return ws, dt, ptrs, sizes
+
+
+def bof4_em_step(weights, block_size: int, norm: int, metric: int, levels,
+                 workspace: Optional[torch.Tensor] = None) -> dict:
+    """One accumulation pass; returns the ``bof4_em_stats`` record as a dict of numpy arrays."""
+    ws, dt, ptrs, sizes = _tensor_list(weights)
+    dev = ws[0].device
+    cb = _codebook(levels, dev)
+    wsp = workspace if workspace is not None else _workspace(
+        OP_EM, max(w.numel() for w in ws), block_size, metric, dev)
+    stats = torch.zeros(ctypes.sizeof(EmStats), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().bof4_em_step(ptrs, sizes, len(ws), dt, block_size, norm, metric, _ptr(cb),
+                                  _ptr(stats), _ptr(wsp), wsp.numel(), _stream()))
+    rec = EmStats.from_buffer_copy(stats.cpu().numpy().tobytes())
+    return dict(s1=np.array(rec.s1), s0=np.array(rec.s0), count=np.array(rec.count, dtype=np.uint64),
+                err_sum=float(rec.err_sum), n=int(rec.n_total), median=np.array(rec.median, dtype=np.float32))
+
+
+def bof4_fit_codebook(weights, block_size: int, norm: int, metric: int, levels, fixed_mask: int,
+                      iters: int, workspace: Optional[torch.Tensor] = None,
+                      sync: bool = True):
+    """``iters`` Lloyd iterations; returns (levels, err_log) as device tensors (fp32[16],
+    fp64[iters]).  With sync=False nothing waits for the stream."""
+    ws, dt, ptrs, sizes = _tensor_list(weights)
+    dev = ws[0].device
+    cb = _codebook(levels, dev).clone()
+    wsp = workspace if workspace is not None else _workspace(
+        OP_EM, max(w.numel() for w in ws), block_size, metric, dev)
+    log = torch.zeros(max(iters, 1), dtype=torch.float64, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().bof4_fit_codebook(ptrs, sizes, len(ws), dt, block_size, norm, metric, _ptr(cb),
+                                       fixed_mask, iters, _ptr(log), _ptr(wsp), wsp.numel(), _stream()))
+    if sync:
+        torch.cuda.current_stream(dev).synchronize()
+    return cb, log[:iters]
+
+
+# --------------------------------------------------------------------------- quantise / dequantise
+
+
+def bof4_quantize(w: torch.Tensor, block_size: int, norm: int, levels,
+                  scale_dtype: Optional[int] = None,
+                  out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None):
+    """-> (codes uint8[n/2], scales [n/block_size])."""
+    w = _dev(w, "w").reshape(-1)
+    n, dt = w.numel(), _dt(w)
+    sd = dt if scale_dtype is None else scale_dtype
+    cb = _codebook(levels, w.device)
+    if out is None:
+        codes = torch.empty(n // 2, dtype=torch.uint8, device=w.device)
+        scales = torch.empty(max(n // max(block_size, 1), 0), dtype=_torch_dt(sd), device=w.device)
+    else:
+        codes, scales = out
+    with torch.cuda.device(w.device):
+        _check(lib().bof4_quantize(_ptr(w), dt, n, block_size, norm, _ptr(cb), _ptr(codes),
+                                   _ptr(scales), sd, _stream()))
+    return codes, scales
+
+
+def bof4_dequantize(codes: torch.Tensor, scales: torch.Tensor, block_size: int, levels,
+                    out_dtype: int, outliers: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
+                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """-> dequantised tensor [n]; `outliers` = (idx int32, val bf16, n_out int64[1]) for OPQ."""
+    codes = _dev(codes, "codes")
+    scales = _dev(scales, "scales")
+    n = codes.numel() * 2
+    cb = _codebook(levels, codes.device)
+    if out is None:
+        out = torch.empty(n, dtype=_torch_dt(out_dtype), device=codes.device)
+    idx = val = cnt = None
+    cap = 0
+    if outliers is not None:
+        idx, val, cnt = outliers
+        cap = idx.numel()
+    with torch.cuda.device(codes.device):
+        _check(lib().bof4_dequantize(_ptr(codes), _ptr(scales), _dt(scales), n, block_size, _ptr(cb),
+                                     _ptr(idx), _ptr(val), _ptr(cnt), cap, _ptr(out), out_dtype,
+                                     _stream()))
+    return out
+
+
+def opq_split(w: torch.Tensor, block_size: int, tau: float, capacity: int,
+              want_clean: bool = True, workspace: Optional[torch.Tensor] = None):
+    """-> (w_clean or None, idx int32[capacity], val bf16[capacity], n_out int64[1])."""
+    w = _dev(w, "w").reshape(-1)
+    n, dt = w.numel(), _dt(w)
+    dev = w.device
+    wsp = workspace if workspace is not None else _workspace(OP_OPQ, n, block_size, 0, dev)
+    clean = torch.empty_like(w) if want_clean else None
+    idx = torch.empty(capacity, dtype=torch.int32, device=dev)
+    val = torch.empty(capacity, dtype=torch.bfloat16, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().opq_split(_ptr(w), dt, n, block_size, tau, _ptr(clean), _ptr(idx), _ptr(val),
+                               capacity, _ptr(cnt), _ptr(wsp), wsp.numel(), _stream()))
+    return clean, idx, val, cnt
+
+
+def bof4_quantize_opq(w: torch.Tensor, block_size: int, norm: int, levels, tau: float,
+                      capacity: int, scale_dtype: Optional[int] = None,
+                      workspace: Optional[torch.Tensor] = None, out=None):
+    """-> (codes, scales, idx int32[capacity], val bf16[capacity], n_out int64[1])."""
+    w = _dev(w, "w").reshape(-1)
+    n, dt = w.numel(), _dt(w)
+    dev = w.device
+    sd = dt if scale_dtype is None else scale_dtype
+    cb = _codebook(levels, dev)
+    wsp = workspace if workspace is not None else _workspace(OP_OPQ, n, block_size, 0, dev)
+    if out is None:
+        codes = torch.empty(n // 2, dtype=torch.uint8, device=dev)
+        scales = torch.empty(n // max(block_size, 1), dtype=_torch_dt(sd), device=dev)
+        idx = torch.empty(capacity, dtype=torch.int32, device=dev)
+        val = torch.empty(capacity, dtype=torch.bfloat16, device=dev)
+        cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+    else:
+        codes, scales, idx, val, cnt = out
+    with torch.cuda.device(dev):
+        _check(lib().bof4_quantize_opq(_ptr(w), dt, n, block_size, norm, _ptr(cb), tau, _ptr(codes),
+                                       _ptr(scales), sd, _ptr(idx), _ptr(val), capacity, _ptr(cnt),
+                                       _ptr(wsp), wsp.numel(), _stream()))
+    return codes, scales, idx, val, cnt

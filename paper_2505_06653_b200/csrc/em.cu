@@ -1,0 +1,405 @@
+// Data-driven EM / Lloyd codebook fit (Sec. 3.2, App. B.3): one streaming pass per iteration.
+//
+// MSE pass (Eq. 6): every lane owns 8 consecutive weights, a block is a group of I/8 lanes.
+// Per weight: x = w / m, region c by threshold search, then
+//     s1[c] += m^2 x,  s0[c] += m^2,  count[c] += 1,  err += (w - m xhat[c])^2.
+// The level-indexed sums live in shared memory as one private column per thread (no atomics,
+// no bank conflicts: the bank is the lane), are folded into fp64 per-CTA totals in a fixed
+// order, written as one partial record per CTA, and combined by a single-CTA kernel that also
+// updates the free levels.  Nothing depends on scheduling, so results are bit-reproducible.
+#include "common.cuh"
+#include "layout.h"
+
+namespace bof4 {
+
+constexpr int kEmThreads = 256;
+constexpr int kEmRow = kEmThreads * 8;  // weights per CTA row
+constexpr int kEmUnroll = 2;            // rows in flight per CTA iteration
+constexpr int kEmMaxTensors = 64;       // tensors per launch (kernel parameter table)
+constexpr int kEmFlushIters = 128;      // loop iterations between fp32 -> fp64 folds
+constexpr size_t kEmSmemBytes = (size_t)kLevels * kEmThreads * (sizeof(float2) + sizeof(uint32_t));
+
+struct EmTensors {
+    const void* ptr[kEmMaxTensors];
+    int64_t n[kEmMaxTensors];
+    int64_t row_end[kEmMaxTensors];  // cumulative number of CTA rows up to and including tensor t
+    int count;
+    int accumulate;  // 0: this launch overwrites the partial records, 1: adds to them
+};
+
+// Record layout in doubles: [0,16) s1, [16,32) s0, [32,48) count (uint64 bits), [48] err.
+constexpr int kRecS1 = 0, kRecS0 = 16, kRecCnt = 32, kRecErr = 48;
+
+template <class DT, int I, bool SIGNED>
+__global__ void __launch_bounds__(kEmThreads, 4)
+em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __restrict__ partials)
+{
+    constexpr int LPB = I / 8;
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    float2* s_acc = reinterpret_cast<float2*>(s_raw);                              // [16][threads]
+    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_raw + kLevels * kEmThreads * sizeof(float2));
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ double s_tot[3 * kLevels];  // s1, s0, count (as uint64 bits)
+    __shared__ double s_err[kEmThreads / 32];
+    __shared__ const void* s_ptr[kEmMaxTensors];
+    __shared__ int64_t s_n[kEmMaxTensors], s_row_end[kEmMaxTensors];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    make_thresholds(levels, s_xi, s_lv, tid);
+    if (tid < 3 * kLevels) s_tot[tid] = 0.0;  // all-zero bits are also uint64 zero
+    if (tid < T.count) {
+        s_ptr[tid] = T.ptr[tid];
+        s_n[tid] = T.n[tid];
+        s_row_end[tid] = T.row_end[tid];
+    }
+#pragma unroll
+    for (int l = 0; l < kLevels; ++l) {
+        s_acc[l * kEmThreads + tid] = make_float2(0.0f, 0.0f);
+        s_cnt[l * kEmThreads + tid] = 0u;
+    }
+    __syncthreads();
+
+    const int64_t total_rows = T.row_end[T.count - 1];
+    const int64_t stride = (int64_t)gridDim.x * kEmUnroll;
+    double err = 0.0;
+    int t_cur = 0;
+    int since_flush = 0;
+
+    // Folds the private fp32 columns into the fp64 CTA totals (fixed order) and clears them.
+    auto flush = [&]() {
+        __syncthreads();
+        for (int l = warp; l < kLevels; l += kEmThreads / 32) {
+            double a1 = 0.0, a0 = 0.0;
+            unsigned long long ac = 0;
+#pragma unroll
+            for (int k = 0; k < kEmThreads / 32; ++k) {
+                const int col = l * kEmThreads + k * 32 + lane;
+                const float2 a = s_acc[col];
+                a1 += (double)a.x;
+                a0 += (double)a.y;
+                ac += s_cnt[col];
+                s_acc[col] = make_float2(0.0f, 0.0f);
+                s_cnt[col] = 0u;
+            }
+#pragma unroll
+            for (int off = 16; off; off >>= 1) {
+                a1 += __shfl_xor_sync(kFull, a1, off);
+                a0 += __shfl_xor_sync(kFull, a0, off);
+                ac += __shfl_xor_sync(kFull, ac, off);
+            }
+            if (lane == 0) {
+                s_tot[l] += a1;
+                s_tot[kLevels + l] += a0;
+                reinterpret_cast<unsigned long long*>(s_tot)[2 * kLevels + l] += ac;
+            }
+        }
+        __syncthreads();
+    };
+
+    for (int64_t g0 = (int64_t)blockIdx.x * kEmUnroll; g0 < total_rows; g0 += stride) {
+        float v[kEmUnroll][8];
+        bool ok[kEmUnroll];
+#pragma unroll
+        for (int u = 0; u < kEmUnroll; ++u) {
+            const int64_t g = g0 + u;
+            ok[u] = false;
+            if (g < total_rows) {
+                while (g >= s_row_end[t_cur]) ++t_cur;
+                const int64_t r = g - (t_cur ? s_row_end[t_cur - 1] : 0);
+                const int64_t idx = (r * kEmThreads + tid) * 8;
+                ok[u] = idx < s_n[t_cur];
+                if (ok[u]) load8<DT>(s_ptr[t_cur], idx, v[u]);
+            }
+            if (!ok[u]) zero8<DT>(v[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < kEmUnroll; ++u) {
+            const float m = block_constant<LPB, SIGNED>(v[u]);
+            if (ok[u]) {
+                const float m2 = m * m;
+                float e = 0.0f;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float x = normalise(v[u][k], m);
+                    const int c = region_of(x, s_xi);
+                    const float d = fmaf(-m, s_lv[c], v[u][k]);
+                    e = fmaf(d, d, e);
+                    const int col = c * kEmThreads + tid;
+                    float2 a = s_acc[col];
+                    a.x = fmaf(m2, x, a.x);
+                    a.y += m2;
+                    s_acc[col] = a;
+                    s_cnt[col] += 1u;
+                }
+                err += (double)e;
+            }
+        }
+        if (++since_flush == kEmFlushIters) {
+            flush();
+            since_flush = 0;
+        }
+    }
+    flush();
+
+    // error: fixed-order fold over the CTA
+#pragma unroll
+    for (int off = 16; off; off >>= 1) err += __shfl_xor_sync(kFull, err, off);
+    if (lane == 0) s_err[warp] = err;
+    __syncthreads();
+    double* rec = partials + (size_t)blockIdx.x * kEmRecordDoubles;
+    if (tid < kLevels) {
+        unsigned long long* rc = reinterpret_cast<unsigned long long*>(rec);
+        const unsigned long long cnt = reinterpret_cast<unsigned long long*>(s_tot)[2 * kLevels + tid];
+        if (T.accumulate) {
+            rec[kRecS1 + tid] += s_tot[tid];
+            rec[kRecS0 + tid] += s_tot[kLevels + tid];
+            rc[kRecCnt + tid] += cnt;
+        } else {
+            rec[kRecS1 + tid] = s_tot[tid];
+            rec[kRecS0 + tid] = s_tot[kLevels + tid];
+            rc[kRecCnt + tid] = cnt;
+        }
+    }
+    if (tid == 0) {
+        double e = 0.0;
+        for (int k = 0; k < kEmThreads / 32; ++k) e += s_err[k];
+        rec[kRecErr] = T.accumulate ? rec[kRecErr] + e : e;
+    }
+}
+
+// Combines the per-CTA records in a fixed order and, if asked, performs the M step.
+//   stats    != NULL: receives the combined record
+//   codebook != NULL: every free level with s0 > 0 becomes (float)(s1 / s0)      (Eq. 6)
+//   err_slot != NULL: receives err_sum / n_total
+__global__ void __launch_bounds__(1024)
+em_mse_finalize_kernel(const double* __restrict__ partials, int n_records, int64_t n_total,
+                       const float* levels_in, bof4_em_stats* __restrict__ stats,
+                       float* codebook, uint32_t fixed_mask, double* __restrict__ err_slot)
+{
+    __shared__ double s_q[kRecErr + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int q = warp; q <= kRecErr; q += 32) {
+        const bool is_count = q >= kRecCnt && q < kRecErr;
+        double a = 0.0;
+        unsigned long long c = 0;
+        for (int r = lane; r < n_records; r += 32) {
+            const double* rec = partials + (size_t)r * kEmRecordDoubles;
+            if (is_count)
+                c += reinterpret_cast<const unsigned long long*>(rec)[q];
+            else
+                a += rec[q];
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) {
+            a += __shfl_xor_sync(kFull, a, off);
+            c += __shfl_xor_sync(kFull, c, off);
+        }
+        if (lane == 0) {
+            if (is_count)
+                reinterpret_cast<unsigned long long*>(s_q)[q] = c;
+            else
+                s_q[q] = a;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < kLevels) {
+        const int l = threadIdx.x;
+        const double s1 = s_q[kRecS1 + l], s0 = s_q[kRecS0 + l];
+        const float old = levels_in[l];
+        const float cen = (s0 > 0.0) ? (float)(s1 / s0) : old;
+        if (stats) {
+            stats->s1[l] = s1;
+            stats->s0[l] = s0;
+            stats->count[l] = reinterpret_cast<unsigned long long*>(s_q)[kRecCnt + l];
+            stats->median[l] = cen;
+        }
+        if (codebook && !((fixed_mask >> l) & 1u)) codebook[l] = cen;
+    }
+    if (threadIdx.x == 0) {
+        if (stats) {
+            stats->err_sum = s_q[kRecErr];
+            stats->n_total = n_total;
+        }
+        if (err_slot) *err_slot = (n_total > 0) ? s_q[kRecErr] / (double)n_total : 0.0;
+    }
+}
+
+}  // namespace bof4
+
+// ================================================================= launchers (C ABI)
+
+namespace {
+
+using namespace bof4;
+
+struct EmArgs {
+    const void* const* h_w;
+    const int64_t* h_n;
+    int n_tensors, w_dtype, block_size, norm, metric;
+    int64_t n_total;
+};
+
+int check_em(const char* fn, const EmArgs& a, const void* d_codebook, void* d_ws, size_t ws_bytes,
+             int64_t* n_total)
+{
+    if (a.n_tensors < 0 || (a.n_tensors > 0 && (!a.h_w || !a.h_n))) {
+        set_error("%s: bad tensor list", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (!valid_block_size(a.block_size)) {
+        set_error("%s: block_size %d is not one of 32, 64, 128, 256", fn, a.block_size);
+        return BOF4_ERR_SHAPE;
+    }
+    if (a.w_dtype != BOF4_F32 && a.w_dtype != BOF4_BF16) {
+        set_error("%s: unknown weight dtype %d", fn, a.w_dtype);
+        return BOF4_ERR_DTYPE;
+    }
+    if ((a.norm != BOF4_NORM_ABS && a.norm != BOF4_NORM_SIGNED) ||
+        (a.metric != BOF4_METRIC_MSE && a.metric != BOF4_METRIC_MAE)) {
+        set_error("%s: bad norm or metric", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    int64_t tot = 0;
+    for (int t = 0; t < a.n_tensors; ++t) {
+        if (a.h_n[t] < 0 || (a.h_n[t] > 0 && !a.h_w[t])) {
+            set_error("%s: tensor %d has a negative size or a NULL pointer", fn, t);
+            return BOF4_ERR_INVALID_ARG;
+        }
+        if (a.h_n[t] % a.block_size) {
+            set_error("%s: tensor %d has %lld elements, not a multiple of block_size %d", fn, t,
+                      (long long)a.h_n[t], a.block_size);
+            return BOF4_ERR_SHAPE;
+        }
+        tot += a.h_n[t];
+    }
+    if (!d_codebook) {
+        set_error("%s: NULL codebook", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (!d_ws || ((uintptr_t)d_ws & 255u) || ws_bytes < em_workspace_bytes()) {
+        set_error("%s: workspace NULL, not 256-byte aligned, or smaller than %zu bytes", fn,
+                  em_workspace_bytes());
+        return BOF4_ERR_WORKSPACE;
+    }
+    *n_total = tot;
+    return BOF4_OK;
+}
+
+template <class DT, int I, bool SG>
+int launch_mse_chunk(const EmTensors& T, const float* d_codebook, double* partials, cudaStream_t st)
+{
+    static bool attr_done = false;  // per instantiation; setting it twice is harmless
+    if (!attr_done) {
+        BOF4_CUDA_TRY(cudaFuncSetAttribute(em_mse_kernel<DT, I, SG>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEmSmemBytes));
+        attr_done = true;
+    }
+    em_mse_kernel<DT, I, SG><<<kEmGrid, kEmThreads, kEmSmemBytes, st>>>(T, d_codebook, partials);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
+}
+
+// Enqueues the accumulation launches of one MSE pass over all tensors (non-empty ones, in
+// list order, kEmMaxTensors per launch).  With no weights at all the records are zeroed.
+int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials, cudaStream_t st)
+{
+    EmTensors T;
+    T.count = 0;
+    T.accumulate = 0;
+    int64_t rows = 0;
+    bool launched = false;
+    auto fire = [&]() -> int {
+        if (T.count == 0) return BOF4_OK;
+        int rc = BOF4_OK;
+        const bool sg = a.norm == BOF4_NORM_SIGNED;
+#define BOF4_EM_GO(DT_)                                                                          \
+    switch (a.block_size) {                                                                      \
+        case 32: rc = sg ? launch_mse_chunk<DT_, 32, true>(T, d_codebook, partials, st)          \
+                         : launch_mse_chunk<DT_, 32, false>(T, d_codebook, partials, st); break; \
+        case 64: rc = sg ? launch_mse_chunk<DT_, 64, true>(T, d_codebook, partials, st)          \
+                         : launch_mse_chunk<DT_, 64, false>(T, d_codebook, partials, st); break; \
+        case 128: rc = sg ? launch_mse_chunk<DT_, 128, true>(T, d_codebook, partials, st)        \
+                          : launch_mse_chunk<DT_, 128, false>(T, d_codebook, partials, st); break; \
+        default: rc = sg ? launch_mse_chunk<DT_, 256, true>(T, d_codebook, partials, st)         \
+                         : launch_mse_chunk<DT_, 256, false>(T, d_codebook, partials, st); break; \
+    }
+        if (a.w_dtype == BOF4_F32) { BOF4_EM_GO(F32) } else { BOF4_EM_GO(BF16) }
+#undef BOF4_EM_GO
+        launched = true;
+        T.count = 0;
+        T.accumulate = 1;
+        rows = 0;
+        return rc;
+    };
+    for (int t = 0; t < a.n_tensors; ++t) {
+        if (a.h_n[t] == 0) continue;
+        rows += (a.h_n[t] + kEmRow - 1) / kEmRow;
+        T.ptr[T.count] = a.h_w[t];
+        T.n[T.count] = a.h_n[t];
+        T.row_end[T.count] = rows;
+        if (++T.count == kEmMaxTensors) {
+            const int rc = fire();
+            if (rc) return rc;
+        }
+    }
+    const int rc = fire();
+    if (rc) return rc;
+    if (!launched) BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));
+    return BOF4_OK;
+}
+
+}  // namespace
+
+extern "C" int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_tensors, int w_dtype,
+                            int block_size, int norm, int metric, const float* d_codebook,
+                            bof4_em_stats* d_stats, void* d_ws, size_t ws_bytes, void* stream)
+{
+    EmArgs a{h_w, h_n, n_tensors, w_dtype, block_size, norm, metric, 0};
+    int rc = check_em("bof4_em_step", a, d_codebook, d_ws, ws_bytes, &a.n_total);
+    if (rc) return rc;
+    if (!d_stats) {
+        set_error("bof4_em_step: NULL stats");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double* partials = static_cast<double*>(d_ws);
+    if (metric == BOF4_METRIC_MSE) {
+        rc = enqueue_mse_pass(a, d_codebook, partials, st);
+        if (rc) return rc;
+        em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, kEmGrid, a.n_total, d_codebook, d_stats,
+                                                   nullptr, 0u, nullptr);
+        BOF4_CUDA_TRY(cudaGetLastError());
+        return BOF4_OK;
+    }
+    set_error("bof4_em_step: MAE not available in this build");
+    return BOF4_ERR_INVALID_ARG;
+}
+
+extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int n_tensors,
+                                 int w_dtype, int block_size, int norm, int metric,
+                                 float* d_codebook, uint32_t fixed_mask, int iters,
+                                 double* d_err_log, void* d_ws, size_t ws_bytes, void* stream)
+{
+    EmArgs a{h_w, h_n, n_tensors, w_dtype, block_size, norm, metric, 0};
+    int rc = check_em("bof4_fit_codebook", a, d_codebook, d_ws, ws_bytes, &a.n_total);
+    if (rc) return rc;
+    if (iters < 0) {
+        set_error("bof4_fit_codebook: negative iteration count");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double* partials = static_cast<double*>(d_ws);
+    if (metric == BOF4_METRIC_MSE) {
+        for (int t = 0; t < iters; ++t) {
+            rc = enqueue_mse_pass(a, d_codebook, partials, st);
+            if (rc) return rc;
+            em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, kEmGrid, a.n_total, d_codebook, nullptr,
+                                                       d_codebook, fixed_mask,
+                                                       d_err_log ? d_err_log + t : nullptr);
+            BOF4_CUDA_TRY(cudaGetLastError());
+        }
+        return BOF4_OK;
+    }
+    set_error("bof4_fit_codebook: MAE not available in this build");
+    return BOF4_ERR_INVALID_ARG;
+}

@@ -1,0 +1,54 @@
+// Workspace layouts (host-side arithmetic only; used by the size query and by the launchers).
+#pragma once
+
+#include <stddef.h>
+#include <stdint.h>
+
+namespace bof4 {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---------------------------------------------------------------- EM workspace
+// [0, kEmPartialBytes)            per-CTA partial records of the MSE / error reduction
+// [kEmMaeOffset, +kEmMaeBytes)    weighted-median selection state and histograms (MAE)
+constexpr int kEmGrid = 148 * 4;          // CTAs of the accumulation kernels (4 per SM)
+constexpr int kEmRecordDoubles = 64;      // 16 s1 + 16 s0 + 16 count + err, padded to 512 B
+constexpr size_t kEmPartialBytes = (size_t)kEmGrid * kEmRecordDoubles * 8;
+constexpr int kMaeBins = 1024;            // bins per level and selection pass
+constexpr size_t kEmMaeOffset = 512 * 1024;
+constexpr size_t kEmMaeHistBytes = (size_t)16 * kMaeBins * 8;
+constexpr size_t kEmMaeBytes = 4096 + kEmMaeHistBytes;
+
+inline size_t em_workspace_bytes() { return kEmMaeOffset + align_up(kEmMaeBytes, 256); }
+
+// ---------------------------------------------------------------- OPQ workspace
+// The weights are cut into tiles of kOpqTile elements (one warp iteration).  Each tile has a
+// count and a staging slot of kOpqStage outliers; tiles are scanned in chunks of kOpqChunk.
+constexpr int kOpqTile = 256;
+constexpr int kOpqStage = 8;
+constexpr int kOpqChunk = 4096;
+
+struct OpqLayout {
+    int64_t tiles, chunks;
+    size_t counts, chunk_off, stage_idx, stage_val, total;
+};
+
+inline OpqLayout opq_layout(int64_t n)
+{
+    OpqLayout L;
+    L.tiles = (n + kOpqTile - 1) / kOpqTile;
+    L.chunks = (L.tiles + kOpqChunk - 1) / kOpqChunk;
+    size_t off = 0;
+    L.counts = off;
+    off = align_up(off + (size_t)L.tiles * 4, 256);
+    L.chunk_off = off;
+    off = align_up(off + (size_t)(L.chunks + 1) * 8, 256);
+    L.stage_idx = off;
+    off = align_up(off + (size_t)L.tiles * kOpqStage * 4, 256);
+    L.stage_val = off;
+    off = align_up(off + (size_t)L.tiles * kOpqStage * 2, 256);
+    L.total = off < 256 ? 256 : off;
+    return L;
+}
+
+}  // namespace bof4

@@ -1,0 +1,651 @@
+// Block-wise quantiser and dequantiser (Sec. 2.1 Eq. 1-3, Sec. 3.1 Eq. 4): streaming kernels.
+//
+// quantize: one lane owns 8 consecutive weights (16-byte load), a block is a group of I/8
+// lanes; shuffle butterfly for the block constant, IEEE division, 4-probe threshold search,
+// 8 codes packed into one 32-bit store per lane (128 contiguous bytes per warp).
+// dequantize: one lane owns 16 outputs (8 code bytes in, 32 or 64 bytes out).
+#include "common.cuh"
+#include "layout.h"
+
+namespace bof4 {
+
+constexpr int kQThreads = 256;
+constexpr int kQRow = kQThreads * 8;   // weights per CTA row (quantise)
+constexpr int kQUnroll = 2;            // rows in flight per CTA iteration
+constexpr int kDRow = kQThreads * 16;  // outputs per CTA row (dequantise)
+
+__device__ __forceinline__ void st_stream32(void* p, uint32_t v)
+{
+    asm volatile("st.global.cs.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_stream128(void* p, uint4 v)
+{
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y),
+                 "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+template <class ST>
+__device__ __forceinline__ void store_scale(void* scales, int64_t b, float m);
+template <>
+__device__ __forceinline__ void store_scale<F32>(void* scales, int64_t b, float m)
+{
+    static_cast<float*>(scales)[b] = m;
+}
+template <>
+__device__ __forceinline__ void store_scale<BF16>(void* scales, int64_t b, float m)
+{
+    static_cast<uint16_t*>(scales)[b] = (uint16_t)(__float_as_uint(m) >> 16);  // exact: m is a bf16 value
+}
+
+// Codes of 8 normalised weights packed as 4 bytes, even element in the high nibble.
+__device__ __forceinline__ uint32_t encode8(const float (&v)[8], float m, const float* s_xi)
+{
+    uint32_t word = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int c0 = region_of(normalise(v[2 * k], m), s_xi);
+        const int c1 = region_of(normalise(v[2 * k + 1], m), s_xi);
+        word |= (uint32_t)((c0 << 4) | c1) << (8 * k);
+    }
+    return word;
+}
+
+template <class DT, int I, bool SIGNED, class ST>
+__global__ void __launch_bounds__(kQThreads)
+quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels,
+                uint8_t* __restrict__ codes, void* __restrict__ scales)
+{
+    constexpr int LPB = I / 8;
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    make_thresholds(levels, s_xi, s_lv, threadIdx.x);
+    __syncthreads();
+    const int64_t rows = (n + kQRow - 1) / kQRow;
+    const int lane = threadIdx.x & 31;
+    for (int64_t r0 = (int64_t)blockIdx.x * kQUnroll; r0 < rows; r0 += (int64_t)gridDim.x * kQUnroll) {
+        float v[kQUnroll][8];
+        int64_t idx[kQUnroll];
+#pragma unroll
+        for (int u = 0; u < kQUnroll; ++u) {
+            idx[u] = ((r0 + u) * kQThreads + threadIdx.x) * 8;
+            if (idx[u] < n)
+                load8<DT>(w, idx[u], v[u]);
+            else
+                zero8<DT>(v[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < kQUnroll; ++u) {
+            const float m = block_constant<LPB, SIGNED>(v[u]);
+            const uint32_t word = encode8(v[u], m, s_xi);
+            if (idx[u] < n) {
+                st_stream32(codes + idx[u] / 2, word);
+                if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx[u] / I, m);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- dequantise
+
+template <class ST>
+__device__ __forceinline__ float load_scale(const void* scales, int64_t b);
+template <>
+__device__ __forceinline__ float load_scale<F32>(const void* scales, int64_t b)
+{
+    return __ldg(static_cast<const float*>(scales) + b);
+}
+template <>
+__device__ __forceinline__ float load_scale<BF16>(const void* scales, int64_t b)
+{
+    return __uint_as_float((uint32_t)__ldg(static_cast<const uint16_t*>(scales) + b) << 16);
+}
+
+template <class ST, class OT, int I>
+__global__ void __launch_bounds__(kQThreads)
+dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t n,
+                  const float* __restrict__ levels, void* __restrict__ out)
+{
+    __shared__ float s_lv[kLevels];
+    if (threadIdx.x < kLevels) s_lv[threadIdx.x] = levels[threadIdx.x];
+    __syncthreads();
+    const int64_t rows = (n + kDRow - 1) / kDRow;
+    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+        const int64_t idx = (r * kQThreads + threadIdx.x) * 16;
+        if (idx >= n) continue;
+        uint2 cc;
+        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];"
+                     : "=r"(cc.x), "=r"(cc.y)
+                     : "l"(codes + idx / 2));
+        const float m = load_scale<ST>(scales, idx / I);
+        float o[16];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t byte = ((k < 4 ? cc.x : cc.y) >> (8 * (k & 3))) & 0xffu;
+            o[2 * k] = __fmul_rn(m, s_lv[byte >> 4]);
+            o[2 * k + 1] = __fmul_rn(m, s_lv[byte & 15u]);
+        }
+        if (OT::code == BF16::code) {
+            uint32_t p[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) p[k] = bf16_rne(o[2 * k]) | (bf16_rne(o[2 * k + 1]) << 16);
+            uint16_t* dst = static_cast<uint16_t*>(out) + idx;
+            st_stream128(dst, make_uint4(p[0], p[1], p[2], p[3]));
+            st_stream128(dst + 8, make_uint4(p[4], p[5], p[6], p[7]));
+        } else {
+            float* dst = static_cast<float*>(out) + idx;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                st_stream128(dst + 4 * k, make_uint4(__float_as_uint(o[4 * k]), __float_as_uint(o[4 * k + 1]),
+                                                     __float_as_uint(o[4 * k + 2]), __float_as_uint(o[4 * k + 3])));
+        }
+    }
+}
+
+// Outliers written back over the dequantised tensor (Sec. 3.3, decoding side).
+template <class OT>
+__global__ void scatter_outliers_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict__ val,
+                                        const int64_t* __restrict__ n_out, int64_t capacity, int64_t n,
+                                        void* __restrict__ out)
+{
+    int64_t k_end = *n_out;
+    if (k_end > capacity) k_end = capacity;
+    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < k_end;
+         k += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = idx[k];
+        if (i < 0 || i >= n) continue;
+        if (OT::code == BF16::code)
+            static_cast<uint16_t*>(out)[i] = val[k];
+        else
+            static_cast<float*>(out)[i] = __uint_as_float((uint32_t)val[k] << 16);
+    }
+}
+
+// ---------------------------------------------------------------- OPQ (Sec. 3.3, App. E)
+
+// Balanced binary summation tree over the block: neighbours first inside the lane, then the
+// lane butterfly.  Every addition is a separate fp32 RN operation.
+template <int LPB>
+__device__ __forceinline__ float tree_sum(const float (&t)[8])
+{
+    float s = __fadd_rn(__fadd_rn(__fadd_rn(t[0], t[1]), __fadd_rn(t[2], t[3])),
+                        __fadd_rn(__fadd_rn(t[4], t[5]), __fadd_rn(t[6], t[7])));
+#pragma unroll
+    for (int off = 1; off < LPB; off <<= 1) s = __fadd_rn(s, __shfl_xor_sync(kFull, s, off));
+    return s;
+}
+
+// Bit k of the result is set iff element k of this lane is an outlier of its block:
+// |w| > sigma_b * tau, sigma_b the corrected sample standard deviation (two-pass, fp32).
+template <int I>
+__device__ __forceinline__ unsigned outlier_mask(const float (&v)[8], float tau)
+{
+    constexpr int LPB = I / 8;
+    const float mean = __fdiv_rn(tree_sum<LPB>(v), (float)I);
+    float q[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const float d = __fsub_rn(v[k], mean);
+        q[k] = __fmul_rn(d, d);
+    }
+    const float sigma = __fsqrt_rn(__fdiv_rn(tree_sum<LPB>(q), (float)(I - 1)));
+    const float thr = __fmul_rn(sigma, tau);
+    unsigned o = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) o |= (fabsf(v[k]) > thr) ? (1u << k) : 0u;
+    return o;
+}
+
+// Exclusive prefix of a per-lane count over the warp, and the warp total.
+__device__ __forceinline__ int warp_excl_scan(int cnt, int lane, int& total)
+{
+    int inc = cnt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(kFull, inc, off);
+        if (lane >= off) inc += t;
+    }
+    total = __shfl_sync(kFull, inc, 31);
+    return inc - cnt;
+}
+
+template <class DT>
+__device__ __forceinline__ void store8(void* base, int64_t idx, const float (&v)[8]);
+template <>
+__device__ __forceinline__ void store8<BF16>(void* base, int64_t idx, const float (&v)[8])
+{
+    uint32_t p[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        p[k] = (__float_as_uint(v[2 * k]) >> 16) | (__float_as_uint(v[2 * k + 1]) & 0xffff0000u);
+    st_stream128(static_cast<uint16_t*>(base) + idx, make_uint4(p[0], p[1], p[2], p[3]));
+}
+template <>
+__device__ __forceinline__ void store8<F32>(void* base, int64_t idx, const float (&v)[8])
+{
+    float* d = static_cast<float*>(base) + idx;
+    st_stream128(d, make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])));
+    st_stream128(d + 4, make_uint4(__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7])));
+}
+
+// Pass 1 of OPQ.  Each warp iteration is one tile of kOpqTile weights: outliers are detected,
+// counted (counts[tile]) and the first kOpqStage of the tile staged in ascending index order;
+// the cleaned weights are quantised (QUANT) or stored (w_clean != NULL).
+template <class DT, int I, bool SIGNED, class ST, bool QUANT>
+__global__ void __launch_bounds__(kQThreads)
+opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels, float tau,
+                 uint8_t* __restrict__ codes, void* __restrict__ scales, void* __restrict__ w_clean,
+                 int32_t* __restrict__ counts, int32_t* __restrict__ stage_idx,
+                 uint16_t* __restrict__ stage_val)
+{
+    constexpr int LPB = I / 8;
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    if (QUANT) make_thresholds(levels, s_xi, s_lv, threadIdx.x);
+    __syncthreads();
+    const int64_t rows = (n + kQRow - 1) / kQRow;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+        const int64_t idx = (r * kQThreads + threadIdx.x) * 8;
+        const int64_t tile = r * (kQThreads / 32) + warp;
+        const bool tile_ok = tile * kOpqTile < n;  // warp-uniform
+        float v[8];
+        if (idx < n)
+            load8<DT>(w, idx, v);
+        else
+            zero8<DT>(v);
+        const unsigned o = outlier_mask<I>(v, tau);
+        const unsigned any = __ballot_sync(kFull, o != 0u);
+        if (any) {
+            int total;
+            int pos = warp_excl_scan(__popc(o), lane, total);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if ((o >> k) & 1u) {
+                    if (pos < kOpqStage) {
+                        stage_idx[tile * kOpqStage + pos] = (int32_t)(idx + k);
+                        stage_val[tile * kOpqStage + pos] = (uint16_t)bf16_rne(v[k]);
+                    }
+                    ++pos;
+                    v[k] = 0.0f;
+                }
+            if (lane == 0) counts[tile] = total;
+        } else if (lane == 0 && tile_ok) {
+            counts[tile] = 0;
+        }
+        if (QUANT) {
+            const float m = block_constant<LPB, SIGNED>(v);
+            const uint32_t word = encode8(v, m, s_xi);
+            if (idx < n) {
+                st_stream32(codes + idx / 2, word);
+                if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx / I, m);
+            }
+        } else if (w_clean != nullptr && idx < n) {
+            store8<DT>(w_clean, idx, v);
+        }
+    }
+}
+
+// Pass 2a: outlier count of every chunk of kOpqChunk tiles.
+__global__ void __launch_bounds__(256)
+opq_chunk_sum_kernel(const int32_t* __restrict__ counts, int64_t tiles, int64_t* __restrict__ chunk_off)
+{
+    __shared__ int64_t s_part[8];
+    const int64_t t0 = (int64_t)blockIdx.x * kOpqChunk;
+    int64_t s = 0;
+    for (int k = threadIdx.x; k < kOpqChunk; k += 256)
+        if (t0 + k < tiles) s += counts[t0 + k];
+#pragma unroll
+    for (int off = 16; off; off >>= 1) s += __shfl_xor_sync(kFull, s, off);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t t = 0;
+        for (int k = 0; k < 8; ++k) t += s_part[k];
+        chunk_off[blockIdx.x] = t;
+    }
+}
+
+// Pass 2b: exclusive scan of the chunk sums in place (one CTA); total -> chunk_off[chunks], *n_out.
+__global__ void __launch_bounds__(1024)
+opq_chunk_scan_kernel(int64_t* __restrict__ chunk_off, int64_t chunks, int64_t* __restrict__ n_out)
+{
+    __shared__ int64_t s_sum[1024];
+    const int64_t per = (chunks + 1023) / 1024;
+    const int64_t lo = threadIdx.x * per, hi = (lo + per < chunks) ? lo + per : chunks;
+    int64_t s = 0;
+    for (int64_t k = lo; k < hi; ++k) s += chunk_off[k];
+    s_sum[threadIdx.x] = s;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+        const int64_t t = (threadIdx.x >= off) ? s_sum[threadIdx.x - off] : 0;
+        __syncthreads();
+        s_sum[threadIdx.x] += t;
+        __syncthreads();
+    }
+    int64_t run = s_sum[threadIdx.x] - s;
+    for (int64_t k = lo; k < hi; ++k) {
+        const int64_t c = chunk_off[k];
+        chunk_off[k] = run;
+        run += c;
+    }
+    if (threadIdx.x == 1023) {
+        chunk_off[chunks] = s_sum[1023];
+        *n_out = s_sum[1023];
+    }
+}
+
+// Pass 3: every tile's staged outliers are copied to their final, globally ascending position;
+// a tile with more than kOpqStage outliers is re-derived from the weights by one warp.
+template <class DT, int I>
+__global__ void __launch_bounds__(256)
+opq_gather_kernel(const void* __restrict__ w, int64_t n, float tau, const int32_t* __restrict__ counts,
+                  int64_t tiles, const int64_t* __restrict__ chunk_off,
+                  const int32_t* __restrict__ stage_idx, const uint16_t* __restrict__ stage_val,
+                  int32_t* __restrict__ out_idx, uint16_t* __restrict__ out_val, int64_t capacity)
+{
+    constexpr int PER = kOpqChunk / 256;  // consecutive tiles per thread
+    __shared__ int64_t s_warp[8];
+    __shared__ int32_t s_ovf_tile[kOpqChunk];  // tile index relative to the chunk
+    __shared__ int32_t s_ovf_off[kOpqChunk];   // offset relative to the chunk's first output
+    __shared__ int s_novf;
+    if (threadIdx.x == 0) s_novf = 0;
+    __syncthreads();
+    const int64_t t0 = (int64_t)blockIdx.x * kOpqChunk + (int64_t)threadIdx.x * PER;
+    int c[PER];
+    int local = 0;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+        c[k] = (t0 + k < tiles) ? counts[t0 + k] : 0;
+        local += c[k];
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int wtotal;
+    int excl = warp_excl_scan(local, lane, wtotal);
+    if (lane == 0) s_warp[warp] = wtotal;
+    __syncthreads();
+    int rel = excl;
+    for (int k = 0; k < warp; ++k) rel += (int)s_warp[k];
+    const int64_t base = chunk_off[blockIdx.x];
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+        if (c[k] > 0) {
+            if (c[k] <= kOpqStage) {
+                for (int j = 0; j < c[k]; ++j) {
+                    const int64_t dst = base + rel + j;
+                    if (dst < capacity) {
+                        out_idx[dst] = stage_idx[(t0 + k) * kOpqStage + j];
+                        out_val[dst] = stage_val[(t0 + k) * kOpqStage + j];
+                    }
+                }
+            } else {
+                const int slot = atomicAdd(&s_novf, 1);
+                s_ovf_tile[slot] = threadIdx.x * PER + k;
+                s_ovf_off[slot] = rel;
+            }
+        }
+        rel += c[k];
+    }
+    __syncthreads();
+    const int novf = s_novf;
+    for (int s = warp; s < novf; s += 8) {
+        const int64_t tile = (int64_t)blockIdx.x * kOpqChunk + s_ovf_tile[s];
+        const int64_t idx = tile * kOpqTile + lane * 8;
+        float v[8];
+        if (idx < n)
+            load8<DT>(w, idx, v);
+        else
+            zero8<DT>(v);
+        const unsigned o = outlier_mask<I>(v, tau);
+        int total;
+        int pos = warp_excl_scan(__popc(o), lane, total);
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if ((o >> k) & 1u) {
+                const int64_t dst = base + s_ovf_off[s] + pos;
+                if (dst < capacity) {
+                    out_idx[dst] = (int32_t)(idx + k);
+                    out_val[dst] = (uint16_t)bf16_rne(v[k]);
+                }
+                ++pos;
+            }
+    }
+}
+
+}  // namespace bof4
+
+// ================================================================= launchers (C ABI)
+
+namespace {
+
+using namespace bof4;
+
+int grid_for(int64_t rows, int per_sm)
+{
+    const int64_t cap = (int64_t)kSMs * per_sm;
+    return (int)(rows < 1 ? 1 : (rows < cap ? rows : cap));
+}
+
+int check_common(const char* fn, int64_t n, int block_size)
+{
+    if (n < 0) {
+        set_error("%s: n is negative", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (!valid_block_size(block_size)) {
+        set_error("%s: block_size %d is not one of 32, 64, 128, 256", fn, block_size);
+        return BOF4_ERR_SHAPE;
+    }
+    if (n % block_size) {
+        set_error("%s: n = %lld is not a multiple of block_size %d", fn, (long long)n, block_size);
+        return BOF4_ERR_SHAPE;
+    }
+    return BOF4_OK;
+}
+
+int check_quant_dtypes(const char* fn, int w_dtype, int scale_dtype, int norm)
+{
+    if (norm != BOF4_NORM_ABS && norm != BOF4_NORM_SIGNED) {
+        set_error("%s: norm must be BOF4_NORM_ABS or BOF4_NORM_SIGNED", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (w_dtype != BOF4_F32 && w_dtype != BOF4_BF16) {
+        set_error("%s: unknown weight dtype %d", fn, w_dtype);
+        return BOF4_ERR_DTYPE;
+    }
+    if (scale_dtype != BOF4_F32 && scale_dtype != BOF4_BF16) {
+        set_error("%s: unknown scale dtype %d", fn, scale_dtype);
+        return BOF4_ERR_DTYPE;
+    }
+    if (w_dtype == BOF4_F32 && scale_dtype == BOF4_BF16) {
+        set_error("%s: fp32 weights need fp32 scales (the block constant is stored exactly)", fn);
+        return BOF4_ERR_DTYPE;
+    }
+    return BOF4_OK;
+}
+
+// Expands BODY with DT, I_, SG, ST bound to the template arguments of the runtime configuration.
+#define BOF4_DISPATCH_I(I_VAL, ...)                    \
+    switch (I_VAL) {                                   \
+        case 32: { constexpr int I_ = 32; __VA_ARGS__; } break;   \
+        case 64: { constexpr int I_ = 64; __VA_ARGS__; } break;   \
+        case 128: { constexpr int I_ = 128; __VA_ARGS__; } break; \
+        default: { constexpr int I_ = 256; __VA_ARGS__; } break;  \
+    }
+#define BOF4_DISPATCH_BOOL(FLAG, NAME, ...)                \
+    if (FLAG) { constexpr bool NAME = true; __VA_ARGS__; } \
+    else { constexpr bool NAME = false; __VA_ARGS__; }
+// (weight dtype, scale dtype) in {(f32,f32), (bf16,bf16), (bf16,f32)}
+#define BOF4_DISPATCH_WS(WD, SD, ...)                                               \
+    if ((WD) == BOF4_F32) { using DT = F32; using ST = F32; __VA_ARGS__; }          \
+    else if ((SD) == BOF4_BF16) { using DT = BF16; using ST = BF16; __VA_ARGS__; }  \
+    else { using DT = BF16; using ST = F32; __VA_ARGS__; }
+
+}  // namespace
+
+extern "C" int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_size, int norm,
+                             const float* d_codebook, uint8_t* d_codes, void* d_scales,
+                             int scale_dtype, void* stream)
+{
+    int rc = check_common("bof4_quantize", n, block_size);
+    if (rc) return rc;
+    rc = check_quant_dtypes("bof4_quantize", w_dtype, scale_dtype, norm);
+    if (rc) return rc;
+    if (n == 0) return BOF4_OK;
+    if (!d_w || !d_codebook || !d_codes || !d_scales) {
+        set_error("bof4_quantize: NULL pointer");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t rows = (n + kQRow - 1) / kQRow;
+    const int grid = grid_for((rows + kQUnroll - 1) / kQUnroll, 8);
+    BOF4_DISPATCH_WS(w_dtype, scale_dtype,
+        BOF4_DISPATCH_I(block_size,
+            BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                (quantize_kernel<DT, I_, SG, ST><<<grid, kQThreads, 0, st>>>(d_w, n, d_codebook, d_codes, d_scales)))));
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
+}
+
+extern "C" int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int scale_dtype,
+                               int64_t n, int block_size, const float* d_codebook,
+                               const int32_t* d_out_idx, const void* d_out_val,
+                               const int64_t* d_n_out, int64_t capacity, void* d_out,
+                               int out_dtype, void* stream)
+{
+    int rc = check_common("bof4_dequantize", n, block_size);
+    if (rc) return rc;
+    if ((scale_dtype != BOF4_F32 && scale_dtype != BOF4_BF16) ||
+        (out_dtype != BOF4_F32 && out_dtype != BOF4_BF16)) {
+        set_error("bof4_dequantize: unknown dtype");
+        return BOF4_ERR_DTYPE;
+    }
+    const bool opq = d_out_idx != nullptr;
+    if (opq && (!d_out_val || !d_n_out)) {
+        set_error("bof4_dequantize: outlier list needs d_out_idx, d_out_val and d_n_out together");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (opq && capacity < 0) {
+        set_error("bof4_dequantize: negative capacity");
+        return BOF4_ERR_CAPACITY;
+    }
+    if (n == 0) return BOF4_OK;
+    if (!d_codes || !d_scales || !d_codebook || !d_out) {
+        set_error("bof4_dequantize: NULL pointer");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t rows = (n + kDRow - 1) / kDRow;
+    const int grid = grid_for(rows, 8);
+#define BOF4_DEQ(ST_, OT_) \
+    BOF4_DISPATCH_I(block_size, (dequantize_kernel<ST_, OT_, I_><<<grid, kQThreads, 0, st>>>(d_codes, d_scales, n, d_codebook, d_out)))
+    if (scale_dtype == BOF4_F32 && out_dtype == BOF4_F32) { BOF4_DEQ(F32, F32) }
+    else if (scale_dtype == BOF4_F32) { BOF4_DEQ(F32, BF16) }
+    else if (out_dtype == BOF4_F32) { BOF4_DEQ(BF16, F32) }
+    else { BOF4_DEQ(BF16, BF16) }
+#undef BOF4_DEQ
+    BOF4_CUDA_TRY(cudaGetLastError());
+    if (opq && capacity > 0) {
+        const uint16_t* val = static_cast<const uint16_t*>(d_out_val);
+        if (out_dtype == BOF4_F32)
+            scatter_outliers_kernel<F32><<<kSMs, 256, 0, st>>>(d_out_idx, val, d_n_out, capacity, n, d_out);
+        else
+            scatter_outliers_kernel<BF16><<<kSMs, 256, 0, st>>>(d_out_idx, val, d_n_out, capacity, n, d_out);
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
+    return BOF4_OK;
+}
+
+namespace {
+
+// Shared launcher of opq_split (QUANT = false) and bof4_quantize_opq (QUANT = true).
+template <bool QUANT>
+int launch_opq(const char* fn, const void* d_w, int w_dtype, int64_t n, int block_size, int norm,
+               const float* d_codebook, float tau, uint8_t* d_codes, void* d_scales, int scale_dtype,
+               void* d_w_clean, int32_t* d_out_idx, void* d_out_val, int64_t capacity,
+               int64_t* d_n_out, void* d_ws, size_t ws_bytes, void* stream)
+{
+    int rc = check_common(fn, n, block_size);
+    if (rc) return rc;
+    rc = check_quant_dtypes(fn, w_dtype, scale_dtype, norm);
+    if (rc) return rc;
+    if (n >= ((int64_t)1 << 31)) {
+        set_error("%s: n must be below 2^31 (int32 outlier indices)", fn);
+        return BOF4_ERR_SHAPE;
+    }
+    if (capacity < 0 || capacity >= ((int64_t)1 << 31)) {
+        set_error("%s: capacity out of range", fn);
+        return BOF4_ERR_CAPACITY;
+    }
+    if (!(tau >= 0.0f)) {
+        set_error("%s: tau must be a non-negative number", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (!d_n_out || (capacity > 0 && (!d_out_idx || !d_out_val))) {
+        set_error("%s: NULL outlier output", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    const OpqLayout L = opq_layout(n);
+    if (!d_ws || ((uintptr_t)d_ws & 255u) || ws_bytes < L.total) {
+        set_error("%s: workspace NULL, not 256-byte aligned, or smaller than %zu bytes", fn, L.total);
+        return BOF4_ERR_WORKSPACE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n == 0) {
+        BOF4_CUDA_TRY(cudaMemsetAsync(d_n_out, 0, sizeof(int64_t), st));
+        return BOF4_OK;
+    }
+    if (!d_w || (QUANT && (!d_codebook || !d_codes || !d_scales))) {
+        set_error("%s: NULL pointer", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    char* ws = static_cast<char*>(d_ws);
+    int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
+    int64_t* chunk_off = reinterpret_cast<int64_t*>(ws + L.chunk_off);
+    int32_t* stage_idx = reinterpret_cast<int32_t*>(ws + L.stage_idx);
+    uint16_t* stage_val = reinterpret_cast<uint16_t*>(ws + L.stage_val);
+    uint16_t* out_val = static_cast<uint16_t*>(d_out_val);
+    const int64_t rows = (n + kQRow - 1) / kQRow;
+    const int grid = grid_for(rows, 8);
+    BOF4_DISPATCH_WS(w_dtype, scale_dtype,
+        BOF4_DISPATCH_I(block_size,
+            BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                (opq_pass1_kernel<DT, I_, SG, ST, QUANT><<<grid, kQThreads, 0, st>>>(
+                    d_w, n, d_codebook, tau, d_codes, d_scales, d_w_clean, counts, stage_idx, stage_val)))));
+    BOF4_CUDA_TRY(cudaGetLastError());
+    opq_chunk_sum_kernel<<<(int)L.chunks, 256, 0, st>>>(counts, L.tiles, chunk_off);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    opq_chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_off, L.chunks, d_n_out);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    if (capacity > 0) {
+        if (w_dtype == BOF4_F32) {
+            BOF4_DISPATCH_I(block_size, (opq_gather_kernel<F32, I_><<<(int)L.chunks, 256, 0, st>>>(
+                d_w, n, tau, counts, L.tiles, chunk_off, stage_idx, stage_val, d_out_idx, out_val, capacity)));
+        } else {
+            BOF4_DISPATCH_I(block_size, (opq_gather_kernel<BF16, I_><<<(int)L.chunks, 256, 0, st>>>(
+                d_w, n, tau, counts, L.tiles, chunk_off, stage_idx, stage_val, d_out_idx, out_val, capacity)));
+        }
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
+    return BOF4_OK;
+}
+
+}  // namespace
+
+extern "C" int opq_split(const void* d_w, int w_dtype, int64_t n, int block_size, float tau,
+                         void* d_w_clean, int32_t* d_out_idx, void* d_out_val, int64_t capacity,
+                         int64_t* d_n_out, void* d_ws, size_t ws_bytes, void* stream)
+{
+    return launch_opq<false>("opq_split", d_w, w_dtype, n, block_size, BOF4_NORM_ABS, nullptr, tau,
+                             nullptr, nullptr, w_dtype, d_w_clean, d_out_idx, d_out_val, capacity,
+                             d_n_out, d_ws, ws_bytes, stream);
+}
+
+extern "C" int bof4_quantize_opq(const void* d_w, int w_dtype, int64_t n, int block_size, int norm,
+                                 const float* d_codebook, float tau, uint8_t* d_codes,
+                                 void* d_scales, int scale_dtype, int32_t* d_out_idx,
+                                 void* d_out_val, int64_t capacity, int64_t* d_n_out, void* d_ws,
+                                 size_t ws_bytes, void* stream)
+{
+    return launch_opq<true>("bof4_quantize_opq", d_w, w_dtype, n, block_size, norm, d_codebook, tau,
+                            d_codes, d_scales, scale_dtype, nullptr, d_out_idx, d_out_val, capacity,
+                            d_n_out, d_ws, ws_bytes, stream);
+}
