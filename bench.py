@@ -139,8 +139,10 @@ class Step:
         self.cnt = torch.zeros(1, dtype=torch.int64, device=dev)
         self.out = torch.empty(n, dtype=torch.bfloat16, device=dev)
         self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-        self.cb_mse = self.cb_mae = None
+        self.cb_mse = self.cb_mae = self.cb0
+        self.log_mse = torch.zeros(1, dtype=torch.float64, device=dev)
         self.have_mae = True
+        self.only = None
 
     def flush_l2(self):
         self.flush_buf.zero_()
@@ -169,7 +171,10 @@ class Step:
     def components(self):
         comps = [("em_mse", self.em_mse, 2), ("em_mae", self.em_mae, None), ("quantize_opq", self.quant, 4),
                  ("dequantize", self.dequant, 2)]
-        return [c for c in comps if c[0] != "em_mae" or self.have_mae]
+        comps = [c for c in comps if c[0] != "em_mae" or self.have_mae]
+        if self.only:
+            comps = [c for c in comps if c[0] in self.only]
+        return comps
 
     def run_timed(self):
         """One step; returns {component: ms} from CUDA events on the current stream."""
@@ -222,6 +227,9 @@ def run_gpu(args):
 
     st = Step(bof4, dev, seed_offset=rank)       # independent problem per rank: no collective
     st.have_mae = hasattr(binding, "MAE_LAUNCHES_PER_ITERATION")
+    if args.only:
+        st.only = set(args.only.split(","))
+        args.no_e2e = args.no_cpu_baseline = True
     K, W = args.steps, args.warmup
     for _ in range(W):
         st.run_timed()
@@ -278,17 +286,16 @@ def run_gpu(args):
     ms_per_step = total_ms / K
     peak, peak_kind = measured_peak()
     avg = {k: sum(v) / len(v) for k, v in comp_ms.items()}
-    comp = {
-        "em_mse_ms": avg["em_mse"], "em_mse_gweights_s": n / avg["em_mse"] / 1e6,
-        "em_mse_gbs": BYTES_EM * n / avg["em_mse"] / 1e6,
-        "quantize_opq_ms": avg["quantize_opq"], "quantize_opq_gbs": BYTES_QUANT * n / avg["quantize_opq"] / 1e6,
-        "dequantize_ms": avg["dequantize"], "dequantize_gbs": BYTES_DEQUANT * n / avg["dequantize"] / 1e6,
-    }
-    launches = 2 + 4 + 2
-    if "em_mae" in avg:
-        comp["em_mae_ms"] = avg["em_mae"]
-        comp["em_mae_gweights_s"] = n / avg["em_mae"] / 1e6
-        launches += mae_launches(bof4)
+    bytes_per_w = {"em_mse": BYTES_EM, "em_mae": None, "quantize_opq": BYTES_QUANT, "dequantize": BYTES_DEQUANT}
+    kernels = {"em_mse": 2, "em_mae": mae_launches(bof4), "quantize_opq": 4, "dequantize": 2}
+    comp, launches = {}, 0
+    for name, ms in avg.items():
+        comp[name + "_ms"] = ms
+        if name.startswith("em_"):
+            comp[name + "_gweights_s"] = n / ms / 1e6
+        if bytes_per_w[name]:
+            comp[name + "_gbs"] = bytes_per_w[name] * n / ms / 1e6
+        launches += kernels[name]
     for k in list(comp):
         if k.endswith("_gbs"):
             comp[k.replace("_gbs", "_frac_of_%s_hbm" % peak_kind)] = comp[k] / peak
@@ -395,6 +402,8 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--only", default="", help="comma list of components to run (profiling runs only; "
+                    "the JSON line is then not a bench result)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":

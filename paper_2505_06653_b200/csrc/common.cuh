@@ -154,4 +154,106 @@ __device__ __forceinline__ int region_of(float x, const float* s_xi)
     return c;
 }
 
+// ---------------------------------------------------------------- one-probe region search
+//
+// The interval [-1, 1] of normalised weights is cut into 257 bins by the monotone map
+//     bin(x) = bits(fma(x, 128, 1.5 * 2^23 + 128)) - bits(1.5 * 2^23)  =  RN(128 x) + 128,
+// and a table gives, per bin, base = the number of thresholds that fall into LOWER bins and
+// thr = xi[base] (xi[15] = +inf).  Because bin() is monotone, every threshold in a lower bin
+// is <= x and every threshold in a higher bin is > x, so when no bin holds two thresholds
+//     region(x) = base + (x >= thr)
+// exactly.  A codebook with two thresholds in one bin (levels closer than 1/128) makes the
+// kernels fall back to the binary search.  Each table row is replicated for the 32 lanes
+// ([bin][lane], 8 bytes each) so that the shared-memory bank only depends on the lane.
+constexpr int kLutBins = 257;
+constexpr uint32_t kLutMagicBits = 0x4B400000u;  // bits of 1.5 * 2^23
+constexpr int kLutRowBytes = 32 * 8;
+constexpr int kLutBytes = kLutBins * kLutRowBytes;
+
+__device__ __forceinline__ float lut_key(float x) { return fmaf(x, 128.0f, 12583040.0f); }
+
+// Byte offset of the lane's table entry for normalised weight x; key = lut_key(x).  The
+// unsigned minimum also sends NaN / infinite keys (non-finite input) to the last row.
+__device__ __forceinline__ uint32_t lut_offset(float key, uint32_t lane_off)
+{
+    const uint32_t b = min(__float_as_uint(key), kLutMagicBits + (uint32_t)(kLutBins - 1));
+    return b * (uint32_t)kLutRowBytes + (lane_off - kLutMagicBits * (uint32_t)kLutRowBytes);
+}
+
+// Builds the table in shared memory from the thresholds; payload[base] is stored next to
+// thr (a code, or a byte offset).  Returns through *s_multi whether some bin holds two
+// thresholds.  Call with all threads of the CTA, then __syncthreads().
+template <class PayloadFn>
+__device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lut, int* s_multi,
+                                          PayloadFn payload)
+{
+    if (threadIdx.x == 0) *s_multi = 0;
+    __syncthreads();
+    for (int b = threadIdx.x; b < kLutBins; b += blockDim.x) {
+        int base = 0, inside = 0;
+#pragma unroll
+        for (int j = 0; j < kLevels - 1; ++j) {
+            int bj = (int)(__float_as_uint(lut_key(s_xi[j])) - kLutMagicBits);
+            bj = bj < 0 ? 0 : (bj > kLutBins - 1 ? kLutBins - 1 : bj);
+            base += (bj < b) ? 1 : 0;
+            inside += (bj == b) ? 1 : 0;
+        }
+        if (inside > 1) *s_multi = 1;
+        const uint2 ent = make_uint2(__float_as_uint(s_xi[base]), payload(base));
+        for (int l = 0; l < 32; ++l)
+            *reinterpret_cast<uint2*>(s_lut + b * kLutRowBytes + l * 8) = ent;
+    }
+}
+
+// ---------------------------------------------------------------- division for bf16 inputs
+//
+// For bfloat16 operands with 2^-60 <= |m| <= 2^60 the sequence
+//     r = RN(1/m);  q0 = RN(w r);  e = fma(-q0, m, w);  q = fma(e, r, q0)
+// returns exactly RN(w / m) whenever the quotient is a normal number (checked exhaustively
+// over all operand pairs on the CPU by the test-suite).  It costs three (packed) operations
+// per weight plus one reciprocal per block.
+__device__ __forceinline__ bool div_safe(float m)
+{
+    const float a = fabsf(m);
+    return a >= 0x1p-60f && a <= 0x1p60f;
+}
+
+__device__ __forceinline__ float2 fast_div2(float2 w, float m, float r)
+{
+    const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
+    const float2 q0 = __fmul2_rn(w, rr);
+    const float2 e = __ffma2_rn(q0, nm, w);
+    return __ffma2_rn(e, rr, q0);
+}
+
+// x[k] = RN(v[k] / m) for the 8 weights of a lane (x = 0 when m = 0).  FAST selects the
+// reciprocal sequence (bf16 operands only; the caller has checked div_safe for the whole
+// warp).  With GUARD, quotients below 2^-100 in magnitude are recomputed by the IEEE
+// division so that subnormal results are rounded once.
+template <bool FAST, bool GUARD>
+__device__ __forceinline__ void normalise8(const float (&v)[8], float m, float (&x)[8])
+{
+    if (FAST) {
+        const float r = __frcp_rn(m);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float2 q = fast_div2(make_float2(v[2 * k], v[2 * k + 1]), m, r);
+            x[2 * k] = q.x;
+            x[2 * k + 1] = q.y;
+        }
+        if (GUARD) {
+            const float lo = fminf(fminf(fminf(fabsf(x[0]), fabsf(x[1])), fminf(fabsf(x[2]), fabsf(x[3]))),
+                                   fminf(fminf(fabsf(x[4]), fabsf(x[5])), fminf(fabsf(x[6]), fabsf(x[7]))));
+            if (lo < 0x1p-100f) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (fabsf(x[k]) < 0x1p-100f && v[k] != 0.0f) x[k] = normalise(v[k], m);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = normalise(v[k], m);
+    }
+}
+
 }  // namespace bof4

@@ -1,23 +1,31 @@
 // Data-driven EM / Lloyd codebook fit (Sec. 3.2, App. B.3): one streaming pass per iteration.
 //
 // MSE pass (Eq. 6): every lane owns 8 consecutive weights, a block is a group of I/8 lanes.
-// Per weight: x = w / m, region c by threshold search, then
-//     s1[c] += m^2 x,  s0[c] += m^2,  count[c] += 1,  err += (w - m xhat[c])^2.
-// The level-indexed sums live in shared memory as one private column per thread (no atomics,
-// no bank conflicts: the bank is the lane), are folded into fp64 per-CTA totals in a fixed
-// order, written as one partial record per CTA, and combined by a single-CTA kernel that also
-// updates the free levels.  Nothing depends on scheduling, so results are bit-reproducible.
+// Per weight: x = w / m, region c by the one-probe table search, then
+//     s1[c] += m^2 x,   s0[c] += m^2            (one packed read-modify-write)
+// and, per lane, w2 += w^2.  The error of App. B.3 follows in the combine step from
+//     sum (w - m xhat[c])^2 = w2 - sum_l xhat[l] (2 s1[l] - xhat[l] s0[l]),
+// evaluated in fp64.  The level-indexed sums live in shared memory as one private column per
+// thread (no atomics, no bank conflicts: the bank is the lane), are folded into fp64 per-CTA
+// totals in a fixed order, written as one partial record per CTA, and combined by a single-CTA
+// kernel that also updates the free levels.  Nothing depends on scheduling, so results are
+// bit-reproducible.  The COUNT variant also keeps the member count of every region.
 #include "common.cuh"
 #include "layout.h"
 
 namespace bof4 {
 
-constexpr int kEmThreads = 256;
-constexpr int kEmRow = kEmThreads * 8;  // weights per CTA row
 constexpr int kEmUnroll = 2;            // rows in flight per CTA iteration
 constexpr int kEmMaxTensors = 64;       // tensors per launch (kernel parameter table)
 constexpr int kEmFlushIters = 128;      // loop iterations between fp32 -> fp64 folds
-constexpr size_t kEmSmemBytes = (size_t)kLevels * kEmThreads * (sizeof(float2) + sizeof(uint32_t));
+
+template <bool COUNT>
+struct EmGeo {
+    static constexpr int threads = COUNT ? 512 : 1024;
+    static constexpr int row = threads * 8;                 // weights per CTA row
+    static constexpr uint32_t acc_row_bytes = threads * 8;  // one level's float2 columns
+    static constexpr size_t smem = (size_t)kLutBytes + (size_t)kLevels * threads * (COUNT ? 12 : 8);
+};
 
 struct EmTensors {
     const void* ptr[kEmMaxTensors];
@@ -27,20 +35,25 @@ struct EmTensors {
     int accumulate;  // 0: this launch overwrites the partial records, 1: adds to them
 };
 
-// Record layout in doubles: [0,16) s1, [16,32) s0, [32,48) count (uint64 bits), [48] err.
-constexpr int kRecS1 = 0, kRecS0 = 16, kRecCnt = 32, kRecErr = 48;
+// Record layout in doubles: [0,16) s1, [16,32) s0, [32,48) count (uint64 bits), [48] sum w^2.
+constexpr int kRecS1 = 0, kRecS0 = 16, kRecCnt = 32, kRecW2 = 48;
 
-template <class DT, int I, bool SIGNED>
-__global__ void __launch_bounds__(kEmThreads, 4)
+template <class DT, int I, bool SIGNED, bool COUNT>
+__global__ void __launch_bounds__(EmGeo<COUNT>::threads, 1)
 em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __restrict__ partials)
 {
+    using G = EmGeo<COUNT>;
     constexpr int LPB = I / 8;
+    constexpr int NT = G::threads, NW = NT / 32, NSEG = NW / kLevels;
     extern __shared__ __align__(16) unsigned char s_raw[];
-    float2* s_acc = reinterpret_cast<float2*>(s_raw);                              // [16][threads]
-    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_raw + kLevels * kEmThreads * sizeof(float2));
+    unsigned char* s_lut = s_raw;
+    unsigned char* s_acc = s_raw + kLutBytes;                           // float2 [16][NT]
+    unsigned char* s_cnt = s_acc + (size_t)kLevels * G::acc_row_bytes;  // uint32 [16][NT] (COUNT)
     __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ int s_multi;
+    __shared__ double s_part[NSEG][3][kLevels];
     __shared__ double s_tot[3 * kLevels];  // s1, s0, count (as uint64 bits)
-    __shared__ double s_err[kEmThreads / 32];
+    __shared__ double s_w2[NW];
     __shared__ const void* s_ptr[kEmMaxTensors];
     __shared__ int64_t s_n[kEmMaxTensors], s_row_end[kEmMaxTensors];
 
@@ -54,43 +67,67 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
     }
 #pragma unroll
     for (int l = 0; l < kLevels; ++l) {
-        s_acc[l * kEmThreads + tid] = make_float2(0.0f, 0.0f);
-        s_cnt[l * kEmThreads + tid] = 0u;
+        *reinterpret_cast<float2*>(s_acc + l * G::acc_row_bytes + tid * 8) = make_float2(0.0f, 0.0f);
+        if (COUNT) *reinterpret_cast<uint32_t*>(s_cnt + l * (G::acc_row_bytes / 2) + tid * 4) = 0u;
     }
     __syncthreads();
+    build_lut(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base * G::acc_row_bytes; });
+    __syncthreads();
+    const bool lut_ok = s_multi == 0;
 
     const int64_t total_rows = T.row_end[T.count - 1];
     const int64_t stride = (int64_t)gridDim.x * kEmUnroll;
-    double err = 0.0;
+    const uint32_t lane_off = lane * 8, tid_off = tid * 8;
+    double w2sum = 0.0;
     int t_cur = 0;
     int since_flush = 0;
 
     // Folds the private fp32 columns into the fp64 CTA totals (fixed order) and clears them.
     auto flush = [&]() {
         __syncthreads();
-        for (int l = warp; l < kLevels; l += kEmThreads / 32) {
+        {
+            const int l = warp & (kLevels - 1), seg = warp >> 4;
             double a1 = 0.0, a0 = 0.0;
             unsigned long long ac = 0;
-#pragma unroll
-            for (int k = 0; k < kEmThreads / 32; ++k) {
-                const int col = l * kEmThreads + k * 32 + lane;
-                const float2 a = s_acc[col];
+            constexpr int PER = NT / NSEG / 32;  // columns per lane
+#pragma unroll 4
+            for (int k = 0; k < PER; ++k) {
+                const int col = seg * (NT / NSEG) + k * 32 + lane;
+                float2* pa = reinterpret_cast<float2*>(s_acc + l * G::acc_row_bytes + col * 8);
+                const float2 a = *pa;
                 a1 += (double)a.x;
                 a0 += (double)a.y;
-                ac += s_cnt[col];
-                s_acc[col] = make_float2(0.0f, 0.0f);
-                s_cnt[col] = 0u;
+                *pa = make_float2(0.0f, 0.0f);
+                if (COUNT) {
+                    uint32_t* pc = reinterpret_cast<uint32_t*>(s_cnt + l * (G::acc_row_bytes / 2) + col * 4);
+                    ac += *pc;
+                    *pc = 0u;
+                }
             }
 #pragma unroll
             for (int off = 16; off; off >>= 1) {
                 a1 += __shfl_xor_sync(kFull, a1, off);
                 a0 += __shfl_xor_sync(kFull, a0, off);
-                ac += __shfl_xor_sync(kFull, ac, off);
+                if (COUNT) ac += __shfl_xor_sync(kFull, ac, off);
             }
             if (lane == 0) {
-                s_tot[l] += a1;
-                s_tot[kLevels + l] += a0;
-                reinterpret_cast<unsigned long long*>(s_tot)[2 * kLevels + l] += ac;
+                s_part[seg][0][l] = a1;
+                s_part[seg][1][l] = a0;
+                s_part[seg][2][l] = __longlong_as_double((long long)ac);
+            }
+        }
+        __syncthreads();
+        if (tid < 3 * kLevels) {
+            const int q = tid / kLevels, l = tid % kLevels;
+            if (q < 2) {
+                double a = s_tot[tid];
+                for (int sg = 0; sg < NSEG; ++sg) a += s_part[sg][q][l];
+                s_tot[tid] = a;
+            } else {
+                unsigned long long a = (unsigned long long)__double_as_longlong(s_tot[tid]);
+                for (int sg = 0; sg < NSEG; ++sg)
+                    a += (unsigned long long)__double_as_longlong(s_part[sg][2][l]);
+                s_tot[tid] = __longlong_as_double((long long)a);
             }
         }
         __syncthreads();
@@ -106,7 +143,7 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
             if (g < total_rows) {
                 while (g >= s_row_end[t_cur]) ++t_cur;
                 const int64_t r = g - (t_cur ? s_row_end[t_cur - 1] : 0);
-                const int64_t idx = (r * kEmThreads + tid) * 8;
+                const int64_t idx = (r * NT + tid) * 8;
                 ok[u] = idx < s_n[t_cur];
                 if (ok[u]) load8<DT>(s_ptr[t_cur], idx, v[u]);
             }
@@ -115,23 +152,36 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
 #pragma unroll
         for (int u = 0; u < kEmUnroll; ++u) {
             const float m = block_constant<LPB, SIGNED>(v[u]);
+            const bool fast = __all_sync(kFull, div_safe(m) || !ok[u]);
+            float x[8];
+            if (DT::code == BF16::code && fast)
+                normalise8<true, false>(v[u], m, x);
+            else
+                normalise8<false, false>(v[u], m, x);
+            float2 sq = make_float2(0.0f, 0.0f);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 vv = make_float2(v[u][2 * k], v[u][2 * k + 1]);
+                sq = __ffma2_rn(vv, vv, sq);
+            }
+            w2sum += (double)(sq.x + sq.y);  // invalid lanes hold zeros
             if (ok[u]) {
                 const float m2 = m * m;
-                float e = 0.0f;
+                const float2 mm = make_float2(m2, m2);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    const float x = normalise(v[u][k], m);
-                    const int c = region_of(x, s_xi);
-                    const float d = fmaf(-m, s_lv[c], v[u][k]);
-                    e = fmaf(d, d, e);
-                    const int col = c * kEmThreads + tid;
-                    float2 a = s_acc[col];
-                    a.x = fmaf(m2, x, a.x);
-                    a.y += m2;
-                    s_acc[col] = a;
-                    s_cnt[col] += 1u;
+                    uint32_t off;
+                    if (lut_ok) {
+                        const uint2 ent =
+                            *reinterpret_cast<const uint2*>(s_lut + lut_offset(lut_key(x[k]), lane_off));
+                        off = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? G::acc_row_bytes : 0u) + tid_off;
+                    } else {
+                        off = (uint32_t)region_of(x[k], s_xi) * G::acc_row_bytes + tid_off;
+                    }
+                    float2* pa = reinterpret_cast<float2*>(s_acc + off);
+                    *pa = __ffma2_rn(mm, make_float2(x[k], 1.0f), *pa);
+                    if (COUNT) *reinterpret_cast<uint32_t*>(s_cnt + (off >> 1)) += 1u;
                 }
-                err += (double)e;
             }
         }
         if (++since_flush == kEmFlushIters) {
@@ -141,15 +191,15 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
     }
     flush();
 
-    // error: fixed-order fold over the CTA
+    // sum of squares: fixed-order fold over the CTA
 #pragma unroll
-    for (int off = 16; off; off >>= 1) err += __shfl_xor_sync(kFull, err, off);
-    if (lane == 0) s_err[warp] = err;
+    for (int off = 16; off; off >>= 1) w2sum += __shfl_xor_sync(kFull, w2sum, off);
+    if (lane == 0) s_w2[warp] = w2sum;
     __syncthreads();
     double* rec = partials + (size_t)blockIdx.x * kEmRecordDoubles;
     if (tid < kLevels) {
         unsigned long long* rc = reinterpret_cast<unsigned long long*>(rec);
-        const unsigned long long cnt = reinterpret_cast<unsigned long long*>(s_tot)[2 * kLevels + tid];
+        const unsigned long long cnt = (unsigned long long)__double_as_longlong(s_tot[2 * kLevels + tid]);
         if (T.accumulate) {
             rec[kRecS1 + tid] += s_tot[tid];
             rec[kRecS0 + tid] += s_tot[kLevels + tid];
@@ -162,8 +212,8 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
     }
     if (tid == 0) {
         double e = 0.0;
-        for (int k = 0; k < kEmThreads / 32; ++k) e += s_err[k];
-        rec[kRecErr] = T.accumulate ? rec[kRecErr] + e : e;
+        for (int k = 0; k < NW; ++k) e += s_w2[k];
+        rec[kRecW2] = T.accumulate ? rec[kRecW2] + e : e;
     }
 }
 
@@ -171,15 +221,17 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
 //   stats    != NULL: receives the combined record
 //   codebook != NULL: every free level with s0 > 0 becomes (float)(s1 / s0)      (Eq. 6)
 //   err_slot != NULL: receives err_sum / n_total
+// err_sum = w2 - sum_l xhat[l] (2 s1[l] - xhat[l] s0[l]) with the levels that produced the sums.
 __global__ void __launch_bounds__(1024)
 em_mse_finalize_kernel(const double* __restrict__ partials, int n_records, int64_t n_total,
                        const float* levels_in, bof4_em_stats* __restrict__ stats,
                        float* codebook, uint32_t fixed_mask, double* __restrict__ err_slot)
 {
-    __shared__ double s_q[kRecErr + 1];
+    __shared__ double s_q[kRecW2 + 1];
+    __shared__ double s_corr[kLevels];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int q = warp; q <= kRecErr; q += 32) {
-        const bool is_count = q >= kRecCnt && q < kRecErr;
+    for (int q = warp; q <= kRecW2; q += 32) {
+        const bool is_count = q >= kRecCnt && q < kRecW2;
         double a = 0.0;
         unsigned long long c = 0;
         for (int r = lane; r < n_records; r += 32) {
@@ -207,6 +259,7 @@ em_mse_finalize_kernel(const double* __restrict__ partials, int n_records, int64
         const double s1 = s_q[kRecS1 + l], s0 = s_q[kRecS0 + l];
         const float old = levels_in[l];
         const float cen = (s0 > 0.0) ? (float)(s1 / s0) : old;
+        s_corr[l] = (double)old * (2.0 * s1 - (double)old * s0);
         if (stats) {
             stats->s1[l] = s1;
             stats->s0[l] = s0;
@@ -215,12 +268,17 @@ em_mse_finalize_kernel(const double* __restrict__ partials, int n_records, int64
         }
         if (codebook && !((fixed_mask >> l) & 1u)) codebook[l] = cen;
     }
+    __syncthreads();
     if (threadIdx.x == 0) {
+        double corr = 0.0;
+        for (int l = 0; l < kLevels; ++l) corr += s_corr[l];
+        double err = s_q[kRecW2] - corr;
+        if (err < 0.0) err = 0.0;
         if (stats) {
-            stats->err_sum = s_q[kRecErr];
+            stats->err_sum = err;
             stats->n_total = n_total;
         }
-        if (err_slot) *err_slot = (n_total > 0) ? s_q[kRecErr] / (double)n_total : 0.0;
+        if (err_slot) *err_slot = (n_total > 0) ? err / (double)n_total : 0.0;
     }
 }
 
@@ -285,24 +343,23 @@ int check_em(const char* fn, const EmArgs& a, const void* d_codebook, void* d_ws
     return BOF4_OK;
 }
 
-template <class DT, int I, bool SG>
+template <class DT, int I, bool SG, bool COUNT>
 int launch_mse_chunk(const EmTensors& T, const float* d_codebook, double* partials, cudaStream_t st)
 {
-    static bool attr_done = false;  // per instantiation; setting it twice is harmless
-    if (!attr_done) {
-        BOF4_CUDA_TRY(cudaFuncSetAttribute(em_mse_kernel<DT, I, SG>,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEmSmemBytes));
-        attr_done = true;
-    }
-    em_mse_kernel<DT, I, SG><<<kEmGrid, kEmThreads, kEmSmemBytes, st>>>(T, d_codebook, partials);
+    using G = EmGeo<COUNT>;
+    auto kern = em_mse_kernel<DT, I, SG, COUNT>;
+    BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::smem));
+    kern<<<kEmGrid, G::threads, G::smem, st>>>(T, d_codebook, partials);
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }
 
 // Enqueues the accumulation launches of one MSE pass over all tensors (non-empty ones, in
 // list order, kEmMaxTensors per launch).  With no weights at all the records are zeroed.
+template <bool COUNT>
 int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials, cudaStream_t st)
 {
+    constexpr int kEmRow = EmGeo<COUNT>::row;
     EmTensors T;
     T.count = 0;
     T.accumulate = 0;
@@ -314,14 +371,14 @@ int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials,
         const bool sg = a.norm == BOF4_NORM_SIGNED;
 #define BOF4_EM_GO(DT_)                                                                          \
     switch (a.block_size) {                                                                      \
-        case 32: rc = sg ? launch_mse_chunk<DT_, 32, true>(T, d_codebook, partials, st)          \
-                         : launch_mse_chunk<DT_, 32, false>(T, d_codebook, partials, st); break; \
-        case 64: rc = sg ? launch_mse_chunk<DT_, 64, true>(T, d_codebook, partials, st)          \
-                         : launch_mse_chunk<DT_, 64, false>(T, d_codebook, partials, st); break; \
-        case 128: rc = sg ? launch_mse_chunk<DT_, 128, true>(T, d_codebook, partials, st)        \
-                          : launch_mse_chunk<DT_, 128, false>(T, d_codebook, partials, st); break; \
-        default: rc = sg ? launch_mse_chunk<DT_, 256, true>(T, d_codebook, partials, st)         \
-                         : launch_mse_chunk<DT_, 256, false>(T, d_codebook, partials, st); break; \
+        case 32: rc = sg ? launch_mse_chunk<DT_, 32, true, COUNT>(T, d_codebook, partials, st)          \
+                         : launch_mse_chunk<DT_, 32, false, COUNT>(T, d_codebook, partials, st); break; \
+        case 64: rc = sg ? launch_mse_chunk<DT_, 64, true, COUNT>(T, d_codebook, partials, st)          \
+                         : launch_mse_chunk<DT_, 64, false, COUNT>(T, d_codebook, partials, st); break; \
+        case 128: rc = sg ? launch_mse_chunk<DT_, 128, true, COUNT>(T, d_codebook, partials, st)        \
+                          : launch_mse_chunk<DT_, 128, false, COUNT>(T, d_codebook, partials, st); break; \
+        default: rc = sg ? launch_mse_chunk<DT_, 256, true, COUNT>(T, d_codebook, partials, st)         \
+                         : launch_mse_chunk<DT_, 256, false, COUNT>(T, d_codebook, partials, st); break; \
     }
         if (a.w_dtype == BOF4_F32) { BOF4_EM_GO(F32) } else { BOF4_EM_GO(BF16) }
 #undef BOF4_EM_GO
@@ -364,7 +421,7 @@ extern "C" int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_te
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partials = static_cast<double*>(d_ws);
     if (metric == BOF4_METRIC_MSE) {
-        rc = enqueue_mse_pass(a, d_codebook, partials, st);
+        rc = enqueue_mse_pass<true>(a, d_codebook, partials, st);
         if (rc) return rc;
         em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, kEmGrid, a.n_total, d_codebook, d_stats,
                                                    nullptr, 0u, nullptr);
@@ -391,7 +448,7 @@ extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int
     double* partials = static_cast<double*>(d_ws);
     if (metric == BOF4_METRIC_MSE) {
         for (int t = 0; t < iters; ++t) {
-            rc = enqueue_mse_pass(a, d_codebook, partials, st);
+            rc = enqueue_mse_pass<false>(a, d_codebook, partials, st);
             if (rc) return rc;
             em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, kEmGrid, a.n_total, d_codebook, nullptr,
                                                        d_codebook, fixed_mask,

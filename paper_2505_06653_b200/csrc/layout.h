@@ -11,8 +11,8 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // ---------------------------------------------------------------- EM workspace
 // [0, kEmPartialBytes)            per-CTA partial records of the MSE / error reduction
 // [kEmMaeOffset, +kEmMaeBytes)    weighted-median selection state and histograms (MAE)
-constexpr int kEmGrid = 148 * 4;          // CTAs of the accumulation kernels (4 per SM)
-constexpr int kEmRecordDoubles = 64;      // 16 s1 + 16 s0 + 16 count + err, padded to 512 B
+constexpr int kEmGrid = 148;              // CTAs of the accumulation kernels (1 per SM)
+constexpr int kEmRecordDoubles = 64;      // 16 s1 + 16 s0 + 16 count + sum w^2, padded to 512 B
 constexpr size_t kEmPartialBytes = (size_t)kEmGrid * kEmRecordDoubles * 8;
 constexpr int kMaeBins = 1024;            // bins per level and selection pass
 constexpr size_t kEmMaeOffset = 512 * 1024;

@@ -1,18 +1,21 @@
 // Block-wise quantiser and dequantiser (Sec. 2.1 Eq. 1-3, Sec. 3.1 Eq. 4): streaming kernels.
 //
 // quantize: one lane owns 8 consecutive weights (16-byte load), a block is a group of I/8
-// lanes; shuffle butterfly for the block constant, IEEE division, 4-probe threshold search,
-// 8 codes packed into one 32-bit store per lane (128 contiguous bytes per warp).
+// lanes; shuffle butterfly for the block constant, exact division (reciprocal sequence for
+// bf16, IEEE divide otherwise), one-probe table search of the region, 8 codes packed into one
+// 32-bit store per lane (128 contiguous bytes per warp).
 // dequantize: one lane owns 16 outputs (8 code bytes in, 32 or 64 bytes out).
 #include "common.cuh"
 #include "layout.h"
 
 namespace bof4 {
 
-constexpr int kQThreads = 256;
+constexpr int kQThreads = 512;         // quantise / OPQ pass 1: 2 CTAs per SM share 2 tables
 constexpr int kQRow = kQThreads * 8;   // weights per CTA row (quantise)
 constexpr int kQUnroll = 2;            // rows in flight per CTA iteration
-constexpr int kDRow = kQThreads * 16;  // outputs per CTA row (dequantise)
+constexpr int kDThreads = 256;         // dequantise
+constexpr int kDRow = kDThreads * 16;  // outputs per CTA row (dequantise)
+constexpr int kQCtasPerSm = 2;
 
 __device__ __forceinline__ void st_stream32(void* p, uint32_t v)
 {
@@ -38,30 +41,63 @@ __device__ __forceinline__ void store_scale<BF16>(void* scales, int64_t b, float
     static_cast<uint16_t*>(scales)[b] = (uint16_t)(__float_as_uint(m) >> 16);  // exact: m is a bf16 value
 }
 
-// Codes of 8 normalised weights packed as 4 bytes, even element in the high nibble.
-__device__ __forceinline__ uint32_t encode8(const float (&v)[8], float m, const float* s_xi)
+// Region setup shared by the quantising kernels: thresholds, levels and the one-probe table.
+struct QuantTables {
+    float* xi;
+    unsigned char* lut;
+    bool lut_ok;
+};
+
+__device__ __forceinline__ QuantTables setup_tables(const float* __restrict__ levels, float* s_xi,
+                                                    float* s_lv, unsigned char* s_lut, int* s_multi)
 {
+    make_thresholds(levels, s_xi, s_lv, threadIdx.x);
+    __syncthreads();
+    build_lut(s_xi, s_lut, s_multi, [](int base) { return (uint32_t)base; });
+    __syncthreads();
+    return QuantTables{s_xi, s_lut, *s_multi == 0};
+}
+
+// Codes of the 8 weights of a lane packed as 4 bytes, even element in the high nibble.
+// `fast` (warp-uniform) selects the reciprocal division; it is only ever true for bf16 input.
+template <class DT>
+__device__ __forceinline__ uint32_t encode8(const float (&v)[8], float m, bool fast, const QuantTables& T,
+                                            uint32_t lane_off)
+{
+    float x[8];
+    if (DT::code == BF16::code && fast)
+        normalise8<true, true>(v, m, x);
+    else
+        normalise8<false, false>(v, m, x);
     uint32_t word = 0;
+    if (T.lut_ok) {
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int c0 = region_of(normalise(v[2 * k], m), s_xi);
-        const int c1 = region_of(normalise(v[2 * k + 1], m), s_xi);
-        word |= (uint32_t)((c0 << 4) | c1) << (8 * k);
+        for (int k = 0; k < 8; ++k) {
+            const uint2 ent = *reinterpret_cast<const uint2*>(T.lut + lut_offset(lut_key(x[k]), lane_off));
+            const uint32_t c = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? 1u : 0u);
+            word |= c << (8 * (k >> 1) + ((k & 1) ? 0 : 4));
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            word |= (uint32_t)region_of(x[k], T.xi) << (8 * (k >> 1) + ((k & 1) ? 0 : 4));
     }
     return word;
 }
 
 template <class DT, int I, bool SIGNED, class ST>
-__global__ void __launch_bounds__(kQThreads)
+__global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
 quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels,
                 uint8_t* __restrict__ codes, void* __restrict__ scales)
 {
     constexpr int LPB = I / 8;
+    extern __shared__ __align__(16) unsigned char s_lut[];
     __shared__ float s_xi[kLevels], s_lv[kLevels];
-    make_thresholds(levels, s_xi, s_lv, threadIdx.x);
-    __syncthreads();
+    __shared__ int s_multi;
+    const QuantTables T = setup_tables(levels, s_xi, s_lv, s_lut, &s_multi);
     const int64_t rows = (n + kQRow - 1) / kQRow;
     const int lane = threadIdx.x & 31;
+    const uint32_t lane_off = lane * 8;
     for (int64_t r0 = (int64_t)blockIdx.x * kQUnroll; r0 < rows; r0 += (int64_t)gridDim.x * kQUnroll) {
         float v[kQUnroll][8];
         int64_t idx[kQUnroll];
@@ -76,7 +112,8 @@ quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__
 #pragma unroll
         for (int u = 0; u < kQUnroll; ++u) {
             const float m = block_constant<LPB, SIGNED>(v[u]);
-            const uint32_t word = encode8(v[u], m, s_xi);
+            const bool fast = __all_sync(kFull, div_safe(m) || idx[u] >= n);
+            const uint32_t word = encode8<DT>(v[u], m, fast, T, lane_off);
             if (idx[u] < n) {
                 st_stream32(codes + idx[u] / 2, word);
                 if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx[u] / I, m);
@@ -101,7 +138,7 @@ __device__ __forceinline__ float load_scale<BF16>(const void* scales, int64_t b)
 }
 
 template <class ST, class OT, int I>
-__global__ void __launch_bounds__(kQThreads)
+__global__ void __launch_bounds__(kDThreads)
 dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t n,
                   const float* __restrict__ levels, void* __restrict__ out)
 {
@@ -110,7 +147,7 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ sc
     __syncthreads();
     const int64_t rows = (n + kDRow - 1) / kDRow;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
-        const int64_t idx = (r * kQThreads + threadIdx.x) * 16;
+        const int64_t idx = (r * kDThreads + threadIdx.x) * 16;
         if (idx >= n) continue;
         uint2 cc;
         asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];"
@@ -231,18 +268,21 @@ __device__ __forceinline__ void store8<F32>(void* base, int64_t idx, const float
 // counted (counts[tile]) and the first kOpqStage of the tile staged in ascending index order;
 // the cleaned weights are quantised (QUANT) or stored (w_clean != NULL).
 template <class DT, int I, bool SIGNED, class ST, bool QUANT>
-__global__ void __launch_bounds__(kQThreads)
+__global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
 opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels, float tau,
                  uint8_t* __restrict__ codes, void* __restrict__ scales, void* __restrict__ w_clean,
                  int32_t* __restrict__ counts, int32_t* __restrict__ stage_idx,
                  uint16_t* __restrict__ stage_val)
 {
     constexpr int LPB = I / 8;
+    extern __shared__ __align__(16) unsigned char s_lut[];
     __shared__ float s_xi[kLevels], s_lv[kLevels];
-    if (QUANT) make_thresholds(levels, s_xi, s_lv, threadIdx.x);
-    __syncthreads();
+    __shared__ int s_multi;
+    QuantTables T{s_xi, s_lut, false};
+    if (QUANT) T = setup_tables(levels, s_xi, s_lv, s_lut, &s_multi);
     const int64_t rows = (n + kQRow - 1) / kQRow;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lane_off = lane * 8;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
         const int64_t idx = (r * kQThreads + threadIdx.x) * 8;
         const int64_t tile = r * (kQThreads / 32) + warp;
@@ -273,7 +313,8 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
         }
         if (QUANT) {
             const float m = block_constant<LPB, SIGNED>(v);
-            const uint32_t word = encode8(v, m, s_xi);
+            const bool fast = __all_sync(kFull, div_safe(m) || idx >= n);
+            const uint32_t word = encode8<DT>(v, m, fast, T, lane_off);
             if (idx < n) {
                 st_stream32(codes + idx / 2, word);
                 if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx / I, m);
@@ -496,11 +537,13 @@ extern "C" int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t rows = (n + kQRow - 1) / kQRow;
-    const int grid = grid_for((rows + kQUnroll - 1) / kQUnroll, 8);
+    const int grid = grid_for((rows + kQUnroll - 1) / kQUnroll, kQCtasPerSm);
     BOF4_DISPATCH_WS(w_dtype, scale_dtype,
         BOF4_DISPATCH_I(block_size,
             BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
-                (quantize_kernel<DT, I_, SG, ST><<<grid, kQThreads, 0, st>>>(d_w, n, d_codebook, d_codes, d_scales)))));
+                { auto kern = quantize_kernel<DT, I_, SG, ST>;
+                  BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
+                  kern<<<grid, kQThreads, kLutBytes, st>>>(d_w, n, d_codebook, d_codes, d_scales); })));
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }
@@ -536,7 +579,7 @@ extern "C" int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int
     const int64_t rows = (n + kDRow - 1) / kDRow;
     const int grid = grid_for(rows, 8);
 #define BOF4_DEQ(ST_, OT_) \
-    BOF4_DISPATCH_I(block_size, (dequantize_kernel<ST_, OT_, I_><<<grid, kQThreads, 0, st>>>(d_codes, d_scales, n, d_codebook, d_out)))
+    BOF4_DISPATCH_I(block_size, (dequantize_kernel<ST_, OT_, I_><<<grid, kDThreads, 0, st>>>(d_codes, d_scales, n, d_codebook, d_out)))
     if (scale_dtype == BOF4_F32 && out_dtype == BOF4_F32) { BOF4_DEQ(F32, F32) }
     else if (scale_dtype == BOF4_F32) { BOF4_DEQ(F32, BF16) }
     else if (out_dtype == BOF4_F32) { BOF4_DEQ(BF16, F32) }
@@ -604,12 +647,15 @@ int launch_opq(const char* fn, const void* d_w, int w_dtype, int64_t n, int bloc
     uint16_t* stage_val = reinterpret_cast<uint16_t*>(ws + L.stage_val);
     uint16_t* out_val = static_cast<uint16_t*>(d_out_val);
     const int64_t rows = (n + kQRow - 1) / kQRow;
-    const int grid = grid_for(rows, 8);
+    const int grid = grid_for(rows, kQCtasPerSm);
+    const int smem = QUANT ? kLutBytes : 0;
     BOF4_DISPATCH_WS(w_dtype, scale_dtype,
         BOF4_DISPATCH_I(block_size,
             BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
-                (opq_pass1_kernel<DT, I_, SG, ST, QUANT><<<grid, kQThreads, 0, st>>>(
-                    d_w, n, d_codebook, tau, d_codes, d_scales, d_w_clean, counts, stage_idx, stage_val)))));
+                { auto kern = opq_pass1_kernel<DT, I_, SG, ST, QUANT>;
+                  BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
+                  kern<<<grid, kQThreads, smem, st>>>(
+                      d_w, n, d_codebook, tau, d_codes, d_scales, d_w_clean, counts, stage_idx, stage_val); })));
     BOF4_CUDA_TRY(cudaGetLastError());
     opq_chunk_sum_kernel<<<(int)L.chunks, 256, 0, st>>>(counts, L.tiles, chunk_off);
     BOF4_CUDA_TRY(cudaGetLastError());
