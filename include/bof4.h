@@ -13,6 +13,8 @@
  *    the stream has reached the end of the enqueued work.
  *  - Weights are a flattened tensor of n elements cut into B = n / block_size contiguous blocks
  *    (Sec. 2.1).  block_size is one of 32, 64, 128, 256 and n must be a multiple of it.
+ *  - Weight tensors, code arrays and dequantised outputs are accessed with 32-byte vector
+ *    instructions: their device pointers must be 32-byte aligned (BOF4_ERR_INVALID_ARG if not).
  *  - A codebook is 16 fp32 reconstruction levels in ASCENDING order, device resident.  Code c
  *    (0..15) is the 0-based rank of the level; decision thresholds are the fp32 midpoints
  *    (xhat[j] + xhat[j+1]) * 0.5f and a value equal to a threshold belongs to the upper level

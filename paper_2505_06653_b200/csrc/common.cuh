@@ -1,10 +1,11 @@
-// Shared device helpers of the BOF4 kernels: 16-byte weight loads, block constant (Eq. 1 / Eq. 4),
+// Shared device helpers of the BOF4 kernels: 32-byte weight loads, block constant (Eq. 1 / Eq. 4),
 // normalisation (Eq. 2), region search (Sec. 3.2), plus the host-side status plumbing.
 //
-// Work layout used by every streaming kernel: one lane owns 8 consecutive weights (one 16-byte
-// load for bf16, two for fp32), so a block of I weights is owned by LPB = I / 8 neighbouring
-// lanes of one warp (4, 8, 16 or 32 lanes) and every per-block reduction is a shuffle butterfly
-// inside that lane group.
+// Work layout used by every streaming kernel: one lane owns kLaneW = 16 consecutive weights
+// (one 32-byte load for bf16, two for fp32), so a block of I weights is owned by
+// LPB = I / 16 neighbouring lanes of one warp (2, 4, 8 or 16 lanes) and every per-block
+// reduction is a shuffle butterfly inside that lane group.  One warp iteration covers
+// kWarpW = 512 consecutive weights.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -17,6 +18,8 @@ namespace bof4 {
 constexpr int kLevels = 16;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kSMs = 148;  // B200: grids are sized in multiples of this
+constexpr int kLaneW = 16;
+constexpr int kWarpW = 32 * kLaneW;
 
 // ---------------------------------------------------------------- host status plumbing
 
@@ -30,59 +33,98 @@ int cuda_fail(cudaError_t e, const char* what);
     } while (0)
 
 inline bool valid_block_size(int I) { return I == 32 || I == 64 || I == 128 || I == 256; }
+inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
-// ---------------------------------------------------------------- loads
+// ---------------------------------------------------------------- loads and stores
 
 struct F32 {
-    using scalar = float;
     static constexpr int code = BOF4_F32;
 };
 struct BF16 {
-    using scalar = uint16_t;
     static constexpr int code = BOF4_BF16;
 };
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p)
+struct Raw8 {
+    uint32_t u[8];
+};
+
+// 32 bytes, read once: no L1 allocation.
+__device__ __forceinline__ Raw8 ld_stream256(const void* p)
 {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+    Raw8 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.u[0]), "=r"(r.u[1]), "=r"(r.u[2]), "=r"(r.u[3]), "=r"(r.u[4]), "=r"(r.u[5]),
+                   "=r"(r.u[6]), "=r"(r.u[7])
                  : "l"(p));
     return r;
 }
-
-// 8 consecutive weights starting at element index idx (idx a multiple of 8), widened to fp32.
-template <class DT>
-__device__ __forceinline__ void load8(const void* base, int64_t idx, float (&v)[8]);
-
-template <>
-__device__ __forceinline__ void load8<BF16>(const void* base, int64_t idx, float (&v)[8])
+__device__ __forceinline__ void st_stream256(void* p, const Raw8& r)
 {
-    const uint4 q = ld_stream(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(base) + idx));
-    const uint32_t u[4] = {q.x, q.y, q.z, q.w};
+    asm volatile("st.global.cs.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(r.u[0]), "r"(r.u[1]),
+                 "r"(r.u[2]), "r"(r.u[3]), "r"(r.u[4]), "r"(r.u[5]), "r"(r.u[6]), "r"(r.u[7])
+                 : "memory");
+}
+__device__ __forceinline__ void st_stream64(void* p, uint32_t a, uint32_t b)
+{
+    asm volatile("st.global.cs.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(a), "r"(b) : "memory");
+}
+
+// The raw bits of the 16 weights of a lane, as loaded (1 or 2 vectors of 32 bytes).
+template <class DT>
+struct RawRow;
+template <>
+struct RawRow<BF16> {
+    Raw8 a;
+};
+template <>
+struct RawRow<F32> {
+    Raw8 a, b;
+};
+
+// idx = element index of the lane's first weight (a multiple of 16).
+template <class DT>
+__device__ __forceinline__ RawRow<DT> load_raw(const void* base, int64_t idx);
+template <>
+__device__ __forceinline__ RawRow<BF16> load_raw<BF16>(const void* base, int64_t idx)
+{
+    return RawRow<BF16>{ld_stream256(static_cast<const uint16_t*>(base) + idx)};
+}
+template <>
+__device__ __forceinline__ RawRow<F32> load_raw<F32>(const void* base, int64_t idx)
+{
+    const float* p = static_cast<const float*>(base) + idx;
+    return RawRow<F32>{ld_stream256(p), ld_stream256(p + 8)};
+}
+
+template <class DT>
+__device__ __forceinline__ RawRow<DT> zero_raw()
+{
+    RawRow<DT> r;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        v[2 * k] = __uint_as_float(u[k] << 16);
-        v[2 * k + 1] = __uint_as_float(u[k] & 0xffff0000u);
+    for (int k = 0; k < 8; ++k) r.a.u[k] = 0u;
+    if constexpr (DT::code == BOF4_F32) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) r.b.u[k] = 0u;
+    }
+    return r;
+}
+
+// Widening to fp32 (exact).
+__device__ __forceinline__ void widen(const RawRow<BF16>& r, float (&v)[kLaneW])
+{
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        v[2 * k] = __uint_as_float(r.a.u[k] << 16);
+        v[2 * k + 1] = __uint_as_float(r.a.u[k] & 0xffff0000u);
     }
 }
-
-template <>
-__device__ __forceinline__ void load8<F32>(const void* base, int64_t idx, float (&v)[8])
-{
-    const uint4* p = reinterpret_cast<const uint4*>(static_cast<const float*>(base) + idx);
-    const uint4 a = ld_stream(p), b = ld_stream(p + 1);
-    v[0] = __uint_as_float(a.x); v[1] = __uint_as_float(a.y);
-    v[2] = __uint_as_float(a.z); v[3] = __uint_as_float(a.w);
-    v[4] = __uint_as_float(b.x); v[5] = __uint_as_float(b.y);
-    v[6] = __uint_as_float(b.z); v[7] = __uint_as_float(b.w);
-}
-
-template <class DT>
-__device__ __forceinline__ void zero8(float (&v)[8])
+__device__ __forceinline__ void widen(const RawRow<F32>& r, float (&v)[kLaneW])
 {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) v[k] = 0.0f;
+    for (int k = 0; k < 8; ++k) {
+        v[k] = __uint_as_float(r.a.u[k]);
+        v[8 + k] = __uint_as_float(r.b.u[k]);
+    }
 }
 
 // fp32 -> bf16 bits, round to nearest even (finite inputs).
@@ -92,35 +134,64 @@ __device__ __forceinline__ uint32_t bf16_rne(float f)
     return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
 }
 
-// ---------------------------------------------------------------- block constant
-
-template <int LPB>
-__device__ __forceinline__ float group_max(float a)
+__device__ __forceinline__ float max3(float a, float b, float c)
 {
-#pragma unroll
-    for (int off = 1; off < LPB; off <<= 1) a = fmaxf(a, __shfl_xor_sync(kFull, a, off));
-    return a;
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
+__device__ __forceinline__ float min3(float a, float b, float c)
+{
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// ---------------------------------------------------------------- block constant
 
 // Block constant of the lane group that owns the block.  SIGNED = false: max |w| (Eq. 1).
 // SIGNED = true: the element of largest magnitude with its sign, lowest index on ties (Eq. 4).
 // An all-zero block gives +0.  Must be called by all 32 lanes.
+//
+// The signed constant is found from the block's largest and smallest element: the larger
+// magnitude wins.  Only when both +g and -g occur does the position matter; that case is
+// settled by two ballots (which lane holds the first +g, which the first -g) and, where one
+// lane holds both, by that lane's elements in index order.
 template <int LPB, bool SIGNED>
-__device__ __forceinline__ float block_constant(const float (&v)[8])
+__device__ __forceinline__ float block_constant(const float (&v)[kLaneW])
 {
-    float a = fmaxf(fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3]))),
-                    fmaxf(fmaxf(fabsf(v[4]), fabsf(v[5])), fmaxf(fabsf(v[6]), fabsf(v[7]))));
-    const float g = group_max<LPB>(a);
-    if (!SIGNED) return g;
-    float cand = v[7];
+    float mx = max3(v[0], v[1], v[2]), mn = min3(v[0], v[1], v[2]);
 #pragma unroll
-    for (int j = 6; j >= 0; --j) cand = (fabsf(v[j]) == a) ? v[j] : cand;
-    const unsigned hit = __ballot_sync(kFull, a == g);
-    const int lane = threadIdx.x & 31;
-    const int base = lane & ~(LPB - 1);
-    const unsigned grp = (LPB == 32) ? hit : ((hit >> base) & ((1u << LPB) - 1u));
-    const int src = base + __ffs(grp) - 1;
-    const float m = __shfl_sync(kFull, cand, src);
+    for (int k = 3; k < 15; k += 2) {
+        mx = max3(mx, v[k], v[k + 1]);
+        mn = min3(mn, v[k], v[k + 1]);
+    }
+    mx = fmaxf(mx, v[15]);
+    mn = fminf(mn, v[15]);
+    float gx = mx, gn = mn;
+#pragma unroll
+    for (int off = 1; off < LPB; off <<= 1) {
+        gx = fmaxf(gx, __shfl_xor_sync(kFull, gx, off));
+        gn = fminf(gn, __shfl_xor_sync(kFull, gn, off));
+    }
+    const float g = fmaxf(gx, -gn);
+    if (!SIGNED) return g;
+    float m = (gx > -gn) ? gx : gn;
+    const bool tie = (gx == -gn) && (g != 0.0f);
+    if (__any_sync(kFull, tie)) {
+        const int lane = threadIdx.x & 31;
+        const int base = lane & ~(LPB - 1);
+        const unsigned gmask = ((1u << LPB) - 1u) << base;
+        const unsigned hp = __ballot_sync(kFull, mx == g) & gmask;   // lanes holding +g
+        const unsigned hn = __ballot_sync(kFull, mn == -g) & gmask;  // lanes holding -g
+        const int lp = __ffs(hp) - 1, ln = __ffs(hn) - 1;            // -1: none
+        float first = 0.0f;  // this lane's first element of magnitude g
+#pragma unroll
+        for (int k = kLaneW - 1; k >= 0; --k) first = (fabsf(v[k]) == g) ? v[k] : first;
+        const int src = (lp >= 0 && (ln < 0 || lp <= ln)) ? lp : ln;  // lane of the block's first +-g
+        const float pick = __shfl_sync(kFull, first, src < 0 ? 0 : src);
+        if (tie) m = pick;
+    }
     return (g == 0.0f) ? 0.0f : m;
 }
 
@@ -167,22 +238,27 @@ __device__ __forceinline__ int region_of(float x, const float* s_xi)
 // ([bin][lane], 8 bytes each) so that the shared-memory bank only depends on the lane.
 constexpr int kLutBins = 257;
 constexpr uint32_t kLutMagicBits = 0x4B400000u;  // bits of 1.5 * 2^23
+constexpr float kLutMagic = 12583040.0f;         // 1.5 * 2^23 + 128
 constexpr int kLutRowBytes = 32 * 8;
 constexpr int kLutBytes = kLutBins * kLutRowBytes;
 
-__device__ __forceinline__ float lut_key(float x) { return fmaf(x, 128.0f, 12583040.0f); }
+__device__ __forceinline__ float lut_key(float x) { return fmaf(x, 128.0f, kLutMagic); }
+__device__ __forceinline__ float2 lut_key2(float2 x)
+{
+    return __ffma2_rn(x, make_float2(128.0f, 128.0f), make_float2(kLutMagic, kLutMagic));
+}
 
-// Byte offset of the lane's table entry for normalised weight x; key = lut_key(x).  The
-// unsigned minimum also sends NaN / infinite keys (non-finite input) to the last row.
+// Byte offset of the lane's table entry; key = lut_key(x).  The unsigned minimum also sends
+// NaN / infinite keys (non-finite input) to the last row, so the read stays inside the table.
 __device__ __forceinline__ uint32_t lut_offset(float key, uint32_t lane_off)
 {
     const uint32_t b = min(__float_as_uint(key), kLutMagicBits + (uint32_t)(kLutBins - 1));
     return b * (uint32_t)kLutRowBytes + (lane_off - kLutMagicBits * (uint32_t)kLutRowBytes);
 }
 
-// Builds the table in shared memory from the thresholds; payload[base] is stored next to
-// thr (a code, or a byte offset).  Returns through *s_multi whether some bin holds two
-// thresholds.  Call with all threads of the CTA, then __syncthreads().
+// Builds the table in shared memory from the thresholds; payload(base) is stored next to
+// thr (a code, or a byte offset).  *s_multi tells whether some bin holds two thresholds.
+// Call with all threads of the CTA, then __syncthreads().
 template <class PayloadFn>
 __device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lut, int* s_multi,
                                           PayloadFn payload)
@@ -210,49 +286,48 @@ __device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lu
 // For bfloat16 operands with 2^-60 <= |m| <= 2^60 the sequence
 //     r = RN(1/m);  q0 = RN(w r);  e = fma(-q0, m, w);  q = fma(e, r, q0)
 // returns exactly RN(w / m) whenever the quotient is a normal number (checked exhaustively
-// over all operand pairs on the CPU by the test-suite).  It costs three (packed) operations
-// per weight plus one reciprocal per block.
+// over all operand pairs on the CPU by the test-suite).  It costs three packed operations
+// per two weights plus one reciprocal per lane and block.
 __device__ __forceinline__ bool div_safe(float m)
 {
     const float a = fabsf(m);
     return a >= 0x1p-60f && a <= 0x1p60f;
 }
 
-__device__ __forceinline__ float2 fast_div2(float2 w, float m, float r)
+// x[k] = RN(v[k] / m) for the 16 weights of a lane (x = 0 when m = 0).  `fast` (warp-uniform;
+// only ever true for bf16 input whose block constants all pass div_safe) selects the
+// reciprocal sequence.  With GUARD, quotients below 2^-100 in magnitude are recomputed by the
+// IEEE division so that subnormal results are rounded once.
+template <bool GUARD>
+__device__ __forceinline__ void normalise16(const float (&v)[kLaneW], float m, bool fast,
+                                            float (&x)[kLaneW])
 {
-    const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
-    const float2 q0 = __fmul2_rn(w, rr);
-    const float2 e = __ffma2_rn(q0, nm, w);
-    return __ffma2_rn(e, rr, q0);
-}
-
-// x[k] = RN(v[k] / m) for the 8 weights of a lane (x = 0 when m = 0).  FAST selects the
-// reciprocal sequence (bf16 operands only; the caller has checked div_safe for the whole
-// warp).  With GUARD, quotients below 2^-100 in magnitude are recomputed by the IEEE
-// division so that subnormal results are rounded once.
-template <bool FAST, bool GUARD>
-__device__ __forceinline__ void normalise8(const float (&v)[8], float m, float (&x)[8])
-{
-    if (FAST) {
+    if (fast) {
         const float r = __frcp_rn(m);
+        const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float2 q = fast_div2(make_float2(v[2 * k], v[2 * k + 1]), m, r);
+        for (int k = 0; k < kLaneW / 2; ++k) {
+            const float2 w = make_float2(v[2 * k], v[2 * k + 1]);
+            const float2 q0 = __fmul2_rn(w, rr);
+            const float2 e = __ffma2_rn(q0, nm, w);
+            const float2 q = __ffma2_rn(e, rr, q0);
             x[2 * k] = q.x;
             x[2 * k + 1] = q.y;
         }
         if (GUARD) {
-            const float lo = fminf(fminf(fminf(fabsf(x[0]), fabsf(x[1])), fminf(fabsf(x[2]), fabsf(x[3]))),
-                                   fminf(fminf(fabsf(x[4]), fabsf(x[5])), fminf(fabsf(x[6]), fabsf(x[7]))));
+            float lo = min3(fabsf(x[0]), fabsf(x[1]), fabsf(x[2]));
+#pragma unroll
+            for (int k = 3; k < 15; k += 2) lo = min3(lo, fabsf(x[k]), fabsf(x[k + 1]));
+            lo = fminf(lo, fabsf(x[15]));
             if (lo < 0x1p-100f) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
+                for (int k = 0; k < kLaneW; ++k)
                     if (fabsf(x[k]) < 0x1p-100f && v[k] != 0.0f) x[k] = normalise(v[k], m);
             }
         }
     } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) x[k] = normalise(v[k], m);
+        for (int k = 0; k < kLaneW; ++k) x[k] = normalise(v[k], m);
     }
 }
 

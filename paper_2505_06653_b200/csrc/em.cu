@@ -1,6 +1,6 @@
 // Data-driven EM / Lloyd codebook fit (Sec. 3.2, App. B.3): one streaming pass per iteration.
 //
-// MSE pass (Eq. 6): every lane owns 8 consecutive weights, a block is a group of I/8 lanes.
+// MSE pass (Eq. 6): every lane owns 16 consecutive weights, a block is a group of I/16 lanes.
 // Per weight: x = w / m, region c by the one-probe table search, then
 //     s1[c] += m^2 x,   s0[c] += m^2            (one packed read-modify-write)
 // and, per lane, w2 += w^2.  The error of App. B.3 follows in the combine step from
@@ -15,14 +15,13 @@
 
 namespace bof4 {
 
-constexpr int kEmUnroll = 2;            // rows in flight per CTA iteration
 constexpr int kEmMaxTensors = 64;       // tensors per launch (kernel parameter table)
 constexpr int kEmFlushIters = 128;      // loop iterations between fp32 -> fp64 folds
 
 template <bool COUNT>
 struct EmGeo {
     static constexpr int threads = COUNT ? 512 : 1024;
-    static constexpr int row = threads * 8;                 // weights per CTA row
+    static constexpr int row = threads * kLaneW;            // weights per CTA row
     static constexpr uint32_t acc_row_bytes = threads * 8;  // one level's float2 columns
     static constexpr size_t smem = (size_t)kLutBytes + (size_t)kLevels * threads * (COUNT ? 12 : 8);
 };
@@ -43,7 +42,7 @@ __global__ void __launch_bounds__(EmGeo<COUNT>::threads, 1)
 em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __restrict__ partials)
 {
     using G = EmGeo<COUNT>;
-    constexpr int LPB = I / 8;
+    constexpr int LPB = I / kLaneW;
     constexpr int NT = G::threads, NW = NT / 32, NSEG = NW / kLevels;
     extern __shared__ __align__(16) unsigned char s_raw[];
     unsigned char* s_lut = s_raw;
@@ -76,7 +75,6 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
     const bool lut_ok = s_multi == 0;
 
     const int64_t total_rows = T.row_end[T.count - 1];
-    const int64_t stride = (int64_t)gridDim.x * kEmUnroll;
     const uint32_t lane_off = lane * 8, tid_off = tid * 8;
     double w2sum = 0.0;
     int t_cur = 0;
@@ -133,57 +131,68 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
         __syncthreads();
     };
 
-    for (int64_t g0 = (int64_t)blockIdx.x * kEmUnroll; g0 < total_rows; g0 += stride) {
-        float v[kEmUnroll][8];
-        bool ok[kEmUnroll];
-#pragma unroll
-        for (int u = 0; u < kEmUnroll; ++u) {
-            const int64_t g = g0 + u;
-            ok[u] = false;
-            if (g < total_rows) {
-                while (g >= s_row_end[t_cur]) ++t_cur;
-                const int64_t r = g - (t_cur ? s_row_end[t_cur - 1] : 0);
-                const int64_t idx = (r * NT + tid) * 8;
-                ok[u] = idx < s_n[t_cur];
-                if (ok[u]) load8<DT>(s_ptr[t_cur], idx, v[u]);
-            }
-            if (!ok[u]) zero8<DT>(v[u]);
+    // Loads the lane's 16 weights of global row g (zeros beyond the end of the row's tensor).
+    auto fetch = [&](int64_t g, bool& ok) -> RawRow<DT> {
+        ok = false;
+        if (g < total_rows) {
+            while (g >= s_row_end[t_cur]) ++t_cur;
+            const int64_t r = g - (t_cur ? s_row_end[t_cur - 1] : 0);
+            const int64_t idx = (r * NT + tid) * kLaneW;
+            ok = idx < s_n[t_cur];
+            if (ok) return load_raw<DT>(s_ptr[t_cur], idx);
         }
+        return zero_raw<DT>();
+    };
+
+    bool ok;
+    RawRow<DT> raw = fetch(blockIdx.x, ok);
+    for (int64_t g = blockIdx.x; g < total_rows; g += gridDim.x) {
+        bool ok_next;
+        const RawRow<DT> next = fetch(g + gridDim.x, ok_next);
+        float v[kLaneW];
+        widen(raw, v);
+        const float m = block_constant<LPB, SIGNED>(v);
+        const bool fast = (DT::code == BF16::code) && __all_sync(kFull, div_safe(m) || !ok);
+        float2 sq = make_float2(0.0f, 0.0f);
 #pragma unroll
-        for (int u = 0; u < kEmUnroll; ++u) {
-            const float m = block_constant<LPB, SIGNED>(v[u]);
-            const bool fast = __all_sync(kFull, div_safe(m) || !ok[u]);
-            float x[8];
-            if (DT::code == BF16::code && fast)
-                normalise8<true, false>(v[u], m, x);
-            else
-                normalise8<false, false>(v[u], m, x);
-            float2 sq = make_float2(0.0f, 0.0f);
+        for (int k = 0; k < kLaneW / 2; ++k) {
+            const float2 vv = make_float2(v[2 * k], v[2 * k + 1]);
+            sq = __ffma2_rn(vv, vv, sq);
+        }
+        w2sum += (double)(sq.x + sq.y);  // lanes beyond the end hold zeros
+        float x[kLaneW];
+        normalise16<false>(v, m, fast, x);
+        if (ok) {
+            const float m2 = m * m;
+            const float2 mm = make_float2(m2, m2);
+            if (lut_ok) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float2 vv = make_float2(v[u][2 * k], v[u][2 * k + 1]);
-                sq = __ffma2_rn(vv, vv, sq);
-            }
-            w2sum += (double)(sq.x + sq.y);  // invalid lanes hold zeros
-            if (ok[u]) {
-                const float m2 = m * m;
-                const float2 mm = make_float2(m2, m2);
+                for (int k = 0; k < kLaneW / 2; ++k) {
+                    const float2 key = lut_key2(make_float2(x[2 * k], x[2 * k + 1]));
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    uint32_t off;
-                    if (lut_ok) {
-                        const uint2 ent =
-                            *reinterpret_cast<const uint2*>(s_lut + lut_offset(lut_key(x[k]), lane_off));
-                        off = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? G::acc_row_bytes : 0u) + tid_off;
-                    } else {
-                        off = (uint32_t)region_of(x[k], s_xi) * G::acc_row_bytes + tid_off;
+                    for (int h = 0; h < 2; ++h) {
+                        const float xv = x[2 * k + h];
+                        const uint2 ent = *reinterpret_cast<const uint2*>(
+                            s_lut + lut_offset(h ? key.y : key.x, lane_off));
+                        const uint32_t off =
+                            ent.y + ((xv >= __uint_as_float(ent.x)) ? G::acc_row_bytes : 0u) + tid_off;
+                        float2* pa = reinterpret_cast<float2*>(s_acc + off);
+                        *pa = __ffma2_rn(mm, make_float2(xv, 1.0f), *pa);
+                        if (COUNT) *reinterpret_cast<uint32_t*>(s_cnt + (off >> 1)) += 1u;
                     }
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < kLaneW; ++k) {
+                    const uint32_t off = (uint32_t)region_of(x[k], s_xi) * G::acc_row_bytes + tid_off;
                     float2* pa = reinterpret_cast<float2*>(s_acc + off);
                     *pa = __ffma2_rn(mm, make_float2(x[k], 1.0f), *pa);
                     if (COUNT) *reinterpret_cast<uint32_t*>(s_cnt + (off >> 1)) += 1u;
                 }
             }
         }
+        raw = next;
+        ok = ok_next;
         if (++since_flush == kEmFlushIters) {
             flush();
             since_flush = 0;
@@ -321,6 +330,10 @@ int check_em(const char* fn, const EmArgs& a, const void* d_codebook, void* d_ws
     for (int t = 0; t < a.n_tensors; ++t) {
         if (a.h_n[t] < 0 || (a.h_n[t] > 0 && !a.h_w[t])) {
             set_error("%s: tensor %d has a negative size or a NULL pointer", fn, t);
+            return BOF4_ERR_INVALID_ARG;
+        }
+        if (a.h_n[t] > 0 && !aligned32(a.h_w[t])) {
+            set_error("%s: tensor %d is not 32-byte aligned", fn, t);
             return BOF4_ERR_INVALID_ARG;
         }
         if (a.h_n[t] % a.block_size) {

@@ -24,9 +24,9 @@ inline size_t em_workspace_bytes() { return kEmMaeOffset + align_up(kEmMaeBytes,
 // ---------------------------------------------------------------- OPQ workspace
 // The weights are cut into tiles of kOpqTile elements (one warp iteration).  Each tile has a
 // count and a staging slot of kOpqStage outliers; tiles are scanned in chunks of kOpqChunk.
-constexpr int kOpqTile = 256;
-constexpr int kOpqStage = 8;
-constexpr int kOpqChunk = 4096;
+constexpr int kOpqTile = 512;
+constexpr int kOpqStage = 16;
+constexpr int kOpqChunk = 2048;
 
 struct OpqLayout {
     int64_t tiles, chunks;

@@ -1,32 +1,22 @@
-// Block-wise quantiser and dequantiser (Sec. 2.1 Eq. 1-3, Sec. 3.1 Eq. 4): streaming kernels.
+// Block-wise quantiser and dequantiser (Sec. 2.1 Eq. 1-3, Sec. 3.1 Eq. 4) and the OPQ outlier
+// split (Sec. 3.3, App. E): streaming kernels.
 //
-// quantize: one lane owns 8 consecutive weights (16-byte load), a block is a group of I/8
+// quantize: one lane owns 16 consecutive weights (32-byte load), a block is a group of I/16
 // lanes; shuffle butterfly for the block constant, exact division (reciprocal sequence for
-// bf16, IEEE divide otherwise), one-probe table search of the region, 8 codes packed into one
-// 32-bit store per lane (128 contiguous bytes per warp).
+// bf16, IEEE divide otherwise), one-probe table search of the region, 16 codes packed into one
+// 64-bit store per lane (256 contiguous bytes per warp).  The next row's load is issued before
+// the current row is processed.
 // dequantize: one lane owns 16 outputs (8 code bytes in, 32 or 64 bytes out).
 #include "common.cuh"
 #include "layout.h"
 
 namespace bof4 {
 
-constexpr int kQThreads = 512;         // quantise / OPQ pass 1: 2 CTAs per SM share 2 tables
-constexpr int kQRow = kQThreads * 8;   // weights per CTA row (quantise)
-constexpr int kQUnroll = 2;            // rows in flight per CTA iteration
-constexpr int kDThreads = 256;         // dequantise
-constexpr int kDRow = kDThreads * 16;  // outputs per CTA row (dequantise)
-constexpr int kQCtasPerSm = 2;
-
-__device__ __forceinline__ void st_stream32(void* p, uint32_t v)
-{
-    asm volatile("st.global.cs.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ void st_stream128(void* p, uint4 v)
-{
-    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y),
-                 "r"(v.z), "r"(v.w)
-                 : "memory");
-}
+constexpr int kQThreads = 512;              // quantise / OPQ pass 1
+constexpr int kQRow = kQThreads * kLaneW;   // weights per CTA row
+constexpr int kQCtasPerSm = 2;              // two CTAs, each with its own region table
+constexpr int kDThreads = 256;              // dequantise
+constexpr int kDRow = kDThreads * 16;       // outputs per CTA row (dequantise)
 
 template <class ST>
 __device__ __forceinline__ void store_scale(void* scales, int64_t b, float m);
@@ -58,31 +48,50 @@ __device__ __forceinline__ QuantTables setup_tables(const float* __restrict__ le
     return QuantTables{s_xi, s_lut, *s_multi == 0};
 }
 
-// Codes of the 8 weights of a lane packed as 4 bytes, even element in the high nibble.
-// `fast` (warp-uniform) selects the reciprocal division; it is only ever true for bf16 input.
-template <class DT>
-__device__ __forceinline__ uint32_t encode8(const float (&v)[8], float m, bool fast, const QuantTables& T,
-                                            uint32_t lane_off)
+// Codes of the 16 normalised weights of a lane packed as 8 bytes (two words), even element in
+// the high nibble of its byte.
+__device__ __forceinline__ void encode16(const float (&x)[kLaneW], const QuantTables& T, uint32_t lane_off,
+                                         uint32_t& w0, uint32_t& w1)
 {
-    float x[8];
-    if (DT::code == BF16::code && fast)
-        normalise8<true, true>(v, m, x);
-    else
-        normalise8<false, false>(v, m, x);
-    uint32_t word = 0;
+    uint32_t word[2] = {0u, 0u};
     if (T.lut_ok) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint2 ent = *reinterpret_cast<const uint2*>(T.lut + lut_offset(lut_key(x[k]), lane_off));
-            const uint32_t c = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? 1u : 0u);
-            word |= c << (8 * (k >> 1) + ((k & 1) ? 0 : 4));
+        for (int k = 0; k < kLaneW / 2; ++k) {
+            const float2 key = lut_key2(make_float2(x[2 * k], x[2 * k + 1]));
+            const uint2 e0 = *reinterpret_cast<const uint2*>(T.lut + lut_offset(key.x, lane_off));
+            const uint2 e1 = *reinterpret_cast<const uint2*>(T.lut + lut_offset(key.y, lane_off));
+            const uint32_t c0 = e0.y + ((x[2 * k] >= __uint_as_float(e0.x)) ? 1u : 0u);
+            const uint32_t c1 = e1.y + ((x[2 * k + 1] >= __uint_as_float(e1.x)) ? 1u : 0u);
+            word[k >> 2] |= ((c0 << 4) | c1) << (8 * (k & 3));
         }
     } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-            word |= (uint32_t)region_of(x[k], T.xi) << (8 * (k >> 1) + ((k & 1) ? 0 : 4));
+        for (int k = 0; k < kLaneW / 2; ++k) {
+            const uint32_t c0 = (uint32_t)region_of(x[2 * k], T.xi), c1 = (uint32_t)region_of(x[2 * k + 1], T.xi);
+            word[k >> 2] |= ((c0 << 4) | c1) << (8 * (k & 3));
+        }
     }
-    return word;
+    w0 = word[0];
+    w1 = word[1];
+}
+
+// Block constant, normalisation, codes and stores for one lane-row of (cleaned) weights.
+template <class DT, int I, bool SIGNED, class ST>
+__device__ __forceinline__ void quantize_row(const float (&v)[kLaneW], int64_t idx, bool ok,
+                                             const QuantTables& T, uint32_t lane_off, int lane,
+                                             uint8_t* __restrict__ codes, void* __restrict__ scales)
+{
+    constexpr int LPB = I / kLaneW;
+    const float m = block_constant<LPB, SIGNED>(v);
+    const bool fast = (DT::code == BF16::code) && __all_sync(kFull, div_safe(m) || !ok);
+    float x[kLaneW];
+    normalise16<true>(v, m, fast, x);
+    uint32_t w0, w1;
+    encode16(x, T, lane_off, w0, w1);
+    if (ok) {
+        st_stream64(codes + idx / 2, w0, w1);
+        if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx / I, m);
+    }
 }
 
 template <class DT, int I, bool SIGNED, class ST>
@@ -90,7 +99,6 @@ __global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
 quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels,
                 uint8_t* __restrict__ codes, void* __restrict__ scales)
 {
-    constexpr int LPB = I / 8;
     extern __shared__ __align__(16) unsigned char s_lut[];
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
@@ -98,27 +106,18 @@ quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__
     const int64_t rows = (n + kQRow - 1) / kQRow;
     const int lane = threadIdx.x & 31;
     const uint32_t lane_off = lane * 8;
-    for (int64_t r0 = (int64_t)blockIdx.x * kQUnroll; r0 < rows; r0 += (int64_t)gridDim.x * kQUnroll) {
-        float v[kQUnroll][8];
-        int64_t idx[kQUnroll];
-#pragma unroll
-        for (int u = 0; u < kQUnroll; ++u) {
-            idx[u] = ((r0 + u) * kQThreads + threadIdx.x) * 8;
-            if (idx[u] < n)
-                load8<DT>(w, idx[u], v[u]);
-            else
-                zero8<DT>(v[u]);
-        }
-#pragma unroll
-        for (int u = 0; u < kQUnroll; ++u) {
-            const float m = block_constant<LPB, SIGNED>(v[u]);
-            const bool fast = __all_sync(kFull, div_safe(m) || idx[u] >= n);
-            const uint32_t word = encode8<DT>(v[u], m, fast, T, lane_off);
-            if (idx[u] < n) {
-                st_stream32(codes + idx[u] / 2, word);
-                if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx[u] / I, m);
-            }
-        }
+    int64_t r = blockIdx.x;
+    if (r >= rows) return;
+    int64_t idx = (r * kQThreads + threadIdx.x) * kLaneW;
+    RawRow<DT> raw = (idx < n) ? load_raw<DT>(w, idx) : zero_raw<DT>();
+    for (; r < rows; r += gridDim.x) {
+        const int64_t idx_next = ((r + gridDim.x) * kQThreads + threadIdx.x) * kLaneW;
+        const RawRow<DT> next = (idx_next < n) ? load_raw<DT>(w, idx_next) : zero_raw<DT>();
+        float v[kLaneW];
+        widen(raw, v);
+        quantize_row<DT, I, SIGNED, ST>(v, idx, idx < n, T, lane_off, lane, codes, scales);
+        raw = next;
+        idx = idx_next;
     }
 }
 
@@ -162,18 +161,19 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ sc
             o[2 * k + 1] = __fmul_rn(m, s_lv[byte & 15u]);
         }
         if (OT::code == BF16::code) {
-            uint32_t p[8];
+            Raw8 p;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) p[k] = bf16_rne(o[2 * k]) | (bf16_rne(o[2 * k + 1]) << 16);
-            uint16_t* dst = static_cast<uint16_t*>(out) + idx;
-            st_stream128(dst, make_uint4(p[0], p[1], p[2], p[3]));
-            st_stream128(dst + 8, make_uint4(p[4], p[5], p[6], p[7]));
+            for (int k = 0; k < 8; ++k) p.u[k] = bf16_rne(o[2 * k]) | (bf16_rne(o[2 * k + 1]) << 16);
+            st_stream256(static_cast<uint16_t*>(out) + idx, p);
         } else {
-            float* dst = static_cast<float*>(out) + idx;
+            Raw8 p, q;
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                st_stream128(dst + 4 * k, make_uint4(__float_as_uint(o[4 * k]), __float_as_uint(o[4 * k + 1]),
-                                                     __float_as_uint(o[4 * k + 2]), __float_as_uint(o[4 * k + 3])));
+            for (int k = 0; k < 8; ++k) {
+                p.u[k] = __float_as_uint(o[k]);
+                q.u[k] = __float_as_uint(o[8 + k]);
+            }
+            st_stream256(static_cast<float*>(out) + idx, p);
+            st_stream256(static_cast<float*>(out) + idx + 8, q);
         }
     }
 }
@@ -202,10 +202,13 @@ __global__ void scatter_outliers_kernel(const int32_t* __restrict__ idx, const u
 // Balanced binary summation tree over the block: neighbours first inside the lane, then the
 // lane butterfly.  Every addition is a separate fp32 RN operation.
 template <int LPB>
-__device__ __forceinline__ float tree_sum(const float (&t)[8])
+__device__ __forceinline__ float tree_sum(const float (&t)[kLaneW])
 {
-    float s = __fadd_rn(__fadd_rn(__fadd_rn(t[0], t[1]), __fadd_rn(t[2], t[3])),
-                        __fadd_rn(__fadd_rn(t[4], t[5]), __fadd_rn(t[6], t[7])));
+    float a[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) a[k] = __fadd_rn(t[2 * k], t[2 * k + 1]);
+    float s = __fadd_rn(__fadd_rn(__fadd_rn(a[0], a[1]), __fadd_rn(a[2], a[3])),
+                        __fadd_rn(__fadd_rn(a[4], a[5]), __fadd_rn(a[6], a[7])));
 #pragma unroll
     for (int off = 1; off < LPB; off <<= 1) s = __fadd_rn(s, __shfl_xor_sync(kFull, s, off));
     return s;
@@ -214,13 +217,13 @@ __device__ __forceinline__ float tree_sum(const float (&t)[8])
 // Bit k of the result is set iff element k of this lane is an outlier of its block:
 // |w| > sigma_b * tau, sigma_b the corrected sample standard deviation (two-pass, fp32).
 template <int I>
-__device__ __forceinline__ unsigned outlier_mask(const float (&v)[8], float tau)
+__device__ __forceinline__ unsigned outlier_mask(const float (&v)[kLaneW], float tau)
 {
-    constexpr int LPB = I / 8;
-    const float mean = __fdiv_rn(tree_sum<LPB>(v), (float)I);
-    float q[8];
+    constexpr int LPB = I / kLaneW;
+    const float mean = __fmul_rn(tree_sum<LPB>(v), 1.0f / (float)I);  // exact: I is a power of two
+    float q[kLaneW];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < kLaneW; ++k) {
         const float d = __fsub_rn(v[k], mean);
         q[k] = __fmul_rn(d, d);
     }
@@ -228,7 +231,7 @@ __device__ __forceinline__ unsigned outlier_mask(const float (&v)[8], float tau)
     const float thr = __fmul_rn(sigma, tau);
     unsigned o = 0;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) o |= (fabsf(v[k]) > thr) ? (1u << k) : 0u;
+    for (int k = 0; k < kLaneW; ++k) o |= (fabsf(v[k]) > thr) ? (1u << k) : 0u;
     return o;
 }
 
@@ -245,23 +248,26 @@ __device__ __forceinline__ int warp_excl_scan(int cnt, int lane, int& total)
     return inc - cnt;
 }
 
-template <class DT>
-__device__ __forceinline__ void store8(void* base, int64_t idx, const float (&v)[8]);
-template <>
-__device__ __forceinline__ void store8<BF16>(void* base, int64_t idx, const float (&v)[8])
+// The 16 (cleaned) weights of a lane back to their storage type (exact: values are the
+// original ones or zero).
+__device__ __forceinline__ void store_row(BF16, void* base, int64_t idx, const float (&v)[kLaneW])
 {
-    uint32_t p[4];
+    Raw8 p;
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
-        p[k] = (__float_as_uint(v[2 * k]) >> 16) | (__float_as_uint(v[2 * k + 1]) & 0xffff0000u);
-    st_stream128(static_cast<uint16_t*>(base) + idx, make_uint4(p[0], p[1], p[2], p[3]));
+    for (int k = 0; k < 8; ++k)
+        p.u[k] = (__float_as_uint(v[2 * k]) >> 16) | (__float_as_uint(v[2 * k + 1]) & 0xffff0000u);
+    st_stream256(static_cast<uint16_t*>(base) + idx, p);
 }
-template <>
-__device__ __forceinline__ void store8<F32>(void* base, int64_t idx, const float (&v)[8])
+__device__ __forceinline__ void store_row(F32, void* base, int64_t idx, const float (&v)[kLaneW])
 {
-    float* d = static_cast<float*>(base) + idx;
-    st_stream128(d, make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3])));
-    st_stream128(d + 4, make_uint4(__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7])));
+    Raw8 p, q;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        p.u[k] = __float_as_uint(v[k]);
+        q.u[k] = __float_as_uint(v[8 + k]);
+    }
+    st_stream256(static_cast<float*>(base) + idx, p);
+    st_stream256(static_cast<float*>(base) + idx + 8, q);
 }
 
 // Pass 1 of OPQ.  Each warp iteration is one tile of kOpqTile weights: outliers are detected,
@@ -274,7 +280,7 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
                  int32_t* __restrict__ counts, int32_t* __restrict__ stage_idx,
                  uint16_t* __restrict__ stage_val)
 {
-    constexpr int LPB = I / 8;
+    static_assert(kOpqTile == kWarpW, "one tile per warp iteration");
     extern __shared__ __align__(16) unsigned char s_lut[];
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
@@ -283,22 +289,24 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
     const int64_t rows = (n + kQRow - 1) / kQRow;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lane_off = lane * 8;
-    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
-        const int64_t idx = (r * kQThreads + threadIdx.x) * 8;
+    int64_t r = blockIdx.x;
+    if (r >= rows) return;
+    int64_t idx = (r * kQThreads + threadIdx.x) * kLaneW;
+    RawRow<DT> raw = (idx < n) ? load_raw<DT>(w, idx) : zero_raw<DT>();
+    for (; r < rows; r += gridDim.x) {
+        const int64_t idx_next = ((r + gridDim.x) * kQThreads + threadIdx.x) * kLaneW;
+        const RawRow<DT> next = (idx_next < n) ? load_raw<DT>(w, idx_next) : zero_raw<DT>();
         const int64_t tile = r * (kQThreads / 32) + warp;
         const bool tile_ok = tile * kOpqTile < n;  // warp-uniform
-        float v[8];
-        if (idx < n)
-            load8<DT>(w, idx, v);
-        else
-            zero8<DT>(v);
+        float v[kLaneW];
+        widen(raw, v);
         const unsigned o = outlier_mask<I>(v, tau);
         const unsigned any = __ballot_sync(kFull, o != 0u);
         if (any) {
             int total;
             int pos = warp_excl_scan(__popc(o), lane, total);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
+            for (int k = 0; k < kLaneW; ++k)
                 if ((o >> k) & 1u) {
                     if (pos < kOpqStage) {
                         stage_idx[tile * kOpqStage + pos] = (int32_t)(idx + k);
@@ -312,16 +320,12 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
             counts[tile] = 0;
         }
         if (QUANT) {
-            const float m = block_constant<LPB, SIGNED>(v);
-            const bool fast = __all_sync(kFull, div_safe(m) || idx >= n);
-            const uint32_t word = encode8<DT>(v, m, fast, T, lane_off);
-            if (idx < n) {
-                st_stream32(codes + idx / 2, word);
-                if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx / I, m);
-            }
+            quantize_row<DT, I, SIGNED, ST>(v, idx, idx < n, T, lane_off, lane, codes, scales);
         } else if (w_clean != nullptr && idx < n) {
-            store8<DT>(w_clean, idx, v);
+            store_row(DT{}, w_clean, idx, v);
         }
+        raw = next;
+        idx = idx_next;
     }
 }
 
@@ -429,17 +433,14 @@ opq_gather_kernel(const void* __restrict__ w, int64_t n, float tau, const int32_
     const int novf = s_novf;
     for (int s = warp; s < novf; s += 8) {
         const int64_t tile = (int64_t)blockIdx.x * kOpqChunk + s_ovf_tile[s];
-        const int64_t idx = tile * kOpqTile + lane * 8;
-        float v[8];
-        if (idx < n)
-            load8<DT>(w, idx, v);
-        else
-            zero8<DT>(v);
+        const int64_t idx = tile * kOpqTile + lane * kLaneW;
+        float v[kLaneW];
+        widen((idx < n) ? load_raw<DT>(w, idx) : zero_raw<DT>(), v);
         const unsigned o = outlier_mask<I>(v, tau);
         int total;
         int pos = warp_excl_scan(__popc(o), lane, total);
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
+        for (int k = 0; k < kLaneW; ++k)
             if ((o >> k) & 1u) {
                 const int64_t dst = base + s_ovf_off[s] + pos;
                 if (dst < capacity) {
@@ -503,7 +504,16 @@ int check_quant_dtypes(const char* fn, int w_dtype, int scale_dtype, int norm)
     return BOF4_OK;
 }
 
-// Expands BODY with DT, I_, SG, ST bound to the template arguments of the runtime configuration.
+int check_aligned(const char* fn, const char* what, const void* p)
+{
+    if (!aligned32(p)) {
+        set_error("%s: %s is not 32-byte aligned", fn, what);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    return BOF4_OK;
+}
+
+// Expand the body with I_, SG, DT, ST bound to the compile-time configuration.
 #define BOF4_DISPATCH_I(I_VAL, ...)                    \
     switch (I_VAL) {                                   \
         case 32: { constexpr int I_ = 32; __VA_ARGS__; } break;   \
@@ -535,9 +545,11 @@ extern "C" int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_
         set_error("bof4_quantize: NULL pointer");
         return BOF4_ERR_INVALID_ARG;
     }
+    if ((rc = check_aligned("bof4_quantize", "d_w", d_w)) || (rc = check_aligned("bof4_quantize", "d_codes", d_codes)))
+        return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t rows = (n + kQRow - 1) / kQRow;
-    const int grid = grid_for((rows + kQUnroll - 1) / kQUnroll, kQCtasPerSm);
+    const int grid = grid_for(rows, kQCtasPerSm);
     BOF4_DISPATCH_WS(w_dtype, scale_dtype,
         BOF4_DISPATCH_I(block_size,
             BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
@@ -575,6 +587,8 @@ extern "C" int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int
         set_error("bof4_dequantize: NULL pointer");
         return BOF4_ERR_INVALID_ARG;
     }
+    if ((rc = check_aligned("bof4_dequantize", "d_codes", d_codes)) || (rc = check_aligned("bof4_dequantize", "d_out", d_out)))
+        return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t rows = (n + kDRow - 1) / kDRow;
     const int grid = grid_for(rows, 8);
@@ -640,6 +654,9 @@ int launch_opq(const char* fn, const void* d_w, int w_dtype, int64_t n, int bloc
         set_error("%s: NULL pointer", fn);
         return BOF4_ERR_INVALID_ARG;
     }
+    if ((rc = check_aligned(fn, "d_w", d_w)) || (rc = check_aligned(fn, "d_codes", d_codes)) ||
+        (rc = check_aligned(fn, "d_w_clean", d_w_clean)))
+        return rc;
     char* ws = static_cast<char*>(d_ws);
     int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
     int64_t* chunk_off = reinterpret_cast<int64_t*>(ws + L.chunk_off);
