@@ -24,6 +24,9 @@ METRIC_MSE, METRIC_MAE = 0, 1
 OP_EM, OP_OPQ = 0, 1
 LEVELS = 16
 
+# kernels one MAE iteration enqueues: setup, 4 x (data pass + bin selection), level update
+MAE_LAUNCHES_PER_ITERATION = 10
+
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error")

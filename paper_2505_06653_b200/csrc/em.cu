@@ -11,12 +11,12 @@
 // kernel that also updates the free levels.  Nothing depends on scheduling, so results are
 // bit-reproducible.  The COUNT variant also keeps the member count of every region.
 #include "common.cuh"
+#include "em_common.cuh"
 #include "layout.h"
 
 namespace bof4 {
 
-constexpr int kEmMaxTensors = 64;       // tensors per launch (kernel parameter table)
-constexpr int kEmFlushIters = 128;      // loop iterations between fp32 -> fp64 folds
+constexpr int kEmFlushIters = 64;  // loop iterations (16 weights per lane each) between fp32 -> fp64 folds
 
 template <bool COUNT>
 struct EmGeo {
@@ -24,14 +24,6 @@ struct EmGeo {
     static constexpr int row = threads * kLaneW;            // weights per CTA row
     static constexpr uint32_t acc_row_bytes = threads * 8;  // one level's float2 columns
     static constexpr size_t smem = (size_t)kLutBytes + (size_t)kLevels * threads * (COUNT ? 12 : 8);
-};
-
-struct EmTensors {
-    const void* ptr[kEmMaxTensors];
-    int64_t n[kEmMaxTensors];
-    int64_t row_end[kEmMaxTensors];  // cumulative number of CTA rows up to and including tensor t
-    int count;
-    int accumulate;  // 0: this launch overwrites the partial records, 1: adds to them
 };
 
 // Record layout in doubles: [0,16) s1, [16,32) s0, [32,48) count (uint64 bits), [48] sum w^2.
@@ -295,19 +287,9 @@ em_mse_finalize_kernel(const double* __restrict__ partials, int n_records, int64
 
 // ================================================================= launchers (C ABI)
 
-namespace {
+namespace bof4 {
 
-using namespace bof4;
-
-struct EmArgs {
-    const void* const* h_w;
-    const int64_t* h_n;
-    int n_tensors, w_dtype, block_size, norm, metric;
-    int64_t n_total;
-};
-
-int check_em(const char* fn, const EmArgs& a, const void* d_codebook, void* d_ws, size_t ws_bytes,
-             int64_t* n_total)
+int check_em(const char* fn, EmArgs& a, const void* d_codebook, void* d_ws, size_t ws_bytes)
 {
     if (a.n_tensors < 0 || (a.n_tensors > 0 && (!a.h_w || !a.h_n))) {
         set_error("%s: bad tensor list", fn);
@@ -352,9 +334,15 @@ int check_em(const char* fn, const EmArgs& a, const void* d_codebook, void* d_ws
                   em_workspace_bytes());
         return BOF4_ERR_WORKSPACE;
     }
-    *n_total = tot;
+    a.n_total = tot;
     return BOF4_OK;
 }
+
+}  // namespace bof4
+
+namespace {
+
+using namespace bof4;
 
 template <class DT, int I, bool SG, bool COUNT>
 int launch_mse_chunk(const EmTensors& T, const float* d_codebook, double* partials, cudaStream_t st)
@@ -372,49 +360,26 @@ int launch_mse_chunk(const EmTensors& T, const float* d_codebook, double* partia
 template <bool COUNT>
 int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials, cudaStream_t st)
 {
-    constexpr int kEmRow = EmGeo<COUNT>::row;
-    EmTensors T;
-    T.count = 0;
-    T.accumulate = 0;
-    int64_t rows = 0;
-    bool launched = false;
-    auto fire = [&]() -> int {
-        if (T.count == 0) return BOF4_OK;
-        int rc = BOF4_OK;
-        const bool sg = a.norm == BOF4_NORM_SIGNED;
-#define BOF4_EM_GO(DT_)                                                                          \
-    switch (a.block_size) {                                                                      \
-        case 32: rc = sg ? launch_mse_chunk<DT_, 32, true, COUNT>(T, d_codebook, partials, st)          \
-                         : launch_mse_chunk<DT_, 32, false, COUNT>(T, d_codebook, partials, st); break; \
-        case 64: rc = sg ? launch_mse_chunk<DT_, 64, true, COUNT>(T, d_codebook, partials, st)          \
-                         : launch_mse_chunk<DT_, 64, false, COUNT>(T, d_codebook, partials, st); break; \
-        case 128: rc = sg ? launch_mse_chunk<DT_, 128, true, COUNT>(T, d_codebook, partials, st)        \
-                          : launch_mse_chunk<DT_, 128, false, COUNT>(T, d_codebook, partials, st); break; \
-        default: rc = sg ? launch_mse_chunk<DT_, 256, true, COUNT>(T, d_codebook, partials, st)         \
-                         : launch_mse_chunk<DT_, 256, false, COUNT>(T, d_codebook, partials, st); break; \
+    const bool sg = a.norm == BOF4_NORM_SIGNED;
+    auto fire = [&](const EmTensors& T) -> int {
+#define BOF4_EM_GO(DT_)                                                                                 \
+    switch (a.block_size) {                                                                             \
+        case 32: return sg ? launch_mse_chunk<DT_, 32, true, COUNT>(T, d_codebook, partials, st)        \
+                           : launch_mse_chunk<DT_, 32, false, COUNT>(T, d_codebook, partials, st);      \
+        case 64: return sg ? launch_mse_chunk<DT_, 64, true, COUNT>(T, d_codebook, partials, st)        \
+                           : launch_mse_chunk<DT_, 64, false, COUNT>(T, d_codebook, partials, st);      \
+        case 128: return sg ? launch_mse_chunk<DT_, 128, true, COUNT>(T, d_codebook, partials, st)      \
+                            : launch_mse_chunk<DT_, 128, false, COUNT>(T, d_codebook, partials, st);    \
+        default: return sg ? launch_mse_chunk<DT_, 256, true, COUNT>(T, d_codebook, partials, st)       \
+                           : launch_mse_chunk<DT_, 256, false, COUNT>(T, d_codebook, partials, st);     \
     }
         if (a.w_dtype == BOF4_F32) { BOF4_EM_GO(F32) } else { BOF4_EM_GO(BF16) }
 #undef BOF4_EM_GO
-        launched = true;
-        T.count = 0;
-        T.accumulate = 1;
-        rows = 0;
-        return rc;
     };
-    for (int t = 0; t < a.n_tensors; ++t) {
-        if (a.h_n[t] == 0) continue;
-        rows += (a.h_n[t] + kEmRow - 1) / kEmRow;
-        T.ptr[T.count] = a.h_w[t];
-        T.n[T.count] = a.h_n[t];
-        T.row_end[T.count] = rows;
-        if (++T.count == kEmMaxTensors) {
-            const int rc = fire();
-            if (rc) return rc;
-        }
-    }
-    const int rc = fire();
+    int calls = 0;
+    const int rc = for_each_tensor_chunk(a, EmGeo<COUNT>::row, fire, &calls);
     if (rc) return rc;
-    if (!launched) BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));
+    if (calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));
     return BOF4_OK;
 }
 
@@ -425,7 +390,7 @@ extern "C" int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_te
                             bof4_em_stats* d_stats, void* d_ws, size_t ws_bytes, void* stream)
 {
     EmArgs a{h_w, h_n, n_tensors, w_dtype, block_size, norm, metric, 0};
-    int rc = check_em("bof4_em_step", a, d_codebook, d_ws, ws_bytes, &a.n_total);
+    int rc = check_em("bof4_em_step", a, d_codebook, d_ws, ws_bytes);
     if (rc) return rc;
     if (!d_stats) {
         set_error("bof4_em_step: NULL stats");
@@ -441,8 +406,9 @@ extern "C" int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_te
         BOF4_CUDA_TRY(cudaGetLastError());
         return BOF4_OK;
     }
-    set_error("bof4_em_step: MAE not available in this build");
-    return BOF4_ERR_INVALID_ARG;
+    rc = mae_prepare(a, d_ws, st);
+    if (rc) return rc;
+    return mae_iteration(a, d_codebook, nullptr, 0u, d_stats, nullptr, d_ws, st);
 }
 
 extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int n_tensors,
@@ -451,7 +417,7 @@ extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int
                                  double* d_err_log, void* d_ws, size_t ws_bytes, void* stream)
 {
     EmArgs a{h_w, h_n, n_tensors, w_dtype, block_size, norm, metric, 0};
-    int rc = check_em("bof4_fit_codebook", a, d_codebook, d_ws, ws_bytes, &a.n_total);
+    int rc = check_em("bof4_fit_codebook", a, d_codebook, d_ws, ws_bytes);
     if (rc) return rc;
     if (iters < 0) {
         set_error("bof4_fit_codebook: negative iteration count");
@@ -470,6 +436,14 @@ extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int
         }
         return BOF4_OK;
     }
-    set_error("bof4_fit_codebook: MAE not available in this build");
-    return BOF4_ERR_INVALID_ARG;
+    if (iters > 0) {
+        rc = mae_prepare(a, d_ws, st);
+        if (rc) return rc;
+    }
+    for (int t = 0; t < iters; ++t) {
+        rc = mae_iteration(a, d_codebook, d_codebook, fixed_mask, nullptr,
+                           d_err_log ? d_err_log + t : nullptr, d_ws, st);
+        if (rc) return rc;
+    }
+    return BOF4_OK;
 }

@@ -1,0 +1,438 @@
+// MAE variant of the codebook fit (Eq. 8, App. B.3): every free level becomes the weighted
+// median of the normalised weights of its region, the weight of a sample being |m| of its block.
+//
+// The weighted median is found by radix selection on an order-preserving integer key of x.
+// All members of region l have keys in [key(xi[l-1]), key(xi[l])), so only the B_l low bits of
+// rel = key - key(xi[l-1]) differ; each data pass histograms the next (up to) 9 of those bits for
+// the samples that match the digits chosen so far, and a single-CTA kernel picks the bin in
+// which the cumulative weight first reaches half of the region's total.  After ceil(B_l / 9)
+// passes (3 for ordinary regions, 4 at most) the key, hence the sample, is known exactly.
+//
+// Weights enter the histograms as 31-bit fixed-point integers relative to the largest |w| of
+// the data (exact whenever |m| is within 2^-7 of it for fp32 input, 2^-23 for bf16 input), so
+// every sum is an integer sum: independent of the order of the atomics, bit-reproducible, and
+// equal to the exact real-number sums that define the median.
+#include "common.cuh"
+#include "em_common.cuh"
+#include "layout.h"
+
+namespace bof4 {
+
+constexpr int kMaeThreads = 1024;
+constexpr int kMaeRow = kMaeThreads * kLaneW;
+constexpr size_t kMaeSmem = (size_t)kLutBytes + 3u * kLevels * kMaeBins * 4u;  // lo, hi, count
+
+struct MaeState {
+    unsigned long long before[kLevels];  // weight below the current candidate range
+    unsigned long long total[kLevels];   // total weight of the region (after the first pass)
+    unsigned long long count[kLevels];   // members of the region (after the first pass)
+    uint32_t base[kLevels];              // key of the region's lower edge
+    uint32_t prefix[kLevels];            // digits chosen so far
+    int top[kLevels];                    // key bits still unresolved (0: done)
+    uint32_t active;                     // bit l: level l takes part in the selection
+    uint32_t max_bits;                   // bits of the largest |w| of the data
+    int passes_left;                     // max over active levels of the passes still needed
+    int pad;
+};
+static_assert(sizeof(MaeState) <= kEmMaeStateBytes, "state must fit its slot");
+
+struct MaeWs {
+    double* partials;
+    MaeState* state;
+    unsigned long long* hist;   // [16][kMaeBins] weight
+    unsigned long long* chist;  // [16][kMaeBins] count
+};
+
+__host__ __device__ inline MaeWs mae_ws(void* d_ws)
+{
+    char* p = static_cast<char*>(d_ws) + kEmMaeOffset;
+    return MaeWs{static_cast<double*>(d_ws), reinterpret_cast<MaeState*>(p),
+                 reinterpret_cast<unsigned long long*>(p + kEmMaeStateBytes),
+                 reinterpret_cast<unsigned long long*>(p + kEmMaeStateBytes + kEmMaeHistBytes)};
+}
+
+// Order-preserving key: x <= y  <=>  key(x) <= key(y); -0 and +0 share a key.
+__device__ __forceinline__ uint32_t order_key(float x)
+{
+    const uint32_t u = __float_as_uint(x + 0.0f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_to_float(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// |m| as a 31-bit fixed-point integer relative to the largest magnitude of the data.
+__device__ __forceinline__ uint32_t fixed_weight(float m, uint32_t max_bits)
+{
+    const uint32_t b = __float_as_uint(fabsf(m));
+    const int e = max((int)(b >> 23), 1), emax = max((int)(max_bits >> 23), 1);
+    const uint32_t mant = (b & 0x7fffffu) | ((b >> 23) ? 0x800000u : 0u);
+    const int sh = e - emax + 7;
+    if (sh >= 0) return mant << min(sh, 7);
+    return (-sh >= 32) ? 0u : (mant >> (-sh));
+}
+
+// ---------------------------------------------------------------- largest |w|
+
+template <class DT>
+__global__ void __launch_bounds__(kMaeThreads, 1)
+mae_absmax_kernel(const EmTensors T, MaeState* __restrict__ state)
+{
+    __shared__ uint32_t s_max[kMaeThreads / 32];
+    const int tid = threadIdx.x;
+    const int64_t total_rows = T.row_end[T.count - 1];
+    float a = 0.0f;
+    int t_cur = 0;
+    for (int64_t g = blockIdx.x; g < total_rows; g += gridDim.x) {
+        while (g >= T.row_end[t_cur]) ++t_cur;
+        const int64_t r = g - (t_cur ? T.row_end[t_cur - 1] : 0);
+        const int64_t idx = (r * kMaeThreads + tid) * kLaneW;
+        if (idx < T.n[t_cur]) {
+            float v[kLaneW];
+            widen(load_raw<DT>(T.ptr[t_cur], idx), v);
+#pragma unroll
+            for (int k = 0; k < kLaneW; ++k) a = fmaxf(a, fabsf(v[k]));
+        }
+    }
+    uint32_t b = __float_as_uint(a);
+#pragma unroll
+    for (int off = 16; off; off >>= 1) b = max(b, __shfl_xor_sync(kFull, b, off));
+    if ((tid & 31) == 0) s_max[tid >> 5] = b;
+    __syncthreads();
+    if (tid == 0) {
+        for (int k = 1; k < kMaeThreads / 32; ++k) b = max(b, s_max[k]);
+        atomicMax(&state->max_bits, b);  // non-negative floats order like their bits
+    }
+}
+
+// ---------------------------------------------------------------- per-iteration setup
+
+// Region key ranges from the current levels, selection state reset, histograms cleared.
+__global__ void __launch_bounds__(kMaeBins)
+mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
+{
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ int s_need[kLevels];
+    make_thresholds(levels, s_xi, s_lv, threadIdx.x);
+    __syncthreads();
+    if (threadIdx.x < kLevels) {
+        const int l = threadIdx.x;
+        // members of region l lie in [lo, hi] with lo, hi clipped to [-1, 1]
+        const float lo = (l == 0) ? -1.0f : fminf(fmaxf(s_xi[l - 1], -1.0f), 1.0f);
+        const float hi = (l == kLevels - 1) ? 1.0f : fminf(fmaxf(s_xi[l], -1.0f), 1.0f);
+        const uint32_t klo = order_key(lo), khi = order_key(hi);
+        const uint32_t range = (khi > klo) ? khi - klo : 0u;
+        const int bits = 32 - __clz(range | 1u);
+        const bool on = !((skip_mask >> l) & 1u);
+        W.state->base[l] = klo;
+        W.state->prefix[l] = 0u;
+        W.state->top[l] = on ? bits : 0;
+        W.state->before[l] = 0ull;
+        W.state->total[l] = 0ull;
+        W.state->count[l] = 0ull;
+        s_need[l] = on ? (bits + kMaeDigitBits - 1) / kMaeDigitBits : 0;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int need = 0;
+        for (int l = 0; l < kLevels; ++l) need = max(need, s_need[l]);
+        W.state->active = ~skip_mask & 0xffffu;
+        W.state->passes_left = need;
+    }
+    for (int k = threadIdx.x; k < kLevels * kMaeBins; k += blockDim.x) {
+        W.hist[k] = 0ull;
+        W.chist[k] = 0ull;
+    }
+}
+
+// ---------------------------------------------------------------- data pass
+
+// FIRST: also accumulates sum |w - m xhat[c]| (one partial record per CTA) and, with COUNT,
+// the member counts.  Later passes return at once when no level has bits left.
+template <class DT, int I, bool SIGNED, bool FIRST, bool COUNT>
+__global__ void __launch_bounds__(kMaeThreads, 1)
+mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
+{
+    constexpr int LPB = I / kLaneW;
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    unsigned char* s_lut = s_raw;
+    uint32_t* s_lo = reinterpret_cast<uint32_t*>(s_raw + kLutBytes);
+    uint32_t* s_hi = s_lo + kLevels * kMaeBins;
+    uint32_t* s_cn = s_hi + kLevels * kMaeBins;
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ int s_multi;
+    __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
+    __shared__ double s_err[kMaeThreads / 32];
+    __shared__ const void* s_ptr[kEmMaxTensors];
+    __shared__ int64_t s_n[kEmMaxTensors], s_row_end[kEmMaxTensors];
+
+    if (!FIRST && W.state->passes_left <= 0) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    make_thresholds(levels, s_xi, s_lv, tid);
+    if (tid < kLevels) {
+        const int top = W.state->top[tid];
+        const int sh = max(top - kMaeDigitBits, 0);
+        const uint32_t mask = (1u << (top - sh)) - 1u;
+        s_lvl[tid] = make_uint4(W.state->base[tid], W.state->prefix[tid],
+                                (uint32_t)top | ((uint32_t)sh << 8) | (mask << 16), top > 0 ? 1u : 0u);
+    }
+    if (tid < T.count) {
+        s_ptr[tid] = T.ptr[tid];
+        s_n[tid] = T.n[tid];
+        s_row_end[tid] = T.row_end[tid];
+    }
+    for (int k = tid; k < 3 * kLevels * kMaeBins; k += kMaeThreads) s_lo[k] = 0u;
+    const uint32_t max_bits = W.state->max_bits;
+    __syncthreads();
+    build_lut(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base; });
+    __syncthreads();
+    const bool lut_ok = s_multi == 0;
+
+    const int64_t total_rows = T.row_end[T.count - 1];
+    const uint32_t lane_off = lane * 8;
+    double err = 0.0;
+    int t_cur = 0;
+    for (int64_t g = blockIdx.x; g < total_rows; g += gridDim.x) {
+        while (g >= s_row_end[t_cur]) ++t_cur;
+        const int64_t r = g - (t_cur ? s_row_end[t_cur - 1] : 0);
+        const int64_t idx = (r * kMaeThreads + tid) * kLaneW;
+        const bool ok = idx < s_n[t_cur];
+        float v[kLaneW];
+        widen(ok ? load_raw<DT>(s_ptr[t_cur], idx) : zero_raw<DT>(), v);
+        const float m = block_constant<LPB, SIGNED>(v);
+        const bool fast = (DT::code == BF16::code) && __all_sync(kFull, div_safe(m) || !ok);
+        float x[kLaneW];
+        normalise16<false>(v, m, fast, x);
+        if (!ok) continue;
+        const uint32_t a = fixed_weight(m, max_bits);
+        float e = 0.0f;
+#pragma unroll
+        for (int k = 0; k < kLaneW; ++k) {
+            uint32_t c;
+            if (lut_ok) {
+                const uint2 ent = *reinterpret_cast<const uint2*>(s_lut + lut_offset(lut_key(x[k]), lane_off));
+                c = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? 1u : 0u);
+            } else {
+                c = (uint32_t)region_of(x[k], s_xi);
+            }
+            if (FIRST) e += fabsf(fmaf(-m, s_lv[c], v[k]));
+            const uint4 L = s_lvl[c];
+            const uint32_t rel = order_key(x[k]) - L.x;
+            const uint32_t top = L.z & 0xffu, sh = (L.z >> 8) & 0xffu, mask = L.z >> 16;
+            if (L.w && (uint32_t)((unsigned long long)rel >> top) == L.y) {
+                const uint32_t bin = c * kMaeBins + ((rel >> sh) & mask);
+                const uint32_t old = atomicAdd(&s_lo[bin], a);
+                if (old + a < old) atomicAdd(&s_hi[bin], 1u);
+                if (FIRST && COUNT) atomicAdd(&s_cn[bin], 1u);
+            }
+        }
+        if (FIRST) err += (double)e;
+    }
+    __syncthreads();
+    for (int k = tid; k < kLevels * kMaeBins; k += kMaeThreads) {
+        const unsigned long long wsum = ((unsigned long long)s_hi[k] << 32) + s_lo[k];
+        if (wsum) atomicAdd(&W.hist[k], wsum);
+        if (FIRST && COUNT && s_cn[k]) atomicAdd(&W.chist[k], (unsigned long long)s_cn[k]);
+    }
+    if (FIRST) {
+#pragma unroll
+        for (int off = 16; off; off >>= 1) err += __shfl_xor_sync(kFull, err, off);
+        if (lane == 0) s_err[warp] = err;
+        __syncthreads();
+        if (tid == 0) {
+            double t = 0.0;
+            for (int k = 0; k < kMaeThreads / 32; ++k) t += s_err[k];
+            double* rec = W.partials + (size_t)blockIdx.x * kEmRecordDoubles;
+            rec[0] = T.accumulate ? rec[0] + t : t;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- bin selection
+
+// One CTA, one thread per bin.  For every level with bits left: the first bin in which the
+// cumulative weight reaches half of the total (2 (before + cum) >= total) becomes the next
+// digit.  After the first pass the totals (and counts) are those of the whole region.
+__global__ void __launch_bounds__(kMaeBins)
+mae_select_kernel(MaeWs W, int first)
+{
+    __shared__ unsigned long long s_scan[kMaeBins];
+    __shared__ unsigned long long s_cscan[kMaeBins / 32];
+    __shared__ int s_pick;
+    MaeState* S = W.state;
+    if (!first && S->passes_left <= 0) return;
+    const int j = threadIdx.x;
+    int left = 0;
+    for (int l = 0; l < kLevels; ++l) {
+        const int top = S->top[l];
+        if (top <= 0) continue;  // uniform: read from global by every thread
+        const unsigned long long mine = W.hist[l * kMaeBins + j];
+        W.hist[l * kMaeBins + j] = 0ull;
+        s_scan[j] = mine;
+        if (j == 0) s_pick = kMaeBins - 1;
+        __syncthreads();
+        for (int off = 1; off < kMaeBins; off <<= 1) {
+            const unsigned long long t = (j >= off) ? s_scan[j - off] : 0ull;
+            __syncthreads();
+            s_scan[j] += t;
+            __syncthreads();
+        }
+        if (first) {
+            unsigned long long c = W.chist[l * kMaeBins + j];
+            W.chist[l * kMaeBins + j] = 0ull;
+#pragma unroll
+            for (int off = 16; off; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
+            if ((j & 31) == 0) s_cscan[j >> 5] = c;
+        }
+        __syncthreads();
+        const unsigned long long total = first ? s_scan[kMaeBins - 1] : S->total[l];
+        const unsigned long long before = S->before[l];
+        const unsigned long long incl = s_scan[j], excl = incl - mine;
+        const bool reached = 2ull * (before + incl) >= total;
+        const bool prev_reached = (j > 0) && (2ull * (before + excl) >= total);
+        if (reached && !prev_reached) s_pick = j;  // exactly one thread (cumulative is monotone)
+        __syncthreads();
+        const int pick = s_pick;
+        if (j == pick) {
+            const int sh = max(top - kMaeDigitBits, 0);
+            S->before[l] = before + excl;
+            S->prefix[l] = (S->prefix[l] << (top - sh)) | (uint32_t)pick;
+            S->top[l] = sh;
+            if (first) S->total[l] = total;
+        }
+        if (first && j == 0) {
+            unsigned long long c = 0;
+            for (int k = 0; k < kMaeBins / 32; ++k) c += s_cscan[k];
+            S->count[l] = c;
+        }
+        left = max(left, (max(top - kMaeDigitBits, 0) + kMaeDigitBits - 1) / kMaeDigitBits);
+        __syncthreads();
+    }
+    if (j == 0) S->passes_left = left;
+}
+
+// ---------------------------------------------------------------- level update
+
+__global__ void __launch_bounds__(256)
+mae_finalize_kernel(MaeWs W, int n_records, int64_t n_total, const float* levels_in, float* levels_out,
+                    uint32_t skip_mask, bof4_em_stats* __restrict__ stats, double* __restrict__ err_slot)
+{
+    __shared__ double s_part[8];
+    const MaeState* S = W.state;
+    double e = 0.0;
+    for (int r = threadIdx.x; r < n_records; r += blockDim.x) e += W.partials[(size_t)r * kEmRecordDoubles];
+#pragma unroll
+    for (int off = 16; off; off >>= 1) e += __shfl_xor_sync(kFull, e, off);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = e;
+    __syncthreads();
+    if (threadIdx.x < kLevels) {
+        const int l = threadIdx.x;
+        const float old = levels_in[l];
+        const bool on = !((skip_mask >> l) & 1u);
+        const unsigned long long total = S->total[l];
+        const float med = (on && total > 0ull) ? key_to_float(S->base[l] + S->prefix[l]) : old;
+        if (stats) {
+            const int emax = max((int)(S->max_bits >> 23), 1);
+            stats->s1[l] = 0.0;
+            stats->s0[l] = ldexp((double)total, emax - 157);  // undo the fixed-point scale
+            stats->count[l] = S->count[l];
+            stats->median[l] = med;
+        }
+        if (levels_out && on) levels_out[l] = med;
+    }
+    if (threadIdx.x == 0) {
+        double err = 0.0;
+        for (int k = 0; k < 8; ++k) err += s_part[k];
+        if (stats) {
+            stats->err_sum = err;
+            stats->n_total = n_total;
+        }
+        if (err_slot) *err_slot = (n_total > 0) ? err / (double)n_total : 0.0;
+    }
+}
+
+// ================================================================= host side
+
+namespace {
+
+template <class DT, int I, bool SG>
+int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, bool first, bool count,
+                cudaStream_t st)
+{
+#define BOF4_MAE_GO(FIRST_, COUNT_)                                                                     \
+    {                                                                                                   \
+        auto kern = mae_pass_kernel<DT, I, SG, FIRST_, COUNT_>;                                         \
+        BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaeSmem)); \
+        kern<<<kEmGrid, kMaeThreads, kMaeSmem, st>>>(T, d_levels, W);                                   \
+    }
+    if (first && count) BOF4_MAE_GO(true, true)
+    else if (first) BOF4_MAE_GO(true, false)
+    else BOF4_MAE_GO(false, false)
+#undef BOF4_MAE_GO
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
+}
+
+int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, const MaeWs& W, bool first,
+                  bool count, cudaStream_t st)
+{
+    const bool sg = a.norm == BOF4_NORM_SIGNED;
+#define BOF4_MAE_I(DT_, I_)                                                       \
+    return sg ? launch_pass<DT_, I_, true>(T, d_levels, W, first, count, st)      \
+              : launch_pass<DT_, I_, false>(T, d_levels, W, first, count, st);
+#define BOF4_MAE_DT(DT_)                         \
+    switch (a.block_size) {                      \
+        case 32: BOF4_MAE_I(DT_, 32)             \
+        case 64: BOF4_MAE_I(DT_, 64)             \
+        case 128: BOF4_MAE_I(DT_, 128)           \
+        default: BOF4_MAE_I(DT_, 256)            \
+    }
+    if (a.w_dtype == BOF4_F32) { BOF4_MAE_DT(F32) } else { BOF4_MAE_DT(BF16) }
+#undef BOF4_MAE_DT
+#undef BOF4_MAE_I
+}
+
+}  // namespace
+
+int mae_prepare(const EmArgs& a, void* d_ws, cudaStream_t st)
+{
+    const MaeWs W = mae_ws(d_ws);
+    BOF4_CUDA_TRY(cudaMemsetAsync(W.state, 0, sizeof(MaeState), st));
+    auto fire = [&](const EmTensors& T) -> int {
+        if (a.w_dtype == BOF4_F32)
+            mae_absmax_kernel<F32><<<kEmGrid, kMaeThreads, 0, st>>>(T, W.state);
+        else
+            mae_absmax_kernel<BF16><<<kEmGrid, kMaeThreads, 0, st>>>(T, W.state);
+        BOF4_CUDA_TRY(cudaGetLastError());
+        return BOF4_OK;
+    };
+    int calls = 0;
+    return for_each_tensor_chunk(a, kMaeRow, fire, &calls);
+}
+
+int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out, uint32_t skip_mask,
+                  bof4_em_stats* d_stats, double* d_err_slot, void* d_ws, cudaStream_t st)
+{
+    const MaeWs W = mae_ws(d_ws);
+    mae_init_kernel<<<1, kMaeBins, 0, st>>>(d_levels_in, skip_mask, W);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    for (int p = 0; p < kMaeMaxPasses; ++p) {
+        const bool first = p == 0;
+        auto fire = [&](const EmTensors& T) -> int {
+            return dispatch_pass(a, T, d_levels_in, W, first, first && d_stats != nullptr, st);
+        };
+        int calls = 0;
+        const int rc = for_each_tensor_chunk(a, kMaeRow, fire, &calls);
+        if (rc) return rc;
+        if (first && calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(W.partials, 0, kEmPartialBytes, st));
+        mae_select_kernel<<<1, kMaeBins, 0, st>>>(W, first ? 1 : 0);
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
+    mae_finalize_kernel<<<1, 256, 0, st>>>(W, kEmGrid, a.n_total, d_levels_in, d_levels_out, skip_mask,
+                                           d_stats, d_err_slot);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
+}
+
+}  // namespace bof4

@@ -14,10 +14,13 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 constexpr int kEmGrid = 148;              // CTAs of the accumulation kernels (1 per SM)
 constexpr int kEmRecordDoubles = 64;      // 16 s1 + 16 s0 + 16 count + sum w^2, padded to 512 B
 constexpr size_t kEmPartialBytes = (size_t)kEmGrid * kEmRecordDoubles * 8;
-constexpr int kMaeBins = 1024;            // bins per level and selection pass
+constexpr int kMaeDigitBits = 9;          // key bits resolved per selection pass
+constexpr int kMaeBins = 1 << kMaeDigitBits;  // bins per level and selection pass
+constexpr int kMaeMaxPasses = 4;          // 31 key bits / 9 bits per pass
 constexpr size_t kEmMaeOffset = 512 * 1024;
-constexpr size_t kEmMaeHistBytes = (size_t)16 * kMaeBins * 8;
-constexpr size_t kEmMaeBytes = 4096 + kEmMaeHistBytes;
+constexpr size_t kEmMaeStateBytes = 4096;  // selection state (struct MaeState)
+constexpr size_t kEmMaeHistBytes = (size_t)16 * kMaeBins * 8;  // weight histogram, then count histogram
+constexpr size_t kEmMaeBytes = kEmMaeStateBytes + 2 * kEmMaeHistBytes;
 
 inline size_t em_workspace_bytes() { return kEmMaeOffset + align_up(kEmMaeBytes, 256); }
 

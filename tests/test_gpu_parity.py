@@ -285,3 +285,73 @@ def test_fit_zero_iterations_and_empty_input(bof4):
     cb, log = bof4.bof4_fit_codebook([e], I, 1, bof4.METRIC_MSE, LV_INIT, 0, 2)
     assert np.array_equal(cb.cpu().numpy(), LV_INIT)
     assert np.all(log.cpu().numpy() == 0)
+
+
+# --------------------------------------------------------------------------- EM, MAE
+
+
+def _check_mae_stats(got, ref, levels_in):
+    assert got["n"] == ref["n"]
+    assert np.array_equal(got["count"], ref["count"])
+    np.testing.assert_allclose(got["s0"], ref["wsum"], rtol=RTOL)
+    np.testing.assert_allclose(got["err_sum"], ref["err_sum"], rtol=RTOL)
+    # the median is a sample of the data: it must be the same sample, not merely a close one
+    assert np.array_equal(got["median"], ref["median"])
+
+
+@pytest.mark.parametrize("I", [32, 64, 128, 256])
+@pytest.mark.parametrize("norm", [0, 1])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_em_step_mae_matches_oracle(bof4, I, norm, dtype):
+    n = 8192 * 5 + 7 * 512
+    n -= n % I
+    w = special_blocks(make_weights(n, dtype, 140 + I), I)
+    got = bof4.bof4_em_step([w.cuda()], I, norm, bof4.METRIC_MAE, LV_INIT)
+    ref = oracle.em_accumulate_mae(w, I, norm, LV_INIT)
+    _check_mae_stats(got, ref, LV_INIT)
+
+
+def test_em_step_mae_exact_half_ties(bof4):
+    """Equal block constants: cumulative weights hit exactly half of the total for every region
+    with an even member count; the lower of the two middle samples must be returned."""
+    I, nb = 64, 512
+    g = torch.Generator().manual_seed(5)
+    w = (torch.rand(nb, I, generator=g) * 2 - 1) * 0.999
+    w[:, 0] = 1.0                                  # every block has m = 1
+    w = w.reshape(-1).to(torch.bfloat16)
+    got = bof4.bof4_em_step([w.cuda()], I, 0, bof4.METRIC_MAE, LV_INIT)
+    ref = oracle.em_accumulate_mae(w, I, 0, LV_INIT)
+    assert (ref["count"] % 2 == 0).any()
+    _check_mae_stats(got, ref, LV_INIT)
+
+
+def test_em_step_mae_many_tensors(bof4):
+    I = 64
+    sizes = [64 * (1 + (5 * k) % 40) for k in range(70)] + [0, 8192 * 2]
+    ws = [make_weights(max(s, 1), torch.bfloat16, 900 + k)[:s] for k, s in enumerate(sizes)]
+    got = bof4.bof4_em_step([w.cuda() for w in ws], I, 1, bof4.METRIC_MAE, LV_BOF4S)
+    ref = oracle.em_accumulate_mae(torch.cat(ws), I, 1, LV_BOF4S)
+    _check_mae_stats(got, ref, LV_BOF4S)
+
+
+@pytest.mark.parametrize("norm,mask,dtype", [(0, workloads.FIXED_BOF4, torch.float32),
+                                             (1, workloads.FIXED_BOF4S, torch.bfloat16)])
+def test_fit_mae_matches_oracle(bof4, norm, mask, dtype):
+    I, n, iters = 64, 1 << 17, 8
+    w = make_weights(n, dtype, 160 + norm)
+    cb, log = bof4.bof4_fit_codebook([w.cuda()], I, norm, bof4.METRIC_MAE, LV_INIT, mask, iters)
+    rcb, rlog = oracle.fit(w, I, norm, oracle.METRIC_MAE, LV_INIT, mask, iters)
+    cb = cb.cpu().numpy()
+    np.testing.assert_allclose(cb, rcb, rtol=RTOL, atol=1e-7)
+    np.testing.assert_allclose(log.cpu().numpy(), rlog, rtol=RTOL)
+    for l in range(16):
+        if (mask >> l) & 1:
+            assert cb[l] == LV_INIT[l]
+
+
+def test_fit_mae_is_bit_reproducible(bof4):
+    I, n = 64, 1 << 20
+    wd = make_weights(n, torch.bfloat16, 78).cuda()
+    a, la = bof4.bof4_fit_codebook([wd], I, 1, bof4.METRIC_MAE, LV_INIT, workloads.FIXED_BOF4S, 3)
+    b, lb = bof4.bof4_fit_codebook([wd], I, 1, bof4.METRIC_MAE, LV_INIT, workloads.FIXED_BOF4S, 3)
+    assert torch.equal(a, b) and torch.equal(la, lb)
