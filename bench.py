@@ -201,14 +201,38 @@ class Step:
         host_out["log_mse"].copy_(self.log_mse, non_blocking=True)
 
 
+def rank_env():
+    """(rank, local_rank, world_size) as the launcher exports them (1 process per GPU)."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def workload_seed_offset(rank: int) -> int:
+    """Every rank works on its own, independent problem: the path shards by blocks and needs
+    no exchange, so the ranks' workloads differ only by their seed."""
+    return rank
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_gweights_per_s(world: int, n_per_rank: int, ms_per_step: float) -> float:
+    """All ranks' weights per step over the slowest rank's step time."""
+    return world * n_per_rank / ms_per_step / 1e6
+
+
 def mae_launches(bof4) -> int:
     return getattr(bof4.binding, "MAE_LAUNCHES_PER_ITERATION", 0)
 
 
 def run_gpu(args):
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local, world = rank_env()
     import __graft_entry__ as entry
     if local == 0:
         entry.build()
@@ -225,7 +249,7 @@ def run_gpu(args):
     from paper_2505_06653_b200 import binding
     binding.lib()
 
-    st = Step(bof4, dev, seed_offset=rank)       # independent problem per rank: no collective
+    st = Step(bof4, dev, seed_offset=workload_seed_offset(rank))  # no data-path collective
     st.have_mae = hasattr(binding, "MAE_LAUNCHES_PER_ITERATION")
     if args.only:
         st.only = set(args.only.split(","))
@@ -273,10 +297,7 @@ def run_gpu(args):
     h2d = st.w_host.numel() * 2
     d2h = sum(t.numel() * t.element_size() for t in host_out.values())
 
-    if dist:
-        t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, dev)
     if rank != 0:
         if dist:
             dist.destroy_process_group()
@@ -305,7 +326,7 @@ def run_gpu(args):
                  "dequantize": BYTES_DEQUANT}[dom] * n
     achieved = dom_bytes / avg[dom] / 1e6
     line = {
-        "metric": METRIC, "value": world * n / ms_per_step / 1e6, "unit": "Gweights/s",
+        "metric": METRIC, "value": whole_job_gweights_per_s(world, n, ms_per_step), "unit": "Gweights/s",
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
@@ -364,9 +385,9 @@ def cpu_baseline(w_host, have_mae=True, sample=1 << 25, reps=2):
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
+    rank = rank_env()[0]
     if rank != 0:
-        return
+        return None
     import oracle
     oracle.build()
     sample = 1 << 24
