@@ -155,6 +155,33 @@ BOF4_API int opq_split(const void* d_w, int w_dtype, int64_t n, int block_size, 
               int64_t* d_n_out, void* d_ws, size_t ws_bytes, void* stream);
 
 /*
+ * opq_split without a workspace argument and without any allocation.  (The paper has no
+ * counterpart; this is a convenience of the library.)
+ *
+ * Meant for callers that are not in a position to obtain device memory: code that runs while
+ * another component owns the whole device-memory pool, a plug-in whose host framework forbids
+ * cudaMalloc / cudaFree on its streams because those calls synchronise the device, or a
+ * start-up path that runs before the application's allocator exists.  The scratch that
+ * opq_split takes from d_ws (tile counts, chunk offsets, staging slots) lives instead in a
+ * 4 MiB array inside the library image; every GPU that loads the library holds that array
+ * until the process exits.
+ *
+ *   - Same arguments, outputs and bit-exact results as opq_split, minus d_ws / ws_bytes.
+ *   - n is limited to 2^24 weights per call (BOF4_ERR_SHAPE beyond; split larger tensors at
+ *     multiples of block_size and add the chunk's first index to its outlier indices, or use
+ *     opq_split).
+ *   - The first call on each device looks up the array's device address (once per device,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array.  Every call rewrites each cell before it
+ *     reads it, so nothing has to be cleared between calls, but two calls whose kernels
+ *     overlap on the GPU (different streams, no ordering between them) race on it: order them.
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine.
+ */
+BOF4_API int opq_split_static(const void* d_w, int w_dtype, int64_t n, int block_size, float tau,
+                     void* d_w_clean, int32_t* d_out_idx, void* d_out_val, int64_t capacity,
+                     int64_t* d_n_out, void* stream);
+
+/*
  * OPQ fused with quantisation in one read of the weights (Sec. 3.3): outliers are listed as in
  * opq_split and replaced by zero BEFORE the block-constant search; the cleaned block is then
  * quantised as in bof4_quantize.

@@ -28,7 +28,7 @@ LEVELS = 16
 MAE_LAUNCHES_PER_ITERATION = 10
 
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
-           "opq_split", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
+           "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error")
 
 
@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.bof4_quantize.argtypes = [vp, i32, i64, i32, i32, vp, vp, vp, i32, vp]
         L.opq_split.restype = i32
         L.opq_split.argtypes = [vp, i32, i64, i32, ctypes.c_float, vp, vp, vp, i64, vp, vp, sz, vp]
+        L.opq_split_static.restype = i32
+        L.opq_split_static.argtypes = [vp, i32, i64, i32, ctypes.c_float, vp, vp, vp, i64, vp, vp]
         L.bof4_quantize_opq.restype = i32
         L.bof4_quantize_opq.argtypes = [vp, i32, i64, i32, i32, vp, ctypes.c_float, vp, vp, i32,
                                         vp, vp, i64, vp, vp, sz, vp]

@@ -7,6 +7,8 @@
 // 64-bit store per lane (256 contiguous bytes per warp).  The next row's load is issued before
 // the current row is processed.
 // dequantize: one lane owns 16 outputs (8 code bytes in, 32 or 64 bytes out).
+#include <mutex>
+
 #include "common.cuh"
 #include "layout.h"
 
@@ -711,4 +713,64 @@ extern "C" int bof4_quantize_opq(const void* d_w, int w_dtype, int64_t n, int bl
     return launch_opq<true>("bof4_quantize_opq", d_w, w_dtype, n, block_size, norm, d_codebook, tau,
                             d_codes, d_scales, scale_dtype, nullptr, d_out_idx, d_out_val, capacity,
                             d_n_out, d_ws, ws_bytes, stream);
+}
+
+// ================================================================= allocation-free outlier split
+
+namespace {
+
+// Scratch of opq_split_static: the tile counts, chunk offsets and staging slots that opq_split
+// otherwise takes from the caller's workspace.  It lives in the library image, so every GPU
+// that loads the library holds these 4 MiB until the process exits.
+constexpr int64_t kStaticMaxN = (int64_t)1 << 24;
+constexpr size_t kStaticScratchBytes = (size_t)4 << 20;
+static __device__ __align__(256) unsigned char g_opq_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device.  The array's name is only a
+// host-side handle; the address a kernel may use comes from cudaGetSymbolAddress, once per
+// device, with that device current.
+int static_scratch(void** out)
+{
+    int dev = -1;
+    BOF4_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) {
+        set_error("opq_split_static: device ordinal %d is outside 0..%d", dev, kMaxDevices - 1);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        BOF4_CUDA_TRY(cudaGetSymbolAddress(&p, g_opq_static_scratch));
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return BOF4_OK;
+}
+
+}  // namespace
+
+extern "C" int opq_split_static(const void* d_w, int w_dtype, int64_t n, int block_size, float tau,
+                                void* d_w_clean, int32_t* d_out_idx, void* d_out_val,
+                                int64_t capacity, int64_t* d_n_out, void* stream)
+{
+    if (n > kStaticMaxN) {
+        set_error("opq_split_static: n = %lld exceeds the built-in scratch (at most %lld weights per "
+                  "call; use opq_split with a workspace for larger tensors)",
+                  (long long)n, (long long)kStaticMaxN);
+        return BOF4_ERR_SHAPE;
+    }
+    if (n >= 0 && opq_layout(n).total > kStaticScratchBytes) {
+        set_error("opq_split_static: internal scratch too small for n = %lld", (long long)n);
+        return BOF4_ERR_WORKSPACE;
+    }
+    void* scratch = nullptr;
+    const int rc = static_scratch(&scratch);
+    if (rc) return rc;
+    return launch_opq<false>("opq_split_static", d_w, w_dtype, n, block_size, BOF4_NORM_ABS, nullptr, tau,
+                             nullptr, nullptr, w_dtype, d_w_clean, d_out_idx, d_out_val, capacity,
+                             d_n_out, scratch, kStaticScratchBytes, stream);
 }
