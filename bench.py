@@ -42,6 +42,9 @@ METRIC = ("hot-path step Gweights/s (EM iteration MSE + MAE, OPQ quantize, dequa
 BYTES_EM = 2.0
 BYTES_QUANT = 2.0 + 0.5 + 2.0 / I
 BYTES_DEQUANT = 0.5 + 2.0 / I + 2.0
+# data passes of one MAE iteration that stream all weights on this workload: the max-|w| pass
+# and three selection passes (the fourth is only needed for a region that straddles zero)
+MAE_DATA_PASSES = 4
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -163,6 +166,10 @@ class Step:
                             workspace=self.ws_opq,
                             out=(self.codes, self.scales, self.idx, self.val, self.cnt))
 
+    def quant_plain(self):
+        b = self.b
+        b.bof4_quantize(self.w, I, b.NORM_SIGNED, self.cb_mse, out=(self.codes, self.scales))
+
     def dequant(self):
         b = self.b
         b.bof4_dequantize(self.codes, self.scales, I, self.cb_mse, b.BF16, (self.idx, self.val, self.cnt),
@@ -173,6 +180,7 @@ class Step:
                  ("dequantize", self.dequant, 2)]
         comps = [c for c in comps if c[0] != "em_mae" or self.have_mae]
         if self.only:
+            comps.append(("quantize", self.quant_plain, 1))  # profiling runs only
             comps = [c for c in comps if c[0] in self.only]
         return comps
 
@@ -307,8 +315,9 @@ def run_gpu(args):
     ms_per_step = total_ms / K
     peak, peak_kind = measured_peak()
     avg = {k: sum(v) / len(v) for k, v in comp_ms.items()}
-    bytes_per_w = {"em_mse": BYTES_EM, "em_mae": None, "quantize_opq": BYTES_QUANT, "dequantize": BYTES_DEQUANT}
-    kernels = {"em_mse": 2, "em_mae": mae_launches(bof4), "quantize_opq": 4, "dequantize": 2}
+    bytes_per_w = {"em_mse": BYTES_EM, "em_mae": None, "quantize_opq": BYTES_QUANT, "dequantize": BYTES_DEQUANT,
+                   "quantize": BYTES_QUANT}
+    kernels = {"em_mse": 2, "em_mae": mae_launches(bof4), "quantize_opq": 4, "dequantize": 2, "quantize": 1}
     comp, launches = {}, 0
     for name, ms in avg.items():
         comp[name + "_ms"] = ms
@@ -322,8 +331,8 @@ def run_gpu(args):
             comp[k.replace("_gbs", "_frac_of_%s_hbm" % peak_kind)] = comp[k] / peak
     # dominant component = the one with the largest share of the step
     dom = max(avg, key=avg.get)
-    dom_bytes = {"em_mse": BYTES_EM, "em_mae": BYTES_EM * 3, "quantize_opq": BYTES_QUANT,
-                 "dequantize": BYTES_DEQUANT}[dom] * n
+    dom_bytes = {"em_mse": BYTES_EM, "em_mae": BYTES_EM * MAE_DATA_PASSES, "quantize_opq": BYTES_QUANT,
+                 "dequantize": BYTES_DEQUANT, "quantize": BYTES_QUANT}[dom] * n
     achieved = dom_bytes / avg[dom] / 1e6
     line = {
         "metric": METRIC, "value": whole_job_gweights_per_s(world, n, ms_per_step), "unit": "Gweights/s",

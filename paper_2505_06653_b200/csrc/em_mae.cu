@@ -31,8 +31,6 @@ struct MaeState {
     int top[kLevels];                    // key bits still unresolved (0: done)
     uint32_t active;                     // bit l: level l takes part in the selection
     uint32_t max_bits;                   // bits of the largest |w| of the data
-    int passes_left;                     // max over active levels of the passes still needed
-    int pad;
 };
 static_assert(sizeof(MaeState) <= kEmMaeStateBytes, "state must fit its slot");
 
@@ -113,7 +111,6 @@ __global__ void __launch_bounds__(kMaeBins)
 mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
 {
     __shared__ float s_xi[kLevels], s_lv[kLevels];
-    __shared__ int s_need[kLevels];
     make_thresholds(levels, s_xi, s_lv, threadIdx.x);
     __syncthreads();
     if (threadIdx.x < kLevels) {
@@ -131,15 +128,8 @@ mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
         W.state->before[l] = 0ull;
         W.state->total[l] = 0ull;
         W.state->count[l] = 0ull;
-        s_need[l] = on ? (bits + kMaeDigitBits - 1) / kMaeDigitBits : 0;
     }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int need = 0;
-        for (int l = 0; l < kLevels; ++l) need = max(need, s_need[l]);
-        W.state->active = ~skip_mask & 0xffffu;
-        W.state->passes_left = need;
-    }
+    if (threadIdx.x == 0) W.state->active = ~skip_mask & 0xffffu;
     for (int k = threadIdx.x; k < kLevels * kMaeBins; k += blockDim.x) {
         W.hist[k] = 0ull;
         W.chist[k] = 0ull;
@@ -167,7 +157,11 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     __shared__ const void* s_ptr[kEmMaxTensors];
     __shared__ int64_t s_n[kEmMaxTensors], s_row_end[kEmMaxTensors];
 
-    if (!FIRST && W.state->passes_left <= 0) return;
+    if (!FIRST) {  // nothing left to resolve: uniform over the grid
+        int any = 0;
+        for (int l = 0; l < kLevels; ++l) any |= W.state->top[l];
+        if (any <= 0) return;
+    }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     make_thresholds(levels, s_xi, s_lv, tid);
     if (tid < kLevels) {
@@ -251,65 +245,59 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
 
 // ---------------------------------------------------------------- bin selection
 
-// One CTA, one thread per bin.  For every level with bits left: the first bin in which the
-// cumulative weight reaches half of the total (2 (before + cum) >= total) becomes the next
+// One CTA per level, one thread per bin.  For a level with bits left: the first bin in which
+// the cumulative weight reaches half of the total (2 (before + cum) >= total) becomes the next
 // digit.  After the first pass the totals (and counts) are those of the whole region.
 __global__ void __launch_bounds__(kMaeBins)
 mae_select_kernel(MaeWs W, int first)
 {
-    __shared__ unsigned long long s_scan[kMaeBins];
-    __shared__ unsigned long long s_cscan[kMaeBins / 32];
-    __shared__ int s_pick;
+    __shared__ unsigned long long s_wsum[kMaeBins / 32], s_csum[kMaeBins / 32];
     MaeState* S = W.state;
-    if (!first && S->passes_left <= 0) return;
-    const int j = threadIdx.x;
-    int left = 0;
-    for (int l = 0; l < kLevels; ++l) {
-        const int top = S->top[l];
-        if (top <= 0) continue;  // uniform: read from global by every thread
-        const unsigned long long mine = W.hist[l * kMaeBins + j];
-        W.hist[l * kMaeBins + j] = 0ull;
-        s_scan[j] = mine;
-        if (j == 0) s_pick = kMaeBins - 1;
-        __syncthreads();
-        for (int off = 1; off < kMaeBins; off <<= 1) {
-            const unsigned long long t = (j >= off) ? s_scan[j - off] : 0ull;
-            __syncthreads();
-            s_scan[j] += t;
-            __syncthreads();
-        }
-        if (first) {
-            unsigned long long c = W.chist[l * kMaeBins + j];
-            W.chist[l * kMaeBins + j] = 0ull;
-#pragma unroll
-            for (int off = 16; off; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
-            if ((j & 31) == 0) s_cscan[j >> 5] = c;
-        }
-        __syncthreads();
-        const unsigned long long total = first ? s_scan[kMaeBins - 1] : S->total[l];
-        const unsigned long long before = S->before[l];
-        const unsigned long long incl = s_scan[j], excl = incl - mine;
-        const bool reached = 2ull * (before + incl) >= total;
-        const bool prev_reached = (j > 0) && (2ull * (before + excl) >= total);
-        if (reached && !prev_reached) s_pick = j;  // exactly one thread (cumulative is monotone)
-        __syncthreads();
-        const int pick = s_pick;
-        if (j == pick) {
-            const int sh = max(top - kMaeDigitBits, 0);
-            S->before[l] = before + excl;
-            S->prefix[l] = (S->prefix[l] << (top - sh)) | (uint32_t)pick;
-            S->top[l] = sh;
-            if (first) S->total[l] = total;
-        }
-        if (first && j == 0) {
-            unsigned long long c = 0;
-            for (int k = 0; k < kMaeBins / 32; ++k) c += s_cscan[k];
-            S->count[l] = c;
-        }
-        left = max(left, (max(top - kMaeDigitBits, 0) + kMaeDigitBits - 1) / kMaeDigitBits);
-        __syncthreads();
+    const int l = blockIdx.x, j = threadIdx.x, lane = j & 31, warp = j >> 5;
+    const int top = S->top[l];
+    if (top <= 0) return;  // uniform over the CTA
+    const unsigned long long mine = W.hist[l * kMaeBins + j];
+    W.hist[l * kMaeBins + j] = 0ull;
+    unsigned long long c = 0ull;
+    if (first) {
+        c = W.chist[l * kMaeBins + j];
+        W.chist[l * kMaeBins + j] = 0ull;
     }
-    if (j == 0) S->passes_left = left;
+    // inclusive scan of the bin weights: inside the warp, then over the warp totals
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long t = __shfl_up_sync(kFull, incl, off);
+        if (lane >= off) incl += t;
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
+    if (lane == 31) s_wsum[warp] = incl;
+    if (lane == 0) s_csum[warp] = c;
+    __syncthreads();
+    unsigned long long carry = 0ull, all = 0ull, count = 0ull;
+    for (int k = 0; k < kMaeBins / 32; ++k) {
+        if (k < warp) carry += s_wsum[k];
+        all += s_wsum[k];
+        count += s_csum[k];
+    }
+    incl += carry;
+    const unsigned long long total = first ? all : S->total[l];
+    const unsigned long long before = S->before[l];
+    const unsigned long long excl = incl - mine;
+    const bool reached = 2ull * (before + incl) >= total;
+    const bool prev_reached = (j > 0) && (2ull * (before + excl) >= total);
+    __syncthreads();  // every thread has read the state it needs
+    if (reached && !prev_reached) {  // exactly one thread: the cumulative weight is monotone
+        const int sh = max(top - kMaeDigitBits, 0);
+        S->before[l] = before + excl;
+        S->prefix[l] = (S->prefix[l] << (top - sh)) | (uint32_t)j;
+        S->top[l] = sh;
+        if (first) {
+            S->total[l] = total;
+            S->count[l] = count;
+        }
+    }
 }
 
 // ---------------------------------------------------------------- level update
@@ -426,7 +414,7 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
         const int rc = for_each_tensor_chunk(a, kMaeRow, fire, &calls);
         if (rc) return rc;
         if (first && calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(W.partials, 0, kEmPartialBytes, st));
-        mae_select_kernel<<<1, kMaeBins, 0, st>>>(W, first ? 1 : 0);
+        mae_select_kernel<<<kLevels, kMaeBins, 0, st>>>(W, first ? 1 : 0);
         BOF4_CUDA_TRY(cudaGetLastError());
     }
     mae_finalize_kernel<<<1, 256, 0, st>>>(W, kEmGrid, a.n_total, d_levels_in, d_levels_out, skip_mask,

@@ -138,13 +138,24 @@ __device__ __forceinline__ float load_scale<BF16>(const void* scales, int64_t b)
     return __uint_as_float((uint32_t)__ldg(static_cast<const uint16_t*>(scales) + b) << 16);
 }
 
+// Two fp32 values to one packed pair of bf16 (round to nearest even): lo -> bits 0..15.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+// One code byte holds two weights, so the levels are tabulated per byte: entry b is the pair
+// (xhat[b >> 4], xhat[b & 15]); one 8-byte shared-memory read and one packed multiplication by
+// the block constant give both products (Eq. 3).
 template <class ST, class OT, int I>
 __global__ void __launch_bounds__(kDThreads)
 dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t n,
                   const float* __restrict__ levels, void* __restrict__ out)
 {
-    __shared__ float s_lv[kLevels];
-    if (threadIdx.x < kLevels) s_lv[threadIdx.x] = levels[threadIdx.x];
+    __shared__ float2 s_pair[256];
+    s_pair[threadIdx.x] = make_float2(levels[threadIdx.x >> 4], levels[threadIdx.x & 15]);
     __syncthreads();
     const int64_t rows = (n + kDRow - 1) / kDRow;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
@@ -155,24 +166,26 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ sc
                      : "=r"(cc.x), "=r"(cc.y)
                      : "l"(codes + idx / 2));
         const float m = load_scale<ST>(scales, idx / I);
-        float o[16];
+        const float2 mm = make_float2(m, m);
+        float2 o[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            const uint32_t byte = ((k < 4 ? cc.x : cc.y) >> (8 * (k & 3))) & 0xffu;
-            o[2 * k] = __fmul_rn(m, s_lv[byte >> 4]);
-            o[2 * k + 1] = __fmul_rn(m, s_lv[byte & 15u]);
+            const uint32_t byte = __byte_perm(k < 4 ? cc.x : cc.y, 0u, 0x4440u | (uint32_t)(k & 3));
+            o[k] = __fmul2_rn(mm, s_pair[byte]);
         }
         if (OT::code == BF16::code) {
             Raw8 p;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) p.u[k] = bf16_rne(o[2 * k]) | (bf16_rne(o[2 * k + 1]) << 16);
+            for (int k = 0; k < 8; ++k) p.u[k] = pack_bf16x2(o[k].x, o[k].y);
             st_stream256(static_cast<uint16_t*>(out) + idx, p);
         } else {
             Raw8 p, q;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                p.u[k] = __float_as_uint(o[k]);
-                q.u[k] = __float_as_uint(o[8 + k]);
+            for (int k = 0; k < 4; ++k) {
+                p.u[2 * k] = __float_as_uint(o[k].x);
+                p.u[2 * k + 1] = __float_as_uint(o[k].y);
+                q.u[2 * k] = __float_as_uint(o[4 + k].x);
+                q.u[2 * k + 1] = __float_as_uint(o[4 + k].y);
             }
             st_stream256(static_cast<float*>(out) + idx, p);
             st_stream256(static_cast<float*>(out) + idx + 8, q);
