@@ -149,32 +149,47 @@ __device__ __forceinline__ float min3(float a, float b, float c)
 
 // ---------------------------------------------------------------- block constant
 
+__device__ __forceinline__ float max3_nan(float a, float b, float c)
+{
+    float d;
+    asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float max2_nan(float a, float b)
+{
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
 // Block constant of the lane group that owns the block.  SIGNED = false: max |w| (Eq. 1).
 // SIGNED = true: the element of largest magnitude with its sign, lowest index on ties (Eq. 4).
-// An all-zero block gives +0.  Must be called by all 32 lanes.
+// An all-zero block gives +0.  Must be called by all 32 lanes.  `g` receives the largest
+// magnitude of the block, or NaN if the block holds a NaN (the maximum chain propagates NaN),
+// so that one range test on g tells whether every quotient w / m is a finite number in [-1, 1].
 //
 // The signed constant is found from the block's largest and smallest element: the larger
 // magnitude wins.  Only when both +g and -g occur does the position matter; that case is
 // settled by two ballots (which lane holds the first +g, which the first -g) and, where one
 // lane holds both, by that lane's elements in index order.
 template <int LPB, bool SIGNED>
-__device__ __forceinline__ float block_constant(const float (&v)[kLaneW])
+__device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float& g)
 {
-    float mx = max3(v[0], v[1], v[2]), mn = min3(v[0], v[1], v[2]);
+    float mx = max3_nan(v[0], v[1], v[2]), mn = min3(v[0], v[1], v[2]);
 #pragma unroll
     for (int k = 3; k < 15; k += 2) {
-        mx = max3(mx, v[k], v[k + 1]);
+        mx = max3_nan(mx, v[k], v[k + 1]);
         mn = min3(mn, v[k], v[k + 1]);
     }
-    mx = fmaxf(mx, v[15]);
+    mx = max2_nan(mx, v[15]);
     mn = fminf(mn, v[15]);
     float gx = mx, gn = mn;
 #pragma unroll
     for (int off = 1; off < LPB; off <<= 1) {
-        gx = fmaxf(gx, __shfl_xor_sync(kFull, gx, off));
+        gx = max2_nan(gx, __shfl_xor_sync(kFull, gx, off));
         gn = fminf(gn, __shfl_xor_sync(kFull, gn, off));
     }
-    const float g = fmaxf(gx, -gn);
+    g = max2_nan(gx, -gn);
     if (!SIGNED) return g;
     float m = (gx > -gn) ? gx : gn;
     const bool tie = (gx == -gn) && (g != 0.0f);
@@ -236,6 +251,10 @@ __device__ __forceinline__ int region_of(float x, const float* s_xi)
 // exactly.  A codebook with two thresholds in one bin (levels closer than 1/128) makes the
 // kernels fall back to the binary search.  Each table row is replicated for the 32 lanes
 // ([bin][lane], 8 bytes each) so that the shared-memory bank only depends on the lane.
+//
+// The table may only be indexed with finite x in [-1, 1]: callers use it for a warp row only
+// when every block of the row has a finite, non-zero largest magnitude (row_is_safe), which
+// makes every quotient such a number; all other rows take the binary search.
 constexpr int kLutBins = 257;
 constexpr uint32_t kLutMagicBits = 0x4B400000u;  // bits of 1.5 * 2^23
 constexpr float kLutMagic = 12583040.0f;         // 1.5 * 2^23 + 128
@@ -248,12 +267,11 @@ __device__ __forceinline__ float2 lut_key2(float2 x)
     return __ffma2_rn(x, make_float2(128.0f, 128.0f), make_float2(kLutMagic, kLutMagic));
 }
 
-// Byte offset of the lane's table entry; key = lut_key(x).  The unsigned minimum also sends
-// NaN / infinite keys (non-finite input) to the last row, so the read stays inside the table.
+// Byte offset of the lane's table entry; key = lut_key(x) has bits kLutMagicBits + bin.
 __device__ __forceinline__ uint32_t lut_offset(float key, uint32_t lane_off)
 {
-    const uint32_t b = min(__float_as_uint(key), kLutMagicBits + (uint32_t)(kLutBins - 1));
-    return b * (uint32_t)kLutRowBytes + (lane_off - kLutMagicBits * (uint32_t)kLutRowBytes);
+    return __float_as_uint(key) * (uint32_t)kLutRowBytes +
+           (lane_off - kLutMagicBits * (uint32_t)kLutRowBytes);
 }
 
 // Builds the table in shared memory from the thresholds; payload(base) is stored next to
@@ -288,11 +306,14 @@ __device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lu
 // returns exactly RN(w / m) whenever the quotient is a normal number (checked exhaustively
 // over all operand pairs on the CPU by the test-suite).  It costs three packed operations
 // per two weights plus one reciprocal per lane and block.
-__device__ __forceinline__ bool div_safe(float m)
+__device__ __forceinline__ bool div_safe(float g)
 {
-    const float a = fabsf(m);
-    return a >= 0x1p-60f && a <= 0x1p60f;
+    return g >= 0x1p-60f && g <= 0x1p60f;  // false for NaN, infinity and zero
 }
+
+// Warp-uniform: every block of this warp row (lanes beyond the end of the data excepted) has a
+// largest magnitude g inside the safe range.
+__device__ __forceinline__ bool row_is_safe(float g, bool ok) { return __all_sync(kFull, div_safe(g) || !ok); }
 
 // x[k] = RN(v[k] / m) for the 16 weights of a lane (x = 0 when m = 0).  `fast` (warp-uniform;
 // only ever true for bf16 input whose block constants all pass div_safe) selects the
@@ -303,7 +324,8 @@ __device__ __forceinline__ void normalise16(const float (&v)[kLaneW], float m, b
                                             float (&x)[kLaneW])
 {
     if (fast) {
-        const float r = __frcp_rn(m);
+        // lanes beyond the end of the data hold zeros and m = 0: give them x = 0, a valid table index
+        const float r = (m == 0.0f) ? 0.0f : __frcp_rn(m);
         const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
 #pragma unroll
         for (int k = 0; k < kLaneW / 2; ++k) {

@@ -143,8 +143,9 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
         const RawRow<DT> next = fetch(g + gridDim.x, ok_next);
         float v[kLaneW];
         widen(raw, v);
-        const float m = block_constant<LPB, SIGNED>(v);
-        const bool fast = (DT::code == BF16::code) && __all_sync(kFull, div_safe(m) || !ok);
+        float gmax;
+        const float m = block_constant<LPB, SIGNED>(v, gmax);
+        const bool safe = row_is_safe(gmax, ok);
         float2 sq = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int k = 0; k < kLaneW / 2; ++k) {
@@ -153,11 +154,11 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
         }
         w2sum += (double)(sq.x + sq.y);  // lanes beyond the end hold zeros
         float x[kLaneW];
-        normalise16<false>(v, m, fast, x);
+        normalise16<false>(v, m, safe && DT::code == BF16::code, x);
         if (ok) {
             const float m2 = m * m;
             const float2 mm = make_float2(m2, m2);
-            if (lut_ok) {
+            if (lut_ok && safe) {
 #pragma unroll
                 for (int k = 0; k < kLaneW / 2; ++k) {
                     const float2 key = lut_key2(make_float2(x[2 * k], x[2 * k + 1]));

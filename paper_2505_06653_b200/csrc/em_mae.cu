@@ -194,17 +194,19 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         const bool ok = idx < s_n[t_cur];
         float v[kLaneW];
         widen(ok ? load_raw<DT>(s_ptr[t_cur], idx) : zero_raw<DT>(), v);
-        const float m = block_constant<LPB, SIGNED>(v);
-        const bool fast = (DT::code == BF16::code) && __all_sync(kFull, div_safe(m) || !ok);
+        float gmax;
+        const float m = block_constant<LPB, SIGNED>(v, gmax);
+        const bool safe = row_is_safe(gmax, ok);
         float x[kLaneW];
-        normalise16<false>(v, m, fast, x);
+        normalise16<false>(v, m, safe && DT::code == BF16::code, x);
+        const bool use_lut = lut_ok && safe;
         if (!ok) continue;
         const uint32_t a = fixed_weight(m, max_bits);
         float e = 0.0f;
 #pragma unroll
         for (int k = 0; k < kLaneW; ++k) {
             uint32_t c;
-            if (lut_ok) {
+            if (use_lut) {
                 const uint2 ent = *reinterpret_cast<const uint2*>(s_lut + lut_offset(lut_key(x[k]), lane_off));
                 c = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? 1u : 0u);
             } else {

@@ -18,7 +18,8 @@ constexpr int kQThreads = 512;              // quantise / OPQ pass 1
 constexpr int kQRow = kQThreads * kLaneW;   // weights per CTA row
 constexpr int kQCtasPerSm = 2;              // two CTAs, each with its own region table
 constexpr int kDThreads = 256;              // dequantise
-constexpr int kDRow = kDThreads * 16;       // outputs per CTA row (dequantise)
+constexpr int kDLaneW = 32;                 // outputs per lane and row (16 code bytes in)
+constexpr int kDRow = kDThreads * kDLaneW;  // outputs per CTA row (dequantise)
 
 template <class ST>
 __device__ __forceinline__ void store_scale(void* scales, int64_t b, float m);
@@ -51,26 +52,43 @@ __device__ __forceinline__ QuantTables setup_tables(const float* __restrict__ le
 }
 
 // Codes of the 16 normalised weights of a lane packed as 8 bytes (two words), even element in
-// the high nibble of its byte.
-__device__ __forceinline__ void encode16(const float (&x)[kLaneW], const QuantTables& T, uint32_t lane_off,
-                                         uint32_t& w0, uint32_t& w1)
+// the high nibble of its byte.  Each word is built by Horner steps w = 16 w + code over its 8
+// codes in the order 6 7 4 5 2 3 0 1, which leaves byte k = (code[2k] << 4) | code[2k+1].
+// use_lut (warp-uniform) requires finite x in [-1, 1].
+__device__ __forceinline__ void encode16(const float (&x)[kLaneW], const QuantTables& T, bool use_lut,
+                                         uint32_t lane_off, uint32_t& w0, uint32_t& w1)
 {
-    uint32_t word[2] = {0u, 0u};
-    if (T.lut_ok) {
+    uint32_t word[2];
+    if (use_lut) {
+        float key[kLaneW];
 #pragma unroll
         for (int k = 0; k < kLaneW / 2; ++k) {
-            const float2 key = lut_key2(make_float2(x[2 * k], x[2 * k + 1]));
-            const uint2 e0 = *reinterpret_cast<const uint2*>(T.lut + lut_offset(key.x, lane_off));
-            const uint2 e1 = *reinterpret_cast<const uint2*>(T.lut + lut_offset(key.y, lane_off));
-            const uint32_t c0 = e0.y + ((x[2 * k] >= __uint_as_float(e0.x)) ? 1u : 0u);
-            const uint32_t c1 = e1.y + ((x[2 * k + 1] >= __uint_as_float(e1.x)) ? 1u : 0u);
-            word[k >> 2] |= ((c0 << 4) | c1) << (8 * (k & 3));
+            const float2 kk = lut_key2(make_float2(x[2 * k], x[2 * k + 1]));
+            key[2 * k] = kk.x;
+            key[2 * k + 1] = kk.y;
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t w = 0u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int k = 8 * h + (6 - 2 * (j >> 1)) + (j & 1);
+                const uint2 e = *reinterpret_cast<const uint2*>(T.lut + lut_offset(key[k], lane_off));
+                w = w * 16u + e.y;
+                if (x[k] >= __uint_as_float(e.x)) w += 1u;
+            }
+            word[h] = w;
         }
     } else {
 #pragma unroll
-        for (int k = 0; k < kLaneW / 2; ++k) {
-            const uint32_t c0 = (uint32_t)region_of(x[2 * k], T.xi), c1 = (uint32_t)region_of(x[2 * k + 1], T.xi);
-            word[k >> 2] |= ((c0 << 4) | c1) << (8 * (k & 3));
+        for (int h = 0; h < 2; ++h) {
+            uint32_t w = 0u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int k = 8 * h + (6 - 2 * (j >> 1)) + (j & 1);
+                w = w * 16u + (uint32_t)region_of(x[k], T.xi);
+            }
+            word[h] = w;
         }
     }
     w0 = word[0];
@@ -84,12 +102,13 @@ __device__ __forceinline__ void quantize_row(const float (&v)[kLaneW], int64_t i
                                              uint8_t* __restrict__ codes, void* __restrict__ scales)
 {
     constexpr int LPB = I / kLaneW;
-    const float m = block_constant<LPB, SIGNED>(v);
-    const bool fast = (DT::code == BF16::code) && __all_sync(kFull, div_safe(m) || !ok);
+    float g;
+    const float m = block_constant<LPB, SIGNED>(v, g);
+    const bool safe = row_is_safe(g, ok);
     float x[kLaneW];
-    normalise16<true>(v, m, fast, x);
+    normalise16<true>(v, m, safe && DT::code == BF16::code, x);
     uint32_t w0, w1;
-    encode16(x, T, lane_off, w0, w1);
+    encode16(x, T, safe && T.lut_ok, lane_off, w0, w1);
     if (ok) {
         st_stream64(codes + idx / 2, w0, w1);
         if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx / I, m);
@@ -158,38 +177,59 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ sc
     s_pair[threadIdx.x] = make_float2(levels[threadIdx.x >> 4], levels[threadIdx.x & 15]);
     __syncthreads();
     const int64_t rows = (n + kDRow - 1) / kDRow;
-    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
-        const int64_t idx = (r * kDThreads + threadIdx.x) * 16;
-        if (idx >= n) continue;
-        uint2 cc;
-        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];"
-                     : "=r"(cc.x), "=r"(cc.y)
-                     : "l"(codes + idx / 2));
-        const float m = load_scale<ST>(scales, idx / I);
-        const float2 mm = make_float2(m, m);
-        float2 o[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint32_t byte = __byte_perm(k < 4 ? cc.x : cc.y, 0u, 0x4440u | (uint32_t)(k & 3));
-            o[k] = __fmul2_rn(mm, s_pair[byte]);
+    int64_t r = blockIdx.x;
+    if (r >= rows) return;
+    // n is a multiple of 32, so a lane's 32 outputs are all inside the tensor or all outside
+    auto fetch = [&](int64_t row, int64_t& idx, uint4& cc, float& m) {
+        idx = (row * kDThreads + threadIdx.x) * kDLaneW;
+        cc = make_uint4(0u, 0u, 0u, 0u);
+        m = 0.0f;
+        if (idx < n) {
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(cc.x), "=r"(cc.y), "=r"(cc.z), "=r"(cc.w)
+                         : "l"(codes + idx / 2));
+            m = load_scale<ST>(scales, idx / I);
         }
-        if (OT::code == BF16::code) {
-            Raw8 p;
+    };
+    int64_t idx, idx_next;
+    uint4 cc, cc_next;
+    float m, m_next;
+    fetch(r, idx, cc, m);
+    for (; r < rows; r += gridDim.x) {
+        fetch(r + gridDim.x, idx_next, cc_next, m_next);
+        if (idx < n) {
+            const float2 mm = make_float2(m, m);
+            const uint32_t word[4] = {cc.x, cc.y, cc.z, cc.w};
 #pragma unroll
-            for (int k = 0; k < 8; ++k) p.u[k] = pack_bf16x2(o[k].x, o[k].y);
-            st_stream256(static_cast<uint16_t*>(out) + idx, p);
-        } else {
-            Raw8 p, q;
+            for (int h = 0; h < 2; ++h) {  // 16 outputs at a time
+                float2 o[8];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                p.u[2 * k] = __float_as_uint(o[k].x);
-                p.u[2 * k + 1] = __float_as_uint(o[k].y);
-                q.u[2 * k] = __float_as_uint(o[4 + k].x);
-                q.u[2 * k + 1] = __float_as_uint(o[4 + k].y);
+                for (int k = 0; k < 8; ++k) {
+                    const uint32_t byte = __byte_perm(word[2 * h + (k >> 2)], 0u, 0x4440u | (uint32_t)(k & 3));
+                    o[k] = __fmul2_rn(mm, s_pair[byte]);
+                }
+                if (OT::code == BF16::code) {
+                    Raw8 p;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) p.u[k] = pack_bf16x2(o[k].x, o[k].y);
+                    st_stream256(static_cast<uint16_t*>(out) + idx + 16 * h, p);
+                } else {
+                    Raw8 p, q;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        p.u[2 * k] = __float_as_uint(o[k].x);
+                        p.u[2 * k + 1] = __float_as_uint(o[k].y);
+                        q.u[2 * k] = __float_as_uint(o[4 + k].x);
+                        q.u[2 * k + 1] = __float_as_uint(o[4 + k].y);
+                    }
+                    st_stream256(static_cast<float*>(out) + idx + 16 * h, p);
+                    st_stream256(static_cast<float*>(out) + idx + 16 * h + 8, q);
+                }
             }
-            st_stream256(static_cast<float*>(out) + idx, p);
-            st_stream256(static_cast<float*>(out) + idx + 8, q);
         }
+        idx = idx_next;
+        cc = cc_next;
+        m = m_next;
     }
 }
 

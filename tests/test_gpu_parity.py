@@ -355,3 +355,31 @@ def test_fit_mae_is_bit_reproducible(bof4):
     a, la = bof4.bof4_fit_codebook([wd], I, 1, bof4.METRIC_MAE, LV_INIT, workloads.FIXED_BOF4S, 3)
     b, lb = bof4.bof4_fit_codebook([wd], I, 1, bof4.METRIC_MAE, LV_INIT, workloads.FIXED_BOF4S, 3)
     assert torch.equal(a, b) and torch.equal(la, lb)
+
+
+def test_non_finite_weights_do_not_disturb_other_blocks(bof4):
+    """NaN / infinite weights are outside the contract, but they must neither fault nor change
+    the result of any block that holds only finite numbers (rows with a non-finite block take
+    the comparison-only search instead of the table)."""
+    I, n = 64, 8192 * 3
+    w = make_weights(n, torch.bfloat16, 33)
+    bad_blocks = [3, 40, 41, 200]
+    w[3 * I + 5] = float("nan")
+    w[40 * I] = float("inf")
+    w[41 * I + 63] = float("-inf")
+    w[200 * I + 1] = float("nan")
+    w[200 * I + 2] = float("inf")
+    wd = w.cuda()
+    codes, scales = bof4.bof4_quantize(wd, I, 1, LV_BOF4S)
+    out = bof4.bof4_dequantize(codes, scales, I, LV_BOF4S, bof4.BF16)
+    st = bof4.bof4_em_step([wd], I, 1, bof4.METRIC_MSE, LV_BOF4S)
+    torch.cuda.synchronize()
+    clean = w.clone()
+    for b in bad_blocks:
+        clean[b * I:(b + 1) * I] = 0.0
+    rc, rs = oracle.quantize(clean, I, 1, LV_BOF4S)
+    keep = np.ones(n // I, bool)
+    keep[bad_blocks] = False
+    assert np.array_equal(codes.cpu().numpy().reshape(-1, I // 2)[keep], rc.reshape(-1, I // 2)[keep])
+    assert np.array_equal(scales_f32(scales)[keep], rs[keep])
+    assert st["n"] == n
