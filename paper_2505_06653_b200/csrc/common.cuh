@@ -127,6 +127,22 @@ __device__ __forceinline__ void widen(const RawRow<F32>& r, float (&v)[kLaneW])
     }
 }
 
+// Rows of `row` consecutive weights (one CTA iteration each) over a tensor of n weights; the
+// calling thread owns kLaneW weights at offset tid * kLaneW of every row.  Row indices are
+// 32-bit; only the last row can be partial (n is a multiple of the block size, hence of 16).
+struct RowMap {
+    int rows, rows_full, row;
+    int tid_off;
+    bool tail_ok;
+    __device__ __forceinline__ RowMap(int64_t n, int row_, int tid)
+        : rows((int)((n + row_ - 1) / row_)), rows_full((int)(n / row_)), row(row_), tid_off(tid * kLaneW),
+          tail_ok((int64_t)(n / row_) * row_ + tid * kLaneW < n)
+    {
+    }
+    __device__ __forceinline__ bool ok(int r) const { return r < rows_full || (r < rows && tail_ok); }
+    __device__ __forceinline__ int64_t idx(int r) const { return (int64_t)r * row + tid_off; }
+};
+
 // fp32 -> bf16 bits, round to nearest even (finite inputs).
 __device__ __forceinline__ uint32_t bf16_rne(float f)
 {
@@ -267,11 +283,22 @@ __device__ __forceinline__ float2 lut_key2(float2 x)
     return __ffma2_rn(x, make_float2(128.0f, 128.0f), make_float2(kLutMagic, kLutMagic));
 }
 
-// Byte offset of the lane's table entry; key = lut_key(x) has bits kLutMagicBits + bin.
-__device__ __forceinline__ uint32_t lut_offset(float key, uint32_t lane_off)
+// The lane's table entry {thr bits, payload} for key = lut_key(x), whose bits are
+// kLutMagicBits + bin.  lut_base = lut_lane_base(table, lane): a 32-bit shared-memory address
+// with the magic folded in, so that the probe is one multiply-add and one 8-byte read.  The
+// table is constant while it is probed, hence the read may be scheduled freely.
+__device__ __forceinline__ uint32_t lut_lane_base(const unsigned char* s_lut, int lane)
 {
-    return __float_as_uint(key) * (uint32_t)kLutRowBytes +
-           (lane_off - kLutMagicBits * (uint32_t)kLutRowBytes);
+    return (uint32_t)__cvta_generic_to_shared(s_lut) + (uint32_t)lane * 8u -
+           kLutMagicBits * (uint32_t)kLutRowBytes;
+}
+__device__ __forceinline__ uint2 lut_probe(float key, uint32_t lut_base)
+{
+    uint2 e;
+    asm("ld.shared.v2.u32 {%0, %1}, [%2];"
+        : "=r"(e.x), "=r"(e.y)
+        : "r"(__float_as_uint(key) * (uint32_t)kLutRowBytes + lut_base));
+    return e;
 }
 
 // Builds the table in shared memory from the thresholds; payload(base) is stored next to

@@ -67,7 +67,7 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
     const bool lut_ok = s_multi == 0;
 
     const int64_t total_rows = T.row_end[T.count - 1];
-    const uint32_t lane_off = lane * 8, tid_off = tid * 8;
+    const uint32_t lut_base = lut_lane_base(s_lut, lane), tid_off = tid * 8;
     double w2sum = 0.0;
     int t_cur = 0;
     int since_flush = 0;
@@ -165,8 +165,7 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const float xv = x[2 * k + h];
-                        const uint2 ent = *reinterpret_cast<const uint2*>(
-                            s_lut + lut_offset(h ? key.y : key.x, lane_off));
+                        const uint2 ent = lut_probe(h ? key.y : key.x, lut_base);
                         const uint32_t off =
                             ent.y + ((xv >= __uint_as_float(ent.x)) ? G::acc_row_bytes : 0u) + tid_off;
                         float2* pa = reinterpret_cast<float2*>(s_acc + off);

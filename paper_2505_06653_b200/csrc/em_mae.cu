@@ -184,7 +184,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     const bool lut_ok = s_multi == 0;
 
     const int64_t total_rows = T.row_end[T.count - 1];
-    const uint32_t lane_off = lane * 8;
+    const uint32_t lut_base = lut_lane_base(s_lut, lane);
     double err = 0.0;
     int t_cur = 0;
     for (int64_t g = blockIdx.x; g < total_rows; g += gridDim.x) {
@@ -207,7 +207,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         for (int k = 0; k < kLaneW; ++k) {
             uint32_t c;
             if (use_lut) {
-                const uint2 ent = *reinterpret_cast<const uint2*>(s_lut + lut_offset(lut_key(x[k]), lane_off));
+                const uint2 ent = lut_probe(lut_key(x[k]), lut_base);
                 c = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? 1u : 0u);
             } else {
                 c = (uint32_t)region_of(x[k], s_xi);

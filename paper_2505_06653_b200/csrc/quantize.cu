@@ -56,7 +56,7 @@ __device__ __forceinline__ QuantTables setup_tables(const float* __restrict__ le
 // codes in the order 6 7 4 5 2 3 0 1, which leaves byte k = (code[2k] << 4) | code[2k+1].
 // use_lut (warp-uniform) requires finite x in [-1, 1].
 __device__ __forceinline__ void encode16(const float (&x)[kLaneW], const QuantTables& T, bool use_lut,
-                                         uint32_t lane_off, uint32_t& w0, uint32_t& w1)
+                                         uint32_t lut_base, uint32_t& w0, uint32_t& w1)
 {
     uint32_t word[2];
     if (use_lut) {
@@ -73,7 +73,7 @@ __device__ __forceinline__ void encode16(const float (&x)[kLaneW], const QuantTa
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int k = 8 * h + (6 - 2 * (j >> 1)) + (j & 1);
-                const uint2 e = *reinterpret_cast<const uint2*>(T.lut + lut_offset(key[k], lane_off));
+                const uint2 e = lut_probe(key[k], lut_base);
                 w = w * 16u + e.y;
                 if (x[k] >= __uint_as_float(e.x)) w += 1u;
             }
@@ -98,7 +98,7 @@ __device__ __forceinline__ void encode16(const float (&x)[kLaneW], const QuantTa
 // Block constant, normalisation, codes and stores for one lane-row of (cleaned) weights.
 template <class DT, int I, bool SIGNED, class ST>
 __device__ __forceinline__ void quantize_row(const float (&v)[kLaneW], int64_t idx, bool ok,
-                                             const QuantTables& T, uint32_t lane_off, int lane,
+                                             const QuantTables& T, uint32_t lut_base, int lane,
                                              uint8_t* __restrict__ codes, void* __restrict__ scales)
 {
     constexpr int LPB = I / kLaneW;
@@ -108,7 +108,7 @@ __device__ __forceinline__ void quantize_row(const float (&v)[kLaneW], int64_t i
     float x[kLaneW];
     normalise16<true>(v, m, safe && DT::code == BF16::code, x);
     uint32_t w0, w1;
-    encode16(x, T, safe && T.lut_ok, lane_off, w0, w1);
+    encode16(x, T, safe && T.lut_ok, lut_base, w0, w1);
     if (ok) {
         st_stream64(codes + idx / 2, w0, w1);
         if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx / I, m);
@@ -124,21 +124,19 @@ quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
     const QuantTables T = setup_tables(levels, s_xi, s_lv, s_lut, &s_multi);
-    const int64_t rows = (n + kQRow - 1) / kQRow;
     const int lane = threadIdx.x & 31;
-    const uint32_t lane_off = lane * 8;
-    int64_t r = blockIdx.x;
-    if (r >= rows) return;
-    int64_t idx = (r * kQThreads + threadIdx.x) * kLaneW;
-    RawRow<DT> raw = (idx < n) ? load_raw<DT>(w, idx) : zero_raw<DT>();
-    for (; r < rows; r += gridDim.x) {
-        const int64_t idx_next = ((r + gridDim.x) * kQThreads + threadIdx.x) * kLaneW;
-        const RawRow<DT> next = (idx_next < n) ? load_raw<DT>(w, idx_next) : zero_raw<DT>();
+    const uint32_t lut_base = lut_lane_base(s_lut, lane);  // table base of this lane
+    const RowMap map(n, kQRow, threadIdx.x);
+    int r = blockIdx.x;
+    if (r >= map.rows) return;
+    RawRow<DT> raw = map.ok(r) ? load_raw<DT>(w, map.idx(r)) : zero_raw<DT>();
+    for (; r < map.rows; r += gridDim.x) {
+        const int rn = r + gridDim.x;
+        const RawRow<DT> next = map.ok(rn) ? load_raw<DT>(w, map.idx(rn)) : zero_raw<DT>();
         float v[kLaneW];
         widen(raw, v);
-        quantize_row<DT, I, SIGNED, ST>(v, idx, idx < n, T, lane_off, lane, codes, scales);
+        quantize_row<DT, I, SIGNED, ST>(v, map.idx(r), map.ok(r), T, lut_base, lane, codes, scales);
         raw = next;
-        idx = idx_next;
     }
 }
 
@@ -341,17 +339,18 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
     __shared__ int s_multi;
     QuantTables T{s_xi, s_lut, false};
     if (QUANT) T = setup_tables(levels, s_xi, s_lv, s_lut, &s_multi);
-    const int64_t rows = (n + kQRow - 1) / kQRow;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t lane_off = lane * 8;
-    int64_t r = blockIdx.x;
-    if (r >= rows) return;
-    int64_t idx = (r * kQThreads + threadIdx.x) * kLaneW;
-    RawRow<DT> raw = (idx < n) ? load_raw<DT>(w, idx) : zero_raw<DT>();
-    for (; r < rows; r += gridDim.x) {
-        const int64_t idx_next = ((r + gridDim.x) * kQThreads + threadIdx.x) * kLaneW;
-        const RawRow<DT> next = (idx_next < n) ? load_raw<DT>(w, idx_next) : zero_raw<DT>();
-        const int64_t tile = r * (kQThreads / 32) + warp;
+    const uint32_t lut_base = lut_lane_base(s_lut, lane);  // table base of this lane
+    const RowMap map(n, kQRow, threadIdx.x);
+    int r = blockIdx.x;
+    if (r >= map.rows) return;
+    RawRow<DT> raw = map.ok(r) ? load_raw<DT>(w, map.idx(r)) : zero_raw<DT>();
+    for (; r < map.rows; r += gridDim.x) {
+        const int rn = r + gridDim.x;
+        const RawRow<DT> next = map.ok(rn) ? load_raw<DT>(w, map.idx(rn)) : zero_raw<DT>();
+        const int64_t idx = map.idx(r);
+        const bool ok = map.ok(r);
+        const int64_t tile = (int64_t)r * (kQThreads / 32) + warp;
         const bool tile_ok = tile * kOpqTile < n;  // warp-uniform
         float v[kLaneW];
         widen(raw, v);
@@ -375,12 +374,11 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
             counts[tile] = 0;
         }
         if (QUANT) {
-            quantize_row<DT, I, SIGNED, ST>(v, idx, idx < n, T, lane_off, lane, codes, scales);
-        } else if (w_clean != nullptr && idx < n) {
+            quantize_row<DT, I, SIGNED, ST>(v, idx, ok, T, lut_base, lane, codes, scales);
+        } else if (w_clean != nullptr && ok) {
             store_row(DT{}, w_clean, idx, v);
         }
         raw = next;
-        idx = idx_next;
     }
 }
 
