@@ -43,8 +43,8 @@ BYTES_EM = 2.0
 BYTES_QUANT = 2.0 + 0.5 + 2.0 / I
 BYTES_DEQUANT = 0.5 + 2.0 / I + 2.0
 # data passes of one MAE iteration that stream all weights on this workload: the max-|w| pass
-# and three selection passes (the fourth is only needed for a region that straddles zero)
-MAE_DATA_PASSES = 4
+# and two selection passes (the rest of the selection runs on the candidate lists)
+MAE_DATA_PASSES = 3
 FALLBACK_HBM_GBS = 6650.0
 
 

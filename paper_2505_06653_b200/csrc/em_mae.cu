@@ -6,7 +6,11 @@
 // rel = key - key(xi[l-1]) differ; each data pass histograms the next (up to) 9 of those bits for
 // the samples that match the digits chosen so far, and a single-CTA kernel picks the bin in
 // which the cumulative weight first reaches half of the region's total.  After ceil(B_l / 9)
-// passes (3 for ordinary regions, 4 at most) the key, hence the sample, is known exactly.
+// digits the key, hence the sample, is known exactly.  The second data pass also copies the
+// samples that match the first digit (about 1/512 of the region) into a candidate list; when
+// that list fits (64 Ki samples per level) the remaining digits are resolved from the list by
+// one CTA and no further data pass is needed.  Otherwise (very large or degenerate inputs) the
+// third and fourth data passes finish the selection; they return at once when nothing is left.
 //
 // Weights enter the histograms as 31-bit fixed-point integers relative to the largest |w| of
 // the data (exact whenever |m| is within 2^-7 of it for fp32 input, 2^-23 for bf16 input), so
@@ -20,7 +24,9 @@ namespace bof4 {
 
 constexpr int kMaeThreads = 1024;
 constexpr int kMaeRow = kMaeThreads * kLaneW;
-constexpr size_t kMaeSmem = (size_t)kLutBytes + 3u * kLevels * kMaeBins * 4u;  // lo, hi, count
+constexpr int kMaeStage = 256;  // candidates staged per CTA and level in the collecting pass
+constexpr size_t kMaeSmem = (size_t)kLutBytes + 3u * kLevels * kMaeBins * 4u  // table; lo, hi, count
+                            + (size_t)kLevels * kMaeStage * 8u;                // staged candidates
 
 struct MaeState {
     unsigned long long before[kLevels];  // weight below the current candidate range
@@ -29,6 +35,7 @@ struct MaeState {
     uint32_t base[kLevels];              // key of the region's lower edge
     uint32_t prefix[kLevels];            // digits chosen so far
     int top[kLevels];                    // key bits still unresolved (0: done)
+    uint32_t cand_count[kLevels];        // samples offered to the candidate list of level l
     uint32_t active;                     // bit l: level l takes part in the selection
     uint32_t max_bits;                   // bits of the largest |w| of the data
 };
@@ -39,6 +46,7 @@ struct MaeWs {
     MaeState* state;
     unsigned long long* hist;   // [16][kMaeBins] weight
     unsigned long long* chist;  // [16][kMaeBins] count
+    uint2* cand;                // [16][kMaeCand] {rel key, fixed-point weight}
 };
 
 __host__ __device__ inline MaeWs mae_ws(void* d_ws)
@@ -46,7 +54,8 @@ __host__ __device__ inline MaeWs mae_ws(void* d_ws)
     char* p = static_cast<char*>(d_ws) + kEmMaeOffset;
     return MaeWs{static_cast<double*>(d_ws), reinterpret_cast<MaeState*>(p),
                  reinterpret_cast<unsigned long long*>(p + kEmMaeStateBytes),
-                 reinterpret_cast<unsigned long long*>(p + kEmMaeStateBytes + kEmMaeHistBytes)};
+                 reinterpret_cast<unsigned long long*>(p + kEmMaeStateBytes + kEmMaeHistBytes),
+                 reinterpret_cast<uint2*>(p + kEmMaeStateBytes + 2 * kEmMaeHistBytes)};
 }
 
 // Order-preserving key: x <= y  <=>  key(x) <= key(y); -0 and +0 share a key.
@@ -128,6 +137,7 @@ mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
         W.state->before[l] = 0ull;
         W.state->total[l] = 0ull;
         W.state->count[l] = 0ull;
+        W.state->cand_count[l] = 0u;
     }
     if (threadIdx.x == 0) W.state->active = ~skip_mask & 0xffffu;
     for (int k = threadIdx.x; k < kLevels * kMaeBins; k += blockDim.x) {
@@ -140,7 +150,8 @@ mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
 
 // FIRST: also accumulates sum |w - m xhat[c]| (one partial record per CTA) and, with COUNT,
 // the member counts.  Later passes return at once when no level has bits left.
-template <class DT, int I, bool SIGNED, bool FIRST, bool COUNT>
+// COLLECT (second pass): every participating sample is also appended to its level's list.
+template <class DT, int I, bool SIGNED, bool FIRST, bool COUNT, bool COLLECT>
 __global__ void __launch_bounds__(kMaeThreads, 1)
 mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
 {
@@ -150,6 +161,8 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     uint32_t* s_lo = reinterpret_cast<uint32_t*>(s_raw + kLutBytes);
     uint32_t* s_hi = s_lo + kLevels * kMaeBins;
     uint32_t* s_cn = s_hi + kLevels * kMaeBins;
+    uint2* s_cand = reinterpret_cast<uint2*>(s_cn + kLevels * kMaeBins);  // [16][kMaeStage] (COLLECT)
+    __shared__ uint32_t s_ncand[kLevels], s_gbase[kLevels];
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
     __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
@@ -177,6 +190,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         s_row_end[tid] = T.row_end[tid];
     }
     for (int k = tid; k < 3 * kLevels * kMaeBins; k += kMaeThreads) s_lo[k] = 0u;
+    if (tid < kLevels) s_ncand[tid] = 0u;
     const uint32_t max_bits = W.state->max_bits;
     __syncthreads();
     build_lut(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base; });
@@ -221,6 +235,20 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
                 const uint32_t old = atomicAdd(&s_lo[bin], a);
                 if (old + a < old) atomicAdd(&s_hi[bin], 1u);
                 if (FIRST && COUNT) atomicAdd(&s_cn[bin], 1u);
+                if (COLLECT) {
+                    // staged per CTA and level; the rare overflow of a slot goes straight to the
+                    // global list (whose count only needs to stay above the capacity once full)
+                    const uint32_t slot = atomicAdd(&s_ncand[c], 1u);
+                    if (slot < (uint32_t)kMaeStage) {
+                        s_cand[c * kMaeStage + slot] = make_uint2(rel, a);
+                    } else {
+                        uint32_t* cnt = &W.state->cand_count[c];
+                        if (*reinterpret_cast<volatile uint32_t*>(cnt) <= (uint32_t)kMaeCand) {
+                            const uint32_t gslot = atomicAdd(cnt, 1u);
+                            if (gslot < (uint32_t)kMaeCand) W.cand[c * kMaeCand + gslot] = make_uint2(rel, a);
+                        }
+                    }
+                }
             }
         }
         if (FIRST) err += (double)e;
@@ -230,6 +258,20 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         const unsigned long long wsum = ((unsigned long long)s_hi[k] << 32) + s_lo[k];
         if (wsum) atomicAdd(&W.hist[k], wsum);
         if (FIRST && COUNT && s_cn[k]) atomicAdd(&W.chist[k], (unsigned long long)s_cn[k]);
+    }
+    if (COLLECT) {
+        // one reservation per CTA and level, then a plain copy of the staged samples
+        if (tid < kLevels) {
+            const uint32_t k = min(s_ncand[tid], (uint32_t)kMaeStage);
+            s_gbase[tid] = k ? atomicAdd(&W.state->cand_count[tid], k) : 0u;
+        }
+        __syncthreads();
+        for (int k = tid; k < kLevels * kMaeStage; k += kMaeThreads) {
+            const int l = k / kMaeStage, i = k % kMaeStage;
+            const uint32_t dst = s_gbase[l] + (uint32_t)i;
+            if ((uint32_t)i < min(s_ncand[l], (uint32_t)kMaeStage) && dst < (uint32_t)kMaeCand)
+                W.cand[l * kMaeCand + dst] = s_cand[k];
+        }
     }
     if (FIRST) {
 #pragma unroll
@@ -247,13 +289,53 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
 
 // ---------------------------------------------------------------- bin selection
 
-// One CTA per level, one thread per bin.  For a level with bits left: the first bin in which
-// the cumulative weight reaches half of the total (2 (before + cum) >= total) becomes the next
-// digit.  After the first pass the totals (and counts) are those of the whole region.
+// Block-wide step of the selection, one thread per bin: given this thread's bin weight `mine`,
+// finds the first bin j with 2 (before + cumulative(j)) >= total.  Returns through the shared
+// result the bin and the cumulative weight below it.  *all_out = sum of all bins.
+struct PickResult {
+    int bin;
+    unsigned long long excl;
+};
+
+__device__ __forceinline__ PickResult pick_bin(unsigned long long mine, unsigned long long before,
+                                               unsigned long long total, bool total_is_sum,
+                                               unsigned long long* s_wsum, PickResult* s_res,
+                                               unsigned long long* all_out)
+{
+    const int j = threadIdx.x, lane = j & 31, warp = j >> 5;
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long t = __shfl_up_sync(kFull, incl, off);
+        if (lane >= off) incl += t;
+    }
+    __syncthreads();  // s_wsum / s_res may still be read from a previous call
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    unsigned long long carry = 0ull, all = 0ull;
+    for (int k = 0; k < kMaeBins / 32; ++k) {
+        if (k < warp) carry += s_wsum[k];
+        all += s_wsum[k];
+    }
+    incl += carry;
+    if (total_is_sum) total = all;
+    const unsigned long long excl = incl - mine;
+    const bool reached = 2ull * (before + incl) >= total;
+    const bool prev_reached = (j > 0) && (2ull * (before + excl) >= total);
+    if (reached && !prev_reached) *s_res = PickResult{j, excl};  // exactly one thread: monotone
+    __syncthreads();
+    *all_out = all;
+    return *s_res;
+}
+
+// One CTA per level, one thread per bin.  For a level with bits left: the bin in which the
+// cumulative weight first reaches half of the total becomes the next digit.  After the first
+// pass the totals (and counts) are those of the whole region.
 __global__ void __launch_bounds__(kMaeBins)
 mae_select_kernel(MaeWs W, int first)
 {
     __shared__ unsigned long long s_wsum[kMaeBins / 32], s_csum[kMaeBins / 32];
+    __shared__ PickResult s_res;
     MaeState* S = W.state;
     const int l = blockIdx.x, j = threadIdx.x, lane = j & 31, warp = j >> 5;
     const int top = S->top[l];
@@ -264,41 +346,91 @@ mae_select_kernel(MaeWs W, int first)
     if (first) {
         c = W.chist[l * kMaeBins + j];
         W.chist[l * kMaeBins + j] = 0ull;
-    }
-    // inclusive scan of the bin weights: inside the warp, then over the warp totals
-    unsigned long long incl = mine;
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const unsigned long long t = __shfl_up_sync(kFull, incl, off);
-        if (lane >= off) incl += t;
+        for (int off = 16; off; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
+        if (lane == 0) s_csum[warp] = c;
     }
-#pragma unroll
-    for (int off = 16; off; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
-    if (lane == 31) s_wsum[warp] = incl;
-    if (lane == 0) s_csum[warp] = c;
-    __syncthreads();
-    unsigned long long carry = 0ull, all = 0ull, count = 0ull;
-    for (int k = 0; k < kMaeBins / 32; ++k) {
-        if (k < warp) carry += s_wsum[k];
-        all += s_wsum[k];
-        count += s_csum[k];
-    }
-    incl += carry;
-    const unsigned long long total = first ? all : S->total[l];
     const unsigned long long before = S->before[l];
-    const unsigned long long excl = incl - mine;
-    const bool reached = 2ull * (before + incl) >= total;
-    const bool prev_reached = (j > 0) && (2ull * (before + excl) >= total);
-    __syncthreads();  // every thread has read the state it needs
-    if (reached && !prev_reached) {  // exactly one thread: the cumulative weight is monotone
+    unsigned long long all;
+    const PickResult r = pick_bin(mine, before, first ? 0ull : S->total[l], first != 0, s_wsum, &s_res, &all);
+    if (j == 0) {
         const int sh = max(top - kMaeDigitBits, 0);
-        S->before[l] = before + excl;
-        S->prefix[l] = (S->prefix[l] << (top - sh)) | (uint32_t)j;
+        S->before[l] = before + r.excl;
+        S->prefix[l] = (S->prefix[l] << (top - sh)) | (uint32_t)r.bin;
         S->top[l] = sh;
         if (first) {
-            S->total[l] = total;
+            unsigned long long count = 0ull;
+            for (int k = 0; k < kMaeBins / 32; ++k) count += s_csum[k];
+            S->total[l] = all;
             S->count[l] = count;
         }
+    }
+}
+
+// After the collecting (second) pass.  A level whose candidate list holds every sample that
+// matched the first digit is finished here: the remaining digits are selected from the list.
+// A level whose list overflowed takes the ordinary histogram step and goes on to the later
+// passes.
+__global__ void __launch_bounds__(kMaeBins)
+mae_resolve_kernel(MaeWs W)
+{
+    __shared__ unsigned long long s_wsum[kMaeBins / 32];
+    __shared__ uint32_t s_lo[kMaeBins], s_hi[kMaeBins];  // 64-bit bins as two words: native 32-bit atomics
+    __shared__ PickResult s_res;
+    MaeState* S = W.state;
+    const int l = blockIdx.x, j = threadIdx.x;
+    int top = S->top[l];
+    if (top <= 0) return;  // uniform over the CTA
+    const uint32_t m = S->cand_count[l];
+    unsigned long long before = S->before[l];
+    const unsigned long long total = S->total[l];
+    uint32_t prefix = S->prefix[l];
+    unsigned long long all;
+    // the digit of this pass, from the global histogram (also clears it)
+    {
+        const unsigned long long mine = W.hist[l * kMaeBins + j];
+        W.hist[l * kMaeBins + j] = 0ull;
+        const PickResult r = pick_bin(mine, before, total, false, s_wsum, &s_res, &all);
+        const int sh = max(top - kMaeDigitBits, 0);
+        before += r.excl;
+        prefix = (prefix << (top - sh)) | (uint32_t)r.bin;
+        top = sh;
+    }
+    if (m <= (uint32_t)kMaeCand) {
+        const uint2* cand = W.cand + (size_t)l * kMaeCand;
+        while (top > 0) {
+            const int sh = max(top - kMaeDigitBits, 0);
+            const uint32_t mask = (1u << (top - sh)) - 1u;
+            s_lo[j] = 0u;
+            s_hi[j] = 0u;
+            __syncthreads();
+            for (uint32_t i0 = 0; i0 < m; i0 += 8 * kMaeBins) {  // 8 independent loads in flight per thread
+                uint2 c[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t i = i0 + u * kMaeBins + j;
+                    c[u] = (i < m) ? cand[i] : make_uint2(0xffffffffu, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (c[u].y != 0u && (c[u].x >> top) == prefix) {
+                        const uint32_t bin = (c[u].x >> sh) & mask;
+                        const uint32_t old = atomicAdd(&s_lo[bin], c[u].y);
+                        if (old + c[u].y < old) atomicAdd(&s_hi[bin], 1u);
+                    }
+            }
+            __syncthreads();
+            const PickResult r = pick_bin(((unsigned long long)s_hi[j] << 32) + s_lo[j], before, total, false,
+                                          s_wsum, &s_res, &all);
+            before += r.excl;
+            prefix = (prefix << (top - sh)) | (uint32_t)r.bin;
+            top = sh;
+        }
+    }
+    if (j == 0) {
+        S->before[l] = before;
+        S->prefix[l] = prefix;
+        S->top[l] = top;
     }
 }
 
@@ -347,30 +479,31 @@ mae_finalize_kernel(MaeWs W, int n_records, int64_t n_total, const float* levels
 namespace {
 
 template <class DT, int I, bool SG>
-int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, bool first, bool count,
+int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, int pass, bool count,
                 cudaStream_t st)
 {
-#define BOF4_MAE_GO(FIRST_, COUNT_)                                                                     \
+#define BOF4_MAE_GO(FIRST_, COUNT_, COLLECT_)                                                           \
     {                                                                                                   \
-        auto kern = mae_pass_kernel<DT, I, SG, FIRST_, COUNT_>;                                         \
+        auto kern = mae_pass_kernel<DT, I, SG, FIRST_, COUNT_, COLLECT_>;                               \
         BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaeSmem)); \
         kern<<<kEmGrid, kMaeThreads, kMaeSmem, st>>>(T, d_levels, W);                                   \
     }
-    if (first && count) BOF4_MAE_GO(true, true)
-    else if (first) BOF4_MAE_GO(true, false)
-    else BOF4_MAE_GO(false, false)
+    if (pass == 0 && count) BOF4_MAE_GO(true, true, false)
+    else if (pass == 0) BOF4_MAE_GO(true, false, false)
+    else if (pass == 1) BOF4_MAE_GO(false, false, true)
+    else BOF4_MAE_GO(false, false, false)
 #undef BOF4_MAE_GO
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }
 
-int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, const MaeWs& W, bool first,
+int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, const MaeWs& W, int pass,
                   bool count, cudaStream_t st)
 {
     const bool sg = a.norm == BOF4_NORM_SIGNED;
 #define BOF4_MAE_I(DT_, I_)                                                       \
-    return sg ? launch_pass<DT_, I_, true>(T, d_levels, W, first, count, st)      \
-              : launch_pass<DT_, I_, false>(T, d_levels, W, first, count, st);
+    return sg ? launch_pass<DT_, I_, true>(T, d_levels, W, pass, count, st)       \
+              : launch_pass<DT_, I_, false>(T, d_levels, W, pass, count, st);
 #define BOF4_MAE_DT(DT_)                         \
     switch (a.block_size) {                      \
         case 32: BOF4_MAE_I(DT_, 32)             \
@@ -410,13 +543,16 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
     for (int p = 0; p < kMaeMaxPasses; ++p) {
         const bool first = p == 0;
         auto fire = [&](const EmTensors& T) -> int {
-            return dispatch_pass(a, T, d_levels_in, W, first, first && d_stats != nullptr, st);
+            return dispatch_pass(a, T, d_levels_in, W, p, first && d_stats != nullptr, st);
         };
         int calls = 0;
         const int rc = for_each_tensor_chunk(a, kMaeRow, fire, &calls);
         if (rc) return rc;
         if (first && calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(W.partials, 0, kEmPartialBytes, st));
-        mae_select_kernel<<<kLevels, kMaeBins, 0, st>>>(W, first ? 1 : 0);
+        if (p == 1)
+            mae_resolve_kernel<<<kLevels, kMaeBins, 0, st>>>(W);
+        else
+            mae_select_kernel<<<kLevels, kMaeBins, 0, st>>>(W, first ? 1 : 0);
         BOF4_CUDA_TRY(cudaGetLastError());
     }
     mae_finalize_kernel<<<1, 256, 0, st>>>(W, kEmGrid, a.n_total, d_levels_in, d_levels_out, skip_mask,

@@ -20,7 +20,9 @@ constexpr int kMaeMaxPasses = 4;          // 31 key bits / 9 bits per pass
 constexpr size_t kEmMaeOffset = 512 * 1024;
 constexpr size_t kEmMaeStateBytes = 4096;  // selection state (struct MaeState)
 constexpr size_t kEmMaeHistBytes = (size_t)16 * kMaeBins * 8;  // weight histogram, then count histogram
-constexpr size_t kEmMaeBytes = kEmMaeStateBytes + 2 * kEmMaeHistBytes;
+constexpr int kMaeCand = 1 << 16;          // candidate samples kept per level by the second pass
+constexpr size_t kEmMaeCandBytes = (size_t)16 * kMaeCand * 8;
+constexpr size_t kEmMaeBytes = kEmMaeStateBytes + 2 * kEmMaeHistBytes + kEmMaeCandBytes;
 
 inline size_t em_workspace_bytes() { return kEmMaeOffset + align_up(kEmMaeBytes, 256); }
 
