@@ -122,6 +122,8 @@ BOF4_API int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_tens
  *   d_err_log   [iters] fp64 or NULL: entry t = mean error (MSE or MAE over all weights,
  *               un-normalised domain) of the levels that ENTER iteration t
  * No host synchronisation happens inside; the whole loop is enqueued on `stream`.
+ * (MAE only: the environment variable BOF4_MAE_COLLECT_PASS = 1 or 2 overrides which data pass
+ * fills the candidate lists of the median selection; results do not depend on it.)
  */
 BOF4_API int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int n_tensors, int w_dtype,
                       int block_size, int norm, int metric, float* d_codebook,

@@ -16,6 +16,8 @@
 // the data (exact whenever |m| is within 2^-7 of it for fp32 input, 2^-23 for bf16 input), so
 // every sum is an integer sum: independent of the order of the atomics, bit-reproducible, and
 // equal to the exact real-number sums that define the median.
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "em_common.cuh"
 #include "layout.h"
@@ -479,8 +481,8 @@ mae_finalize_kernel(MaeWs W, int n_records, int64_t n_total, const float* levels
 namespace {
 
 template <class DT, int I, bool SG>
-int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, int pass, bool count,
-                cudaStream_t st)
+int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, int pass, bool collect,
+                bool count, cudaStream_t st)
 {
 #define BOF4_MAE_GO(FIRST_, COUNT_, COLLECT_)                                                           \
     {                                                                                                   \
@@ -490,7 +492,7 @@ int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, int p
     }
     if (pass == 0 && count) BOF4_MAE_GO(true, true, false)
     else if (pass == 0) BOF4_MAE_GO(true, false, false)
-    else if (pass == 1) BOF4_MAE_GO(false, false, true)
+    else if (collect) BOF4_MAE_GO(false, false, true)
     else BOF4_MAE_GO(false, false, false)
 #undef BOF4_MAE_GO
     BOF4_CUDA_TRY(cudaGetLastError());
@@ -498,12 +500,12 @@ int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, int p
 }
 
 int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, const MaeWs& W, int pass,
-                  bool count, cudaStream_t st)
+                  bool collect, bool count, cudaStream_t st)
 {
     const bool sg = a.norm == BOF4_NORM_SIGNED;
 #define BOF4_MAE_I(DT_, I_)                                                       \
-    return sg ? launch_pass<DT_, I_, true>(T, d_levels, W, pass, count, st)       \
-              : launch_pass<DT_, I_, false>(T, d_levels, W, pass, count, st);
+    return sg ? launch_pass<DT_, I_, true>(T, d_levels, W, pass, collect, count, st)   \
+              : launch_pass<DT_, I_, false>(T, d_levels, W, pass, collect, count, st);
 #define BOF4_MAE_DT(DT_)                         \
     switch (a.block_size) {                      \
         case 32: BOF4_MAE_I(DT_, 32)             \
@@ -540,16 +542,24 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
     const MaeWs W = mae_ws(d_ws);
     mae_init_kernel<<<1, kMaeBins, 0, st>>>(d_levels_in, skip_mask, W);
     BOF4_CUDA_TRY(cudaGetLastError());
+    // The candidate lists are filled by the first pass after which a region's candidates
+    // (about 1/512 of them survive each digit) are expected to fit: the second pass up to
+    // 2^29 weights, the third beyond.
+    // BOF4_MAE_COLLECT_PASS=1|2 in the environment overrides the choice (tests, tuning).
+    int collect_pass = (a.n_total / kLevels / kMaeBins <= kMaeCand / 8) ? 1 : 2;
+    if (const char* env = getenv("BOF4_MAE_COLLECT_PASS")) {
+        if (env[0] == '1' || env[0] == '2') collect_pass = env[0] - '0';
+    }
     for (int p = 0; p < kMaeMaxPasses; ++p) {
         const bool first = p == 0;
         auto fire = [&](const EmTensors& T) -> int {
-            return dispatch_pass(a, T, d_levels_in, W, p, first && d_stats != nullptr, st);
+            return dispatch_pass(a, T, d_levels_in, W, p, p == collect_pass, first && d_stats != nullptr, st);
         };
         int calls = 0;
         const int rc = for_each_tensor_chunk(a, kMaeRow, fire, &calls);
         if (rc) return rc;
         if (first && calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(W.partials, 0, kEmPartialBytes, st));
-        if (p == 1)
+        if (p == collect_pass)
             mae_resolve_kernel<<<kLevels, kMaeBins, 0, st>>>(W);
         else
             mae_select_kernel<<<kLevels, kMaeBins, 0, st>>>(W, first ? 1 : 0);

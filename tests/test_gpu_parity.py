@@ -383,3 +383,23 @@ def test_non_finite_weights_do_not_disturb_other_blocks(bof4):
     assert np.array_equal(codes.cpu().numpy().reshape(-1, I // 2)[keep], rc.reshape(-1, I // 2)[keep])
     assert np.array_equal(scales_f32(scales)[keep], rs[keep])
     assert st["n"] == n
+
+
+def test_mae_collecting_pass_choice_does_not_change_results(bof4):
+    """The pass that fills the candidate lists is chosen from the data size; forcing the other
+    choice (as for very large inputs) must give the same medians, bit for bit."""
+    import os
+    I, n = 64, 1 << 18
+    w = make_weights(n, torch.bfloat16, 301)
+    ref = oracle.em_accumulate_mae(w, I, 1, LV_INIT)
+    old = os.environ.get("BOF4_MAE_COLLECT_PASS")
+    try:
+        for choice in ("1", "2"):
+            os.environ["BOF4_MAE_COLLECT_PASS"] = choice
+            got = bof4.bof4_em_step([w.cuda()], I, 1, bof4.METRIC_MAE, LV_INIT)
+            _check_mae_stats(got, ref, LV_INIT)
+    finally:
+        if old is None:
+            os.environ.pop("BOF4_MAE_COLLECT_PASS", None)
+        else:
+            os.environ["BOF4_MAE_COLLECT_PASS"] = old
