@@ -303,11 +303,14 @@ __device__ __forceinline__ uint2 lut_probe(float key, uint32_t lut_base)
 
 // Builds the table in shared memory from the thresholds; payload(base) is stored next to
 // thr (a code, or a byte offset).  *s_multi tells whether some bin holds two thresholds.
-// Call with all threads of the CTA, then __syncthreads().
+// Call with all threads of the CTA, then __syncthreads().  The entries are first computed once
+// per bin into the table's own first row slots and then replicated with one warp per row, so
+// that the replicating stores of a warp fall into 32 different lanes' columns (no conflicts).
 template <class PayloadFn>
 __device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lut, int* s_multi,
                                           PayloadFn payload)
 {
+    __shared__ uint2 s_ent[kLutBins];
     if (threadIdx.x == 0) *s_multi = 0;
     __syncthreads();
     for (int b = threadIdx.x; b < kLutBins; b += blockDim.x) {
@@ -320,10 +323,11 @@ __device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lu
             inside += (bj == b) ? 1 : 0;
         }
         if (inside > 1) *s_multi = 1;
-        const uint2 ent = make_uint2(__float_as_uint(s_xi[base]), payload(base));
-        for (int l = 0; l < 32; ++l)
-            *reinterpret_cast<uint2*>(s_lut + b * kLutRowBytes + l * 8) = ent;
+        s_ent[b] = make_uint2(__float_as_uint(s_xi[base]), payload(base));
     }
+    __syncthreads();
+    for (int k = threadIdx.x; k < kLutBins * 32; k += blockDim.x)
+        *reinterpret_cast<uint2*>(s_lut + k * 8) = s_ent[k >> 5];
 }
 
 // ---------------------------------------------------------------- division for bf16 inputs

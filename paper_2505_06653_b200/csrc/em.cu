@@ -29,9 +29,101 @@ struct EmGeo {
 // Record layout in doubles: [0,16) s1, [16,32) s0, [32,48) count (uint64 bits), [48] sum w^2.
 constexpr int kRecS1 = 0, kRecS0 = 16, kRecCnt = 32, kRecW2 = 48;
 
+// What the last accumulation CTA (or the stand-alone combine kernel) does with the records.
+//   stats    != NULL: receives the combined record
+//   codebook != NULL: every free level with s0 > 0 becomes (float)(s1 / s0)      (Eq. 6)
+//   err_slot != NULL: receives err_sum / n_total
+// err_sum = w2 - sum_l xhat[l] (2 s1[l] - xhat[l] s0[l]) with the levels that produced the sums.
+struct MseTail {
+    int enabled;            // the last CTA to arrive combines the records (fused M step)
+    int n_records;
+    int64_t n_total;
+    const float* levels_in;
+    bof4_em_stats* stats;
+    float* codebook;
+    uint32_t fixed_mask;
+    double* err_slot;
+    unsigned int* ticket;   // arrival counter, zero before the pass and reset by the last CTA
+};
+
+// Combines the per-CTA records in a fixed order (the order does not depend on which CTA runs
+// this) and performs the M step.  Called by all threads of one CTA.
+__device__ __forceinline__ void mse_combine(const double* partials, const MseTail& t, double* s_q,
+                                            double* s_corr)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    constexpr int PER = (kEmGrid + 31) / 32;  // records per lane; all loads are issued before any sum
+    for (int q = warp; q <= kRecW2; q += nwarps) {
+        const bool is_count = q >= kRecCnt && q < kRecW2;
+        unsigned long long raw[PER];
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+            const int r = lane + 32 * k;
+            raw[k] = (r < t.n_records)
+                         ? __ldcg(reinterpret_cast<const unsigned long long*>(partials + (size_t)r * kEmRecordDoubles) + q)
+                         : 0ull;  // zero bits are also +0.0
+        }
+        double a = 0.0;
+        unsigned long long c = 0;
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+            if (is_count)
+                c += raw[k];
+            else
+                a += __longlong_as_double((long long)raw[k]);
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) {
+            a += __shfl_xor_sync(kFull, a, off);
+            c += __shfl_xor_sync(kFull, c, off);
+        }
+        if (lane == 0) {
+            if (is_count)
+                reinterpret_cast<unsigned long long*>(s_q)[q] = c;
+            else
+                s_q[q] = a;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < kLevels) {
+        const int l = threadIdx.x;
+        const double s1 = s_q[kRecS1 + l], s0 = s_q[kRecS0 + l];
+        const float old = t.levels_in[l];
+        const float cen = (s0 > 0.0) ? (float)(s1 / s0) : old;
+        s_corr[l] = (double)old * (2.0 * s1 - (double)old * s0);
+        if (t.stats) {
+            t.stats->s1[l] = s1;
+            t.stats->s0[l] = s0;
+            t.stats->count[l] = reinterpret_cast<unsigned long long*>(s_q)[kRecCnt + l];
+            t.stats->median[l] = cen;
+        }
+        if (t.codebook && !((t.fixed_mask >> l) & 1u)) t.codebook[l] = cen;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double corr = 0.0;
+        for (int l = 0; l < kLevels; ++l) corr += s_corr[l];
+        double err = s_q[kRecW2] - corr;
+        if (err < 0.0) err = 0.0;
+        if (t.stats) {
+            t.stats->err_sum = err;
+            t.stats->n_total = t.n_total;
+        }
+        if (t.err_slot) *t.err_slot = (t.n_total > 0) ? err / (double)t.n_total : 0.0;
+    }
+}
+
+// Stand-alone combine (used when a pass launched no accumulation kernel at all).
+__global__ void __launch_bounds__(1024)
+em_mse_finalize_kernel(const double* partials, const MseTail t)
+{
+    __shared__ double s_q[kRecW2 + 1], s_corr[kLevels];
+    mse_combine(partials, t, s_q, s_corr);
+}
+
 template <class DT, int I, bool SIGNED, bool COUNT>
 __global__ void __launch_bounds__(EmGeo<COUNT>::threads, 1)
-em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __restrict__ partials)
+em_mse_kernel(const EmTensors T, const float* levels, double* partials, const MseTail tail)
 {
     using G = EmGeo<COUNT>;
     constexpr int LPB = I / kLaneW;
@@ -216,70 +308,20 @@ em_mse_kernel(const EmTensors T, const float* __restrict__ levels, double* __res
         for (int k = 0; k < NW; ++k) e += s_w2[k];
         rec[kRecW2] = T.accumulate ? rec[kRecW2] + e : e;
     }
-}
-
-// Combines the per-CTA records in a fixed order and, if asked, performs the M step.
-//   stats    != NULL: receives the combined record
-//   codebook != NULL: every free level with s0 > 0 becomes (float)(s1 / s0)      (Eq. 6)
-//   err_slot != NULL: receives err_sum / n_total
-// err_sum = w2 - sum_l xhat[l] (2 s1[l] - xhat[l] s0[l]) with the levels that produced the sums.
-__global__ void __launch_bounds__(1024)
-em_mse_finalize_kernel(const double* __restrict__ partials, int n_records, int64_t n_total,
-                       const float* levels_in, bof4_em_stats* __restrict__ stats,
-                       float* codebook, uint32_t fixed_mask, double* __restrict__ err_slot)
-{
-    __shared__ double s_q[kRecW2 + 1];
-    __shared__ double s_corr[kLevels];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int q = warp; q <= kRecW2; q += 32) {
-        const bool is_count = q >= kRecCnt && q < kRecW2;
-        double a = 0.0;
-        unsigned long long c = 0;
-        for (int r = lane; r < n_records; r += 32) {
-            const double* rec = partials + (size_t)r * kEmRecordDoubles;
-            if (is_count)
-                c += reinterpret_cast<const unsigned long long*>(rec)[q];
-            else
-                a += rec[q];
+    // Fused M step: the CTA that arrives last (no CTA ever waits for another) combines all
+    // records; the fences order every CTA's record writes before its arrival.
+    if (tail.enabled) {
+        __shared__ int s_last;
+        __shared__ double s_q[kRecW2 + 1], s_corr[kLevels];
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = (atomicAdd(tail.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            mse_combine(partials, tail, s_q, s_corr);
+            if (tid == 0) *tail.ticket = 0u;
         }
-#pragma unroll
-        for (int off = 16; off; off >>= 1) {
-            a += __shfl_xor_sync(kFull, a, off);
-            c += __shfl_xor_sync(kFull, c, off);
-        }
-        if (lane == 0) {
-            if (is_count)
-                reinterpret_cast<unsigned long long*>(s_q)[q] = c;
-            else
-                s_q[q] = a;
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x < kLevels) {
-        const int l = threadIdx.x;
-        const double s1 = s_q[kRecS1 + l], s0 = s_q[kRecS0 + l];
-        const float old = levels_in[l];
-        const float cen = (s0 > 0.0) ? (float)(s1 / s0) : old;
-        s_corr[l] = (double)old * (2.0 * s1 - (double)old * s0);
-        if (stats) {
-            stats->s1[l] = s1;
-            stats->s0[l] = s0;
-            stats->count[l] = reinterpret_cast<unsigned long long*>(s_q)[kRecCnt + l];
-            stats->median[l] = cen;
-        }
-        if (codebook && !((fixed_mask >> l) & 1u)) codebook[l] = cen;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        double corr = 0.0;
-        for (int l = 0; l < kLevels; ++l) corr += s_corr[l];
-        double err = s_q[kRecW2] - corr;
-        if (err < 0.0) err = 0.0;
-        if (stats) {
-            stats->err_sum = err;
-            stats->n_total = n_total;
-        }
-        if (err_slot) *err_slot = (n_total > 0) ? err / (double)n_total : 0.0;
     }
 }
 
@@ -345,33 +387,41 @@ namespace {
 using namespace bof4;
 
 template <class DT, int I, bool SG, bool COUNT>
-int launch_mse_chunk(const EmTensors& T, const float* d_codebook, double* partials, cudaStream_t st)
+int launch_mse_chunk(const EmTensors& T, const float* d_codebook, double* partials, MseTail tail,
+                     cudaStream_t st)
 {
+    tail.enabled = T.last;
     using G = EmGeo<COUNT>;
     auto kern = em_mse_kernel<DT, I, SG, COUNT>;
     BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::smem));
-    kern<<<kEmGrid, G::threads, G::smem, st>>>(T, d_codebook, partials);
+    kern<<<kEmGrid, G::threads, G::smem, st>>>(T, d_codebook, partials, tail);
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }
 
-// Enqueues the accumulation launches of one MSE pass over all tensors (non-empty ones, in
-// list order, kEmMaxTensors per launch).  With no weights at all the records are zeroed.
+// Enqueues one MSE pass over all tensors (non-empty ones, in list order, kEmMaxTensors per
+// launch); the last launch also combines the records and performs what `tail` asks for.  With
+// no weights at all the records are zeroed and a stand-alone combine runs.
 template <bool COUNT>
-int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials, cudaStream_t st)
+int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials, MseTail tail,
+                     cudaStream_t st)
 {
+    tail.n_records = kEmGrid;
+    tail.n_total = a.n_total;
+    tail.levels_in = d_codebook;
+    tail.ticket = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(partials) + kEmTicketOffset);
     const bool sg = a.norm == BOF4_NORM_SIGNED;
     auto fire = [&](const EmTensors& T) -> int {
 #define BOF4_EM_GO(DT_)                                                                                 \
     switch (a.block_size) {                                                                             \
-        case 32: return sg ? launch_mse_chunk<DT_, 32, true, COUNT>(T, d_codebook, partials, st)        \
-                           : launch_mse_chunk<DT_, 32, false, COUNT>(T, d_codebook, partials, st);      \
-        case 64: return sg ? launch_mse_chunk<DT_, 64, true, COUNT>(T, d_codebook, partials, st)        \
-                           : launch_mse_chunk<DT_, 64, false, COUNT>(T, d_codebook, partials, st);      \
-        case 128: return sg ? launch_mse_chunk<DT_, 128, true, COUNT>(T, d_codebook, partials, st)      \
-                            : launch_mse_chunk<DT_, 128, false, COUNT>(T, d_codebook, partials, st);    \
-        default: return sg ? launch_mse_chunk<DT_, 256, true, COUNT>(T, d_codebook, partials, st)       \
-                           : launch_mse_chunk<DT_, 256, false, COUNT>(T, d_codebook, partials, st);     \
+        case 32: return sg ? launch_mse_chunk<DT_, 32, true, COUNT>(T, d_codebook, partials, tail, st)        \
+                           : launch_mse_chunk<DT_, 32, false, COUNT>(T, d_codebook, partials, tail, st);      \
+        case 64: return sg ? launch_mse_chunk<DT_, 64, true, COUNT>(T, d_codebook, partials, tail, st)        \
+                           : launch_mse_chunk<DT_, 64, false, COUNT>(T, d_codebook, partials, tail, st);      \
+        case 128: return sg ? launch_mse_chunk<DT_, 128, true, COUNT>(T, d_codebook, partials, tail, st)      \
+                            : launch_mse_chunk<DT_, 128, false, COUNT>(T, d_codebook, partials, tail, st);    \
+        default: return sg ? launch_mse_chunk<DT_, 256, true, COUNT>(T, d_codebook, partials, tail, st)       \
+                           : launch_mse_chunk<DT_, 256, false, COUNT>(T, d_codebook, partials, tail, st);     \
     }
         if (a.w_dtype == BOF4_F32) { BOF4_EM_GO(F32) } else { BOF4_EM_GO(BF16) }
 #undef BOF4_EM_GO
@@ -379,7 +429,18 @@ int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials,
     int calls = 0;
     const int rc = for_each_tensor_chunk(a, EmGeo<COUNT>::row, fire, &calls);
     if (rc) return rc;
-    if (calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));
+    if (calls == 0) {
+        BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));
+        tail.enabled = 0;
+        em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, tail);
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
+    return BOF4_OK;
+}
+
+int reset_ticket(double* partials, cudaStream_t st)
+{
+    BOF4_CUDA_TRY(cudaMemsetAsync(reinterpret_cast<char*>(partials) + kEmTicketOffset, 0, 4, st));
     return BOF4_OK;
 }
 
@@ -399,12 +460,10 @@ extern "C" int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_te
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partials = static_cast<double*>(d_ws);
     if (metric == BOF4_METRIC_MSE) {
-        rc = enqueue_mse_pass<true>(a, d_codebook, partials, st);
-        if (rc) return rc;
-        em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, kEmGrid, a.n_total, d_codebook, d_stats,
-                                                   nullptr, 0u, nullptr);
-        BOF4_CUDA_TRY(cudaGetLastError());
-        return BOF4_OK;
+        if ((rc = reset_ticket(partials, st))) return rc;
+        MseTail tail{};
+        tail.stats = d_stats;
+        return enqueue_mse_pass<true>(a, d_codebook, partials, tail, st);
     }
     rc = mae_prepare(a, d_ws, st);
     if (rc) return rc;
@@ -426,13 +485,14 @@ extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partials = static_cast<double*>(d_ws);
     if (metric == BOF4_METRIC_MSE) {
+        if (iters > 0 && (rc = reset_ticket(partials, st))) return rc;
         for (int t = 0; t < iters; ++t) {
-            rc = enqueue_mse_pass<false>(a, d_codebook, partials, st);
+            MseTail tail{};
+            tail.codebook = d_codebook;
+            tail.fixed_mask = fixed_mask;
+            tail.err_slot = d_err_log ? d_err_log + t : nullptr;
+            rc = enqueue_mse_pass<false>(a, d_codebook, partials, tail, st);
             if (rc) return rc;
-            em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, kEmGrid, a.n_total, d_codebook, nullptr,
-                                                       d_codebook, fixed_mask,
-                                                       d_err_log ? d_err_log + t : nullptr);
-            BOF4_CUDA_TRY(cudaGetLastError());
         }
         return BOF4_OK;
     }

@@ -15,6 +15,7 @@ struct EmTensors {
     int64_t row_end[kEmMaxTensors];  // cumulative number of CTA rows up to and including tensor t
     int count;
     int accumulate;  // 0: this launch overwrites the partial records, 1: adds to them
+    int last;        // 1: no further launch of this pass follows
 };
 
 struct EmArgs {
@@ -37,7 +38,9 @@ int for_each_tensor_chunk(const EmArgs& a, int row, Fire fire, int* n_calls)
     T.count = 0;
     T.accumulate = 0;
     int64_t rows = 0;
-    int calls = 0;
+    int calls = 0, nonempty = 0;
+    for (int t = 0; t < a.n_tensors; ++t) nonempty += a.h_n[t] > 0;
+    const int total_calls = (nonempty + kEmMaxTensors - 1) / kEmMaxTensors;
     for (int t = 0; t <= a.n_tensors; ++t) {
         if (t < a.n_tensors) {
             if (a.h_n[t] == 0) continue;
@@ -48,6 +51,7 @@ int for_each_tensor_chunk(const EmArgs& a, int row, Fire fire, int* n_calls)
             ++T.count;
         }
         if (T.count == kEmMaxTensors || (t == a.n_tensors && T.count > 0)) {
+            T.last = (calls + 1 == total_calls) ? 1 : 0;
             const int rc = fire(T);
             if (rc) return rc;
             ++calls;
