@@ -188,10 +188,11 @@ __device__ __forceinline__ float max2_nan(float a, float b)
 // magnitude wins.  Only when both +g and -g occur does the position matter; that case is
 // settled by two ballots (which lane holds the first +g, which the first -g) and, where one
 // lane holds both, by that lane's elements in index order.
-template <int LPB, bool SIGNED>
-__device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float& g)
+// Largest (NaN-propagating) and smallest of the lane's 16 weights.
+__device__ __forceinline__ void lane_minmax(const float (&v)[kLaneW], float& mx, float& mn)
 {
-    float mx = max3_nan(v[0], v[1], v[2]), mn = min3(v[0], v[1], v[2]);
+    mx = max3_nan(v[0], v[1], v[2]);
+    mn = min3(v[0], v[1], v[2]);
 #pragma unroll
     for (int k = 3; k < 15; k += 2) {
         mx = max3_nan(mx, v[k], v[k + 1]);
@@ -199,6 +200,11 @@ __device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float&
     }
     mx = max2_nan(mx, v[15]);
     mn = fminf(mn, v[15]);
+}
+
+template <int LPB, bool SIGNED>
+__device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float mx, float mn, float& g)
+{
     float gx = mx, gn = mn;
 #pragma unroll
     for (int off = 1; off < LPB; off <<= 1) {
@@ -224,6 +230,14 @@ __device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float&
         if (tie) m = pick;
     }
     return (g == 0.0f) ? 0.0f : m;
+}
+
+template <int LPB, bool SIGNED>
+__device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float& g)
+{
+    float mx, mn;
+    lane_minmax(v, mx, mn);
+    return block_constant<LPB, SIGNED>(v, mx, mn, g);
 }
 
 // Eq. 2 with the 0/0 reading x = 0.  IEEE round-to-nearest division.

@@ -97,13 +97,13 @@ __device__ __forceinline__ void encode16(const float (&x)[kLaneW], const QuantTa
 
 // Block constant, normalisation, codes and stores for one lane-row of (cleaned) weights.
 template <class DT, int I, bool SIGNED, class ST>
-__device__ __forceinline__ void quantize_row(const float (&v)[kLaneW], int64_t idx, bool ok,
-                                             const QuantTables& T, uint32_t lut_base, int lane,
+__device__ __forceinline__ void quantize_row(const float (&v)[kLaneW], float mx, float mn, int64_t idx,
+                                             bool ok, const QuantTables& T, uint32_t lut_base, int lane,
                                              uint8_t* __restrict__ codes, void* __restrict__ scales)
 {
     constexpr int LPB = I / kLaneW;
     float g;
-    const float m = block_constant<LPB, SIGNED>(v, g);
+    const float m = block_constant<LPB, SIGNED>(v, mx, mn, g);
     const bool safe = row_is_safe(g, ok);
     float x[kLaneW];
     normalise16<true>(v, m, safe && DT::code == BF16::code, x);
@@ -133,9 +133,10 @@ quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__
     for (; r < map.rows; r += gridDim.x) {
         const int rn = r + gridDim.x;
         const RawRow<DT> next = map.ok(rn) ? load_raw<DT>(w, map.idx(rn)) : zero_raw<DT>();
-        float v[kLaneW];
+        float v[kLaneW], mx, mn;
         widen(raw, v);
-        quantize_row<DT, I, SIGNED, ST>(v, map.idx(r), map.ok(r), T, lut_base, lane, codes, scales);
+        lane_minmax(v, mx, mn);
+        quantize_row<DT, I, SIGNED, ST>(v, mx, mn, map.idx(r), map.ok(r), T, lut_base, lane, codes, scales);
         raw = next;
     }
 }
@@ -267,10 +268,10 @@ __device__ __forceinline__ float tree_sum(const float (&t)[kLaneW])
     return s;
 }
 
-// Bit k of the result is set iff element k of this lane is an outlier of its block:
-// |w| > sigma_b * tau, sigma_b the corrected sample standard deviation (two-pass, fp32).
+// The outlier threshold of the lane's block: sigma_b * tau, sigma_b the corrected sample
+// standard deviation (two-pass formula in fp32, tree-ordered sums).
 template <int I>
-__device__ __forceinline__ unsigned outlier_mask(const float (&v)[kLaneW], float tau)
+__device__ __forceinline__ float outlier_threshold(const float (&v)[kLaneW], float tau)
 {
     constexpr int LPB = I / kLaneW;
     const float mean = __fmul_rn(tree_sum<LPB>(v), 1.0f / (float)I);  // exact: I is a power of two
@@ -281,11 +282,22 @@ __device__ __forceinline__ unsigned outlier_mask(const float (&v)[kLaneW], float
         q[k] = __fmul_rn(d, d);
     }
     const float sigma = __fsqrt_rn(__fdiv_rn(tree_sum<LPB>(q), (float)(I - 1)));
-    const float thr = __fmul_rn(sigma, tau);
+    return __fmul_rn(sigma, tau);
+}
+
+// Bit k of the result is set iff element k of this lane is an outlier: |w| > thr.
+__device__ __forceinline__ unsigned outlier_bits(const float (&v)[kLaneW], float thr)
+{
     unsigned o = 0;
 #pragma unroll
     for (int k = 0; k < kLaneW; ++k) o |= (fabsf(v[k]) > thr) ? (1u << k) : 0u;
     return o;
+}
+
+template <int I>
+__device__ __forceinline__ unsigned outlier_mask(const float (&v)[kLaneW], float tau)
+{
+    return outlier_bits(v, outlier_threshold<I>(v, tau));
 }
 
 // Exclusive prefix of a per-lane count over the warp, and the warp total.
@@ -354,27 +366,38 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
         const bool tile_ok = tile * kOpqTile < n;  // warp-uniform
         float v[kLaneW];
         widen(raw, v);
-        const unsigned o = outlier_mask<I>(v, tau);
-        const unsigned any = __ballot_sync(kFull, o != 0u);
-        if (any) {
-            int total;
-            int pos = warp_excl_scan(__popc(o), lane, total);
+        // A lane can only hold an outlier if its largest magnitude exceeds the threshold, so the
+        // per-element test runs only in warps where some lane does (a NaN maximum also enters).
+        float mx, mn;
+        lane_minmax(v, mx, mn);
+        const float thr = outlier_threshold<I>(v, tau);
+        const bool maybe = !(fmaxf(mx, -mn) <= thr);
+        if (__any_sync(kFull, maybe)) {
+            const unsigned o = outlier_bits(v, thr);
+            const unsigned any = __ballot_sync(kFull, o != 0u);
+            if (any) {
+                int total;
+                int pos = warp_excl_scan(__popc(o), lane, total);
 #pragma unroll
-            for (int k = 0; k < kLaneW; ++k)
-                if ((o >> k) & 1u) {
-                    if (pos < kOpqStage) {
-                        stage_idx[tile * kOpqStage + pos] = (int32_t)(idx + k);
-                        stage_val[tile * kOpqStage + pos] = (uint16_t)bf16_rne(v[k]);
+                for (int k = 0; k < kLaneW; ++k)
+                    if ((o >> k) & 1u) {
+                        if (pos < kOpqStage) {
+                            stage_idx[tile * kOpqStage + pos] = (int32_t)(idx + k);
+                            stage_val[tile * kOpqStage + pos] = (uint16_t)bf16_rne(v[k]);
+                        }
+                        ++pos;
+                        v[k] = 0.0f;
                     }
-                    ++pos;
-                    v[k] = 0.0f;
-                }
-            if (lane == 0) counts[tile] = total;
+                if (lane == 0) counts[tile] = total;
+                lane_minmax(v, mx, mn);  // of the cleaned weights
+            } else if (lane == 0 && tile_ok) {
+                counts[tile] = 0;
+            }
         } else if (lane == 0 && tile_ok) {
             counts[tile] = 0;
         }
         if (QUANT) {
-            quantize_row<DT, I, SIGNED, ST>(v, idx, ok, T, lut_base, lane, codes, scales);
+            quantize_row<DT, I, SIGNED, ST>(v, mx, mn, idx, ok, T, lut_base, lane, codes, scales);
         } else if (w_clean != nullptr && ok) {
             store_row(DT{}, w_clean, idx, v);
         }
