@@ -317,7 +317,7 @@ def run_gpu(args):
     avg = {k: sum(v) / len(v) for k, v in comp_ms.items()}
     bytes_per_w = {"em_mse": BYTES_EM, "em_mae": None, "quantize_opq": BYTES_QUANT, "dequantize": BYTES_DEQUANT,
                    "quantize": BYTES_QUANT}
-    kernels = {"em_mse": 1, "em_mae": mae_launches(bof4), "quantize_opq": 4, "dequantize": 2, "quantize": 1}
+    kernels = {"em_mse": 1, "em_mae": mae_launches(bof4), "quantize_opq": 2, "dequantize": 2, "quantize": 1}
     comp, launches = {}, 0
     for name, ms in avg.items():
         comp[name + "_ms"] = ms

@@ -342,8 +342,8 @@ template <class DT, int I, bool SIGNED, class ST, bool QUANT>
 __global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
 opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels, float tau,
                  uint8_t* __restrict__ codes, void* __restrict__ scales, void* __restrict__ w_clean,
-                 int32_t* __restrict__ counts, int32_t* __restrict__ stage_idx,
-                 uint16_t* __restrict__ stage_val)
+                 int32_t* __restrict__ counts, unsigned long long* __restrict__ chunk_sum,
+                 int32_t* __restrict__ stage_idx, uint16_t* __restrict__ stage_val)
 {
     static_assert(kOpqTile == kWarpW, "one tile per warp iteration");
     extern __shared__ __align__(16) unsigned char s_lut[];
@@ -388,7 +388,10 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
                         ++pos;
                         v[k] = 0.0f;
                     }
-                if (lane == 0) counts[tile] = total;
+                if (lane == 0) {
+                    counts[tile] = total;
+                    atomicAdd(&chunk_sum[tile / kOpqChunk], (unsigned long long)total);  // integer: order-free
+                }
                 lane_minmax(v, mx, mn);  // of the cleaned weights
             } else if (lane == 0 && tile_ok) {
                 counts[tile] = 0;
@@ -405,66 +408,21 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
     }
 }
 
-// Pass 2a: outlier count of every chunk of kOpqChunk tiles.
-__global__ void __launch_bounds__(256)
-opq_chunk_sum_kernel(const int32_t* __restrict__ counts, int64_t tiles, int64_t* __restrict__ chunk_off)
-{
-    __shared__ int64_t s_part[8];
-    const int64_t t0 = (int64_t)blockIdx.x * kOpqChunk;
-    int64_t s = 0;
-    for (int k = threadIdx.x; k < kOpqChunk; k += 256)
-        if (t0 + k < tiles) s += counts[t0 + k];
-#pragma unroll
-    for (int off = 16; off; off >>= 1) s += __shfl_xor_sync(kFull, s, off);
-    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = s;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int64_t t = 0;
-        for (int k = 0; k < 8; ++k) t += s_part[k];
-        chunk_off[blockIdx.x] = t;
-    }
-}
-
-// Pass 2b: exclusive scan of the chunk sums in place (one CTA); total -> chunk_off[chunks], *n_out.
-__global__ void __launch_bounds__(1024)
-opq_chunk_scan_kernel(int64_t* __restrict__ chunk_off, int64_t chunks, int64_t* __restrict__ n_out)
-{
-    __shared__ int64_t s_sum[1024];
-    const int64_t per = (chunks + 1023) / 1024;
-    const int64_t lo = threadIdx.x * per, hi = (lo + per < chunks) ? lo + per : chunks;
-    int64_t s = 0;
-    for (int64_t k = lo; k < hi; ++k) s += chunk_off[k];
-    s_sum[threadIdx.x] = s;
-    __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
-        const int64_t t = (threadIdx.x >= off) ? s_sum[threadIdx.x - off] : 0;
-        __syncthreads();
-        s_sum[threadIdx.x] += t;
-        __syncthreads();
-    }
-    int64_t run = s_sum[threadIdx.x] - s;
-    for (int64_t k = lo; k < hi; ++k) {
-        const int64_t c = chunk_off[k];
-        chunk_off[k] = run;
-        run += c;
-    }
-    if (threadIdx.x == 1023) {
-        chunk_off[chunks] = s_sum[1023];
-        *n_out = s_sum[1023];
-    }
-}
-
-// Pass 3: every tile's staged outliers are copied to their final, globally ascending position;
-// a tile with more than kOpqStage outliers is re-derived from the weights by one warp.
+// Pass 2: every tile's staged outliers are copied to their final, globally ascending position;
+// a tile with more than kOpqStage outliers is re-derived from the weights by one warp.  Each
+// CTA owns one chunk of tiles; its first output position is the sum of the earlier chunks'
+// outlier counts (accumulated by pass 1), and the last chunk's CTA also reports the total.
 template <class DT, int I>
 __global__ void __launch_bounds__(256)
 opq_gather_kernel(const void* __restrict__ w, int64_t n, float tau, const int32_t* __restrict__ counts,
-                  int64_t tiles, const int64_t* __restrict__ chunk_off,
+                  int64_t tiles, const unsigned long long* __restrict__ chunk_sum,
                   const int32_t* __restrict__ stage_idx, const uint16_t* __restrict__ stage_val,
-                  int32_t* __restrict__ out_idx, uint16_t* __restrict__ out_val, int64_t capacity)
+                  int32_t* __restrict__ out_idx, uint16_t* __restrict__ out_val, int64_t capacity,
+                  int64_t* __restrict__ n_out)
 {
     constexpr int PER = kOpqChunk / 256;  // consecutive tiles per thread
     __shared__ int64_t s_warp[8];
+    __shared__ unsigned long long s_base[8];
     __shared__ int32_t s_ovf_tile[kOpqChunk];  // tile index relative to the chunk
     __shared__ int32_t s_ovf_off[kOpqChunk];   // offset relative to the chunk's first output
     __shared__ int s_novf;
@@ -485,7 +443,17 @@ opq_gather_kernel(const void* __restrict__ w, int64_t n, float tau, const int32_
     __syncthreads();
     int rel = excl;
     for (int k = 0; k < warp; ++k) rel += (int)s_warp[k];
-    const int64_t base = chunk_off[blockIdx.x];
+    // first output position of this chunk: outliers of all earlier chunks
+    unsigned long long before = 0ull;
+    for (int k = threadIdx.x; k < (int)blockIdx.x; k += 256) before += chunk_sum[k];
+#pragma unroll
+    for (int off = 16; off; off >>= 1) before += __shfl_xor_sync(kFull, before, off);
+    if (lane == 0) s_base[warp] = before;
+    __syncthreads();
+    before = 0ull;
+    for (int k = 0; k < 8; ++k) before += s_base[k];
+    const int64_t base = (int64_t)before;
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) *n_out = base + (int64_t)chunk_sum[blockIdx.x];
 #pragma unroll
     for (int k = 0; k < PER; ++k) {
         if (c[k] > 0) {
@@ -735,35 +703,30 @@ int launch_opq(const char* fn, const void* d_w, int w_dtype, int64_t n, int bloc
         return rc;
     char* ws = static_cast<char*>(d_ws);
     int32_t* counts = reinterpret_cast<int32_t*>(ws + L.counts);
-    int64_t* chunk_off = reinterpret_cast<int64_t*>(ws + L.chunk_off);
+    unsigned long long* chunk_sum = reinterpret_cast<unsigned long long*>(ws + L.chunk_off);
     int32_t* stage_idx = reinterpret_cast<int32_t*>(ws + L.stage_idx);
     uint16_t* stage_val = reinterpret_cast<uint16_t*>(ws + L.stage_val);
     uint16_t* out_val = static_cast<uint16_t*>(d_out_val);
     const int64_t rows = (n + kQRow - 1) / kQRow;
     const int grid = grid_for(rows, kQCtasPerSm);
     const int smem = QUANT ? kLutBytes : 0;
+    BOF4_CUDA_TRY(cudaMemsetAsync(chunk_sum, 0, (size_t)L.chunks * 8, st));
     BOF4_DISPATCH_WS(w_dtype, scale_dtype,
         BOF4_DISPATCH_I(block_size,
             BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
                 { auto kern = opq_pass1_kernel<DT, I_, SG, ST, QUANT>;
                   BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
                   kern<<<grid, kQThreads, smem, st>>>(
-                      d_w, n, d_codebook, tau, d_codes, d_scales, d_w_clean, counts, stage_idx, stage_val); })));
+                      d_w, n, d_codebook, tau, d_codes, d_scales, d_w_clean, counts, chunk_sum, stage_idx, stage_val); })));
     BOF4_CUDA_TRY(cudaGetLastError());
-    opq_chunk_sum_kernel<<<(int)L.chunks, 256, 0, st>>>(counts, L.tiles, chunk_off);
-    BOF4_CUDA_TRY(cudaGetLastError());
-    opq_chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_off, L.chunks, d_n_out);
-    BOF4_CUDA_TRY(cudaGetLastError());
-    if (capacity > 0) {
-        if (w_dtype == BOF4_F32) {
-            BOF4_DISPATCH_I(block_size, (opq_gather_kernel<F32, I_><<<(int)L.chunks, 256, 0, st>>>(
-                d_w, n, tau, counts, L.tiles, chunk_off, stage_idx, stage_val, d_out_idx, out_val, capacity)));
-        } else {
-            BOF4_DISPATCH_I(block_size, (opq_gather_kernel<BF16, I_><<<(int)L.chunks, 256, 0, st>>>(
-                d_w, n, tau, counts, L.tiles, chunk_off, stage_idx, stage_val, d_out_idx, out_val, capacity)));
-        }
-        BOF4_CUDA_TRY(cudaGetLastError());
+    if (w_dtype == BOF4_F32) {
+        BOF4_DISPATCH_I(block_size, (opq_gather_kernel<F32, I_><<<(int)L.chunks, 256, 0, st>>>(
+            d_w, n, tau, counts, L.tiles, chunk_sum, stage_idx, stage_val, d_out_idx, out_val, capacity, d_n_out)));
+    } else {
+        BOF4_DISPATCH_I(block_size, (opq_gather_kernel<BF16, I_><<<(int)L.chunks, 256, 0, st>>>(
+            d_w, n, tau, counts, L.tiles, chunk_sum, stage_idx, stage_val, d_out_idx, out_val, capacity, d_n_out)));
     }
+    BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }
 
