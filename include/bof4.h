@@ -12,7 +12,7 @@
  *    enqueued on that stream and the call returns without synchronising; outputs are valid once
  *    the stream has reached the end of the enqueued work.
  *  - Weights are a flattened tensor of n elements cut into B = n / block_size contiguous blocks
- *    (Sec. 2.1).  block_size is one of 32, 64, 128, 256 and n must be a multiple of it.
+ *    (Sec. 2.1).  block_size is a power of two from 32 to 4096 and n must be a multiple of it.
  *  - Weight tensors, code arrays and dequantised outputs are accessed with 32-byte vector
  *    instructions: their device pointers must be 32-byte aligned (BOF4_ERR_INVALID_ARG if not).
  *  - A codebook is 16 fp32 reconstruction levels in ASCENDING order, device resident.  Code c

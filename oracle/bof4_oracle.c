@@ -376,7 +376,7 @@ static float tree_sum(float *v, int len)
  * fp32, tree-ordered sums. */
 static float block_sigma(const float *w, int I)
 {
-    float tmp[1024];
+    float tmp[4096]; /* largest supported block */
     for (int i = 0; i < I; ++i)
         tmp[i] = w[i];
     float mean = tree_sum(tmp, I) / (float)I;

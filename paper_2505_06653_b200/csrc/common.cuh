@@ -2,10 +2,11 @@
 // normalisation (Eq. 2), region search (Sec. 3.2), plus the host-side status plumbing.
 //
 // Work layout used by every streaming kernel: one lane owns kLaneW = 16 consecutive weights
-// (one 32-byte load for bf16, two for fp32), so a block of I weights is owned by
-// LPB = I / 16 neighbouring lanes of one warp (2, 4, 8 or 16 lanes) and every per-block
-// reduction is a shuffle butterfly inside that lane group.  One warp iteration covers
-// kWarpW = 512 consecutive weights.
+// (one 32-byte load for bf16, two for fp32), so a block of I <= 512 weights is owned by
+// LPB = I / 16 neighbouring lanes of one warp and every per-block reduction is a shuffle
+// butterfly inside that lane group; a block of 1024 ... 4096 weights is owned by 2 ... 8
+// neighbouring warps of one CTA, which exchange their per-warp results through shared memory.
+// One warp iteration covers kWarpW = 512 consecutive weights.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -32,7 +33,7 @@ int cuda_fail(cudaError_t e, const char* what);
         if (e__ != cudaSuccess) return ::bof4::cuda_fail(e__, #expr); \
     } while (0)
 
-inline bool valid_block_size(int I) { return I == 32 || I == 64 || I == 128 || I == 256; }
+inline bool valid_block_size(int I) { return I >= 32 && I <= 4096 && (I & (I - 1)) == 0; }
 inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
 // ---------------------------------------------------------------- loads and stores
@@ -202,42 +203,109 @@ __device__ __forceinline__ void lane_minmax(const float (&v)[kLaneW], float& mx,
     mn = fminf(mn, v[15]);
 }
 
-template <int LPB, bool SIGNED>
-__device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float mx, float mn, float& g)
+// A block of I weights is LPB lanes of one warp (I <= 512) or WPB whole, neighbouring warps of
+// one CTA (I = 1024 ... 4096; CTA rows are multiples of 8192 weights, so blocks never straddle
+// CTA rows).  Blocks wider than a warp combine their per-warp results through shared memory.
+template <int I>
+struct BlockGeo {
+    static constexpr int LPB = (I >= kWarpW) ? 32 : I / kLaneW;  // lanes of a warp per block
+    static constexpr int WPB = (I >= kWarpW) ? I / kWarpW : 1;   // warps per block
+};
+
+// One slot per warp of the CTA for the cross-warp steps of wide blocks.
+struct WideScratch {
+    float a[32], b[32];
+    int pos[32];
+};
+
+// Combines one value per warp over the WPB warps of a block, in warp order, with `op`; every
+// thread of the CTA must call it.  Two barriers: publish, then protect the slots for reuse.
+template <int WPB, class Op>
+__device__ __forceinline__ float across_warps(float x, float* slot, Op op)
 {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) slot[warp] = x;
+    __syncthreads();
+    const int base = warp & ~(WPB - 1);
+    float t[WPB];
+#pragma unroll
+    for (int k = 0; k < WPB; ++k) t[k] = slot[base + k];
+#pragma unroll
+    for (int step = 1; step < WPB; step <<= 1)  // neighbours first: the order of a balanced tree
+#pragma unroll
+        for (int k = 0; k < WPB; k += 2 * step) t[k] = op(t[k], t[k + step]);
+    __syncthreads();
+    return t[0];
+}
+
+// Block constant from the lane's largest / smallest weight (lane_minmax).  `ws` is only used
+// by blocks wider than a warp (then every thread of the CTA must take part).
+template <int I, bool SIGNED>
+__device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float mx, float mn, float& g,
+                                                WideScratch* ws)
+{
+    constexpr int LPB = BlockGeo<I>::LPB, WPB = BlockGeo<I>::WPB;
     float gx = mx, gn = mn;
 #pragma unroll
     for (int off = 1; off < LPB; off <<= 1) {
         gx = max2_nan(gx, __shfl_xor_sync(kFull, gx, off));
         gn = fminf(gn, __shfl_xor_sync(kFull, gn, off));
     }
+    if constexpr (WPB > 1) {
+        gx = across_warps<WPB>(gx, ws->a, [](float p, float q) { return max2_nan(p, q); });
+        gn = across_warps<WPB>(gn, ws->b, [](float p, float q) { return fminf(p, q); });
+    }
     g = max2_nan(gx, -gn);
     if (!SIGNED) return g;
     float m = (gx > -gn) ? gx : gn;
     const bool tie = (gx == -gn) && (g != 0.0f);
-    if (__any_sync(kFull, tie)) {
-        const int lane = threadIdx.x & 31;
-        const int base = lane & ~(LPB - 1);
-        const unsigned gmask = ((1u << LPB) - 1u) << base;
-        const unsigned hp = __ballot_sync(kFull, mx == g) & gmask;   // lanes holding +g
-        const unsigned hn = __ballot_sync(kFull, mn == -g) & gmask;  // lanes holding -g
-        const int lp = __ffs(hp) - 1, ln = __ffs(hn) - 1;            // -1: none
-        float first = 0.0f;  // this lane's first element of magnitude g
+    const int lane = threadIdx.x & 31;
+    if constexpr (WPB == 1) {
+        if (__any_sync(kFull, tie)) {
+            const int base = lane & ~(LPB - 1);
+            const unsigned gmask = (LPB == 32) ? kFull : (((1u << (LPB & 31)) - 1u) << base);
+            const unsigned hp = __ballot_sync(kFull, mx == g) & gmask;   // lanes holding +g
+            const unsigned hn = __ballot_sync(kFull, mn == -g) & gmask;  // lanes holding -g
+            const int lp = __ffs(hp) - 1, ln = __ffs(hn) - 1;            // -1: none
+            float first = 0.0f;  // this lane's first element of magnitude g
 #pragma unroll
-        for (int k = kLaneW - 1; k >= 0; --k) first = (fabsf(v[k]) == g) ? v[k] : first;
-        const int src = (lp >= 0 && (ln < 0 || lp <= ln)) ? lp : ln;  // lane of the block's first +-g
-        const float pick = __shfl_sync(kFull, first, src < 0 ? 0 : src);
-        if (tie) m = pick;
+            for (int k = kLaneW - 1; k >= 0; --k) first = (fabsf(v[k]) == g) ? v[k] : first;
+            const int src = (lp >= 0 && (ln < 0 || lp <= ln)) ? lp : ln;  // lane of the block's first +-g
+            const float pick = __shfl_sync(kFull, first, src < 0 ? 0 : src);
+            if (tie) m = pick;
+        }
+    } else {
+        if (__syncthreads_or(tie ? 1 : 0)) {
+            // every warp reports the position and value of its first element of magnitude g
+            float first = 0.0f;
+#pragma unroll
+            for (int k = kLaneW - 1; k >= 0; --k) first = (fabsf(v[k]) == g) ? v[k] : first;
+            const unsigned has = __ballot_sync(kFull, fmaxf(mx, -mn) == g);
+            const int src = __ffs(has) - 1;  // -1: this warp holds no +-g
+            const float val = __shfl_sync(kFull, first, src < 0 ? 0 : src);
+            const int warp = threadIdx.x >> 5;
+            if (lane == 0) {
+                ws->pos[warp] = src;
+                ws->a[warp] = val;
+            }
+            __syncthreads();
+            const int base = warp & ~(WPB - 1);
+            float pick = 0.0f;
+#pragma unroll
+            for (int k = WPB - 1; k >= 0; --k) pick = (ws->pos[base + k] >= 0) ? ws->a[base + k] : pick;
+            __syncthreads();
+            if (tie) m = pick;
+        }
     }
     return (g == 0.0f) ? 0.0f : m;
 }
 
-template <int LPB, bool SIGNED>
-__device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float& g)
+template <int I, bool SIGNED>
+__device__ __forceinline__ float block_constant(const float (&v)[kLaneW], float& g, WideScratch* ws)
 {
     float mx, mn;
     lane_minmax(v, mx, mn);
-    return block_constant<LPB, SIGNED>(v, mx, mn, g);
+    return block_constant<I, SIGNED>(v, mx, mn, g, ws);
 }
 
 // Eq. 2 with the 0/0 reading x = 0.  IEEE round-to-nearest division.

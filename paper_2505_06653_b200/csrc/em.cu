@@ -126,7 +126,6 @@ __global__ void __launch_bounds__(EmGeo<COUNT>::threads, 1)
 em_mse_kernel(const EmTensors T, const float* levels, double* partials, const MseTail tail)
 {
     using G = EmGeo<COUNT>;
-    constexpr int LPB = I / kLaneW;
     constexpr int NT = G::threads, NW = NT / 32, NSEG = NW / kLevels;
     extern __shared__ __align__(16) unsigned char s_raw[];
     unsigned char* s_lut = s_raw;
@@ -134,6 +133,7 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
     unsigned char* s_cnt = s_acc + (size_t)kLevels * G::acc_row_bytes;  // uint32 [16][NT] (COUNT)
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
+    __shared__ WideScratch s_wide;
     __shared__ double s_part[NSEG][3][kLevels];
     __shared__ double s_tot[3 * kLevels];  // s1, s0, count (as uint64 bits)
     __shared__ double s_w2[NW];
@@ -236,7 +236,7 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
         float v[kLaneW];
         widen(raw, v);
         float gmax;
-        const float m = block_constant<LPB, SIGNED>(v, gmax);
+        const float m = block_constant<I, SIGNED>(v, gmax, &s_wide);
         const bool safe = row_is_safe(gmax, ok);
         float2 sq = make_float2(0.0f, 0.0f);
 #pragma unroll
@@ -338,7 +338,7 @@ int check_em(const char* fn, EmArgs& a, const void* d_codebook, void* d_ws, size
         return BOF4_ERR_INVALID_ARG;
     }
     if (!valid_block_size(a.block_size)) {
-        set_error("%s: block_size %d is not one of 32, 64, 128, 256", fn, a.block_size);
+        set_error("%s: block_size %d is not a power of two in 32 ... 4096", fn, a.block_size);
         return BOF4_ERR_SHAPE;
     }
     if (a.w_dtype != BOF4_F32 && a.w_dtype != BOF4_BF16) {
@@ -412,18 +412,18 @@ int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials,
     tail.ticket = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(partials) + kEmTicketOffset);
     const bool sg = a.norm == BOF4_NORM_SIGNED;
     auto fire = [&](const EmTensors& T) -> int {
-#define BOF4_EM_GO(DT_)                                                                                 \
-    switch (a.block_size) {                                                                             \
-        case 32: return sg ? launch_mse_chunk<DT_, 32, true, COUNT>(T, d_codebook, partials, tail, st)        \
-                           : launch_mse_chunk<DT_, 32, false, COUNT>(T, d_codebook, partials, tail, st);      \
-        case 64: return sg ? launch_mse_chunk<DT_, 64, true, COUNT>(T, d_codebook, partials, tail, st)        \
-                           : launch_mse_chunk<DT_, 64, false, COUNT>(T, d_codebook, partials, tail, st);      \
-        case 128: return sg ? launch_mse_chunk<DT_, 128, true, COUNT>(T, d_codebook, partials, tail, st)      \
-                            : launch_mse_chunk<DT_, 128, false, COUNT>(T, d_codebook, partials, tail, st);    \
-        default: return sg ? launch_mse_chunk<DT_, 256, true, COUNT>(T, d_codebook, partials, tail, st)       \
-                           : launch_mse_chunk<DT_, 256, false, COUNT>(T, d_codebook, partials, tail, st);     \
+#define BOF4_EM_CASE(DT_, I_)                                                                        \
+    case I_: return sg ? launch_mse_chunk<DT_, I_, true, COUNT>(T, d_codebook, partials, tail, st)   \
+                       : launch_mse_chunk<DT_, I_, false, COUNT>(T, d_codebook, partials, tail, st);
+#define BOF4_EM_GO(DT_)                                                                              \
+    switch (a.block_size) {                                                                          \
+        BOF4_EM_CASE(DT_, 32) BOF4_EM_CASE(DT_, 64) BOF4_EM_CASE(DT_, 128) BOF4_EM_CASE(DT_, 256)    \
+        BOF4_EM_CASE(DT_, 512) BOF4_EM_CASE(DT_, 1024) BOF4_EM_CASE(DT_, 2048)                       \
+        default: return sg ? launch_mse_chunk<DT_, 4096, true, COUNT>(T, d_codebook, partials, tail, st)  \
+                           : launch_mse_chunk<DT_, 4096, false, COUNT>(T, d_codebook, partials, tail, st); \
     }
         if (a.w_dtype == BOF4_F32) { BOF4_EM_GO(F32) } else { BOF4_EM_GO(BF16) }
+#undef BOF4_EM_CASE
 #undef BOF4_EM_GO
     };
     int calls = 0;

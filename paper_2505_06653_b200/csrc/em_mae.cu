@@ -157,7 +157,6 @@ template <class DT, int I, bool SIGNED, bool FIRST, bool COUNT, bool COLLECT>
 __global__ void __launch_bounds__(kMaeThreads, 1)
 mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
 {
-    constexpr int LPB = I / kLaneW;
     extern __shared__ __align__(16) unsigned char s_raw[];
     unsigned char* s_lut = s_raw;
     uint32_t* s_lo = reinterpret_cast<uint32_t*>(s_raw + kLutBytes);
@@ -167,6 +166,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     __shared__ uint32_t s_ncand[kLevels], s_gbase[kLevels];
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
+    __shared__ WideScratch s_wide;
     __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
     __shared__ double s_err[kMaeThreads / 32];
     __shared__ const void* s_ptr[kEmMaxTensors];
@@ -211,7 +211,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         float v[kLaneW];
         widen(ok ? load_raw<DT>(s_ptr[t_cur], idx) : zero_raw<DT>(), v);
         float gmax;
-        const float m = block_constant<LPB, SIGNED>(v, gmax);
+        const float m = block_constant<I, SIGNED>(v, gmax, &s_wide);
         const bool safe = row_is_safe(gmax, ok);
         float x[kLaneW];
         normalise16<false>(v, m, safe && DT::code == BF16::code, x);
@@ -511,7 +511,11 @@ int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, co
         case 32: BOF4_MAE_I(DT_, 32)             \
         case 64: BOF4_MAE_I(DT_, 64)             \
         case 128: BOF4_MAE_I(DT_, 128)           \
-        default: BOF4_MAE_I(DT_, 256)            \
+        case 256: BOF4_MAE_I(DT_, 256)           \
+        case 512: BOF4_MAE_I(DT_, 512)           \
+        case 1024: BOF4_MAE_I(DT_, 1024)         \
+        case 2048: BOF4_MAE_I(DT_, 2048)         \
+        default: BOF4_MAE_I(DT_, 4096)           \
     }
     if (a.w_dtype == BOF4_F32) { BOF4_MAE_DT(F32) } else { BOF4_MAE_DT(BF16) }
 #undef BOF4_MAE_DT

@@ -99,11 +99,11 @@ __device__ __forceinline__ void encode16(const float (&x)[kLaneW], const QuantTa
 template <class DT, int I, bool SIGNED, class ST>
 __device__ __forceinline__ void quantize_row(const float (&v)[kLaneW], float mx, float mn, int64_t idx,
                                              bool ok, const QuantTables& T, uint32_t lut_base, int lane,
-                                             uint8_t* __restrict__ codes, void* __restrict__ scales)
+                                             uint8_t* __restrict__ codes, void* __restrict__ scales,
+                                             WideScratch* ws)
 {
-    constexpr int LPB = I / kLaneW;
     float g;
-    const float m = block_constant<LPB, SIGNED>(v, mx, mn, g);
+    const float m = block_constant<I, SIGNED>(v, mx, mn, g, ws);
     const bool safe = row_is_safe(g, ok);
     float x[kLaneW];
     normalise16<true>(v, m, safe && DT::code == BF16::code, x);
@@ -111,7 +111,7 @@ __device__ __forceinline__ void quantize_row(const float (&v)[kLaneW], float mx,
     encode16(x, T, safe && T.lut_ok, lut_base, w0, w1);
     if (ok) {
         st_stream64(codes + idx / 2, w0, w1);
-        if ((lane & (LPB - 1)) == 0) store_scale<ST>(scales, idx / I, m);
+        if ((idx & (I - 1)) == 0) store_scale<ST>(scales, idx / I, m);  // the block's first lane
     }
 }
 
@@ -123,6 +123,7 @@ quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__
     extern __shared__ __align__(16) unsigned char s_lut[];
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
+    __shared__ WideScratch s_wide;
     const QuantTables T = setup_tables(levels, s_xi, s_lv, s_lut, &s_multi);
     const int lane = threadIdx.x & 31;
     const uint32_t lut_base = lut_lane_base(s_lut, lane);  // table base of this lane
@@ -136,7 +137,8 @@ quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__
         float v[kLaneW], mx, mn;
         widen(raw, v);
         lane_minmax(v, mx, mn);
-        quantize_row<DT, I, SIGNED, ST>(v, mx, mn, map.idx(r), map.ok(r), T, lut_base, lane, codes, scales);
+        quantize_row<DT, I, SIGNED, ST>(v, mx, mn, map.idx(r), map.ok(r), T, lut_base, lane, codes, scales,
+                                        &s_wide);
         raw = next;
     }
 }
@@ -254,10 +256,12 @@ __global__ void scatter_outliers_kernel(const int32_t* __restrict__ idx, const u
 // ---------------------------------------------------------------- OPQ (Sec. 3.3, App. E)
 
 // Balanced binary summation tree over the block: neighbours first inside the lane, then the
-// lane butterfly.  Every addition is a separate fp32 RN operation.
-template <int LPB>
-__device__ __forceinline__ float tree_sum(const float (&t)[kLaneW])
+// lane butterfly, then (blocks wider than a warp) the warps of the block pairwise in order.
+// Every addition is a separate fp32 RN operation.
+template <int I>
+__device__ __forceinline__ float tree_sum(const float (&t)[kLaneW], float* slot)
 {
+    constexpr int LPB = BlockGeo<I>::LPB, WPB = BlockGeo<I>::WPB;
     float a[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) a[k] = __fadd_rn(t[2 * k], t[2 * k + 1]);
@@ -265,23 +269,24 @@ __device__ __forceinline__ float tree_sum(const float (&t)[kLaneW])
                         __fadd_rn(__fadd_rn(a[4], a[5]), __fadd_rn(a[6], a[7])));
 #pragma unroll
     for (int off = 1; off < LPB; off <<= 1) s = __fadd_rn(s, __shfl_xor_sync(kFull, s, off));
+    if constexpr (WPB > 1) s = across_warps<WPB>(s, slot, [](float p, float q) { return __fadd_rn(p, q); });
     return s;
 }
 
 // The outlier threshold of the lane's block: sigma_b * tau, sigma_b the corrected sample
-// standard deviation (two-pass formula in fp32, tree-ordered sums).
+// standard deviation (two-pass formula in fp32, tree-ordered sums).  For blocks wider than a
+// warp every thread of the CTA must call it.
 template <int I>
-__device__ __forceinline__ float outlier_threshold(const float (&v)[kLaneW], float tau)
+__device__ __forceinline__ float outlier_threshold(const float (&v)[kLaneW], float tau, WideScratch* ws)
 {
-    constexpr int LPB = I / kLaneW;
-    const float mean = __fmul_rn(tree_sum<LPB>(v), 1.0f / (float)I);  // exact: I is a power of two
+    const float mean = __fmul_rn(tree_sum<I>(v, ws ? ws->a : nullptr), 1.0f / (float)I);  // exact: I = 2^k
     float q[kLaneW];
 #pragma unroll
     for (int k = 0; k < kLaneW; ++k) {
         const float d = __fsub_rn(v[k], mean);
         q[k] = __fmul_rn(d, d);
     }
-    const float sigma = __fsqrt_rn(__fdiv_rn(tree_sum<LPB>(q), (float)(I - 1)));
+    const float sigma = __fsqrt_rn(__fdiv_rn(tree_sum<I>(q, ws ? ws->b : nullptr), (float)(I - 1)));
     return __fmul_rn(sigma, tau);
 }
 
@@ -294,10 +299,47 @@ __device__ __forceinline__ unsigned outlier_bits(const float (&v)[kLaneW], float
     return o;
 }
 
-template <int I>
-__device__ __forceinline__ unsigned outlier_mask(const float (&v)[kLaneW], float tau)
+// The outlier threshold of the block that contains tile `tile`, computed by ONE warp alone (the
+// re-derivation of an overflowed tile in the gather kernel): a block wider than a warp is read
+// tile by tile, twice, and its per-tile sums are combined in the same tree order.
+template <class DT, int I>
+__device__ __forceinline__ float outlier_threshold_one_warp(const void* __restrict__ w, int64_t tile, float tau,
+                                                            int lane, const float (&v)[kLaneW])
 {
-    return outlier_bits(v, outlier_threshold<I>(v, tau));
+    constexpr int WPB = BlockGeo<I>::WPB;
+    if constexpr (WPB == 1) {
+        return outlier_threshold<I>(v, tau, nullptr);
+    } else {
+        const int64_t first = (tile / WPB) * WPB;  // first tile of the block
+        float part[WPB];
+        float u[kLaneW];
+#pragma unroll
+        for (int t = 0; t < WPB; ++t) {
+            widen(load_raw<DT>(w, (first + t) * kWarpW + lane * kLaneW), u);
+            part[t] = tree_sum<kWarpW>(u, nullptr);
+        }
+#pragma unroll
+        for (int step = 1; step < WPB; step <<= 1)
+#pragma unroll
+            for (int k = 0; k < WPB; k += 2 * step) part[k] = __fadd_rn(part[k], part[k + step]);
+        const float mean = __fmul_rn(part[0], 1.0f / (float)I);
+#pragma unroll
+        for (int t = 0; t < WPB; ++t) {
+            widen(load_raw<DT>(w, (first + t) * kWarpW + lane * kLaneW), u);
+#pragma unroll
+            for (int k = 0; k < kLaneW; ++k) {
+                const float d = __fsub_rn(u[k], mean);
+                u[k] = __fmul_rn(d, d);
+            }
+            part[t] = tree_sum<kWarpW>(u, nullptr);
+        }
+#pragma unroll
+        for (int step = 1; step < WPB; step <<= 1)
+#pragma unroll
+            for (int k = 0; k < WPB; k += 2 * step) part[k] = __fadd_rn(part[k], part[k + step]);
+        const float sigma = __fsqrt_rn(__fdiv_rn(part[0], (float)(I - 1)));
+        return __fmul_rn(sigma, tau);
+    }
 }
 
 // Exclusive prefix of a per-lane count over the warp, and the warp total.
@@ -349,6 +391,7 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
     extern __shared__ __align__(16) unsigned char s_lut[];
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
+    __shared__ WideScratch s_wide;
     QuantTables T{s_xi, s_lut, false};
     if (QUANT) T = setup_tables(levels, s_xi, s_lv, s_lut, &s_multi);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -370,7 +413,7 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
         // per-element test runs only in warps where some lane does (a NaN maximum also enters).
         float mx, mn;
         lane_minmax(v, mx, mn);
-        const float thr = outlier_threshold<I>(v, tau);
+        const float thr = outlier_threshold<I>(v, tau, &s_wide);
         const bool maybe = !(fmaxf(mx, -mn) <= thr);
         if (__any_sync(kFull, maybe)) {
             const unsigned o = outlier_bits(v, thr);
@@ -400,7 +443,7 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
             counts[tile] = 0;
         }
         if (QUANT) {
-            quantize_row<DT, I, SIGNED, ST>(v, mx, mn, idx, ok, T, lut_base, lane, codes, scales);
+            quantize_row<DT, I, SIGNED, ST>(v, mx, mn, idx, ok, T, lut_base, lane, codes, scales, &s_wide);
         } else if (w_clean != nullptr && ok) {
             store_row(DT{}, w_clean, idx, v);
         }
@@ -480,7 +523,7 @@ opq_gather_kernel(const void* __restrict__ w, int64_t n, float tau, const int32_
         const int64_t idx = tile * kOpqTile + lane * kLaneW;
         float v[kLaneW];
         widen((idx < n) ? load_raw<DT>(w, idx) : zero_raw<DT>(), v);
-        const unsigned o = outlier_mask<I>(v, tau);
+        const unsigned o = outlier_bits(v, outlier_threshold_one_warp<DT, I>(w, tile, tau, lane, v));
         int total;
         int pos = warp_excl_scan(__popc(o), lane, total);
 #pragma unroll
@@ -517,7 +560,7 @@ int check_common(const char* fn, int64_t n, int block_size)
         return BOF4_ERR_INVALID_ARG;
     }
     if (!valid_block_size(block_size)) {
-        set_error("%s: block_size %d is not one of 32, 64, 128, 256", fn, block_size);
+        set_error("%s: block_size %d is not a power of two in 32 ... 4096", fn, block_size);
         return BOF4_ERR_SHAPE;
     }
     if (n % block_size) {
@@ -563,7 +606,11 @@ int check_aligned(const char* fn, const char* what, const void* p)
         case 32: { constexpr int I_ = 32; __VA_ARGS__; } break;   \
         case 64: { constexpr int I_ = 64; __VA_ARGS__; } break;   \
         case 128: { constexpr int I_ = 128; __VA_ARGS__; } break; \
-        default: { constexpr int I_ = 256; __VA_ARGS__; } break;  \
+        case 256: { constexpr int I_ = 256; __VA_ARGS__; } break; \
+        case 512: { constexpr int I_ = 512; __VA_ARGS__; } break; \
+        case 1024: { constexpr int I_ = 1024; __VA_ARGS__; } break; \
+        case 2048: { constexpr int I_ = 2048; __VA_ARGS__; } break; \
+        default: { constexpr int I_ = 4096; __VA_ARGS__; } break;  \
     }
 #define BOF4_DISPATCH_BOOL(FLAG, NAME, ...)                \
     if (FLAG) { constexpr bool NAME = true; __VA_ARGS__; } \

@@ -68,6 +68,8 @@ def test_workspace_sizes(L):
     assert b.bof4_workspace_bytes(b.OP_EM, 1 << 20, 64, b.METRIC_MSE) > 0
     assert b.bof4_workspace_bytes(b.OP_EM, 1 << 20, 64, 5) == 0
     assert b.bof4_workspace_bytes(b.OP_OPQ, 1 << 20, 48, 0) == 0
+    assert b.bof4_workspace_bytes(b.OP_OPQ, 1 << 20, 8192, 0) == 0
+    assert b.bof4_workspace_bytes(b.OP_OPQ, 1 << 20, 4096, 0) > 0
     assert b.bof4_workspace_bytes(9, 1 << 20, 64, 0) == 0
     small = b.bof4_workspace_bytes(b.OP_OPQ, 1 << 20, 64, 0)
     big = b.bof4_workspace_bytes(b.OP_OPQ, 1 << 24, 64, 0)

@@ -403,3 +403,83 @@ def test_mae_collecting_pass_choice_does_not_change_results(bof4):
             os.environ.pop("BOF4_MAE_COLLECT_PASS", None)
         else:
             os.environ["BOF4_MAE_COLLECT_PASS"] = old
+
+
+# --------------------------------------------------------------------------- blocks wider than a warp
+
+
+WIDE = [512, 1024, 2048, 4096]
+
+
+def wide_special(w, I):
+    """Plants, at warp-crossing positions of wide blocks: a tie of +max / -max whose first
+    occurrence sits in a later warp than ... the other sign (lower index must win), an all-zero
+    block and a constant block."""
+    w = w.clone()
+    B = w.numel() // I
+    assert B >= 5
+    w[0:I] = 0.0
+    blk = w[I:2 * I]
+    m = blk.abs().max() * 2
+    blk[I - 7] = m          # last warp of the block
+    blk[I // 2 + 3] = -m    # an earlier warp: the negative one comes first
+    blk = w[2 * I:3 * I]
+    m = blk.abs().max() * 2
+    blk[5] = m              # first warp
+    blk[I - 1] = -m
+    w[3 * I:4 * I] = 0.0123
+    return w
+
+
+@pytest.mark.parametrize("I", WIDE)
+@pytest.mark.parametrize("norm", [0, 1])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_wide_blocks_quantize_dequantize_bit_exact(bof4, I, norm, dtype):
+    n = 8192 * 5 + 4096 * 3     # several CTA rows and a partial one
+    w = wide_special(make_weights(n, dtype, 400 + I + norm), I)
+    codes, scales = bof4.bof4_quantize(w.cuda(), I, norm, LV_BOF4S)
+    out = bof4.bof4_dequantize(codes, scales, I, LV_BOF4S, bof4.BF16)
+    rc, rs = oracle.quantize(w, I, norm, LV_BOF4S)
+    assert np.array_equal(scales_f32(scales).view(np.uint32), rs.view(np.uint32))
+    assert np.array_equal(codes.cpu().numpy(), rc)
+    assert np.array_equal(bits16(out), oracle.f32_to_bf16_bits(oracle.dequantize(rc, rs, I, LV_BOF4S)))
+
+
+@pytest.mark.parametrize("I", WIDE)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_wide_blocks_opq_bit_exact(bof4, I, dtype):
+    n = 8192 * 6 + 4096
+    w = workloads.inject_outliers(make_weights(n, dtype, 500 + I, "gauss"), 0.02, 2e-3, 10.0, 40.0, 17)
+    w = wide_special(w, I)
+    w[8192 * 2 + 100: 8192 * 2 + 140] = torch.tensor([(-1.0) ** k * (3.0 + k) for k in range(40)]).to(dtype)
+    tau = float(np.float32(bof4.bof4_opq_threshold(0.95, I)))
+    clean, ridx, rval, rk, rc, rs, rout = _opq_reference(w, I, 1, LV_BOF4S, tau)
+    codes, scales, idx, val, cnt = bof4.bof4_quantize_opq(w.cuda(), I, 1, LV_BOF4S, tau, n)
+    out = bof4.bof4_dequantize(codes, scales, I, LV_BOF4S, bof4.BF16, (idx, val, cnt))
+    k = int(cnt.item())
+    assert k == rk and rk > 40
+    assert np.array_equal(idx[:k].cpu().numpy().astype(np.int64), ridx)
+    assert np.array_equal(bits16(val[:k]), rval)
+    assert np.array_equal(codes.cpu().numpy(), rc)
+    assert np.array_equal(scales_f32(scales), rs)
+    assert np.array_equal(bits16(out), oracle.f32_to_bf16_bits(rout))
+    c2, idx2, val2, cnt2 = bof4.opq_split(w.cuda(), I, tau, n)
+    assert int(cnt2.item()) == rk
+    assert np.array_equal(c2.float().cpu().numpy().view(np.uint32), clean.view(np.uint32))
+
+
+@pytest.mark.parametrize("I", WIDE)
+@pytest.mark.parametrize("norm", [0, 1])
+def test_wide_blocks_em_steps_match_oracle(bof4, I, norm):
+    n = 16384 * 3 + 8192
+    w = wide_special(make_weights(n, torch.bfloat16, 600 + I), I)
+    wd = w.cuda()
+    _check_stats(bof4.bof4_em_step([wd], I, norm, bof4.METRIC_MSE, LV_INIT),
+                 oracle.em_accumulate_mse(w, I, norm, LV_INIT))
+    _check_mae_stats(bof4.bof4_em_step([wd], I, norm, bof4.METRIC_MAE, LV_INIT),
+                     oracle.em_accumulate_mae(w, I, norm, LV_INIT), LV_INIT)
+    mask = workloads.FIXED_BOF4S if norm else workloads.FIXED_BOF4
+    cb, log = bof4.bof4_fit_codebook([wd], I, norm, bof4.METRIC_MSE, LV_INIT, mask, 4)
+    rcb, rlog = oracle.fit(w, I, norm, oracle.METRIC_MSE, LV_INIT, mask, 4)
+    np.testing.assert_allclose(cb.cpu().numpy(), rcb, rtol=RTOL, atol=1e-7)
+    np.testing.assert_allclose(log.cpu().numpy(), rlog, rtol=RTOL)
