@@ -358,9 +358,11 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
-# dram bytes per launch of the dominant kernel from the committed ncu capture (profiles/), or
-# None while the kernel has changed since the counters were taken
-TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant component's data-carrying kernels
+# per step, from the committed ncu captures (profiles/); None for a component whose kernels have
+# changed since the counters were taken
+TRAFFIC = {"em_mae": 406.9e6,   # max-|w| pass 137.8 MB + first pass 134.8 MB + collecting pass 134.4 MB
+           "em_mse": 138.3e6}
 
 
 # --------------------------------------------------------------------------- CPU arm (oracle)
