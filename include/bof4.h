@@ -60,6 +60,10 @@ extern "C" {
 
 #define BOF4_METRIC_MSE 0 /* weighted-mean centroid   (Eq. 6) */
 #define BOF4_METRIC_MAE 1 /* weighted-median centroid (Eq. 8) */
+/* The same two criteria on the NORMALISED weights (App. D): every sample has weight 1, i.e. the
+ * plain mean / plain median of textbook Lloyd, and the error is measured on x, not on w. */
+#define BOF4_METRIC_MSE_NORMALIZED 2
+#define BOF4_METRIC_MAE_NORMALIZED 3
 
 #define BOF4_OP_EM 0  /* bof4_em_step / bof4_fit_codebook workspace */
 #define BOF4_OP_OPQ 1 /* opq_split / bof4_quantize_opq workspace    */
@@ -76,6 +80,7 @@ extern "C" {
  *     median[l] = weighted median of the members (the first sample, in ascending order, whose
  *     cumulative weight reaches half of s0[l]); the input level where s0[l] == 0,
  *     err_sum = sum over all weights of |w - m * xhat[code]|.
+ * For the normalised-domain metrics m^2 and |m| are replaced by 1 and w by x in these sums.
  * count[l] is the number of members of region l, n_total the number of weights seen.
  * For MSE median[l] is the centroid s1[l]/s0[l] rounded to fp32 (input level where s0[l] == 0).
  */

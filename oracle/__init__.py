@@ -25,6 +25,7 @@ _LIB = os.path.join(_HERE, "libbof4_oracle.so")
 _lib = None
 
 METRIC_MSE, METRIC_MAE = 0, 1
+METRIC_MSE_NORMDOM, METRIC_MAE_NORMDOM = 2, 3  # App. D: errors of the normalised weights
 NORM_ABS, NORM_SIGNED = 0, 1
 
 
@@ -142,8 +143,8 @@ def bf16_bits_to_f32(h: np.ndarray) -> np.ndarray:
     return out.reshape(h.shape)
 
 
-def em_accumulate_mse(w, I: int, norm: int, xhat):
-    """-> dict(s1[16] f64, s0[16] f64, count[16] u64, err_sum f64, n)."""
+def em_accumulate_mse(w, I: int, norm: int, xhat, normdom: bool = False):
+    """-> dict(s1[16] f64, s0[16] f64, count[16] u64, err_sum f64, n).  normdom: App. D variant."""
     a = as_f32(w)
     _check(a.size, I)
     lv = _levels(xhat)
@@ -151,13 +152,13 @@ def em_accumulate_mse(w, I: int, norm: int, xhat):
     s0 = np.zeros(16, np.float64)
     cnt = np.zeros(16, np.uint64)
     err = ctypes.c_double(0.0)
-    _load().orc_em_accumulate_mse(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv),
-                                  _p(s1), _p(s0), _p(cnt), ctypes.byref(err))
+    fn = _load().orc_em_accumulate_mse_normdom if normdom else _load().orc_em_accumulate_mse
+    fn(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv), _p(s1), _p(s0), _p(cnt), ctypes.byref(err))
     return dict(s1=s1, s0=s0, count=cnt, err_sum=err.value, n=a.size)
 
 
-def em_accumulate_mae(w, I: int, norm: int, xhat):
-    """-> dict(median[16] f32, wsum[16] f64, count[16] u64, err_sum f64, n)."""
+def em_accumulate_mae(w, I: int, norm: int, xhat, normdom: bool = False):
+    """-> dict(median[16] f32, wsum[16] f64, count[16] u64, err_sum f64, n).  normdom: App. D variant."""
     a = as_f32(w)
     _check(a.size, I)
     lv = _levels(xhat)
@@ -165,8 +166,8 @@ def em_accumulate_mae(w, I: int, norm: int, xhat):
     ws = np.zeros(16, np.float64)
     cnt = np.zeros(16, np.uint64)
     err = ctypes.c_double(0.0)
-    _load().orc_em_accumulate_mae(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv),
-                                  _p(med), _p(ws), _p(cnt), ctypes.byref(err))
+    fn = _load().orc_em_accumulate_mae_normdom if normdom else _load().orc_em_accumulate_mae
+    fn(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv), _p(med), _p(ws), _p(cnt), ctypes.byref(err))
     return dict(median=med, wsum=ws, count=cnt, err_sum=err.value, n=a.size)
 
 

@@ -171,8 +171,25 @@ void orc_dequantize(const uint8_t *codes, const float *scales, int64_t n, int I,
 /* One expectation + accumulation pass with the levels held fixed (Eq. 6 and the first line
  * of the un-normalised-domain error, App. B.3):
  *   s1[l] = sum m^2 x,  s0[l] = sum m^2,  cnt[l] = K_l,  err = sum (w - m xhat(l))^2. */
+static void em_accumulate_mse_impl(const float *w, int64_t n, int I, int norm, const float *xhat,
+                                   int unit, double *s1, double *s0, uint64_t *cnt, double *err);
+
 void orc_em_accumulate_mse(const float *w, int64_t n, int I, int norm, const float *xhat,
                            double *s1, double *s0, uint64_t *cnt, double *err)
+{
+    em_accumulate_mse_impl(w, n, I, norm, xhat, 0, s1, s0, cnt, err);
+}
+
+/* The same pass for the quantisation error of the NORMALISED weights (App. D, the plain-mean
+ * centroid): every sample has weight 1, s1[l] = sum x, s0[l] = K_l, err = sum (x - xhat(l))^2. */
+void orc_em_accumulate_mse_normdom(const float *w, int64_t n, int I, int norm, const float *xhat,
+                                   double *s1, double *s0, uint64_t *cnt, double *err)
+{
+    em_accumulate_mse_impl(w, n, I, norm, xhat, 1, s1, s0, cnt, err);
+}
+
+static void em_accumulate_mse_impl(const float *w, int64_t n, int I, int norm, const float *xhat,
+                                   int unit, double *s1, double *s0, uint64_t *cnt, double *err)
 {
     float xi[L - 1];
     orc_thresholds(xhat, xi);
@@ -197,11 +214,19 @@ void orc_em_accumulate_mse(const float *w, int64_t n, int I, int norm, const flo
             for (int i = 0; i < I; ++i) {
                 float x = normalise(wb[i], m);
                 int c = region_of(x, xi);
-                a1[c] += md * md * (double)x;
-                a0[c] += md * md;
-                ac[c] += 1;
-                double d = (double)wb[i] - md * (double)xhat[c];
-                e += d * d;
+                if (unit) {
+                    a1[c] += (double)x;
+                    a0[c] += 1.0;
+                    ac[c] += 1;
+                    double d = (double)x - (double)xhat[c];
+                    e += d * d;
+                } else {
+                    a1[c] += md * md * (double)x;
+                    a0[c] += md * md;
+                    ac[c] += 1;
+                    double d = (double)wb[i] - md * (double)xhat[c];
+                    e += d * d;
+                }
             }
         }
         pe[ch] = e;
@@ -244,8 +269,24 @@ static int cmp_member(const void *p, const void *q)
  * the minimiser of f(xh) = sum a_k |x_k - xh| (objective of App. B.3, "MAE Optimization").
  *   med[l]  = that sample (unchanged input level when the region's total weight is 0),
  *   wsum[l] = total weight of the region, cnt[l] = K_l, err = sum |w - m xhat(l)|. */
+static void em_accumulate_mae_impl(const float *w, int64_t n, int I, int norm, const float *xhat,
+                                   int unit, float *med, double *wsum, uint64_t *cnt, double *err);
+
 void orc_em_accumulate_mae(const float *w, int64_t n, int I, int norm, const float *xhat,
                            float *med, double *wsum, uint64_t *cnt, double *err)
+{
+    em_accumulate_mae_impl(w, n, I, norm, xhat, 0, med, wsum, cnt, err);
+}
+
+/* Normalised-domain variant (App. D, the plain median): all weights 1, err = sum |x - xhat(l)|. */
+void orc_em_accumulate_mae_normdom(const float *w, int64_t n, int I, int norm, const float *xhat,
+                                   float *med, double *wsum, uint64_t *cnt, double *err)
+{
+    em_accumulate_mae_impl(w, n, I, norm, xhat, 1, med, wsum, cnt, err);
+}
+
+static void em_accumulate_mae_impl(const float *w, int64_t n, int I, int norm, const float *xhat,
+                                   int unit, float *med, double *wsum, uint64_t *cnt, double *err)
 {
     float xi[L - 1];
     orc_thresholds(xhat, xi);
@@ -266,7 +307,8 @@ void orc_em_accumulate_mae(const float *w, int64_t n, int I, int norm, const flo
             xs[b * I + i] = x;
             code[b * I + i] = (uint8_t)c;
             cnt[c] += 1;
-            e += fabs((double)wb[i] - (double)m * (double)xhat[c]);
+            e += unit ? fabs((double)x - (double)xhat[c])
+                      : fabs((double)wb[i] - (double)m * (double)xhat[c]);
         }
     }
     *err = e;
@@ -281,7 +323,7 @@ void orc_em_accumulate_mae(const float *w, int64_t n, int I, int norm, const flo
         for (int64_t j = 0; j < n; ++j)
             if (code[j] == l) {
                 mem[k].x = xs[j];
-                mem[k].a = fabsf(ms[j / I]);
+                mem[k].a = unit ? 1.0f : fabsf(ms[j / I]);
                 ++k;
             }
         qsort(mem, (size_t)k, sizeof(member_t), cmp_member);
@@ -311,23 +353,24 @@ void orc_em_accumulate_mae(const float *w, int64_t n, int I, int norm, const flo
 /* Lloyd iteration of Sec. 3.2: `iters` times { thresholds from the current levels, assign,
  * recompute every level that is not fixed (bit l of fixed_mask) }.  err_log[t] is the mean
  * error (MSE or MAE over all n weights, un-normalised domain) of the levels that ENTER
- * iteration t.  metric: 0 = MSE (Eq. 6), 1 = MAE (Eq. 8). */
+ * iteration t.  metric: 0 = MSE (Eq. 6), 1 = MAE (Eq. 8); 2 / 3 = the same criteria on the
+ * normalised weights (App. D: plain mean / plain median, error measured on x). */
 void orc_fit(const float *w, int64_t n, int I, int norm, int metric, float *xhat,
              uint32_t fixed_mask, int iters, double *err_log)
 {
     for (int t = 0; t < iters; ++t) {
         uint64_t cnt[L];
         double err;
-        if (metric == 0) {
+        if (metric == 0 || metric == 2) {
             double s1[L], s0[L];
-            orc_em_accumulate_mse(w, n, I, norm, xhat, s1, s0, cnt, &err);
+            em_accumulate_mse_impl(w, n, I, norm, xhat, metric == 2, s1, s0, cnt, &err);
             for (int l = 0; l < L; ++l)
                 if (!((fixed_mask >> l) & 1u) && s0[l] > 0.0)
                     xhat[l] = (float)(s1[l] / s0[l]);
         } else {
             float med[L];
             double ws[L];
-            orc_em_accumulate_mae(w, n, I, norm, xhat, med, ws, cnt, &err);
+            em_accumulate_mae_impl(w, n, I, norm, xhat, metric == 3, med, ws, cnt, &err);
             for (int l = 0; l < L; ++l)
                 if (!((fixed_mask >> l) & 1u) && ws[l] > 0.0)
                     xhat[l] = med[l];

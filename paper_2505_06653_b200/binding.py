@@ -21,6 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libbof4.so")
 F32, BF16 = 0, 1
 NORM_ABS, NORM_SIGNED = 0, 1
 METRIC_MSE, METRIC_MAE = 0, 1
+METRIC_MSE_NORMALIZED, METRIC_MAE_NORMALIZED = 2, 3  # App. D: errors of the normalised weights
 OP_EM, OP_OPQ = 0, 1
 LEVELS = 16
 

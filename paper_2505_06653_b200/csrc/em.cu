@@ -159,6 +159,7 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
     const bool lut_ok = s_multi == 0;
 
     const int64_t total_rows = T.row_end[T.count - 1];
+    const bool unit = T.unit != 0;
     const uint32_t lut_base = lut_lane_base(s_lut, lane), tid_off = tid * 8;
     double w2sum = 0.0;
     int t_cur = 0;
@@ -238,17 +239,25 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
         float gmax;
         const float m = block_constant<I, SIGNED>(v, gmax, &s_wide);
         const bool safe = row_is_safe(gmax, ok);
-        float2 sq = make_float2(0.0f, 0.0f);
-#pragma unroll
-        for (int k = 0; k < kLaneW / 2; ++k) {
-            const float2 vv = make_float2(v[2 * k], v[2 * k + 1]);
-            sq = __ffma2_rn(vv, vv, sq);
-        }
-        w2sum += (double)(sq.x + sq.y);  // lanes beyond the end hold zeros
         float x[kLaneW];
         normalise16<false>(v, m, safe && DT::code == BF16::code, x);
+        float2 sq = make_float2(0.0f, 0.0f);
+        if (unit) {  // App. D variant: the error is measured on x
+#pragma unroll
+            for (int k = 0; k < kLaneW / 2; ++k) {
+                const float2 vv = make_float2(x[2 * k], x[2 * k + 1]);
+                sq = __ffma2_rn(vv, vv, sq);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < kLaneW / 2; ++k) {
+                const float2 vv = make_float2(v[2 * k], v[2 * k + 1]);
+                sq = __ffma2_rn(vv, vv, sq);
+            }
+        }
+        if (ok) w2sum += (double)(sq.x + sq.y);
         if (ok) {
-            const float m2 = m * m;
+            const float m2 = unit ? 1.0f : m * m;
             const float2 mm = make_float2(m2, m2);
             if (lut_ok && safe) {
 #pragma unroll
@@ -346,7 +355,7 @@ int check_em(const char* fn, EmArgs& a, const void* d_codebook, void* d_ws, size
         return BOF4_ERR_DTYPE;
     }
     if ((a.norm != BOF4_NORM_ABS && a.norm != BOF4_NORM_SIGNED) ||
-        (a.metric != BOF4_METRIC_MSE && a.metric != BOF4_METRIC_MAE)) {
+        a.metric < BOF4_METRIC_MSE || a.metric > BOF4_METRIC_MAE_NORMALIZED) {
         set_error("%s: bad norm or metric", fn);
         return BOF4_ERR_INVALID_ARG;
     }
@@ -459,7 +468,7 @@ extern "C" int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_te
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partials = static_cast<double*>(d_ws);
-    if (metric == BOF4_METRIC_MSE) {
+    if (metric == BOF4_METRIC_MSE || metric == BOF4_METRIC_MSE_NORMALIZED) {
         if ((rc = reset_ticket(partials, st))) return rc;
         MseTail tail{};
         tail.stats = d_stats;
@@ -484,7 +493,7 @@ extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partials = static_cast<double*>(d_ws);
-    if (metric == BOF4_METRIC_MSE) {
+    if (metric == BOF4_METRIC_MSE || metric == BOF4_METRIC_MSE_NORMALIZED) {
         if (iters > 0 && (rc = reset_ticket(partials, st))) return rc;
         for (int t = 0; t < iters; ++t) {
             MseTail tail{};

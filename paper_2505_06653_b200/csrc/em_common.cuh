@@ -16,6 +16,7 @@ struct EmTensors {
     int count;
     int accumulate;  // 0: this launch overwrites the partial records, 1: adds to them
     int last;        // 1: no further launch of this pass follows
+    int unit;        // 1: normalised-domain variant (App. D): all sample weights are 1, errors on x
 };
 
 struct EmArgs {
@@ -37,6 +38,7 @@ int for_each_tensor_chunk(const EmArgs& a, int row, Fire fire, int* n_calls)
     EmTensors T;
     T.count = 0;
     T.accumulate = 0;
+    T.unit = (a.metric >= 2) ? 1 : 0;
     int64_t rows = 0;
     int calls = 0, nonempty = 0;
     for (int t = 0; t < a.n_tensors; ++t) nonempty += a.h_n[t] > 0;

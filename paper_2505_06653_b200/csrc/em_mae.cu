@@ -217,7 +217,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         normalise16<false>(v, m, safe && DT::code == BF16::code, x);
         const bool use_lut = lut_ok && safe;
         if (!ok) continue;
-        const uint32_t a = fixed_weight(m, max_bits);
+        const uint32_t a = T.unit ? 1u : fixed_weight(m, max_bits);  // App. D variant: plain median
         float e = 0.0f;
 #pragma unroll
         for (int k = 0; k < kLaneW; ++k) {
@@ -228,11 +228,12 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
             } else {
                 c = (uint32_t)region_of(x[k], s_xi);
             }
-            if (FIRST) e += fabsf(fmaf(-m, s_lv[c], v[k]));
+            if (FIRST) e += T.unit ? fabsf(x[k] - s_lv[c]) : fabsf(fmaf(-m, s_lv[c], v[k]));
             const uint4 L = s_lvl[c];
             const uint32_t rel = order_key(x[k]) - L.x;
             const uint32_t top = L.z & 0xffu, sh = (L.z >> 8) & 0xffu, mask = L.z >> 16;
-            if (L.w && (uint32_t)((unsigned long long)rel >> top) == L.y) {
+            // in the first pass no digit has been chosen: every member of an active level takes part
+            if (L.w && (FIRST || (uint32_t)((unsigned long long)rel >> top) == L.y)) {
                 const uint32_t bin = c * kMaeBins + ((rel >> sh) & mask);
                 const uint32_t old = atomicAdd(&s_lo[bin], a);
                 if (old + a < old) atomicAdd(&s_hi[bin], 1u);
@@ -440,7 +441,8 @@ mae_resolve_kernel(MaeWs W)
 
 __global__ void __launch_bounds__(256)
 mae_finalize_kernel(MaeWs W, int n_records, int64_t n_total, const float* levels_in, float* levels_out,
-                    uint32_t skip_mask, bof4_em_stats* __restrict__ stats, double* __restrict__ err_slot)
+                    uint32_t skip_mask, bof4_em_stats* __restrict__ stats, double* __restrict__ err_slot,
+                    int unit)
 {
     __shared__ double s_part[8];
     const MaeState* S = W.state;
@@ -459,7 +461,7 @@ mae_finalize_kernel(MaeWs W, int n_records, int64_t n_total, const float* levels
         if (stats) {
             const int emax = max((int)(S->max_bits >> 23), 1);
             stats->s1[l] = 0.0;
-            stats->s0[l] = ldexp((double)total, emax - 157);  // undo the fixed-point scale
+            stats->s0[l] = unit ? (double)total : ldexp((double)total, emax - 157);  // undo the fixed-point scale
             stats->count[l] = S->count[l];
             stats->median[l] = med;
         }
@@ -570,7 +572,7 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
         BOF4_CUDA_TRY(cudaGetLastError());
     }
     mae_finalize_kernel<<<1, 256, 0, st>>>(W, kEmGrid, a.n_total, d_levels_in, d_levels_out, skip_mask,
-                                           d_stats, d_err_slot);
+                                           d_stats, d_err_slot, a.metric >= 2 ? 1 : 0);
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }

@@ -483,3 +483,32 @@ def test_wide_blocks_em_steps_match_oracle(bof4, I, norm):
     rcb, rlog = oracle.fit(w, I, norm, oracle.METRIC_MSE, LV_INIT, mask, 4)
     np.testing.assert_allclose(cb.cpu().numpy(), rcb, rtol=RTOL, atol=1e-7)
     np.testing.assert_allclose(log.cpu().numpy(), rlog, rtol=RTOL)
+
+
+# --------------------------------------------------------------------------- App. D variants
+
+
+@pytest.mark.parametrize("I", [64, 256, 2048])
+@pytest.mark.parametrize("norm", [0, 1])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_normalised_domain_steps_match_oracle(bof4, I, norm, dtype):
+    """Textbook Lloyd on the normalised weights (unit sample weights, errors on x)."""
+    n = 16384 * 2 + 4096
+    # blocks of very different scale, so that the weighting matters
+    g = torch.Generator().manual_seed(700 + I)
+    scale = torch.rand(n // I, 1, generator=g) * 3 + 0.01
+    w = (torch.randn(n // I, I, generator=g) * scale).reshape(-1).to(dtype)
+    wd = w.cuda()
+    got = bof4.bof4_em_step([wd], I, norm, bof4.METRIC_MSE_NORMALIZED, LV_INIT)
+    ref = oracle.em_accumulate_mse(w, I, norm, LV_INIT, normdom=True)
+    _check_stats(got, ref)
+    assert np.array_equal(got["s0"], ref["count"].astype(np.float64))   # unit weights: exact
+    got = bof4.bof4_em_step([wd], I, norm, bof4.METRIC_MAE_NORMALIZED, LV_INIT)
+    ref = oracle.em_accumulate_mae(w, I, norm, LV_INIT, normdom=True)
+    _check_mae_stats(got, ref, LV_INIT)
+    mask = workloads.FIXED_BOF4S if norm else workloads.FIXED_BOF4
+    for metric in (bof4.METRIC_MSE_NORMALIZED, bof4.METRIC_MAE_NORMALIZED):
+        cb, log = bof4.bof4_fit_codebook([wd], I, norm, metric, LV_INIT, mask, 3)
+        rcb, rlog = oracle.fit(w, I, norm, metric, LV_INIT, mask, 3)
+        np.testing.assert_allclose(cb.cpu().numpy(), rcb, rtol=RTOL, atol=1e-7)
+        np.testing.assert_allclose(log.cpu().numpy(), rlog, rtol=RTOL)

@@ -491,3 +491,56 @@ def test_opq_zero_variance_block_literal_rule():
     assert k == 64  # sigma_b = 0: every non-zero element exceeds the threshold
     _, idx, _, k = oracle.opq_split(np.zeros(64, np.float32), 64, 3.0)
     assert k == 0
+
+
+# --------------------------------------------------------------------------- App. D variants
+
+
+def _normalised(w, I, signed):
+    """x = w / m by its definition, in numpy (independent of the oracle's code)."""
+    wb = w.reshape(-1, I)
+    j = np.abs(wb).argmax(1)
+    m = wb[np.arange(wb.shape[0]), j] if signed else np.abs(wb).max(1)
+    return (wb / m[:, None]).astype(np.float32).reshape(-1)
+
+
+@pytest.mark.parametrize("norm,signed", [(ABS, False), (SGN, True)])
+def test_normalised_domain_mse_is_library_kmeans_on_x(norm, signed):
+    """Minimising the error of the normalised weights is textbook Lloyd on x (App. D, the
+    plain-mean centroid): a library k-means on x = w / m must give the same levels, also for
+    blocks of very different scale (where the BOF4 centroid differs)."""
+    from sklearn.cluster import KMeans
+    g = np.random.default_rng(9)
+    w = (g.standard_normal((400, 64)) * g.uniform(0.01, 3.0, (400, 1))).astype(np.float32).reshape(-1)
+    init = np.array(workloads.init_levels_linspace(), np.float32)
+    T = 3
+    lv, log = oracle.fit(w, 64, norm, oracle.METRIC_MSE_NORMDOM, init, 0, T)
+    x = _normalised(w, 64, signed).astype(np.float64)
+    km = KMeans(n_clusters=16, init=init.astype(np.float64).reshape(-1, 1), n_init=1, max_iter=T,
+                tol=0.0, algorithm="lloyd").fit(x.reshape(-1, 1))
+    assert np.allclose(lv, km.cluster_centers_.reshape(-1), rtol=0, atol=2e-6)
+    # the logged error is the mean squared error of x under the entering levels
+    xi = oracle.thresholds(init)
+    code = (xi[None, :] <= x[:, None].astype(np.float32)).sum(1)
+    assert np.isclose(log[0], np.mean((x - init[code]) ** 2), rtol=1e-9)
+    # and it differs from the BOF4 centroid on such data
+    lv_bof, _ = oracle.fit(w, 64, norm, MSE, init, 0, T)
+    assert np.abs(lv_bof - lv).max() > 1e-3
+
+
+def test_normalised_domain_mae_is_the_plain_median_of_x():
+    g = np.random.default_rng(10)
+    w = (g.standard_normal((300, 32)) * g.uniform(0.01, 3.0, (300, 1))).astype(np.float32).reshape(-1)
+    init = np.array(workloads.init_levels_linspace(), np.float32)
+    st = oracle.em_accumulate_mae(w, 32, SGN, init, normdom=True)
+    x = _normalised(w, 32, True)
+    xi = oracle.thresholds(init)
+    code = (xi[None, :] <= x[:, None]).sum(1)
+    err = 0.0
+    for l in range(16):
+        mem = x[code == l]
+        assert st["count"][l] == mem.size and st["wsum"][l] == mem.size
+        if mem.size:
+            assert st["median"][l] == np.quantile(mem, 0.5, method="inverted_cdf")
+            err += np.abs(mem.astype(np.float64) - float(init[l])).sum()
+    assert np.isclose(st["err_sum"], err, rtol=1e-9)
