@@ -110,7 +110,7 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, fake, ws, 1 << 40, None) == -2
     ns[0] = 128
     assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, fake, ws, 8, None) == -4
-    assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 3, fake, fake, ws, 1 << 40, None) == -1
+    assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 4, fake, fake, ws, 1 << 40, None) == -1
     assert L.bof4_em_step(ptrs, ns, 1, 7, 64, 0, 0, fake, fake, ws, 1 << 40, None) == -3
     assert L.bof4_fit_codebook(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, 0, -1, None, ws, 1 << 40, None) == -1
     assert L.bof4_fit_codebook(ptrs, ns, 1, b.BF16, 64, 0, 0, None, 0, 1, None, ws, 1 << 40, None) == -1
