@@ -142,3 +142,27 @@ def test_config5_layer_on_reduced_rows(bof4):
         assert np.array_equal(bits16(out), oracle.f32_to_bf16_bits(rout))
         frac = k / n
         assert 2e-4 < frac < 3e-3   # Gaussian tail beyond tau plus the injected 1e-4
+
+
+def test_config5_largest_matrix_full_size(bof4):
+    """The 28672 x 8192 matrix of a 70B-shaped layer at full size (2.3e8 weights, 459 chunks of
+    the ordered compaction): fused OPQ quantise and dequantise against the oracle."""
+    r, c = workloads.llama70b_layer_shapes()[4]
+    s = 4_000_000 + 4
+    w = workloads.gaussian(r * c, 0.015, s, torch.bfloat16)
+    w = workloads.inject_outliers(w, 0.015, 1e-4, 10.0, 40.0, s + 8)
+    n = w.numel()
+    tau = float(np.float32(bof4.bof4_opq_threshold(0.95, 64)))
+    cap = n // 256
+    codes, scales, idx, val, cnt = bof4.bof4_quantize_opq(w.cuda(), 64, bof4.NORM_SIGNED, LV0, tau, cap)
+    out = bof4.bof4_dequantize(codes, scales, 64, LV0, bof4.BF16, (idx, val, cnt))
+    clean, ridx, rval, rk = oracle.opq_split(w, 64, tau)
+    k = int(cnt.item())
+    assert k == rk and k <= cap
+    assert np.array_equal(idx[:k].cpu().numpy().astype(np.int64), ridx)
+    assert np.array_equal(bits16(val[:k]), rval)
+    rc, rs = oracle.quantize(clean, 64, oracle.NORM_SIGNED, LV0)
+    assert np.array_equal(codes.cpu().numpy(), rc)
+    assert np.array_equal(scales.float().cpu().numpy(), rs)
+    rout = oracle.opq_restore(oracle.dequantize(rc, rs, 64, LV0), ridx, rval)
+    assert np.array_equal(bits16(out), oracle.f32_to_bf16_bits(rout))
