@@ -249,7 +249,7 @@ def run_gpu(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     dist = None
-    if world > 1:
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:  # launched by torch.distributed.run
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
         dist.barrier()

@@ -512,3 +512,25 @@ def test_normalised_domain_steps_match_oracle(bof4, I, norm, dtype):
         rcb, rlog = oracle.fit(w, I, norm, metric, LV_INIT, mask, 3)
         np.testing.assert_allclose(cb.cpu().numpy(), rcb, rtol=RTOL, atol=1e-7)
         np.testing.assert_allclose(log.cpu().numpy(), rlog, rtol=RTOL)
+
+
+def test_calls_follow_the_callers_stream(bof4):
+    """Everything is enqueued on the stream handed in (here: torch's current stream, a side
+    stream), in order, without touching the default stream's work."""
+    I, n = 64, 8192 * 4
+    w = make_weights(n, torch.bfloat16, 55)
+    side = torch.cuda.Stream()
+    wd = w.cuda()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        cb, log = bof4.bof4_fit_codebook([wd], I, 1, bof4.METRIC_MSE, LV_INIT, workloads.FIXED_BOF4S, 3,
+                                         sync=False)
+        codes, scales = bof4.bof4_quantize(wd, I, 1, cb)          # consumes the fitted levels in order
+        out = bof4.bof4_dequantize(codes, scales, I, cb, bof4.BF16)
+    side.synchronize()
+    rcb, _ = oracle.fit(w, I, 1, oracle.METRIC_MSE, LV_INIT, workloads.FIXED_BOF4S, 3)
+    cbh = cb.cpu().numpy()
+    np.testing.assert_allclose(cbh, rcb, rtol=RTOL, atol=1e-7)
+    rc, rs = oracle.quantize(w, I, 1, cbh)
+    assert np.array_equal(codes.cpu().numpy(), rc)
+    assert np.array_equal(bits16(out), oracle.f32_to_bf16_bits(oracle.dequantize(rc, rs, I, cbh)))
