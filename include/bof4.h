@@ -210,6 +210,23 @@ BOF4_API int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int s
                     const void* d_out_val, const int64_t* d_n_out, int64_t capacity,
                     void* d_out, int out_dtype, void* stream);
 
+/*
+ * Data-free codebook for unit-variance Gaussian weights (Sec. 3.2 Eq. 5 / Eq. 7; App. B.2): `iters`
+ * Lloyd iterations in which every free level becomes the theoretical centroid of its region,
+ * a ratio (MSE) or root (MAE) of integrals over the absolute block maximum, evaluated by
+ * Simpson quadrature in fp64 on the device.  Thresholds are midpoints of adjacent levels.
+ *   block_size  any I >= 2 (the integrals only need I, not a power of two)
+ *   metric      BOF4_METRIC_MSE or BOF4_METRIC_MAE
+ *   d_codebook  in: starting levels (ascending), out: levels after `iters` iterations
+ *   fixed_mask  must fix level 15 (= 1) and, for BOF4_NORM_ABS, level 0 (= -1): the outermost
+ *               regions hold the point mass of the block maximum (App. B.2)
+ *   d_ws        256 bytes of device workspace, 256-byte aligned (the fp64 state between iterations)
+ * One small launch per iteration on `stream`; no host synchronisation.
+ */
+BOF4_API int bof4_theoretical_codebook(int block_size, int norm, int metric, float* d_codebook,
+                              uint32_t fixed_mask, int iters, void* d_ws, size_t ws_bytes,
+                              void* stream);
+
 /* ---- host helpers (no CUDA call) ---- */
 
 /* tau = F_M^{-1}(q) for unit-variance Gaussian weights, F_M(m) = (2 G(m) - 1)^I the CDF of the

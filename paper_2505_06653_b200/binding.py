@@ -30,7 +30,7 @@ MAE_LAUNCHES_PER_ITERATION = 10
 
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
-           "bof4_default_init", "bof4_last_error")
+           "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook")
 
 
 class Bof4Error(RuntimeError):
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
                                         vp, vp, i64, vp, vp, sz, vp]
         L.bof4_dequantize.restype = i32
         L.bof4_dequantize.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp, i64, vp, i32, vp]
+        L.bof4_theoretical_codebook.restype = i32
+        L.bof4_theoretical_codebook.argtypes = [i32, i32, i32, vp, ctypes.c_uint32, i32, vp, sz, vp]
         L.bof4_opq_threshold.restype = ctypes.c_double
         L.bof4_opq_threshold.argtypes = [ctypes.c_double, i32]
         L.bof4_default_init.restype = i32
@@ -208,6 +210,19 @@ def bof4_fit_codebook(weights, block_size: int, norm: int, metric: int, levels, 
     if sync:
         torch.cuda.current_stream(dev).synchronize()
     return cb, log[:iters]
+
+
+def bof4_theoretical_codebook(block_size: int, norm: int, metric: int, levels, fixed_mask: int,
+                              iters: int, device="cuda") -> torch.Tensor:
+    """Data-free Gaussian codebook: `iters` Lloyd iterations with theoretical centroids.
+    -> levels fp32[16] on the device."""
+    dev = torch.device(device)
+    cb = _codebook(levels, dev).clone()
+    ws = torch.empty(256, dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().bof4_theoretical_codebook(block_size, norm, metric, _ptr(cb), fixed_mask, iters,
+                                               _ptr(ws), ws.numel(), _stream()))
+    return cb
 
 
 # --------------------------------------------------------------------------- quantise / dequantise

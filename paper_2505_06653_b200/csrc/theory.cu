@@ -1,0 +1,161 @@
+// Data-free codebook design for Gaussian weights (Sec. 3.2 Eq. 5 and Eq. 7; App. B.2, "Simplified
+// Solution for Gaussian Network Weights" and "MAE Optimization"): Lloyd iterations whose
+// centroids are ratios (MSE) or roots (MAE) of one-dimensional integrals over the absolute
+// block maximum m, evaluated by Simpson quadrature in fp64.
+//
+// With g, G the pdf / cdf of N(0,1), the block maximum has density proportional to
+// (2G(m)-1)^(I-1) g(m) and, given m, the other normalised weights have cdf
+// (G(m x) - G(-m)) / (2G(m)-1) on (-1, 1).  For a region (lo, hi) inside [-1, 1]:
+//   MSE centroid = - INT m [g(m hi) - g(m lo)] c(m) dm / INT m^2 [G(m hi) - G(m lo)] c(m) dm,
+//   MAE centroid = the x with INT m [G(m x) - G(m lo)] c(m) dm = 1/2 INT m [G(m hi) - G(m lo)] c(m) dm,
+// c(m) = (2G(m)-1)^(I-2) g(m).  (The printed boxed MSE formula has lost the leading minus sign of
+// the two equations it is derived from; it is restored here.)  The outermost regions carry the
+// point mass of the block maximum itself, so their levels must be fixed (-1 and 1 for absolute,
+// 1 for signed normalisation).
+#include <math.h>
+
+#include "common.cuh"
+
+namespace bof4 {
+
+constexpr int kThThreads = 512;
+constexpr int kThIntervals = 8192;  // Simpson intervals on m in [0, kThMax]
+constexpr double kThMax = 12.0;     // g(12) ~ 1e-32: the tail is far below fp64 resolution
+
+__device__ __forceinline__ double gauss_pdf(double x) { return 0.3989422804014326779 * exp(-0.5 * x * x); }
+// G(b) - G(a)
+__device__ __forceinline__ double gauss_mass(double a, double b)
+{
+    return 0.5 * (erf(b * 0.70710678118654752440) - erf(a * 0.70710678118654752440));
+}
+
+// Sum over the CTA, result in every thread.
+__device__ __forceinline__ double cta_sum(double v, double* s_red)
+{
+#pragma unroll
+    for (int off = 16; off; off >>= 1) v += __shfl_xor_sync(kFull, v, off);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double t = 0.0;
+    for (int k = 0; k < kThThreads / 32; ++k) t += s_red[k];
+    return t;
+}
+
+// Simpson weight of node q (0 .. kThIntervals) times the step, and its abscissa.
+__device__ __forceinline__ void node(int q, double& m, double& wq)
+{
+    const double h = kThMax / kThIntervals;
+    m = q * h;
+    wq = (q == 0 || q == kThIntervals) ? h / 3.0 : ((q & 1) ? 4.0 * h / 3.0 : 2.0 * h / 3.0);
+}
+
+// One Lloyd iteration: CTA l recomputes level l from the thresholds of levels_in.
+__global__ void __launch_bounds__(kThThreads)
+theory_step_kernel(const double* __restrict__ levels_in, double* __restrict__ levels_out, int I, int metric,
+                   uint32_t fixed_mask)
+{
+    __shared__ double s_red[kThThreads / 32];
+    const int l = blockIdx.x;
+    const double cur = levels_in[l];
+    if ((fixed_mask >> l) & 1u) {
+        if (threadIdx.x == 0) levels_out[l] = cur;
+        return;
+    }
+    double lo = (l > 0) ? 0.5 * (levels_in[l - 1] + cur) : -1.0;
+    double hi = (l < kLevels - 1) ? 0.5 * (cur + levels_in[l + 1]) : 1.0;
+    lo = fmin(fmax(lo, -1.0), 1.0);
+    hi = fmin(fmax(hi, -1.0), 1.0);
+    const double expo = (double)(I - 2);
+    if (metric == BOF4_METRIC_MSE) {
+        double num = 0.0, den = 0.0;
+        for (int q = threadIdx.x; q <= kThIntervals; q += kThThreads) {
+            double m, wq;
+            node(q, m, wq);
+            const double c = pow(erf(m * 0.70710678118654752440), expo) * gauss_pdf(m) * wq;
+            num -= m * (gauss_pdf(m * hi) - gauss_pdf(m * lo)) * c;
+            den += m * m * gauss_mass(m * lo, m * hi) * c;
+        }
+        num = cta_sum(num, s_red);
+        den = cta_sum(den, s_red);
+        if (threadIdx.x == 0) levels_out[l] = (den > 0.0) ? num / den : cur;
+    } else {
+        // weights m c(m) of the nodes this thread owns stay in registers during the bisection
+        constexpr int PER = kThIntervals / kThThreads + 1;
+        double mm[PER], wc[PER];
+        double full = 0.0;
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+            const int q = threadIdx.x + k * kThThreads;
+            double m = 0.0, wq = 0.0;
+            if (q <= kThIntervals) node(q, m, wq);
+            mm[k] = m;
+            wc[k] = (q <= kThIntervals) ? m * pow(erf(m * 0.70710678118654752440), expo) * gauss_pdf(m) * wq : 0.0;
+            full += wc[k] * gauss_mass(m * lo, m * hi);
+        }
+        const double half = 0.5 * cta_sum(full, s_red);
+        double a = lo, b = hi;
+        for (int it = 0; it < 60; ++it) {  // the mass below x grows with x: bisection
+            const double x = 0.5 * (a + b);
+            double part = 0.0;
+#pragma unroll
+            for (int k = 0; k < PER; ++k) part += wc[k] * gauss_mass(mm[k] * lo, mm[k] * x);
+            if (cta_sum(part, s_red) < half)
+                a = x;
+            else
+                b = x;
+        }
+        if (threadIdx.x == 0) levels_out[l] = (half > 0.0) ? 0.5 * (a + b) : cur;
+    }
+}
+
+__global__ void theory_load_kernel(const float* __restrict__ codebook, double* __restrict__ levels)
+{
+    if (threadIdx.x < kLevels) levels[threadIdx.x] = (double)codebook[threadIdx.x];
+}
+__global__ void theory_store_kernel(const double* __restrict__ levels, float* __restrict__ codebook)
+{
+    if (threadIdx.x < kLevels) codebook[threadIdx.x] = (float)levels[threadIdx.x];
+}
+
+}  // namespace bof4
+
+extern "C" int bof4_theoretical_codebook(int block_size, int norm, int metric, float* d_codebook,
+                                         uint32_t fixed_mask, int iters, void* d_ws, size_t ws_bytes,
+                                         void* stream)
+{
+    using namespace bof4;
+    if (block_size < 2 || block_size > (1 << 20)) {
+        set_error("bof4_theoretical_codebook: block_size must be in 2 ... 2^20");
+        return BOF4_ERR_SHAPE;
+    }
+    if ((norm != BOF4_NORM_ABS && norm != BOF4_NORM_SIGNED) ||
+        (metric != BOF4_METRIC_MSE && metric != BOF4_METRIC_MAE) || iters < 0 || !d_codebook) {
+        set_error("bof4_theoretical_codebook: bad norm, metric, iteration count or NULL codebook");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (!((fixed_mask >> 15) & 1u) || (norm == BOF4_NORM_ABS && !(fixed_mask & 1u))) {
+        set_error("bof4_theoretical_codebook: the outermost levels (1, and -1 for absolute normalisation) "
+                  "carry the point mass of the block maximum and must be fixed");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (!d_ws || ((uintptr_t)d_ws & 255u) || ws_bytes < 256) {
+        set_error("bof4_theoretical_codebook: workspace NULL, not 256-byte aligned, or smaller than 256 bytes");
+        return BOF4_ERR_WORKSPACE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double* a = static_cast<double*>(d_ws);
+    double* b = a + kLevels;
+    theory_load_kernel<<<1, 32, 0, st>>>(d_codebook, a);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    for (int t = 0; t < iters; ++t) {
+        theory_step_kernel<<<kLevels, kThThreads, 0, st>>>(a, b, block_size, metric, fixed_mask);
+        BOF4_CUDA_TRY(cudaGetLastError());
+        double* tmp = a;
+        a = b;
+        b = tmp;
+    }
+    theory_store_kernel<<<1, 32, 0, st>>>(a, d_codebook);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
+}

@@ -114,6 +114,13 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     assert L.bof4_em_step(ptrs, ns, 1, 7, 64, 0, 0, fake, fake, ws, 1 << 40, None) == -3
     assert L.bof4_fit_codebook(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, 0, -1, None, ws, 1 << 40, None) == -1
     assert L.bof4_fit_codebook(ptrs, ns, 1, b.BF16, 64, 0, 0, None, 0, 1, None, ws, 1 << 40, None) == -1
+    # theoretical codebook: the outermost levels must be fixed, metric MSE / MAE only
+    full = (1 << 0) | (1 << 7) | (1 << 15)
+    assert L.bof4_theoretical_codebook(64, 0, 0, fake, 1 << 15, 1, ws, 256, None) == -1   # -1 not fixed (abs)
+    assert L.bof4_theoretical_codebook(64, 1, 0, fake, 1 << 7, 1, ws, 256, None) == -1    # +1 not fixed
+    assert L.bof4_theoretical_codebook(64, 0, 2, fake, full, 1, ws, 256, None) == -1
+    assert L.bof4_theoretical_codebook(1, 0, 0, fake, full, 1, ws, 256, None) == -2
+    assert L.bof4_theoretical_codebook(64, 0, 0, fake, full, 1, ws, 8, None) == -4
 
 
 def test_binding_refuses_cpu_tensors(L):

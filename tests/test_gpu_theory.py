@@ -1,0 +1,62 @@
+"""The data-free (theoretical) codebook solver against the paper's printed codebooks and the
+oracle's independent quadrature."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle import theory
+
+pytestmark = pytest.mark.gpu
+
+GOLD = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+TAB8 = np.loadtxt(os.path.join(GOLD, "tab8_bof4_mse_emp_theo.txt"))
+TAB6 = np.loadtxt(os.path.join(GOLD, "tab6_levels_I64.txt"))
+FIX4, FIX4S = workloads.FIXED_BOF4, workloads.FIXED_BOF4S
+
+
+@pytest.fixture(scope="module")
+def bof4():
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2505_06653_b200 as m
+    assert torch.cuda.is_available()
+    return m
+
+
+def test_printed_theoretical_column_is_a_fixed_point(bof4):
+    """Tab. 8, theoretical column (BOF4, MSE, I = 64): one iteration must leave it in place."""
+    theo = TAB8[:, 2].astype(np.float32)
+    one = bof4.bof4_theoretical_codebook(64, bof4.NORM_ABS, bof4.METRIC_MSE, theo, FIX4, 1).cpu().numpy()
+    assert np.abs(one - theo).max() < 3e-7
+
+
+def test_converges_to_the_printed_theoretical_column(bof4):
+    lv = bof4.bof4_theoretical_codebook(64, bof4.NORM_ABS, bof4.METRIC_MSE,
+                                        workloads.init_levels_7_0_8(), FIX4, 1500).cpu().numpy()
+    assert np.abs(lv - TAB8[:, 2]).max() < 5e-6
+    assert lv[0] == -1 and lv[7] == 0 and lv[15] == 1
+
+
+def test_printed_mae_codebooks_are_fixed_points(bof4):
+    """Tab. 6, MAE columns (Monte-Carlo results): residual of one theoretical step within their noise."""
+    for norm, col, mask in ((bof4.NORM_ABS, 1, FIX4), (bof4.NORM_SIGNED, 3, FIX4S)):
+        start = TAB6[:, col].astype(np.float32)
+        one = bof4.bof4_theoretical_codebook(64, norm, bof4.METRIC_MAE, start, mask, 1).cpu().numpy()
+        assert np.abs(one - start).max() < 1.5e-4
+
+
+@pytest.mark.parametrize("I", [32, 100, 256, 2048])
+@pytest.mark.parametrize("signed", [False, True])
+@pytest.mark.parametrize("metric", ["mse", "mae"])
+def test_agrees_with_the_oracles_quadrature(bof4, I, signed, metric):
+    mask = FIX4S if signed else FIX4
+    start = workloads.init_levels_7_0_8()
+    ref = theory.lloyd(I, signed, metric, start, mask, 3, theory.GaussianBlockModel(I, m_max=12.0, points=24001))
+    got = bof4.bof4_theoretical_codebook(I, bof4.NORM_SIGNED if signed else bof4.NORM_ABS,
+                                         bof4.METRIC_MSE if metric == "mse" else bof4.METRIC_MAE,
+                                         start, mask, 3).cpu().numpy()
+    assert np.abs(got - ref).max() < 2e-6
+    assert np.all(np.diff(got) > 0)
