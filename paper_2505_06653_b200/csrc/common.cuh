@@ -393,14 +393,18 @@ __device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lu
                                           PayloadFn payload)
 {
     __shared__ uint2 s_ent[kLutBins];
+    __shared__ int s_bin[kLevels];  // bin of every threshold
     if (threadIdx.x == 0) *s_multi = 0;
+    if (threadIdx.x < kLevels - 1) {
+        int bj = (int)(__float_as_uint(lut_key(s_xi[threadIdx.x])) - kLutMagicBits);
+        s_bin[threadIdx.x] = bj < 0 ? 0 : (bj > kLutBins - 1 ? kLutBins - 1 : bj);
+    }
     __syncthreads();
     for (int b = threadIdx.x; b < kLutBins; b += blockDim.x) {
         int base = 0, inside = 0;
 #pragma unroll
         for (int j = 0; j < kLevels - 1; ++j) {
-            int bj = (int)(__float_as_uint(lut_key(s_xi[j])) - kLutMagicBits);
-            bj = bj < 0 ? 0 : (bj > kLutBins - 1 ? kLutBins - 1 : bj);
+            const int bj = s_bin[j];
             base += (bj < b) ? 1 : 0;
             inside += (bj == b) ? 1 : 0;
         }

@@ -49,28 +49,42 @@ struct MseTail {
 // Combines the per-CTA records in a fixed order (the order does not depend on which CTA runs
 // this) and performs the M step.  Called by all threads of one CTA.
 __device__ __forceinline__ void mse_combine(const double* partials, const MseTail& t, double* s_q,
-                                            double* s_corr)
+                                            double* s_corr, unsigned long long* s_stage)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    constexpr int PER = (kEmGrid + 31) / 32;  // records per lane; all loads are issued before any sum
-    for (int q = warp; q <= kRecW2; q += nwarps) {
-        const bool is_count = q >= kRecCnt && q < kRecW2;
-        unsigned long long raw[PER];
+    constexpr int NQ = kRecW2 + 1;            // quantities per record
+    constexpr int PER = (kEmGrid + 31) / 32;  // records per lane
+    // Stage all records in shared memory first: coalesced, independent loads (every thread has
+    // several in flight), instead of a chain of dependent L2 round trips per quantity.
+    const int total = t.n_records * NQ;
+    for (int i0 = 0; i0 < total; i0 += 8 * (int)blockDim.x) {
+        unsigned long long raw[8];
 #pragma unroll
-        for (int k = 0; k < PER; ++k) {
-            const int r = lane + 32 * k;
-            raw[k] = (r < t.n_records)
-                         ? __ldcg(reinterpret_cast<const unsigned long long*>(partials + (size_t)r * kEmRecordDoubles) + q)
-                         : 0ull;  // zero bits are also +0.0
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * (int)blockDim.x + (int)threadIdx.x;
+            raw[u] = (i < total) ? __ldcg(reinterpret_cast<const unsigned long long*>(partials) +
+                                          (size_t)(i / NQ) * kEmRecordDoubles + (i % NQ))
+                                 : 0ull;
         }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * (int)blockDim.x + (int)threadIdx.x;
+            if (i < total) s_stage[i] = raw[u];
+        }
+    }
+    __syncthreads();
+    for (int q = warp; q < NQ; q += nwarps) {
+        const bool is_count = q >= kRecCnt && q < kRecW2;
         double a = 0.0;
         unsigned long long c = 0;
 #pragma unroll
-        for (int k = 0; k < PER; ++k) {
+        for (int k = 0; k < PER; ++k) {  // fixed order: lane-strided, then the butterfly
+            const int r = lane + 32 * k;
+            const unsigned long long raw = (r < t.n_records) ? s_stage[r * NQ + q] : 0ull;  // zero bits = +0.0
             if (is_count)
-                c += raw[k];
+                c += raw;
             else
-                a += __longlong_as_double((long long)raw[k]);
+                a += __longlong_as_double((long long)raw);
         }
 #pragma unroll
         for (int off = 16; off; off >>= 1) {
@@ -113,12 +127,14 @@ __device__ __forceinline__ void mse_combine(const double* partials, const MseTai
     }
 }
 
-// Stand-alone combine (used when a pass launched no accumulation kernel at all).
+// Stand-alone combine, used when a pass launched no accumulation kernel at all: the records are
+// all zero then and one of them stands for the sum.
 __global__ void __launch_bounds__(1024)
 em_mse_finalize_kernel(const double* partials, const MseTail t)
 {
     __shared__ double s_q[kRecW2 + 1], s_corr[kLevels];
-    mse_combine(partials, t, s_q, s_corr);
+    __shared__ unsigned long long s_stage[kRecW2 + 1];  // the launcher passes a single (zero) record
+    mse_combine(partials, t, s_q, s_corr, s_stage);
 }
 
 template <class DT, int I, bool SIGNED, bool COUNT>
@@ -328,7 +344,8 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
         __syncthreads();
         if (s_last) {
             __threadfence();
-            mse_combine(partials, tail, s_q, s_corr);
+            // the accumulator columns are folded and no longer needed: reuse them as the staging area
+            mse_combine(partials, tail, s_q, s_corr, reinterpret_cast<unsigned long long*>(s_acc));
             if (tid == 0) *tail.ticket = 0u;
         }
     }
@@ -441,6 +458,7 @@ int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials,
     if (calls == 0) {
         BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));
         tail.enabled = 0;
+        tail.n_records = 1;
         em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, tail);
         BOF4_CUDA_TRY(cudaGetLastError());
     }
