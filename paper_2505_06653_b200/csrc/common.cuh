@@ -356,8 +356,13 @@ __device__ __forceinline__ int region_of(float x, const float* s_xi)
 constexpr int kLutBins = 257;
 constexpr uint32_t kLutMagicBits = 0x4B400000u;  // bits of 1.5 * 2^23
 constexpr float kLutMagic = 12583040.0f;         // 1.5 * 2^23 + 128
-constexpr int kLutRowBytes = 32 * 8;
-constexpr int kLutBytes = kLutBins * kLutRowBytes;
+// REP = number of lane columns per row: 32 (one per lane) or 16 (lanes L and L + 16 share a
+// column; an 8-byte read is served half a warp at a time, so this is conflict-free as well and
+// halves the table where shared memory is short).
+__host__ __device__ constexpr int lut_row_bytes(int rep) { return rep * 8; }
+__host__ __device__ constexpr int lut_bytes(int rep) { return kLutBins * rep * 8; }
+constexpr int kLutRowBytes = lut_row_bytes(32);
+constexpr int kLutBytes = lut_bytes(32);
 
 __device__ __forceinline__ float lut_key(float x) { return fmaf(x, 128.0f, kLutMagic); }
 __device__ __forceinline__ float2 lut_key2(float2 x)
@@ -369,17 +374,19 @@ __device__ __forceinline__ float2 lut_key2(float2 x)
 // kLutMagicBits + bin.  lut_base = lut_lane_base(table, lane): a 32-bit shared-memory address
 // with the magic folded in, so that the probe is one multiply-add and one 8-byte read.  The
 // table is constant while it is probed, hence the read may be scheduled freely.
+template <int REP = 32>
 __device__ __forceinline__ uint32_t lut_lane_base(const unsigned char* s_lut, int lane)
 {
-    return (uint32_t)__cvta_generic_to_shared(s_lut) + (uint32_t)lane * 8u -
-           kLutMagicBits * (uint32_t)kLutRowBytes;
+    return (uint32_t)__cvta_generic_to_shared(s_lut) + (uint32_t)(lane & (REP - 1)) * 8u -
+           kLutMagicBits * (uint32_t)lut_row_bytes(REP);
 }
+template <int REP = 32>
 __device__ __forceinline__ uint2 lut_probe(float key, uint32_t lut_base)
 {
     uint2 e;
     asm("ld.shared.v2.u32 {%0, %1}, [%2];"
         : "=r"(e.x), "=r"(e.y)
-        : "r"(__float_as_uint(key) * (uint32_t)kLutRowBytes + lut_base));
+        : "r"(__float_as_uint(key) * (uint32_t)lut_row_bytes(REP) + lut_base));
     return e;
 }
 
@@ -388,7 +395,7 @@ __device__ __forceinline__ uint2 lut_probe(float key, uint32_t lut_base)
 // Call with all threads of the CTA, then __syncthreads().  The entries are first computed once
 // per bin into the table's own first row slots and then replicated with one warp per row, so
 // that the replicating stores of a warp fall into 32 different lanes' columns (no conflicts).
-template <class PayloadFn>
+template <int REP = 32, class PayloadFn>
 __device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lut, int* s_multi,
                                           PayloadFn payload)
 {
@@ -412,8 +419,8 @@ __device__ __forceinline__ void build_lut(const float* s_xi, unsigned char* s_lu
         s_ent[b] = make_uint2(__float_as_uint(s_xi[base]), payload(base));
     }
     __syncthreads();
-    for (int k = threadIdx.x; k < kLutBins * 32; k += blockDim.x)
-        *reinterpret_cast<uint2*>(s_lut + k * 8) = s_ent[k >> 5];
+    for (int k = threadIdx.x; k < kLutBins * REP; k += blockDim.x)
+        *reinterpret_cast<uint2*>(s_lut + k * 8) = s_ent[k / REP];
 }
 
 // ---------------------------------------------------------------- division for bf16 inputs

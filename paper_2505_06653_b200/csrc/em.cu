@@ -18,13 +18,19 @@ namespace bof4 {
 
 constexpr int kEmFlushIters = 64;  // loop iterations (16 weights per lane each) between fp32 -> fp64 folds
 
+// Both variants run 1024 threads per CTA, one CTA per SM.  The COUNT variant also keeps a 16-bit
+// member counter per level and thread (folded before it can overflow) and, to make room for it,
+// shares each table column between two lanes.
 template <bool COUNT>
 struct EmGeo {
-    static constexpr int threads = COUNT ? 512 : 1024;
+    static constexpr int threads = 1024;
     static constexpr int row = threads * kLaneW;            // weights per CTA row
     static constexpr uint32_t acc_row_bytes = threads * 8;  // one level's float2 columns
-    static constexpr size_t smem = (size_t)kLutBytes + (size_t)kLevels * threads * (COUNT ? 12 : 8);
+    static constexpr int lut_rep = COUNT ? 16 : 32;
+    static constexpr size_t smem =
+        (size_t)lut_bytes(lut_rep) + (size_t)kLevels * threads * (COUNT ? 10 : 8);
 };
+static_assert(kEmFlushIters * kLaneW < 65536, "16-bit member counters must not overflow between folds");
 
 // Record layout in doubles: [0,16) s1, [16,32) s0, [32,48) count (uint64 bits), [48] sum w^2.
 constexpr int kRecS1 = 0, kRecS0 = 16, kRecCnt = 32, kRecW2 = 48;
@@ -145,8 +151,8 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
     constexpr int NT = G::threads, NW = NT / 32, NSEG = NW / kLevels;
     extern __shared__ __align__(16) unsigned char s_raw[];
     unsigned char* s_lut = s_raw;
-    unsigned char* s_acc = s_raw + kLutBytes;                           // float2 [16][NT]
-    unsigned char* s_cnt = s_acc + (size_t)kLevels * G::acc_row_bytes;  // uint32 [16][NT] (COUNT)
+    unsigned char* s_acc = s_raw + lut_bytes(G::lut_rep);               // float2 [16][NT]
+    unsigned char* s_cnt = s_acc + (size_t)kLevels * G::acc_row_bytes;  // uint16 [16][NT] (COUNT)
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
     __shared__ WideScratch s_wide;
@@ -167,16 +173,16 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
 #pragma unroll
     for (int l = 0; l < kLevels; ++l) {
         *reinterpret_cast<float2*>(s_acc + l * G::acc_row_bytes + tid * 8) = make_float2(0.0f, 0.0f);
-        if (COUNT) *reinterpret_cast<uint32_t*>(s_cnt + l * (G::acc_row_bytes / 2) + tid * 4) = 0u;
+        if (COUNT) *reinterpret_cast<uint16_t*>(s_cnt + l * (G::acc_row_bytes / 4) + tid * 2) = 0;
     }
     __syncthreads();
-    build_lut(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base * G::acc_row_bytes; });
+    build_lut<G::lut_rep>(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base * G::acc_row_bytes; });
     __syncthreads();
     const bool lut_ok = s_multi == 0;
 
     const int64_t total_rows = T.row_end[T.count - 1];
     const bool unit = T.unit != 0;
-    const uint32_t lut_base = lut_lane_base(s_lut, lane), tid_off = tid * 8;
+    const uint32_t lut_base = lut_lane_base<G::lut_rep>(s_lut, lane), tid_off = tid * 8;
     double w2sum = 0.0;
     int t_cur = 0;
     int since_flush = 0;
@@ -198,9 +204,9 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
                 a0 += (double)a.y;
                 *pa = make_float2(0.0f, 0.0f);
                 if (COUNT) {
-                    uint32_t* pc = reinterpret_cast<uint32_t*>(s_cnt + l * (G::acc_row_bytes / 2) + col * 4);
+                    uint16_t* pc = reinterpret_cast<uint16_t*>(s_cnt + l * (G::acc_row_bytes / 4) + col * 2);
                     ac += *pc;
-                    *pc = 0u;
+                    *pc = 0;
                 }
             }
 #pragma unroll
@@ -282,12 +288,12 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const float xv = x[2 * k + h];
-                        const uint2 ent = lut_probe(h ? key.y : key.x, lut_base);
+                        const uint2 ent = lut_probe<G::lut_rep>(h ? key.y : key.x, lut_base);
                         const uint32_t off =
                             ent.y + ((xv >= __uint_as_float(ent.x)) ? G::acc_row_bytes : 0u) + tid_off;
                         float2* pa = reinterpret_cast<float2*>(s_acc + off);
                         *pa = __ffma2_rn(mm, make_float2(xv, 1.0f), *pa);
-                        if (COUNT) *reinterpret_cast<uint32_t*>(s_cnt + (off >> 1)) += 1u;
+                        if (COUNT) *reinterpret_cast<uint16_t*>(s_cnt + (off >> 2)) += 1;
                     }
                 }
             } else {
@@ -296,7 +302,7 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
                     const uint32_t off = (uint32_t)region_of(x[k], s_xi) * G::acc_row_bytes + tid_off;
                     float2* pa = reinterpret_cast<float2*>(s_acc + off);
                     *pa = __ffma2_rn(mm, make_float2(x[k], 1.0f), *pa);
-                    if (COUNT) *reinterpret_cast<uint32_t*>(s_cnt + (off >> 1)) += 1u;
+                    if (COUNT) *reinterpret_cast<uint16_t*>(s_cnt + (off >> 2)) += 1;
                 }
             }
         }

@@ -164,6 +164,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     uint32_t* s_cn = s_hi + kLevels * kMaeBins;
     uint2* s_cand = reinterpret_cast<uint2*>(s_cn + kLevels * kMaeBins);  // [16][kMaeStage] (COLLECT)
     __shared__ uint32_t s_ncand[kLevels], s_gbase[kLevels];
+    __shared__ volatile uint32_t s_over[kLevels];  // level's global list is known to have overflowed
     __shared__ float s_xi[kLevels], s_lv[kLevels];
     __shared__ int s_multi;
     __shared__ WideScratch s_wide;
@@ -192,7 +193,10 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         s_row_end[tid] = T.row_end[tid];
     }
     for (int k = tid; k < 3 * kLevels * kMaeBins; k += kMaeThreads) s_lo[k] = 0u;
-    if (tid < kLevels) s_ncand[tid] = 0u;
+    if (tid < kLevels) {
+        s_ncand[tid] = 0u;
+        s_over[tid] = 0u;
+    }
     const uint32_t max_bits = W.state->max_bits;
     __syncthreads();
     build_lut(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base; });
@@ -244,11 +248,13 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
                     const uint32_t slot = atomicAdd(&s_ncand[c], 1u);
                     if (slot < (uint32_t)kMaeStage) {
                         s_cand[c * kMaeStage + slot] = make_uint2(rel, a);
-                    } else {
+                    } else if (!s_over[c]) {
                         uint32_t* cnt = &W.state->cand_count[c];
                         if (*reinterpret_cast<volatile uint32_t*>(cnt) <= (uint32_t)kMaeCand) {
                             const uint32_t gslot = atomicAdd(cnt, 1u);
                             if (gslot < (uint32_t)kMaeCand) W.cand[c * kMaeCand + gslot] = make_uint2(rel, a);
+                        } else {
+                            s_over[c] = 1u;  // remembered per CTA: later samples of this level skip the look-up
                         }
                     }
                 }
