@@ -42,6 +42,7 @@ METRIC = ("hot-path step Gweights/s (EM iteration MSE + MAE, OPQ quantize, dequa
 BYTES_EM = 2.0
 BYTES_QUANT = 2.0 + 0.5 + 2.0 / I
 BYTES_DEQUANT = 0.5 + 2.0 / I + 2.0
+BYTES_GEMV = 0.5 + 2.0 / I            # 4-bit codes + bf16 block constants; x and y are negligible
 # data passes of one MAE iteration that stream all weights on this workload: the max-|w| pass
 # and two selection passes (the rest of the selection runs on the candidate lists)
 MAE_DATA_PASSES = 3
@@ -146,6 +147,10 @@ class Step:
         self.log_mse = torch.zeros(1, dtype=torch.float64, device=dev)
         self.have_mae = True
         self.only = None
+        # the decode-side product y = W_q x sees the same codes as a square matrix (profiling runs only)
+        self.gemv_rows = self.gemv_cols = int(round(n ** 0.5))
+        self.x = workloads.gaussian(self.gemv_cols, 1.0, 5 + seed_offset, torch.bfloat16).to(dev)
+        self.y = torch.empty(self.gemv_rows, dtype=torch.float32, device=dev)
 
     def flush_l2(self):
         self.flush_buf.zero_()
@@ -175,12 +180,18 @@ class Step:
         b.bof4_dequantize(self.codes, self.scales, I, self.cb_mse, b.BF16, (self.idx, self.val, self.cnt),
                           out=self.out)
 
+    def gemv(self):
+        b = self.b
+        b.bof4_gemv(self.codes, self.scales, self.gemv_rows, self.gemv_cols, I, self.cb_mse, self.x,
+                    (self.idx, self.val, self.cnt), out=self.y)
+
     def components(self):
         comps = [("em_mse", self.em_mse, 2), ("em_mae", self.em_mae, None), ("quantize_opq", self.quant, 4),
                  ("dequantize", self.dequant, 2)]
         comps = [c for c in comps if c[0] != "em_mae" or self.have_mae]
         if self.only:
             comps.append(("quantize", self.quant_plain, 1))  # profiling runs only
+            comps.append(("gemv", self.gemv, 2))
             comps = [c for c in comps if c[0] in self.only]
         return comps
 
@@ -262,6 +273,9 @@ def run_gpu(args):
     if args.only:
         st.only = set(args.only.split(","))
         args.no_e2e = args.no_cpu_baseline = True
+        if "gemv" in st.only:
+            assert st.gemv_rows * st.gemv_cols == st.n
+            st.quant()  # the matrix the product reads
     K, W = args.steps, args.warmup
     for _ in range(W):
         st.run_timed()
@@ -316,8 +330,9 @@ def run_gpu(args):
     peak, peak_kind = measured_peak()
     avg = {k: sum(v) / len(v) for k, v in comp_ms.items()}
     bytes_per_w = {"em_mse": BYTES_EM, "em_mae": None, "quantize_opq": BYTES_QUANT, "dequantize": BYTES_DEQUANT,
-                   "quantize": BYTES_QUANT}
-    kernels = {"em_mse": 1, "em_mae": mae_launches(bof4), "quantize_opq": 2, "dequantize": 2, "quantize": 1}
+                   "quantize": BYTES_QUANT, "gemv": BYTES_GEMV}
+    kernels = {"em_mse": 1, "em_mae": mae_launches(bof4), "quantize_opq": 2, "dequantize": 2, "quantize": 1,
+               "gemv": 2}
     comp, launches = {}, 0
     for name, ms in avg.items():
         comp[name + "_ms"] = ms
@@ -332,7 +347,7 @@ def run_gpu(args):
     # dominant component = the one with the largest share of the step
     dom = max(avg, key=avg.get)
     dom_bytes = {"em_mse": BYTES_EM, "em_mae": BYTES_EM * MAE_DATA_PASSES, "quantize_opq": BYTES_QUANT,
-                 "dequantize": BYTES_DEQUANT, "quantize": BYTES_QUANT}[dom] * n
+                 "dequantize": BYTES_DEQUANT, "quantize": BYTES_QUANT, "gemv": BYTES_GEMV}[dom] * n
     achieved = dom_bytes / avg[dom] / 1e6
     line = {
         "metric": METRIC, "value": whole_job_gweights_per_s(world, n, ms_per_step), "unit": "Gweights/s",

@@ -211,6 +211,31 @@ BOF4_API int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int s
                     void* d_out, int out_dtype, void* stream);
 
 /*
+ * Matrix-vector product with the 4-bit matrix decoded on the fly: Eq. 3 fused into its consumer,
+ * the operation behind the paper's token-generation timings (App. E.2), with the OPQ outliers
+ * applied as a sparse correction (Sec. 3.3, decoding side).  W is rows x cols, row-major, quantised
+ * as one flat tensor of rows * cols weights (so a block never straddles two rows: block_size
+ * divides cols).  In fp32:
+ *   y[r] = sum over the blocks b of row r of  scale[b] * sum_{i in b} xhat[code[i]] * x[col(i)]
+ *          + sum over the outliers k of row r of  (val[k] - scale[b(k)] * xhat[code[idx[k]]]) * x[col(idx[k])]
+ * i.e. the dequantised weight is not rounded to bf16 in between, and an outlier contributes its
+ * stored value instead of its quantised one.  The summation order is fixed (no atomics), so y is
+ * bit-reproducible; it differs from a sequential sum by fp32 rounding only.
+ *   d_codes     device, rows * cols / 2 bytes, 32-byte aligned
+ *   d_scales    device, rows * cols / block_size block constants of scale_dtype
+ *   cols        multiple of block_size, at most 32768
+ *   d_x         device, cols values of x_dtype (BOF4_BF16 or BOF4_F32)
+ *   d_out_idx / d_out_val / d_n_out / capacity   outlier list as for bof4_dequantize, or all NULL;
+ *               with a list, rows * cols must fit 32-bit indices
+ *   d_y         device, rows fp32 values, written
+ * One launch (two with an outlier list) on `stream`; no workspace, no host synchronisation.
+ */
+BOF4_API int bof4_gemv(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t rows,
+              int64_t cols, int block_size, const float* d_codebook, const void* d_x, int x_dtype,
+              const int32_t* d_out_idx, const void* d_out_val, const int64_t* d_n_out,
+              int64_t capacity, float* d_y, void* stream);
+
+/*
  * Data-free codebook for unit-variance Gaussian weights (Sec. 3.2 Eq. 5 / Eq. 7; App. B.2): `iters`
  * Lloyd iterations in which every free level becomes the theoretical centroid of its region,
  * a ratio (MSE) or root (MAE) of integrals over the absolute block maximum, evaluated by

@@ -228,3 +228,27 @@ def opq_threshold(q: float, I: int) -> float:
     (App. B.1, CDF of the absolute block maximum), hence G(tau) = (1 + q^(1/I)) / 2."""
     from scipy.special import ndtri
     return float(ndtri((1.0 + q ** (1.0 / I)) / 2.0))
+
+
+def gemv(codes: np.ndarray, scales: np.ndarray, rows: int, cols: int, I: int, xhat, x,
+         idx: Optional[np.ndarray] = None, val: Optional[np.ndarray] = None):
+    """y = W x in fp64 for the decoded matrix (Eq. 3; with OPQ the stored outliers replace the
+    decoded values, Sec. 3.3): W[r, c] = scale[block] * xhat[code] exactly (a product of two fp32
+    numbers is exact in fp64), W.flat[idx] = val.  Also returns sum_c |W[r, c] x[c]|, the scale
+    of the rounding error any fp32 evaluation of the same sum may show.
+    -> (y fp64 [rows], mag fp64 [rows])."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8).reshape(-1)
+    scales = np.ascontiguousarray(scales, dtype=np.float32).reshape(-1)
+    n = rows * cols
+    assert codes.size * 2 == n and cols % I == 0 and scales.size == n // I
+    lv = _levels(xhat).astype(np.float64)
+    c = np.empty(n, np.uint8)
+    c[0::2] = codes >> 4
+    c[1::2] = codes & 15
+    W = lv[c] * np.repeat(scales.astype(np.float64), I)
+    if idx is not None and len(idx):
+        W[np.asarray(idx, dtype=np.int64)] = bf16_bits_to_f32(np.asarray(val, dtype=np.uint16)).astype(np.float64)
+    W = W.reshape(rows, cols)
+    xv = np.asarray(x, dtype=np.float64).reshape(-1)
+    assert xv.size == cols
+    return W @ xv, np.abs(W) @ np.abs(xv)

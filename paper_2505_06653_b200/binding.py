@@ -30,7 +30,7 @@ MAE_LAUNCHES_PER_ITERATION = 10
 
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
-           "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook")
+           "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_gemv")
 
 
 class Bof4Error(RuntimeError):
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
                                         vp, vp, i64, vp, vp, sz, vp]
         L.bof4_dequantize.restype = i32
         L.bof4_dequantize.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp, i64, vp, i32, vp]
+        L.bof4_gemv.restype = i32
+        L.bof4_gemv.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, vp, vp, vp, i64, vp, vp]
         L.bof4_theoretical_codebook.restype = i32
         L.bof4_theoretical_codebook.argtypes = [i32, i32, i32, vp, ctypes.c_uint32, i32, vp, sz, vp]
         L.bof4_opq_threshold.restype = ctypes.c_double
@@ -266,6 +268,29 @@ def bof4_dequantize(codes: torch.Tensor, scales: torch.Tensor, block_size: int, 
         _check(lib().bof4_dequantize(_ptr(codes), _ptr(scales), _dt(scales), n, block_size, _ptr(cb),
                                      _ptr(idx), _ptr(val), _ptr(cnt), cap, _ptr(out), out_dtype,
                                      _stream()))
+    return out
+
+
+def bof4_gemv(codes: torch.Tensor, scales: torch.Tensor, rows: int, cols: int, block_size: int, levels,
+              x: torch.Tensor, outliers: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
+              out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """-> y fp32 [rows] = W_q x for the rows x cols matrix held as (codes, scales[, outliers])."""
+    codes = _dev(codes, "codes")
+    scales = _dev(scales, "scales")
+    x = _dev(x, "x")
+    if codes.numel() * 2 != rows * cols or x.numel() != cols:
+        raise ValueError("codes must hold rows * cols weights and x cols values")
+    cb = _codebook(levels, codes.device)
+    if out is None:
+        out = torch.empty(rows, dtype=torch.float32, device=codes.device)
+    idx = val = cnt = None
+    cap = 0
+    if outliers is not None:
+        idx, val, cnt = outliers
+        cap = idx.numel()
+    with torch.cuda.device(codes.device):
+        _check(lib().bof4_gemv(_ptr(codes), _ptr(scales), _dt(scales), rows, cols, block_size, _ptr(cb),
+                               _ptr(x), _dt(x), _ptr(idx), _ptr(val), _ptr(cnt), cap, _ptr(out), _stream()))
     return out
 
 

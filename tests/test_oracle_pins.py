@@ -544,3 +544,60 @@ def test_normalised_domain_mae_is_the_plain_median_of_x():
             assert st["median"][l] == np.quantile(mem, 0.5, method="inverted_cdf")
             err += np.abs(mem.astype(np.float64) - float(init[l])).sum()
     assert np.isclose(st["err_sum"], err, rtol=1e-9)
+
+
+# --------------------------------------------------------------------------- decode fused into y = W x
+
+
+def test_gemv_closed_forms_by_hand():
+    """Eq. 3 inside a matrix-vector product, on a 2 x 64 matrix whose result is known in closed
+    form: a row of codes 15 (level 1) gives scale * sum(x); nibble order (even column = high
+    nibble) and the row / block bookkeeping are fixed by one odd entry per row."""
+    lv = np.linspace(-1, 1, 16).astype(np.float32)
+    lv[7] = 0.0
+    rows, cols, I = 2, 64, 32
+    codes = np.full(rows * cols // 2, 0xFF, np.uint8)
+    scales = np.array([2.0, 3.0, 0.5, 0.25], np.float32)  # blocks (r0,b0) (r0,b1) (r1,b0) (r1,b1)
+    x = np.arange(1, cols + 1, dtype=np.float32)
+    y, mag = oracle.gemv(codes, scales, rows, cols, I, lv, x)
+    assert y[0] == 2.0 * x[:32].sum() + 3.0 * x[32:].sum()
+    assert y[1] == 0.5 * x[:32].sum() + 0.25 * x[32:].sum()
+    assert np.array_equal(y, mag)
+    # column 5 of row 0 -> code 0 (level -1): byte 2 holds columns 4 (high) and 5 (low)
+    codes2 = codes.copy()
+    codes2[2] = 0xF0
+    y2, _ = oracle.gemv(codes2, scales, rows, cols, I, lv, x)
+    assert y2[0] == y[0] - 2 * 2.0 * x[5] and y2[1] == y[1]
+    # column 40 of row 1 -> code 7 (level 0): byte (64 + 40) / 2 = 52, high nibble
+    codes3 = codes.copy()
+    codes3[52] = 0x7F
+    y3, _ = oracle.gemv(codes3, scales, rows, cols, I, lv, x)
+    assert y3[1] == y[1] - 0.25 * x[40] and y3[0] == y[0]
+    # an outlier replaces the decoded value: flat index 64 + 3 gets 10.0 (bf16 bits 0x4120)
+    y4, _ = oracle.gemv(codes, scales, rows, cols, I, lv, x, idx=np.array([67]), val=np.array([0x4120], np.uint16))
+    assert y4[1] == y[1] + (10.0 - 0.5) * x[3]
+
+
+def test_gemv_is_the_library_matvec_of_the_dequantised_matrix():
+    """Against numpy's matvec of the separately dequantised (Eq. 3) and restored (Sec. 3.3) matrix:
+    the only difference is the fp32 rounding of scale * level, 2^-24 relative per term."""
+    rng = np.random.default_rng(5)
+    rows, cols, I = 24, 256, 64
+    w = workloads.gaussian(rows * cols, 0.02, seed=91).numpy()
+    w[rng.integers(0, w.size, 40)] *= 12.0
+    lv = TAB6[:, 2].astype(np.float32)  # BOF4 (MSE), Tab. 6
+    clean, idx, val, k = oracle.opq_split(w, I, oracle.opq_threshold(0.95, I))
+    assert 0 < k == idx.size
+    codes, scales = oracle.quantize(clean, I, oracle.NORM_ABS, lv)
+    x = rng.standard_normal(cols).astype(np.float32)
+    y, mag = oracle.gemv(codes, scales, rows, cols, I, lv, x, idx, val)
+    W = oracle.opq_restore(oracle.dequantize(codes, scales, I, lv), idx, val).reshape(rows, cols).astype(np.float64)
+    ref = W @ x.astype(np.float64)
+    assert np.all(np.abs(y - ref) <= 2.0 ** -23 * mag)
+    assert np.abs(y - ref).max() > 0 or np.array_equal(y, ref)
+    # and it is close to the unquantised product: the quantisation error is small, not absent
+    exact = w.reshape(rows, cols).astype(np.float64) @ x.astype(np.float64)
+    assert 0 < np.abs(y - exact).max() < 0.25 * np.abs(exact).max()
+    # a transposed operand or a dropped outlier list is caught
+    y_no, _ = oracle.gemv(codes, scales, rows, cols, I, lv, x)
+    assert np.abs(y_no - ref).max() > 100 * 2.0 ** -23 * mag.max()
