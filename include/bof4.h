@@ -224,7 +224,7 @@ BOF4_API int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int s
  *   d_codes     device, rows * cols / 2 bytes, 32-byte aligned
  *   d_scales    device, rows * cols / block_size block constants of scale_dtype
  *   cols        multiple of block_size, at most 32768
- *   d_x         device, cols values of x_dtype (BOF4_BF16 or BOF4_F32)
+ *   d_x         device, cols values of x_dtype (BOF4_BF16 or BOF4_F32), 16-byte aligned
  *   d_out_idx / d_out_val / d_n_out / capacity   outlier list as for bof4_dequantize, or all NULL;
  *               with a list, rows * cols must fit 32-bit indices
  *   d_y         device, rows fp32 values, written

@@ -398,8 +398,8 @@ extern "C" int bof4_gemv(const uint8_t* d_codes, const void* d_scales, int scale
         set_error("bof4_gemv: NULL pointer");
         return BOF4_ERR_INVALID_ARG;
     }
-    if (!aligned32(d_codes)) {
-        set_error("bof4_gemv: d_codes must be 32-byte aligned");
+    if (!aligned32(d_codes) || (reinterpret_cast<uintptr_t>(d_x) & 15u)) {
+        set_error("bof4_gemv: d_codes must be 32-byte aligned and d_x 16-byte aligned");
         return BOF4_ERR_INVALID_ARG;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);

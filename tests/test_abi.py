@@ -114,6 +114,20 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     assert L.bof4_em_step(ptrs, ns, 1, 7, 64, 0, 0, fake, fake, ws, 1 << 40, None) == -3
     assert L.bof4_fit_codebook(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, 0, -1, None, ws, 1 << 40, None) == -1
     assert L.bof4_fit_codebook(ptrs, ns, 1, b.BF16, 64, 0, 0, None, 0, 1, None, ws, 1 << 40, None) == -1
+    # fused matrix-vector product: shape, dtype, outlier-list and alignment rules
+    gv = lambda *a: L.bof4_gemv(*a)
+    assert gv(fake, fake, b.BF16, 4, 96, 64, fake, fake, b.BF16, None, None, None, 0, fake, None) == -2
+    assert gv(fake, fake, b.BF16, 4, 65536, 64, fake, fake, b.BF16, None, None, None, 0, fake, None) == -2
+    assert gv(fake, fake, b.BF16, -1, 64, 64, fake, fake, b.BF16, None, None, None, 0, fake, None) == -1
+    assert gv(fake, fake, 5, 4, 64, 64, fake, fake, b.BF16, None, None, None, 0, fake, None) == -3
+    assert gv(fake, fake, b.BF16, 4, 64, 64, fake, fake, b.BF16, fake, None, None, 4, fake, None) == -1
+    assert gv(fake, fake, b.BF16, 4, 64, 64, fake, fake, b.BF16, fake, fake, fake, -1, fake, None) == -5
+    assert gv(fake, fake, b.BF16, 1 << 20, 4096, 64, fake, fake, b.BF16, fake, fake, fake, 4, fake, None) == -2
+    assert gv(fake, fake, b.BF16, 4, 64, 64, fake, ctypes.c_void_p(0x1008), b.BF16, None, None, None, 0, fake, None) == -1
+    assert b"aligned" in L.bof4_last_error()
+    assert gv(ctypes.c_void_p(0x1010), fake, b.BF16, 4, 64, 64, fake, fake, b.BF16, None, None, None, 0, fake, None) == -1
+    assert gv(fake, fake, b.BF16, 4, 64, 64, fake, fake, b.BF16, None, None, None, 0, None, None) == -1
+    assert gv(None, None, b.BF16, 0, 64, 64, None, None, b.BF16, None, None, None, 0, None, None) == 0
     # theoretical codebook: the outermost levels must be fixed, metric MSE / MAE only
     full = (1 << 0) | (1 << 7) | (1 << 15)
     assert L.bof4_theoretical_codebook(64, 0, 0, fake, 1 << 15, 1, ws, 256, None) == -1   # -1 not fixed (abs)

@@ -160,6 +160,11 @@ def test_gemv_degenerate_shapes_and_errors(bof4):
         bof4.bof4_gemv(big, torch.ones(32800 // 32, dtype=torch.bfloat16, device=dev), 1, 32800, 32, lv,
                        torch.ones(32800, dtype=torch.bfloat16, device=dev))
     assert e.value.code == -2
+    xx = torch.ones(72, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(bof4.Bof4Error) as e:  # x must be 16-byte aligned (vector loads)
+        bof4.bof4_gemv(torch.zeros(4 * 64 // 2, dtype=torch.uint8, device=dev),
+                       torch.ones(4 * 64 // 32, dtype=torch.bfloat16, device=dev), 4, 64, 32, lv, xx[3:67])
+    assert e.value.code == -1
     # all-zero blocks: scale 0, y = 0 exactly
     z = torch.zeros(4 * 64, dtype=torch.bfloat16, device=dev)
     c, s = bof4.bof4_quantize(z, 32, bof4.NORM_ABS, lv)
