@@ -150,9 +150,18 @@ mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
 
 // ---------------------------------------------------------------- data pass
 
-// FIRST: also accumulates sum |w - m xhat[c]| (one partial record per CTA) and, with COUNT,
-// the member counts.  Later passes return at once when no level has bits left.
+// FIRST: every member of an active level takes part; also accumulates sum |w - m xhat[c]| (one
+// partial record per CTA) and, with COUNT, the member counts.
+// Later passes return at once when no level has bits left.  Only about one sample in 500 still
+// takes part in them (those whose key carries the digits chosen so far), so their loop over the
+// data does no more than find these: the 257-bin table of the region search holds, instead of
+// thresholds, the hull [lo, hi] of the normalised weights that can still take part in each bin
+// (one 8-byte read and two comparisons per weight), and a hit is appended to a queue in shared
+// memory.  The queue is worked off by all threads after the loop (region search, digit,
+// histogram, candidate list), so that the rare, long path does not run with one lane in 32.
 // COLLECT (second pass): every participating sample is also appended to its level's list.
+constexpr int kMaeQueue = kLevels * kMaeBins * 4 / 8;  // entries {x, weight} in the count histogram's space
+
 template <class DT, int I, bool SIGNED, bool FIRST, bool COUNT, bool COLLECT>
 __global__ void __launch_bounds__(kMaeThreads, 1)
 mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
@@ -162,6 +171,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     uint32_t* s_lo = reinterpret_cast<uint32_t*>(s_raw + kLutBytes);
     uint32_t* s_hi = s_lo + kLevels * kMaeBins;
     uint32_t* s_cn = s_hi + kLevels * kMaeBins;
+    uint2* s_queue = reinterpret_cast<uint2*>(s_cn);  // later passes (which keep no counts)
     uint2* s_cand = reinterpret_cast<uint2*>(s_cn + kLevels * kMaeBins);  // [16][kMaeStage] (COLLECT)
     __shared__ uint32_t s_ncand[kLevels], s_gbase[kLevels];
     __shared__ volatile uint32_t s_over[kLevels];  // level's global list is known to have overflowed
@@ -169,6 +179,9 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     __shared__ int s_multi;
     __shared__ WideScratch s_wide;
     __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
+    __shared__ uint2 s_iv[kLutBins];  // later passes: bits of {lo, hi} per table bin (lo > hi: nothing)
+    __shared__ float2 s_span[kLevels];
+    __shared__ uint32_t s_qn;
     __shared__ double s_err[kMaeThreads / 32];
     __shared__ const void* s_ptr[kEmMaxTensors];
     __shared__ int64_t s_n[kEmMaxTensors], s_row_end[kEmMaxTensors];
@@ -192,16 +205,82 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         s_n[tid] = T.n[tid];
         s_row_end[tid] = T.row_end[tid];
     }
-    for (int k = tid; k < 3 * kLevels * kMaeBins; k += kMaeThreads) s_lo[k] = 0u;
+    for (int k = tid; k < (FIRST ? 3 : 2) * kLevels * kMaeBins; k += kMaeThreads) s_lo[k] = 0u;
     if (tid < kLevels) {
         s_ncand[tid] = 0u;
         s_over[tid] = 0u;
     }
+    if (tid == 0) s_qn = 0u;
     const uint32_t max_bits = W.state->max_bits;
     __syncthreads();
-    build_lut(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base; });
-    __syncthreads();
-    const bool lut_ok = s_multi == 0;
+    bool lut_ok = true;
+    if (FIRST) {
+        build_lut(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base; });
+        __syncthreads();
+        lut_ok = s_multi == 0;
+    } else {
+        // Participants of level l have keys in [base + (prefix << top), base + ((prefix + 1) << top));
+        // keys and normalised weights are ordered alike, so they lie between the weights of the
+        // two end keys (clipped to [-1, 1]), and so do their table bins.
+        if (tid < kLevels) {
+            const uint4 L = s_lvl[tid];
+            const int top = (int)(L.z & 0xffu);
+            float2 span = make_float2(2.0f, -2.0f);
+            if (L.w) {
+                const uint32_t kmin = order_key(-1.0f), kmax = order_key(1.0f);
+                const unsigned long long lo64 = (unsigned long long)L.x + ((unsigned long long)L.y << top);
+                const unsigned long long hi64 = lo64 + ((1ull << top) - 1ull);
+                const uint32_t klo = max(lo64 > kmax ? kmax : (uint32_t)lo64, kmin);
+                const uint32_t khi = max(hi64 > kmax ? kmax : (uint32_t)hi64, kmin);
+                span = make_float2(key_to_float(klo), key_to_float(khi));
+            }
+            s_span[tid] = span;
+        }
+        __syncthreads();
+        for (int b = tid; b < kLutBins; b += kMaeThreads) {
+            float2 iv = make_float2(2.0f, -2.0f);
+            for (int l = 0; l < kLevels; ++l) {
+                const float2 sp = s_span[l];
+                if (sp.x > sp.y) continue;
+                const int blo = (int)(__float_as_uint(lut_key(sp.x)) - kLutMagicBits);
+                const int bhi = (int)(__float_as_uint(lut_key(sp.y)) - kLutMagicBits);
+                if (b >= blo && b <= bhi) iv = make_float2(fminf(iv.x, sp.x), fmaxf(iv.y, sp.y));
+            }
+            s_iv[b] = make_uint2(__float_as_uint(iv.x), __float_as_uint(iv.y));
+        }
+        __syncthreads();
+        for (int k = tid; k < kLutBins * 32; k += kMaeThreads)  // one column per lane, as in the region table
+            *reinterpret_cast<uint2*>(s_lut + k * 8) = s_iv[k >> 5];
+        __syncthreads();
+    }
+
+    // One participating sample of a later pass: digit histogram and (COLLECT) candidate list.
+    auto later_sample = [&](float xk, uint32_t a) {
+        const uint32_t c = (uint32_t)region_of(xk, s_xi);
+        const uint4 L = s_lvl[c];
+        const uint32_t rel = order_key(xk) - L.x;
+        const uint32_t top = L.z & 0xffu, sh = (L.z >> 8) & 0xffu, mask = L.z >> 16;
+        if (!(L.w && (uint32_t)((unsigned long long)rel >> top) == L.y)) return;
+        const uint32_t bin = c * kMaeBins + ((rel >> sh) & mask);
+        const uint32_t old = atomicAdd(&s_lo[bin], a);
+        if (old + a < old) atomicAdd(&s_hi[bin], 1u);
+        if (COLLECT) {
+            // staged per CTA and level; the rare overflow of a slot goes straight to the
+            // global list (whose count only needs to stay above the capacity once full)
+            const uint32_t slot = atomicAdd(&s_ncand[c], 1u);
+            if (slot < (uint32_t)kMaeStage) {
+                s_cand[c * kMaeStage + slot] = make_uint2(rel, a);
+            } else if (!s_over[c]) {
+                uint32_t* cnt = &W.state->cand_count[c];
+                if (*reinterpret_cast<volatile uint32_t*>(cnt) <= (uint32_t)kMaeCand) {
+                    const uint32_t gslot = atomicAdd(cnt, 1u);
+                    if (gslot < (uint32_t)kMaeCand) W.cand[c * kMaeCand + gslot] = make_uint2(rel, a);
+                } else {
+                    s_over[c] = 1u;  // remembered per CTA: later samples of this level skip the look-up
+                }
+            }
+        }
+    };
 
     const int64_t total_rows = T.row_end[T.count - 1];
     const uint32_t lut_base = lut_lane_base(s_lut, lane);
@@ -219,50 +298,67 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         const bool safe = row_is_safe(gmax, ok);
         float x[kLaneW];
         normalise16<false>(v, m, safe && DT::code == BF16::code, x);
-        const bool use_lut = lut_ok && safe;
         if (!ok) continue;
         const uint32_t a = T.unit ? 1u : fixed_weight(m, max_bits);  // App. D variant: plain median
-        float e = 0.0f;
+        if (FIRST) {
+            const bool use_lut = lut_ok && safe;
+            float e = 0.0f;
 #pragma unroll
-        for (int k = 0; k < kLaneW; ++k) {
-            uint32_t c;
-            if (use_lut) {
-                const uint2 ent = lut_probe(lut_key(x[k]), lut_base);
-                c = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? 1u : 0u);
-            } else {
-                c = (uint32_t)region_of(x[k], s_xi);
+            for (int k = 0; k < kLaneW; ++k) {
+                uint32_t c;
+                if (use_lut) {
+                    const uint2 ent = lut_probe(lut_key(x[k]), lut_base);
+                    c = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? 1u : 0u);
+                } else {
+                    c = (uint32_t)region_of(x[k], s_xi);
+                }
+                e += T.unit ? fabsf(x[k] - s_lv[c]) : fabsf(fmaf(-m, s_lv[c], v[k]));
+                const uint4 L = s_lvl[c];
+                if (L.w) {
+                    const uint32_t rel = order_key(x[k]) - L.x;
+                    const uint32_t sh = (L.z >> 8) & 0xffu, mask = L.z >> 16;
+                    const uint32_t bin = c * kMaeBins + ((rel >> sh) & mask);
+                    const uint32_t old = atomicAdd(&s_lo[bin], a);
+                    if (old + a < old) atomicAdd(&s_hi[bin], 1u);
+                    if (COUNT) atomicAdd(&s_cn[bin], 1u);
+                }
             }
-            if (FIRST) e += T.unit ? fabsf(x[k] - s_lv[c]) : fabsf(fmaf(-m, s_lv[c], v[k]));
-            const uint4 L = s_lvl[c];
-            const uint32_t rel = order_key(x[k]) - L.x;
-            const uint32_t top = L.z & 0xffu, sh = (L.z >> 8) & 0xffu, mask = L.z >> 16;
-            // in the first pass no digit has been chosen: every member of an active level takes part
-            if (L.w && (FIRST || (uint32_t)((unsigned long long)rel >> top) == L.y)) {
-                const uint32_t bin = c * kMaeBins + ((rel >> sh) & mask);
-                const uint32_t old = atomicAdd(&s_lo[bin], a);
-                if (old + a < old) atomicAdd(&s_hi[bin], 1u);
-                if (FIRST && COUNT) atomicAdd(&s_cn[bin], 1u);
-                if (COLLECT) {
-                    // staged per CTA and level; the rare overflow of a slot goes straight to the
-                    // global list (whose count only needs to stay above the capacity once full)
-                    const uint32_t slot = atomicAdd(&s_ncand[c], 1u);
-                    if (slot < (uint32_t)kMaeStage) {
-                        s_cand[c * kMaeStage + slot] = make_uint2(rel, a);
-                    } else if (!s_over[c]) {
-                        uint32_t* cnt = &W.state->cand_count[c];
-                        if (*reinterpret_cast<volatile uint32_t*>(cnt) <= (uint32_t)kMaeCand) {
-                            const uint32_t gslot = atomicAdd(cnt, 1u);
-                            if (gslot < (uint32_t)kMaeCand) W.cand[c * kMaeCand + gslot] = make_uint2(rel, a);
-                        } else {
-                            s_over[c] = 1u;  // remembered per CTA: later samples of this level skip the look-up
-                        }
+            err += (double)e;
+        } else {
+            // bit k of `hits`: weight k may take part.  A row that cannot use the table (a non-finite
+            // or extreme block constant makes its quotients unfit as table keys) offers all 16.
+            uint32_t hits = 0xffffu;
+            if (safe) {
+                hits = 0u;
+#pragma unroll
+                for (int k = 0; k < kLaneW; ++k) {
+                    const uint2 iv = lut_probe(lut_key(x[k]), lut_base);
+                    if (x[k] >= __uint_as_float(iv.x) && x[k] <= __uint_as_float(iv.y)) hits |= 1u << k;
+                }
+            }
+            if (hits) {
+#pragma unroll
+                for (int k = 0; k < kLaneW; ++k) {
+                    if ((hits >> k) & 1u) {
+                        const uint32_t slot = atomicAdd(&s_qn, 1u);
+                        if (slot < (uint32_t)kMaeQueue)
+                            s_queue[slot] = make_uint2(__float_as_uint(x[k]), a);
+                        else
+                            later_sample(x[k], a);  // queue full: handled on the spot
                     }
                 }
             }
         }
-        if (FIRST) err += (double)e;
     }
     __syncthreads();
+    if (!FIRST) {
+        const uint32_t q = min(s_qn, (uint32_t)kMaeQueue);
+        for (uint32_t i = tid; i < q; i += kMaeThreads) {
+            const uint2 ent = s_queue[i];
+            later_sample(__uint_as_float(ent.x), ent.y);
+        }
+        __syncthreads();
+    }
     for (int k = tid; k < kLevels * kMaeBins; k += kMaeThreads) {
         const unsigned long long wsum = ((unsigned long long)s_hi[k] << 32) + s_lo[k];
         if (wsum) atomicAdd(&W.hist[k], wsum);
