@@ -11,6 +11,10 @@
 // that list fits (64 Ki samples per level) the remaining digits are resolved from the list by
 // one CTA and no further data pass is needed.  Otherwise (very large or degenerate inputs) the
 // third and fourth data passes finish the selection; they return at once when nothing is left.
+// In every pass after the first only the samples that carry the digits chosen so far matter:
+// the pass finds them with one table read and two comparisons per weight (the table bins hold
+// the range of normalised weights that can still take part) and queues them in shared memory;
+// the queue is worked off by all threads once the data has been read.
 //
 // Weights enter the histograms as 31-bit fixed-point integers relative to the largest |w| of
 // the data (exact whenever |m| is within 2^-7 of it for fp32 input, 2^-23 for bf16 input), so
@@ -179,6 +183,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     __shared__ int s_multi;
     __shared__ WideScratch s_wide;
     __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
+    __shared__ uint2 s_lvl1[kLevels];  // first pass: {base, shift | mask << 8 | on << 31}
     __shared__ uint2 s_iv[kLutBins];  // later passes: bits of {lo, hi} per table bin (lo > hi: nothing)
     __shared__ float2 s_span[kLevels];
     __shared__ uint32_t s_qn;
@@ -199,6 +204,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         const uint32_t mask = (1u << (top - sh)) - 1u;
         s_lvl[tid] = make_uint4(W.state->base[tid], W.state->prefix[tid],
                                 (uint32_t)top | ((uint32_t)sh << 8) | (mask << 16), top > 0 ? 1u : 0u);
+        s_lvl1[tid] = make_uint2(W.state->base[tid], (uint32_t)sh | (mask << 8) | (top > 0 ? 0x80000000u : 0u));
     }
     if (tid < T.count) {
         s_ptr[tid] = T.ptr[tid];
@@ -286,13 +292,23 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     const uint32_t lut_base = lut_lane_base(s_lut, lane);
     double err = 0.0;
     int t_cur = 0;
-    for (int64_t g = blockIdx.x; g < total_rows; g += gridDim.x) {
+    // row g of the concatenated tensors: this thread's 16 weights, or zeros past the end (ok = false)
+    auto fetch = [&](int64_t g, bool& ok) -> RawRow<DT> {
+        ok = false;
+        if (g >= total_rows) return zero_raw<DT>();
         while (g >= s_row_end[t_cur]) ++t_cur;
         const int64_t r = g - (t_cur ? s_row_end[t_cur - 1] : 0);
         const int64_t idx = (r * kMaeThreads + tid) * kLaneW;
-        const bool ok = idx < s_n[t_cur];
+        ok = idx < s_n[t_cur];
+        return ok ? load_raw<DT>(s_ptr[t_cur], idx) : zero_raw<DT>();
+    };
+    bool ok, ok_next;
+    RawRow<DT> raw = fetch(blockIdx.x, ok);
+    for (int64_t g = blockIdx.x; g < total_rows; g += gridDim.x, ok = ok_next) {
+        const RawRow<DT> next = fetch(g + gridDim.x, ok_next);  // in flight while this row is processed
         float v[kLaneW];
-        widen(ok ? load_raw<DT>(s_ptr[t_cur], idx) : zero_raw<DT>(), v);
+        widen(raw, v);
+        raw = next;
         float gmax;
         const float m = block_constant<I, SIGNED>(v, gmax, &s_wide);
         const bool safe = row_is_safe(gmax, ok);
@@ -313,10 +329,10 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
                     c = (uint32_t)region_of(x[k], s_xi);
                 }
                 e += T.unit ? fabsf(x[k] - s_lv[c]) : fabsf(fmaf(-m, s_lv[c], v[k]));
-                const uint4 L = s_lvl[c];
-                if (L.w) {
+                const uint2 L = s_lvl1[c];
+                if (L.y >> 31) {
                     const uint32_t rel = order_key(x[k]) - L.x;
-                    const uint32_t sh = (L.z >> 8) & 0xffu, mask = L.z >> 16;
+                    const uint32_t sh = L.y & 0xffu, mask = (L.y >> 8) & 0x1ffu;
                     const uint32_t bin = c * kMaeBins + ((rel >> sh) & mask);
                     const uint32_t old = atomicAdd(&s_lo[bin], a);
                     if (old + a < old) atomicAdd(&s_hi[bin], 1u);
@@ -325,26 +341,26 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
             }
             err += (double)e;
         } else {
-            // bit k of `hits`: weight k may take part.  A row that cannot use the table (a non-finite
-            // or extreme block constant makes its quotients unfit as table keys) offers all 16.
-            uint32_t hits = 0xffffu;
-            if (safe) {
-                hits = 0u;
+            // A weight inside its bin's hull may take part and is queued.  A row that cannot use the
+            // table (a non-finite or extreme block constant makes its quotients unfit as table
+            // keys) offers all 16.
 #pragma unroll
-                for (int k = 0; k < kLaneW; ++k) {
-                    const uint2 iv = lut_probe(lut_key(x[k]), lut_base);
-                    if (x[k] >= __uint_as_float(iv.x) && x[k] <= __uint_as_float(iv.y)) hits |= 1u << k;
-                }
-            }
-            if (hits) {
+            for (int k = 0; k < kLaneW; k += 2) {
+                const float2 key = lut_key2(make_float2(x[k], x[k + 1]));
+                const float kk[2] = {key.x, key.y};
 #pragma unroll
-                for (int k = 0; k < kLaneW; ++k) {
-                    if ((hits >> k) & 1u) {
+                for (int h = 0; h < 2; ++h) {
+                    bool hit = true;
+                    if (safe) {
+                        const uint2 iv = lut_probe(kk[h], lut_base);
+                        hit = x[k + h] >= __uint_as_float(iv.x) && x[k + h] <= __uint_as_float(iv.y);
+                    }
+                    if (hit) {
                         const uint32_t slot = atomicAdd(&s_qn, 1u);
                         if (slot < (uint32_t)kMaeQueue)
-                            s_queue[slot] = make_uint2(__float_as_uint(x[k]), a);
+                            s_queue[slot] = make_uint2(__float_as_uint(x[k + h]), a);
                         else
-                            later_sample(x[k], a);  // queue full: handled on the spot
+                            later_sample(x[k + h], a);  // queue full: handled on the spot
                     }
                 }
             }
