@@ -4,6 +4,10 @@ TEST INFRASTRUCTURE ONLY: the plain, slow definition of what the CUDA library mu
 Nothing in the product package imports this module, and this module imports nothing from
 the product package.  Inputs are CPU torch tensors or numpy arrays; bf16 inputs are widened
 to fp32 (exact) before they reach the C code.
+
+Parity pins: the C functions as listed in ``bof4_oracle.c``; ``gemv`` (fp64 numpy, the plain
+definition of the decoded matrix-vector product) by hand-built closed forms and numpy's matvec
+of the separately dequantised and restored matrix (tests/test_oracle_pins.py).
 """
 from __future__ import annotations
 
