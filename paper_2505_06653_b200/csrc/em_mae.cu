@@ -68,7 +68,7 @@ __host__ __device__ inline MaeWs mae_ws(void* d_ws)
 __device__ __forceinline__ uint32_t order_key(float x)
 {
     const uint32_t u = __float_as_uint(x + 0.0f);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);  // negative: all bits flip, else only the sign
 }
 __device__ __forceinline__ float key_to_float(uint32_t k)
 {
@@ -183,7 +183,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     __shared__ int s_multi;
     __shared__ WideScratch s_wide;
     __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
-    __shared__ uint2 s_lvl1[kLevels];  // first pass: {base, shift | mask << 8 | on << 31}
+    __shared__ uint2 s_lvl1[kLevels];  // first pass: {base, shift | on << 31}
     __shared__ uint2 s_iv[kLutBins];  // later passes: bits of {lo, hi} per table bin (lo > hi: nothing)
     __shared__ float2 s_span[kLevels];
     __shared__ uint32_t s_qn;
@@ -204,7 +204,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         const uint32_t mask = (1u << (top - sh)) - 1u;
         s_lvl[tid] = make_uint4(W.state->base[tid], W.state->prefix[tid],
                                 (uint32_t)top | ((uint32_t)sh << 8) | (mask << 16), top > 0 ? 1u : 0u);
-        s_lvl1[tid] = make_uint2(W.state->base[tid], (uint32_t)sh | (mask << 8) | (top > 0 ? 0x80000000u : 0u));
+        s_lvl1[tid] = make_uint2(W.state->base[tid], (uint32_t)sh | (top > 0 ? 0x80000000u : 0u));
     }
     if (tid < T.count) {
         s_ptr[tid] = T.ptr[tid];
@@ -320,23 +320,31 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
             const bool use_lut = lut_ok && safe;
             float e = 0.0f;
 #pragma unroll
-            for (int k = 0; k < kLaneW; ++k) {
-                uint32_t c;
-                if (use_lut) {
-                    const uint2 ent = lut_probe(lut_key(x[k]), lut_base);
-                    c = ent.y + ((x[k] >= __uint_as_float(ent.x)) ? 1u : 0u);
-                } else {
-                    c = (uint32_t)region_of(x[k], s_xi);
-                }
-                e += T.unit ? fabsf(x[k] - s_lv[c]) : fabsf(fmaf(-m, s_lv[c], v[k]));
-                const uint2 L = s_lvl1[c];
-                if (L.y >> 31) {
-                    const uint32_t rel = order_key(x[k]) - L.x;
-                    const uint32_t sh = L.y & 0xffu, mask = (L.y >> 8) & 0x1ffu;
-                    const uint32_t bin = c * kMaeBins + ((rel >> sh) & mask);
-                    const uint32_t old = atomicAdd(&s_lo[bin], a);
-                    if (old + a < old) atomicAdd(&s_hi[bin], 1u);
-                    if (COUNT) atomicAdd(&s_cn[bin], 1u);
+            for (int k = 0; k < kLaneW; k += 2) {
+                const float2 key = lut_key2(make_float2(x[k], x[k + 1]));
+                const float kk[2] = {key.x, key.y};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float xk = x[k + h];
+                    uint32_t c;
+                    if (use_lut) {
+                        const uint2 ent = lut_probe(kk[h], lut_base);
+                        c = ent.y + ((xk >= __uint_as_float(ent.x)) ? 1u : 0u);
+                    } else {
+                        c = (uint32_t)region_of(xk, s_xi);
+                    }
+                    e += T.unit ? fabsf(xk - s_lv[c]) : fabsf(fmaf(-m, s_lv[c], v[k + h]));
+                    const uint2 L = s_lvl1[c];
+                    if ((int32_t)L.y < 0) {
+                        // a member's rel is below 2^top, so its digit is rel >> (top - 9) as it stands; the
+                        // constant mask only keeps a non-finite input's garbage inside the level's bins.
+                        // The funnel shift takes the shift count from the low five bits of L.y.
+                        const uint32_t rel = order_key(xk) - L.x;
+                        const uint32_t bin = c * kMaeBins + (__funnelshift_r(rel, 0u, L.y) & (kMaeBins - 1u));
+                        const uint32_t old = atomicAdd(&s_lo[bin], a);
+                        if (old + a < old) atomicAdd(&s_hi[bin], 1u);
+                        if (COUNT) atomicAdd(&s_cn[bin], 1u);
+                    }
                 }
             }
             err += (double)e;
