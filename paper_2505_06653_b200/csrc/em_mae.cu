@@ -183,7 +183,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     __shared__ int s_multi;
     __shared__ WideScratch s_wide;
     __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
-    __shared__ uint2 s_lvl1[kLevels];  // first pass: {base, shift | on << 31}
+    __shared__ uint4 s_lvl1[kLevels];  // first pass: {base, shift | on << 31, level, -}
     __shared__ uint2 s_iv[kLutBins];  // later passes: bits of {lo, hi} per table bin (lo > hi: nothing)
     __shared__ float2 s_span[kLevels];
     __shared__ uint32_t s_qn;
@@ -204,7 +204,8 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         const uint32_t mask = (1u << (top - sh)) - 1u;
         s_lvl[tid] = make_uint4(W.state->base[tid], W.state->prefix[tid],
                                 (uint32_t)top | ((uint32_t)sh << 8) | (mask << 16), top > 0 ? 1u : 0u);
-        s_lvl1[tid] = make_uint2(W.state->base[tid], (uint32_t)sh | (top > 0 ? 0x80000000u : 0u));
+        s_lvl1[tid] = make_uint4(W.state->base[tid], (uint32_t)sh | (top > 0 ? 0x80000000u : 0u),
+                                 __float_as_uint(levels[tid]), 0u);
     }
     if (tid < T.count) {
         s_ptr[tid] = T.ptr[tid];
@@ -319,6 +320,13 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         if (FIRST) {
             const bool use_lut = lut_ok && safe;
             float e = 0.0f;
+            // error of a weight: |v - m xhat|; the normalised-domain variant measures |x - xhat|
+            float scale = m;
+            if (T.unit) {
+                scale = 1.0f;
+#pragma unroll
+                for (int k = 0; k < kLaneW; ++k) v[k] = x[k];
+            }
 #pragma unroll
             for (int k = 0; k < kLaneW; k += 2) {
                 const float2 key = lut_key2(make_float2(x[k], x[k + 1]));
@@ -333,8 +341,8 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
                     } else {
                         c = (uint32_t)region_of(xk, s_xi);
                     }
-                    e += T.unit ? fabsf(xk - s_lv[c]) : fabsf(fmaf(-m, s_lv[c], v[k + h]));
-                    const uint2 L = s_lvl1[c];
+                    const uint4 L = s_lvl1[c];
+                    e += fabsf(fmaf(-scale, __uint_as_float(L.z), v[k + h]));
                     if ((int32_t)L.y < 0) {
                         // a member's rel is below 2^top, so its digit is rel >> (top - 9) as it stands; the
                         // constant mask only keeps a non-finite input's garbage inside the level's bins.
