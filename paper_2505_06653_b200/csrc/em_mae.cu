@@ -183,7 +183,9 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     __shared__ int s_multi;
     __shared__ WideScratch s_wide;
     __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
-    __shared__ uint4 s_lvl1[kLevels];  // first pass: {base, shift | on << 31, level, -}
+    // first pass: {base, shift | on << 31, level, -}, one column per lane of a quarter warp (the unit
+    // a 16-byte shared-memory read is served in), so that the read never meets a bank conflict
+    __shared__ uint4 s_lvl1[kLevels * 8];
     __shared__ uint2 s_iv[kLutBins];  // later passes: bits of {lo, hi} per table bin (lo > hi: nothing)
     __shared__ float2 s_span[kLevels];
     __shared__ uint32_t s_qn;
@@ -204,8 +206,9 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
         const uint32_t mask = (1u << (top - sh)) - 1u;
         s_lvl[tid] = make_uint4(W.state->base[tid], W.state->prefix[tid],
                                 (uint32_t)top | ((uint32_t)sh << 8) | (mask << 16), top > 0 ? 1u : 0u);
-        s_lvl1[tid] = make_uint4(W.state->base[tid], (uint32_t)sh | (top > 0 ? 0x80000000u : 0u),
-                                 __float_as_uint(levels[tid]), 0u);
+        for (int q = 0; q < 8; ++q)
+            s_lvl1[tid * 8 + q] = make_uint4(W.state->base[tid], (uint32_t)sh | (top > 0 ? 0x80000000u : 0u),
+                                             __float_as_uint(levels[tid]), 0u);
     }
     if (tid < T.count) {
         s_ptr[tid] = T.ptr[tid];
@@ -341,7 +344,7 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
                     } else {
                         c = (uint32_t)region_of(xk, s_xi);
                     }
-                    const uint4 L = s_lvl1[c];
+                    const uint4 L = s_lvl1[c * 8 + (lane & 7)];
                     e += fabsf(fmaf(-scale, __uint_as_float(L.z), v[k + h]));
                     if ((int32_t)L.y < 0) {
                         // a member's rel is below 2^top, so its digit is rel >> (top - 9) as it stands; the
