@@ -19,10 +19,12 @@
 // against 128 bytes per clock and SM bound it to 16 code bytes per clock and SM, about two
 // thirds of what HBM could deliver.
 //
-// The codes travel global -> shared memory by asynchronous 16-byte copies into a ring that each
-// warp owns (kGvStages batches of kGvRows rows): a lane later reads back exactly the 16 bytes it
-// copied itself, so the ring needs no barrier, costs no registers, and keeps kGvStages - 1
-// batches per warp in flight whatever the arithmetic is doing.  The per-lane partial sums of a
+// A CTA of up to 16 warps (cols <= 16384) runs with 128 registers per thread and requests the
+// next batch of kGvRows rows straight into registers before it uses the current one.  The
+// 32-warp CTA of wider matrices has 64 registers per thread and no room for that: its codes
+// travel global -> shared memory by asynchronous 16-byte copies into a ring that each warp owns
+// (kGvStages batches); a lane later reads back exactly the 16 bytes it copied itself, so the
+// ring needs no barrier and costs no registers.  The per-lane partial sums of a
 // batch are reduced over the warp with a halving butterfly, then every kGvDefer batches over the
 // stripes through shared memory in a fixed order.  Nothing is accumulated with atomics, so y is
 // bit-reproducible.
@@ -135,7 +137,9 @@ __device__ __forceinline__ void load_x<F32>(const void* x, int64_t c0, bool live
 
 // MAXT = 512 (up to 16 stripes; 128 registers per thread keep many look-ups of a warp in flight,
 // which measured faster than twice the warps) or 1024 (17 ... 32 stripes).  One CTA per SM.
-template <class ST, class XT, int MAXT>
+constexpr bool kGvRing512 = false;  // the 512-thread variant prefetches into registers (measured 8 % faster)
+
+template <class ST, class XT, int MAXT, bool RING>
 __global__ void __launch_bounds__(MAXT, 1)
 gemv_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t rows, int64_t cols,
             int block_shift, const float* __restrict__ levels, const void* __restrict__ x, float* __restrict__ y,
@@ -163,6 +167,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, 
     // codes for this lane start at src.  Nothing is copied for rows past the end or dead lanes:
     // whatever the slot then holds is multiplied by a zero block constant.
     auto issue = [&](const uint8_t* src, int64_t left, int stage) {
+        if (!RING) return;
 #pragma unroll
         for (int u = 0; u < R; ++u) {
             if (live && u < left)
@@ -171,6 +176,17 @@ gemv_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, 
                              : "memory");
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    // Without the ring: the same 16 bytes per row straight into registers (zeros past the end).
+    auto fetch = [&](const uint8_t* src, int64_t left, uint4(&c)[R]) {
+#pragma unroll
+        for (int u = 0; u < R; ++u) {
+            c[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (live && u < left)
+                asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(c[u].x), "=r"(c[u].y), "=r"(c[u].z), "=r"(c[u].w)
+                             : "l"(src + u * row_bytes));
+        }
     };
     // block constants of a batch; index = that of this lane's block in the batch's first row
     auto block_constants = [&](int64_t index, int64_t left, float(&m)[R]) {
@@ -185,9 +201,15 @@ gemv_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, 
     const uint8_t* src = codes + ((r_first * cols + c0) >> 1);               // codes of the next batch to request
     int64_t blk = (r_first * cols + c0) >> block_shift;                      // block of the next batch's constants
     // The first codes, x and the levels are requested together: the cold misses overlap.
+    uint4 cc[R];
+    if (RING) {
 #pragma unroll
-    for (int sI = 0; sI < S - 1; ++sI) {
-        issue(src, left - sI * step_rows, sI);
+        for (int sI = 0; sI < S - 1; ++sI) {
+            issue(src, left - sI * step_rows, sI);
+            src += step_bytes;
+        }
+    } else {
+        fetch(src, left, cc);
         src += step_bytes;
     }
     float m[R];
@@ -207,19 +229,30 @@ gemv_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, 
     int k = 0, buf = 0, stage = 0;
     for (; b0 < batches; b0 += bstep) {
         // refill the slot consumed in the previous iteration, then wait for this iteration's batch
-        issue(src, left - (S - 1) * step_rows, stage == 0 ? S - 1 : stage - 1);
+        // (registers: request the next batch before this one is used)
+        uint4 cn[R];
+        if (RING)
+            issue(src, left - (S - 1) * step_rows, stage == 0 ? S - 1 : stage - 1);
+        else
+            fetch(src, left - step_rows, cn);
         src += step_bytes;
         float mn[R];
         block_constants(blk, left - step_rows, mn);  // block constants run one batch ahead in registers
         blk += step_blocks;
         left -= step_rows;
-        asm volatile("cp.async.wait_group %0;" ::"n"(S - 1) : "memory");
         uint32_t word[R][4];
+        if (RING) {
+            asm volatile("cp.async.wait_group %0;" ::"n"(S - 1) : "memory");
 #pragma unroll
-        for (int u = 0; u < R; ++u)
-            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                         : "=r"(word[u][0]), "=r"(word[u][1]), "=r"(word[u][2]), "=r"(word[u][3])
-                         : "r"(ring + (uint32_t)(stage * R + u) * 512u));
+            for (int u = 0; u < R; ++u)
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(word[u][0]), "=r"(word[u][1]), "=r"(word[u][2]), "=r"(word[u][3])
+                             : "r"(ring + (uint32_t)(stage * R + u) * 512u));
+        } else {
+#pragma unroll
+            for (int u = 0; u < R; ++u)
+                word[u][0] = cc[u].x, word[u][1] = cc[u].y, word[u][2] = cc[u].z, word[u][3] = cc[u].w;
+        }
         uint64_t a2[R];
 #pragma unroll
         for (int u = 0; u < R; ++u) a2[u] = 0ull;
@@ -262,9 +295,12 @@ gemv_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, 
         }
         stage = (stage == S - 1) ? 0 : stage + 1;
 #pragma unroll
-        for (int u = 0; u < R; ++u) m[u] = mn[u];
+        for (int u = 0; u < R; ++u) {
+            m[u] = mn[u];
+            if (!RING) cc[u] = cn[u];
+        }
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");  // nothing of this CTA is in flight when it ends
+    if (RING) asm volatile("cp.async.wait_group 0;" ::: "memory");  // nothing of this CTA is in flight when it ends
 }
 
 // Sparse correction: y[row] += sum over the row's outliers of (val - scale * xhat[code]) * x.
@@ -331,9 +367,11 @@ static int launch_gemv_kernel(const uint8_t* d_codes, const void* d_scales, int6
     const int grid = (int)(want < kSMs ? want : kSMs);  // one CTA per SM (its shared memory fills the SM)
     int block_shift = 0;
     while ((1 << block_shift) < block_size) ++block_shift;
-    auto kern = gemv_kernel<ST, XT, MAXT>;
-    BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, gv_smem(MAXT)));
-    kern<<<grid, 32 * stripes * groups, gv_smem(MAXT), st>>>(d_codes, d_scales, rows, cols, block_shift, d_codebook,
+    constexpr bool RING = MAXT > 512 || kGvRing512;
+    constexpr int smem = RING ? gv_smem(MAXT) : kGvTabBytes;
+    auto kern = gemv_kernel<ST, XT, MAXT, RING>;
+    BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kern<<<grid, 32 * stripes * groups, smem, st>>>(d_codes, d_scales, rows, cols, block_shift, d_codebook,
                                                              d_x, d_y, stripes, groups);
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
