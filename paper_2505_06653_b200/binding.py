@@ -25,8 +25,9 @@ METRIC_MSE_NORMALIZED, METRIC_MAE_NORMALIZED = 2, 3  # App. D: errors of the nor
 OP_EM, OP_OPQ = 0, 1
 LEVELS = 16
 
-# kernels one MAE iteration enqueues: setup, 4 x (data pass + bin selection), level update
-MAE_LAUNCHES_PER_ITERATION = 10
+# kernels one MAE iteration enqueues: setup, 2 x (data pass + bin selection), then 2 data passes
+# that carry their own selection and the level update
+MAE_LAUNCHES_PER_ITERATION = 7
 
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",

@@ -44,6 +44,7 @@ struct MaeState {
     uint32_t cand_count[kLevels];        // samples offered to the candidate list of level l
     uint32_t active;                     // bit l: level l takes part in the selection
     uint32_t max_bits;                   // bits of the largest |w| of the data
+    uint32_t ticket;                     // CTAs of a pass with a fused selection that have finished
 };
 static_assert(sizeof(MaeState) <= kEmMaeStateBytes, "state must fit its slot");
 
@@ -152,6 +153,124 @@ mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
     }
 }
 
+// ---------------------------------------------------------------- bin selection
+
+// Block-wide step of the selection, one thread per bin (threads beyond the bins pass 0): given this thread's bin weight `mine`,
+// finds the first bin j with 2 (before + cumulative(j)) >= total.  Returns through the shared
+// result the bin and the cumulative weight below it.  *all_out = sum of all bins.
+struct PickResult {
+    int bin;
+    unsigned long long excl;
+};
+
+template <int NT = kMaeBins>
+__device__ __forceinline__ PickResult pick_bin(unsigned long long mine, unsigned long long before,
+                                               unsigned long long total, bool total_is_sum,
+                                               unsigned long long* s_wsum, PickResult* s_res,
+                                               unsigned long long* all_out)
+{
+    const int j = threadIdx.x, lane = j & 31, warp = j >> 5;
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long t = __shfl_up_sync(kFull, incl, off);
+        if (lane >= off) incl += t;
+    }
+    __syncthreads();  // s_wsum / s_res may still be read from a previous call
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    unsigned long long carry = 0ull, all = 0ull;
+    for (int k = 0; k < NT / 32; ++k) {
+        if (k < warp) carry += s_wsum[k];
+        all += s_wsum[k];
+    }
+    incl += carry;
+    if (total_is_sum) total = all;
+    const unsigned long long excl = incl - mine;
+    const bool reached = 2ull * (before + incl) >= total;
+    const bool prev_reached = (j > 0) && (2ull * (before + excl) >= total);
+    if (reached && !prev_reached) *s_res = PickResult{j, excl};  // exactly one thread: monotone
+    __syncthreads();
+    *all_out = all;
+    return *s_res;
+}
+
+// The next digit of level l after a pass that was not the first: the bin of the global
+// histogram (cleared on the way) in which the cumulative weight reaches half of the region's
+// total.  Called by all NT threads of a CTA; threads beyond the bins only take part in the scan.
+template <int NT>
+__device__ __forceinline__ void select_body(const MaeWs& W, int l, unsigned long long* s_wsum, PickResult* s_res)
+{
+    MaeState* S = W.state;
+    const int j = threadIdx.x;
+    const int top = S->top[l];
+    if (top <= 0) return;  // uniform over the CTA
+    unsigned long long mine = 0ull;
+    if (j < kMaeBins) {
+        mine = __ldcg(&W.hist[l * kMaeBins + j]);
+        W.hist[l * kMaeBins + j] = 0ull;
+    }
+    const unsigned long long before = S->before[l];
+    unsigned long long all;
+    const PickResult r = pick_bin<NT>(mine, before, S->total[l], false, s_wsum, s_res, &all);
+    if (j == 0) {
+        const int sh = max(top - kMaeDigitBits, 0);
+        S->before[l] = before + r.excl;
+        S->prefix[l] = (S->prefix[l] << (top - sh)) | (uint32_t)r.bin;
+        S->top[l] = sh;
+    }
+}
+
+// What the level update needs beside the selection state.
+struct MaeFinal {
+    int enabled;  // the pass that carries this is the iteration's last launch and ends with the update
+    int n_records;
+    int64_t n_total;
+    const float* levels_in;
+    float* levels_out;
+    uint32_t skip_mask;
+    bof4_em_stats* stats;
+    double* err_slot;
+    int unit;
+};
+
+// Level update and statistics of one iteration, by all threads of one CTA (s_part: one double per warp).
+__device__ __forceinline__ void finalize_body(const MaeWs& W, const MaeFinal& F, double* s_part)
+{
+    const MaeState* S = W.state;
+    double e = 0.0;
+    for (int r = threadIdx.x; r < F.n_records; r += blockDim.x) e += __ldcg(&W.partials[(size_t)r * kEmRecordDoubles]);
+#pragma unroll
+    for (int off = 16; off; off >>= 1) e += __shfl_xor_sync(kFull, e, off);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = e;
+    __syncthreads();
+    if (threadIdx.x < kLevels) {
+        const int l = threadIdx.x;
+        const float old = F.levels_in[l];
+        const bool on = !((F.skip_mask >> l) & 1u);
+        const unsigned long long total = S->total[l];
+        const float med = (on && total > 0ull) ? key_to_float(S->base[l] + S->prefix[l]) : old;
+        if (F.stats) {
+            const int emax = max((int)(S->max_bits >> 23), 1);
+            F.stats->s1[l] = 0.0;
+            F.stats->s0[l] = F.unit ? (double)total : ldexp((double)total, emax - 157);  // undo the fixed-point scale
+            F.stats->count[l] = S->count[l];
+            F.stats->median[l] = med;
+        }
+        if (F.levels_out && on) F.levels_out[l] = med;
+    }
+    if (threadIdx.x == 0) {
+        double err = 0.0;
+        for (int k = 0; k < (int)(blockDim.x >> 5); ++k) err += s_part[k];  // warp order: fixed
+        if (F.stats) {
+            F.stats->err_sum = err;
+            F.stats->n_total = F.n_total;
+        }
+        if (F.err_slot) *F.err_slot = (F.n_total > 0) ? err / (double)F.n_total : 0.0;
+    }
+}
+
 // ---------------------------------------------------------------- data pass
 
 // FIRST: every member of an active level takes part; also accumulates sum |w - m xhat[c]| (one
@@ -166,9 +285,13 @@ mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
 // COLLECT (second pass): every participating sample is also appended to its level's list.
 constexpr int kMaeQueue = kLevels * kMaeBins * 4 / 8;  // entries {x, weight} in the count histogram's space
 
-template <class DT, int I, bool SIGNED, bool FIRST, bool COUNT, bool COLLECT>
+// TAIL (a later pass without a candidate list): the CTA that finishes last, found by an atomic
+// ticket so that nobody waits, also selects the next digit of every level and, if F.enabled,
+// updates the levels: one launch instead of three.  When nothing is left the whole grid
+// returns at once and CTA 0 does the update.
+template <class DT, int I, bool SIGNED, bool FIRST, bool COUNT, bool COLLECT, bool TAIL>
 __global__ void __launch_bounds__(kMaeThreads, 1)
-mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
+mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W, const MaeFinal F)
 {
     extern __shared__ __align__(16) unsigned char s_raw[];
     unsigned char* s_lut = s_raw;
@@ -193,10 +316,16 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
     __shared__ const void* s_ptr[kEmMaxTensors];
     __shared__ int64_t s_n[kEmMaxTensors], s_row_end[kEmMaxTensors];
 
+    __shared__ unsigned long long s_wsum[kMaeThreads / 32];
+    __shared__ PickResult s_res;
+    __shared__ int s_last;
     if (!FIRST) {  // nothing left to resolve: uniform over the grid
         int any = 0;
         for (int l = 0; l < kLevels; ++l) any |= W.state->top[l];
-        if (any <= 0) return;
+        if (any <= 0) {
+            if (TAIL && F.enabled && T.last && blockIdx.x == 0) finalize_body(W, F, s_err);
+            return;
+        }
     }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     make_thresholds(levels, s_xi, s_lv, tid);
@@ -425,47 +554,23 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
             rec[0] = T.accumulate ? rec[0] + t : t;
         }
     }
-}
-
-// ---------------------------------------------------------------- bin selection
-
-// Block-wide step of the selection, one thread per bin: given this thread's bin weight `mine`,
-// finds the first bin j with 2 (before + cumulative(j)) >= total.  Returns through the shared
-// result the bin and the cumulative weight below it.  *all_out = sum of all bins.
-struct PickResult {
-    int bin;
-    unsigned long long excl;
-};
-
-__device__ __forceinline__ PickResult pick_bin(unsigned long long mine, unsigned long long before,
-                                               unsigned long long total, bool total_is_sum,
-                                               unsigned long long* s_wsum, PickResult* s_res,
-                                               unsigned long long* all_out)
-{
-    const int j = threadIdx.x, lane = j & 31, warp = j >> 5;
-    unsigned long long incl = mine;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const unsigned long long t = __shfl_up_sync(kFull, incl, off);
-        if (lane >= off) incl += t;
+    if (TAIL && T.last) {
+        // every thread's histogram atomics are ordered before the ticket of its CTA
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = (atomicAdd(&W.state->ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            for (int l = 0; l < kLevels; ++l) select_body<kMaeThreads>(W, l, s_wsum, &s_res);
+            if (tid == 0) W.state->ticket = 0u;
+            if (F.enabled) {
+                __threadfence();
+                __syncthreads();  // the state written by thread 0 is read by the update
+                finalize_body(W, F, s_err);
+            }
+        }
     }
-    __syncthreads();  // s_wsum / s_res may still be read from a previous call
-    if (lane == 31) s_wsum[warp] = incl;
-    __syncthreads();
-    unsigned long long carry = 0ull, all = 0ull;
-    for (int k = 0; k < kMaeBins / 32; ++k) {
-        if (k < warp) carry += s_wsum[k];
-        all += s_wsum[k];
-    }
-    incl += carry;
-    if (total_is_sum) total = all;
-    const unsigned long long excl = incl - mine;
-    const bool reached = 2ull * (before + incl) >= total;
-    const bool prev_reached = (j > 0) && (2ull * (before + excl) >= total);
-    if (reached && !prev_reached) *s_res = PickResult{j, excl};  // exactly one thread: monotone
-    __syncthreads();
-    *all_out = all;
-    return *s_res;
 }
 
 // One CTA per level, one thread per bin.  For a level with bits left: the bin in which the
@@ -577,42 +682,10 @@ mae_resolve_kernel(MaeWs W)
 // ---------------------------------------------------------------- level update
 
 __global__ void __launch_bounds__(256)
-mae_finalize_kernel(MaeWs W, int n_records, int64_t n_total, const float* levels_in, float* levels_out,
-                    uint32_t skip_mask, bof4_em_stats* __restrict__ stats, double* __restrict__ err_slot,
-                    int unit)
+mae_finalize_kernel(MaeWs W, const MaeFinal F)
 {
     __shared__ double s_part[8];
-    const MaeState* S = W.state;
-    double e = 0.0;
-    for (int r = threadIdx.x; r < n_records; r += blockDim.x) e += W.partials[(size_t)r * kEmRecordDoubles];
-#pragma unroll
-    for (int off = 16; off; off >>= 1) e += __shfl_xor_sync(kFull, e, off);
-    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = e;
-    __syncthreads();
-    if (threadIdx.x < kLevels) {
-        const int l = threadIdx.x;
-        const float old = levels_in[l];
-        const bool on = !((skip_mask >> l) & 1u);
-        const unsigned long long total = S->total[l];
-        const float med = (on && total > 0ull) ? key_to_float(S->base[l] + S->prefix[l]) : old;
-        if (stats) {
-            const int emax = max((int)(S->max_bits >> 23), 1);
-            stats->s1[l] = 0.0;
-            stats->s0[l] = unit ? (double)total : ldexp((double)total, emax - 157);  // undo the fixed-point scale
-            stats->count[l] = S->count[l];
-            stats->median[l] = med;
-        }
-        if (levels_out && on) levels_out[l] = med;
-    }
-    if (threadIdx.x == 0) {
-        double err = 0.0;
-        for (int k = 0; k < 8; ++k) err += s_part[k];
-        if (stats) {
-            stats->err_sum = err;
-            stats->n_total = n_total;
-        }
-        if (err_slot) *err_slot = (n_total > 0) ? err / (double)n_total : 0.0;
-    }
+    finalize_body(W, F, s_part);
 }
 
 // ================================================================= host side
@@ -621,30 +694,32 @@ namespace {
 
 template <class DT, int I, bool SG>
 int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, int pass, bool collect,
-                bool count, cudaStream_t st)
+                bool count, const MaeFinal* tail, cudaStream_t st)
 {
-#define BOF4_MAE_GO(FIRST_, COUNT_, COLLECT_)                                                           \
+    const MaeFinal F = tail ? *tail : MaeFinal{};
+#define BOF4_MAE_GO(FIRST_, COUNT_, COLLECT_, TAIL_)                                                    \
     {                                                                                                   \
-        auto kern = mae_pass_kernel<DT, I, SG, FIRST_, COUNT_, COLLECT_>;                               \
+        auto kern = mae_pass_kernel<DT, I, SG, FIRST_, COUNT_, COLLECT_, TAIL_>;                        \
         BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaeSmem)); \
-        kern<<<kEmGrid, kMaeThreads, kMaeSmem, st>>>(T, d_levels, W);                                   \
+        kern<<<kEmGrid, kMaeThreads, kMaeSmem, st>>>(T, d_levels, W, F);                                \
     }
-    if (pass == 0 && count) BOF4_MAE_GO(true, true, false)
-    else if (pass == 0) BOF4_MAE_GO(true, false, false)
-    else if (collect) BOF4_MAE_GO(false, false, true)
-    else BOF4_MAE_GO(false, false, false)
+    if (pass == 0 && count) BOF4_MAE_GO(true, true, false, false)
+    else if (pass == 0) BOF4_MAE_GO(true, false, false, false)
+    else if (collect) BOF4_MAE_GO(false, false, true, false)
+    else if (tail) BOF4_MAE_GO(false, false, false, true)
+    else BOF4_MAE_GO(false, false, false, false)
 #undef BOF4_MAE_GO
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }
 
 int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, const MaeWs& W, int pass,
-                  bool collect, bool count, cudaStream_t st)
+                  bool collect, bool count, const MaeFinal* tail, cudaStream_t st)
 {
     const bool sg = a.norm == BOF4_NORM_SIGNED;
-#define BOF4_MAE_I(DT_, I_)                                                       \
-    return sg ? launch_pass<DT_, I_, true>(T, d_levels, W, pass, collect, count, st)   \
-              : launch_pass<DT_, I_, false>(T, d_levels, W, pass, collect, count, st);
+#define BOF4_MAE_I(DT_, I_)                                                             \
+    return sg ? launch_pass<DT_, I_, true>(T, d_levels, W, pass, collect, count, tail, st)   \
+              : launch_pass<DT_, I_, false>(T, d_levels, W, pass, collect, count, tail, st);
 #define BOF4_MAE_DT(DT_)                         \
     switch (a.block_size) {                      \
         case 32: BOF4_MAE_I(DT_, 32)             \
@@ -693,24 +768,45 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
     if (const char* env = getenv("BOF4_MAE_COLLECT_PASS")) {
         if (env[0] == '1' || env[0] == '2') collect_pass = env[0] - '0';
     }
+    MaeFinal fin{};
+    fin.n_records = kEmGrid;
+    fin.n_total = a.n_total;
+    fin.levels_in = d_levels_in;
+    fin.levels_out = d_levels_out;
+    fin.skip_mask = skip_mask;
+    fin.stats = d_stats;
+    fin.err_slot = d_err_slot;
+    fin.unit = a.metric >= 2 ? 1 : 0;
+    bool updated = false;
     for (int p = 0; p < kMaeMaxPasses; ++p) {
         const bool first = p == 0;
+        // From the third pass on (they usually find nothing left to do) the selection and, in the
+        // last pass, the level update ride in the pass kernel itself.
+        const bool fused = p >= 2 && p != collect_pass;
+        fin.enabled = (fused && p == kMaeMaxPasses - 1) ? 1 : 0;
         auto fire = [&](const EmTensors& T) -> int {
-            return dispatch_pass(a, T, d_levels_in, W, p, p == collect_pass, first && d_stats != nullptr, st);
+            return dispatch_pass(a, T, d_levels_in, W, p, p == collect_pass, first && d_stats != nullptr,
+                                 fused ? &fin : nullptr, st);
         };
         int calls = 0;
         const int rc = for_each_tensor_chunk(a, kMaeRow, fire, &calls);
         if (rc) return rc;
         if (first && calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(W.partials, 0, kEmPartialBytes, st));
+        if (fused && calls > 0) {
+            updated = fin.enabled != 0;
+            continue;
+        }
         if (p == collect_pass)
             mae_resolve_kernel<<<kLevels, kMaeBins, 0, st>>>(W);
         else
             mae_select_kernel<<<kLevels, kMaeBins, 0, st>>>(W, first ? 1 : 0);
         BOF4_CUDA_TRY(cudaGetLastError());
     }
-    mae_finalize_kernel<<<1, 256, 0, st>>>(W, kEmGrid, a.n_total, d_levels_in, d_levels_out, skip_mask,
-                                           d_stats, d_err_slot, a.metric >= 2 ? 1 : 0);
-    BOF4_CUDA_TRY(cudaGetLastError());
+    if (!updated) {
+        fin.enabled = 1;
+        mae_finalize_kernel<<<1, 256, 0, st>>>(W, fin);
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
     return BOF4_OK;
 }
 

@@ -385,6 +385,27 @@ def test_non_finite_weights_do_not_disturb_other_blocks(bof4):
     assert st["n"] == n
 
 
+def test_mae_candidate_list_overflow_takes_the_later_data_passes(bof4):
+    """Two million normalised weights within one first-digit bin of a free level (four distinct
+    values around 0.5): the candidate list of that level overflows, so the third and fourth data
+    passes, which carry their own selection and the level update, have to finish the median."""
+    I, nb = 32, 1 << 16
+    g = torch.Generator().manual_seed(77)
+    k = torch.randint(0, 4, (nb, I), generator=g).float()
+    x = 0.5 + k * 2.0 ** -13
+    x[:, 0] = 1.0                                            # the block maximum
+    x[:, 1] = -(0.25 + torch.randint(0, 64, (nb,), generator=g).float() * 2.0 ** -9)  # some spread elsewhere
+    scale = 2.0 ** (torch.arange(nb) % 5 - 2).float()        # block constants 1/4 ... 4: unequal weights
+    w = (x * scale[:, None]).reshape(-1).contiguous()        # exact in fp32
+    ref = oracle.em_accumulate_mae(w, I, 1, LV_INIT)
+    assert ref["count"][11] > 65536 * 16                     # level 0.5 holds the 2 M samples
+    got = bof4.bof4_em_step([w.cuda()], I, 1, bof4.METRIC_MAE, LV_INIT)
+    _check_mae_stats(got, ref, LV_INIT)
+    # the same through the fit entry point: one iteration moves level 11 to that median
+    lv, log = bof4.bof4_fit_codebook([w.cuda()], I, 1, bof4.METRIC_MAE, LV_INIT, 0, 1)
+    assert lv.cpu().numpy()[11] == ref["median"][11]
+
+
 def test_mae_collecting_pass_choice_does_not_change_results(bof4):
     """The pass that fills the candidate lists is chosen from the data size; forcing the other
     choice (as for very large inputs) must give the same medians, bit for bit."""
