@@ -143,6 +143,9 @@ class Step:
         self.cnt = torch.zeros(1, dtype=torch.int64, device=dev)
         self.out = torch.empty(n, dtype=torch.bfloat16, device=dev)
         self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        # result buffers of the two fits (levels, error log): no allocation inside the timed region
+        self.fit_out = [(torch.empty(16, dtype=torch.float32, device=dev),
+                         torch.zeros(1, dtype=torch.float64, device=dev)) for _ in range(2)]
         self.cb_mse = self.cb_mae = self.cb0
         self.log_mse = torch.zeros(1, dtype=torch.float64, device=dev)
         self.have_mae = True
@@ -158,12 +161,14 @@ class Step:
     def em_mse(self):
         b = self.b
         self.cb_mse, self.log_mse = b.bof4_fit_codebook([self.w], I, b.NORM_SIGNED, b.METRIC_MSE, self.cb0,
-                                                        self.mask, 1, workspace=self.ws_em, sync=False)
+                                                        self.mask, 1, workspace=self.ws_em, sync=False,
+                                                        out=self.fit_out[0])
 
     def em_mae(self):
         b = self.b
         self.cb_mae, self.log_mae = b.bof4_fit_codebook([self.w], I, b.NORM_SIGNED, b.METRIC_MAE, self.cb0,
-                                                        self.mask, 1, workspace=self.ws_em, sync=False)
+                                                        self.mask, 1, workspace=self.ws_em, sync=False,
+                                                        out=self.fit_out[1])
 
     def quant(self):
         b = self.b

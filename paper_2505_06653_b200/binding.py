@@ -198,15 +198,22 @@ def bof4_em_step(weights, block_size: int, norm: int, metric: int, levels,
 
 def bof4_fit_codebook(weights, block_size: int, norm: int, metric: int, levels, fixed_mask: int,
                       iters: int, workspace: Optional[torch.Tensor] = None,
-                      sync: bool = True):
+                      sync: bool = True, out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None):
     """``iters`` Lloyd iterations; returns (levels, err_log) as device tensors (fp32[16],
-    fp64[iters]).  With sync=False nothing waits for the stream."""
+    fp64[iters]).  With sync=False nothing waits for the stream.  `out` = (fp32[16], fp64[>= iters])
+    device tensors to hold the results instead of fresh allocations."""
     ws, dt, ptrs, sizes = _tensor_list(weights)
     dev = ws[0].device
-    cb = _codebook(levels, dev).clone()
+    if out is not None:
+        cb, log = _dev(out[0], "out[0]"), _dev(out[1], "out[1]")
+        if cb.dtype != torch.float32 or cb.numel() != LEVELS or log.dtype != torch.float64 or log.numel() < iters:
+            raise ValueError("out must be (float32[16], float64[>= iters])")
+        cb.copy_(_codebook(levels, dev))
+    else:
+        cb = _codebook(levels, dev).clone()
+        log = torch.zeros(max(iters, 1), dtype=torch.float64, device=dev)
     wsp = workspace if workspace is not None else _workspace(
         OP_EM, max(w.numel() for w in ws), block_size, metric, dev)
-    log = torch.zeros(max(iters, 1), dtype=torch.float64, device=dev)
     with torch.cuda.device(dev):
         _check(lib().bof4_fit_codebook(ptrs, sizes, len(ws), dt, block_size, norm, metric, _ptr(cb),
                                        fixed_mask, iters, _ptr(log), _ptr(wsp), wsp.numel(), _stream()))

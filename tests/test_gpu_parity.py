@@ -385,6 +385,20 @@ def test_non_finite_weights_do_not_disturb_other_blocks(bof4):
     assert st["n"] == n
 
 
+def test_fit_into_caller_buffers(bof4):
+    """`out=` makes the binding write levels and error log into the caller's tensors."""
+    I, n = 64, 1 << 16
+    w = make_weights(n, torch.bfloat16, 88).cuda()
+    lv, log = bof4.bof4_fit_codebook([w], I, 1, bof4.METRIC_MSE, LV_INIT, workloads.FIXED_BOF4S, 3)
+    cb = torch.empty(16, dtype=torch.float32, device="cuda")
+    lg = torch.full((5,), -1.0, dtype=torch.float64, device="cuda")
+    lv2, log2 = bof4.bof4_fit_codebook([w], I, 1, bof4.METRIC_MSE, LV_INIT, workloads.FIXED_BOF4S, 3, out=(cb, lg))
+    assert lv2.data_ptr() == cb.data_ptr() and log2.numel() == 3
+    assert torch.equal(lv, cb) and torch.equal(log, lg[:3]) and float(lg[3]) == -1.0
+    with pytest.raises(ValueError):
+        bof4.bof4_fit_codebook([w], I, 1, bof4.METRIC_MSE, LV_INIT, 0, 3, out=(cb, lg[:2]))
+
+
 def test_mae_candidate_list_overflow_takes_the_later_data_passes(bof4):
     """Two million normalised weights within one first-digit bin of a free level (four distinct
     values around 0.5): the candidate list of that level overflows, so the third and fourth data
