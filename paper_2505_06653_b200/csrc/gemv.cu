@@ -167,15 +167,17 @@ gemv_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, 
     // codes for this lane start at src.  Nothing is copied for rows past the end or dead lanes:
     // whatever the slot then holds is multiplied by a zero block constant.
     auto issue = [&](const uint8_t* src, int64_t left, int stage) {
-        if (!RING) return;
+        if constexpr (RING) {
 #pragma unroll
-        for (int u = 0; u < R; ++u) {
-            if (live && u < left)
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring + (uint32_t)(stage * R + u) * 512u),
-                             "l"(src + u * row_bytes)
-                             : "memory");
+            for (int u = 0; u < R; ++u) {
+                if (live && u < left)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring +
+                                                                                  (uint32_t)(stage * R + u) * 512u),
+                                 "l"(src + u * row_bytes)
+                                 : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
     };
     // Without the ring: the same 16 bytes per row straight into registers (zeros past the end).
     auto fetch = [&](const uint8_t* src, int64_t left, uint4(&c)[R]) {
