@@ -12,7 +12,13 @@
  *    enqueued on that stream and the call returns without synchronising; outputs are valid once
  *    the stream has reached the end of the enqueued work.
  *  - Weights are a flattened tensor of n elements cut into B = n / block_size contiguous blocks
- *    (Sec. 2.1).  block_size is a power of two from 32 to 4096 and n must be a multiple of it.
+ *    (Sec. 2.1).  block_size is a power of two from 32 to 4096.  The EM entry points and
+ *    opq_split_static need n to be a multiple of it.  bof4_quantize, bof4_dequantize, opq_split
+ *    and bof4_quantize_opq also take a ragged tensor: its last block is simply shorter (its own
+ *    maximum; its own mean and deviation over its own length, the two tree sums padded with
+ *    zeros to the next power of two; a one-weight block has no outliers), there are
+ *    ceil(n / block_size) block constants and (n + 1) / 2 code bytes, and a code byte that holds a
+ *    single weight has a zero low nibble.  The paper only uses whole blocks.
  *  - Weight tensors, code arrays and dequantised outputs are accessed with 32-byte vector
  *    instructions: their device pointers must be 32-byte aligned (BOF4_ERR_INVALID_ARG if not).
  *  - A codebook is 16 fp32 reconstruction levels in ASCENDING order, device resident.  Code c
@@ -45,7 +51,7 @@ extern "C" {
 /* ---- status codes ---- */
 #define BOF4_OK 0
 #define BOF4_ERR_INVALID_ARG (-1) /* NULL pointer, negative size, bad enum value            */
-#define BOF4_ERR_SHAPE (-2)       /* block size unsupported, n not a multiple, n too large  */
+#define BOF4_ERR_SHAPE (-2)       /* block size unsupported, n not a multiple where it must be, n too large */
 #define BOF4_ERR_DTYPE (-3)       /* dtype code unknown or combination not supported        */
 #define BOF4_ERR_WORKSPACE (-4)   /* workspace NULL, misaligned or smaller than required    */
 #define BOF4_ERR_CAPACITY (-5)    /* outlier list capacity is negative or too large         */
@@ -138,8 +144,8 @@ BOF4_API int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int n
 /*
  * Block-wise quantisation (Sec. 2.1 Eq. 1-3, Sec. 3.1 Eq. 4): per block the constant m,
  * x = w / m (x = 0 for an all-zero block), code = region of x.
- *   d_codes   out [n/2] bytes; byte k = (code[2k] << 4) | code[2k+1]
- *   d_scales  out [n/block_size] block constants, dtype scale_dtype.  The constant is stored
+ *   d_codes   out [(n+1)/2] bytes; byte k = (code[2k] << 4) | code[2k+1]
+ *   d_scales  out [ceil(n/block_size)] block constants, dtype scale_dtype.  The constant is stored
  *             exactly: scale_dtype must equal w_dtype, or be BOF4_F32 for bf16 weights.
  */
 BOF4_API int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_size, int norm,

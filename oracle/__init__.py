@@ -86,9 +86,14 @@ def _levels(xhat) -> np.ndarray:
     return a.copy()
 
 
-def _check(n: int, I: int):
-    if I <= 0 or n % I:
+def _check(n: int, I: int, ragged: bool = False):
+    """Whole blocks only, unless the function takes a shorter last block (ragged)."""
+    if I <= 0 or (n % I and not ragged):
         raise ValueError("n must be a multiple of the block size")
+
+
+def _blocks(n: int, I: int) -> int:
+    return (n + I - 1) // I
 
 
 # --------------------------------------------------------------------------- functions
@@ -103,8 +108,8 @@ def thresholds(xhat) -> np.ndarray:
 
 def block_constants(w, I: int, norm: int) -> np.ndarray:
     a = as_f32(w)
-    _check(a.size, I)
-    m = np.empty(a.size // I, np.float32)
+    _check(a.size, I, ragged=True)
+    m = np.empty(_blocks(a.size, I), np.float32)
     _load().orc_block_constants(_p(a), ctypes.c_int64(a.size), I, norm, _p(m))
     return m
 
@@ -112,21 +117,23 @@ def block_constants(w, I: int, norm: int) -> np.ndarray:
 def quantize(w, I: int, norm: int, xhat) -> Tuple[np.ndarray, np.ndarray]:
     """-> (codes uint8 [n/2], scales fp32 [n/I])."""
     a = as_f32(w)
-    _check(a.size, I)
+    _check(a.size, I, ragged=True)
     lv = _levels(xhat)
-    codes = np.empty(a.size // 2, np.uint8)
-    scales = np.empty(a.size // I, np.float32)
+    codes = np.empty((a.size + 1) // 2, np.uint8)
+    scales = np.empty(_blocks(a.size, I), np.float32)
     _load().orc_quantize(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv), _p(codes), _p(scales))
     return codes, scales
 
 
-def dequantize(codes: np.ndarray, scales: np.ndarray, I: int, xhat) -> np.ndarray:
-    """-> fp32 products m * xhat(code), before any rounding to the output type."""
+def dequantize(codes: np.ndarray, scales: np.ndarray, I: int, xhat, n: Optional[int] = None) -> np.ndarray:
+    """-> fp32 products m * xhat(code), before any rounding to the output type.  `n` = number of
+    weights when it is not twice the number of code bytes (an odd count)."""
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
     scales = np.ascontiguousarray(scales, dtype=np.float32)
-    n = codes.size * 2
-    _check(n, I)
-    assert scales.size == n // I
+    n = codes.size * 2 if n is None else int(n)
+    assert (n + 1) // 2 == codes.size
+    _check(n, I, ragged=True)
+    assert scales.size == _blocks(n, I)
     lv = _levels(xhat)
     out = np.empty(n, np.float32)
     _load().orc_dequantize(_p(codes), _p(scales), ctypes.c_int64(n), I, _p(lv), _p(out))
@@ -199,8 +206,8 @@ def quant_error(w, I: int, norm: int, xhat) -> Tuple[float, float]:
 
 def block_sigmas(w, I: int) -> np.ndarray:
     a = as_f32(w)
-    _check(a.size, I)
-    s = np.empty(a.size // I, np.float32)
+    _check(a.size, I, ragged=True)
+    s = np.empty(_blocks(a.size, I), np.float32)
     _load().orc_block_sigmas(_p(a), ctypes.c_int64(a.size), I, _p(s))
     return s
 
@@ -208,7 +215,7 @@ def block_sigmas(w, I: int) -> np.ndarray:
 def opq_split(w, I: int, tau: float, capacity: Optional[int] = None):
     """-> (w_clean fp32[n], idx int64[k], val bf16-bits uint16[k], n_out)."""
     a = as_f32(w)
-    _check(a.size, I)
+    _check(a.size, I, ragged=True)
     cap = a.size if capacity is None else int(capacity)
     clean = np.empty(a.size, np.float32)
     idx = np.empty(max(cap, 1), np.int64)

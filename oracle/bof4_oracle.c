@@ -25,7 +25,11 @@
  *  - the weighted median returned is the minimiser of the stated MAE objective, i.e. the
  *    first sorted sample whose cumulative weight reaches half of the total;
  *  - OPQ block statistics are the two-pass formulas of App. E in fp32 with a balanced binary
- *    summation tree over the block.
+ *    summation tree over the block;
+ *  - quantise / dequantise / OPQ accept n that is not a multiple of I: the last block is simply
+ *    shorter (its own maximum, its own mean and deviation over its own length; for the tree
+ *    sums it is padded with zeros to the next power of two; a code byte that has only one
+ *    weight carries 0 in its low nibble).  The EM functions need whole blocks.
  *
  * Parity pins: every function here is pinned by tests/test_oracle_pins.py (printed codebooks
  * of Tab. 6-8 as fixed points, exact DP optimum on tiny inputs, library k-means / medians in
@@ -118,12 +122,19 @@ static int region_of(float x, const float *xi)
     return c;
 }
 
+/* Length of block b of a tensor of n weights: I, or the remainder for a ragged last block. */
+static int block_len(int64_t n, int I, int64_t b)
+{
+    int64_t left = n - b * I;
+    return (int)(left < I ? left : I);
+}
+
 void orc_block_constants(const float *w, int64_t n, int I, int norm, float *m_out)
 {
-    int64_t B = n / I;
+    int64_t B = (n + I - 1) / I;
 #pragma omp parallel for schedule(static)
     for (int64_t b = 0; b < B; ++b)
-        m_out[b] = block_constant(w + b * I, I, norm);
+        m_out[b] = block_constant(w + b * I, block_len(n, I, b), norm);
 }
 
 /* ---------------------------------------------------------------- quantise ------------ */
@@ -135,15 +146,16 @@ void orc_quantize(const float *w, int64_t n, int I, int norm, const float *xhat,
 {
     float xi[L - 1];
     orc_thresholds(xhat, xi);
-    int64_t B = n / I;
+    int64_t B = (n + I - 1) / I;
 #pragma omp parallel for schedule(static)
     for (int64_t b = 0; b < B; ++b) {
         const float *wb = w + b * I;
-        float m = block_constant(wb, I, norm);
+        int len = block_len(n, I, b);
+        float m = block_constant(wb, len, norm);
         scales[b] = m;
-        for (int i = 0; i < I; i += 2) {
+        for (int i = 0; i < len; i += 2) {
             int c0 = region_of(normalise(wb[i], m), xi);
-            int c1 = region_of(normalise(wb[i + 1], m), xi);
+            int c1 = (i + 1 < len) ? region_of(normalise(wb[i + 1], m), xi) : 0;
             codes[(b * I + i) / 2] = (uint8_t)((c0 << 4) | c1);
         }
     }
@@ -153,11 +165,12 @@ void orc_quantize(const float *w, int64_t n, int I, int norm, const float *xhat,
 void orc_dequantize(const uint8_t *codes, const float *scales, int64_t n, int I,
                     const float *xhat, float *out)
 {
-    int64_t B = n / I;
+    int64_t B = (n + I - 1) / I;
 #pragma omp parallel for schedule(static)
     for (int64_t b = 0; b < B; ++b) {
         float m = scales[b];
-        for (int i = 0; i < I; ++i) {
+        int len = block_len(n, I, b);
+        for (int i = 0; i < len; ++i) {
             int64_t k = b * I + i;
             uint8_t byte = codes[k / 2];
             int c = (k & 1) ? (byte & 15) : (byte >> 4);
@@ -415,27 +428,32 @@ static float tree_sum(float *v, int len)
     return v[0];
 }
 
-/* Corrected sample standard deviation of one block (App. E, the sigma_b equation): two-pass,
- * fp32, tree-ordered sums. */
-static float block_sigma(const float *w, int I)
+/* Corrected sample standard deviation of one block of len weights (App. E, the sigma_b
+ * equation): two-pass, fp32, tree-ordered sums.  A ragged block (len not a power of two) is
+ * padded with zeros for the two tree sums only; mean and variance divide by its own length.
+ * A block of one weight gives 0/0 = NaN, and no weight compares greater than NaN. */
+static float block_sigma(const float *w, int len)
 {
     float tmp[4096]; /* largest supported block */
-    for (int i = 0; i < I; ++i)
-        tmp[i] = w[i];
-    float mean = tree_sum(tmp, I) / (float)I;
-    for (int i = 0; i < I; ++i) {
-        float d = w[i] - mean;
+    int P = 1;
+    while (P < len)
+        P *= 2;
+    for (int i = 0; i < P; ++i)
+        tmp[i] = (i < len) ? w[i] : 0.0f;
+    float mean = tree_sum(tmp, P) / (float)len;
+    for (int i = 0; i < P; ++i) {
+        float d = (i < len) ? w[i] - mean : 0.0f;
         tmp[i] = d * d;
     }
-    float ss = tree_sum(tmp, I);
-    return sqrtf(ss / (float)(I - 1));
+    float ss = tree_sum(tmp, P);
+    return sqrtf(ss / (float)(len - 1));
 }
 
 void orc_block_sigmas(const float *w, int64_t n, int I, float *sigma)
 {
-    int64_t B = n / I;
+    int64_t B = (n + I - 1) / I;
     for (int64_t b = 0; b < B; ++b)
-        sigma[b] = block_sigma(w + b * I, I);
+        sigma[b] = block_sigma(w + b * I, block_len(n, I, b));
 }
 
 /* Outlier split of Sec. 3.3 / Eq. 9: |w| > sigma_b * tau with tau = F_M^{-1}(q).  Outliers are
@@ -444,11 +462,12 @@ void orc_block_sigmas(const float *w, int64_t n, int I, float *sigma)
 int64_t orc_opq_split(const float *w, int64_t n, int I, float tau, float *w_clean,
                       int64_t *idx, uint16_t *val, int64_t cap)
 {
-    int64_t B = n / I, count = 0;
+    int64_t B = (n + I - 1) / I, count = 0;
     for (int64_t b = 0; b < B; ++b) {
         const float *wb = w + b * I;
-        float thr = block_sigma(wb, I) * tau;
-        for (int i = 0; i < I; ++i) {
+        int len = block_len(n, I, b);
+        float thr = block_sigma(wb, len) * tau;
+        for (int i = 0; i < len; ++i) {
             int64_t k = b * I + i;
             if (fabsf(wb[i]) > thr) {
                 if (count < cap) {

@@ -247,8 +247,8 @@ def bof4_quantize(w: torch.Tensor, block_size: int, norm: int, levels,
     sd = dt if scale_dtype is None else scale_dtype
     cb = _codebook(levels, w.device)
     if out is None:
-        codes = torch.empty(n // 2, dtype=torch.uint8, device=w.device)
-        scales = torch.empty(max(n // max(block_size, 1), 0), dtype=_torch_dt(sd), device=w.device)
+        codes = torch.empty((n + 1) // 2, dtype=torch.uint8, device=w.device)
+        scales = torch.empty(-(-n // max(block_size, 1)), dtype=_torch_dt(sd), device=w.device)
     else:
         codes, scales = out
     with torch.cuda.device(w.device):
@@ -259,11 +259,14 @@ def bof4_quantize(w: torch.Tensor, block_size: int, norm: int, levels,
 
 def bof4_dequantize(codes: torch.Tensor, scales: torch.Tensor, block_size: int, levels,
                     out_dtype: int, outliers: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
-                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """-> dequantised tensor [n]; `outliers` = (idx int32, val bf16, n_out int64[1]) for OPQ."""
+                    out: Optional[torch.Tensor] = None, n: Optional[int] = None) -> torch.Tensor:
+    """-> dequantised tensor [n]; `outliers` = (idx int32, val bf16, n_out int64[1]) for OPQ.
+    `n` = number of weights when it is odd (default: twice the number of code bytes)."""
     codes = _dev(codes, "codes")
     scales = _dev(scales, "scales")
-    n = codes.numel() * 2
+    n = codes.numel() * 2 if n is None else int(n)
+    if (n + 1) // 2 != codes.numel():
+        raise ValueError("codes must hold (n + 1) // 2 bytes")
     cb = _codebook(levels, codes.device)
     if out is None:
         out = torch.empty(n, dtype=_torch_dt(out_dtype), device=codes.device)
@@ -330,8 +333,8 @@ def bof4_quantize_opq(w: torch.Tensor, block_size: int, norm: int, levels, tau: 
     cb = _codebook(levels, dev)
     wsp = workspace if workspace is not None else _workspace(OP_OPQ, n, block_size, 0, dev)
     if out is None:
-        codes = torch.empty(n // 2, dtype=torch.uint8, device=dev)
-        scales = torch.empty(n // max(block_size, 1), dtype=_torch_dt(sd), device=dev)
+        codes = torch.empty((n + 1) // 2, dtype=torch.uint8, device=dev)
+        scales = torch.empty(-(-n // max(block_size, 1)), dtype=_torch_dt(sd), device=dev)
         idx = torch.empty(capacity, dtype=torch.int32, device=dev)
         val = torch.empty(capacity, dtype=torch.bfloat16, device=dev)
         cnt = torch.zeros(1, dtype=torch.int64, device=dev)

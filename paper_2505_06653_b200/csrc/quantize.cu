@@ -547,13 +547,152 @@ namespace {
 
 using namespace bof4;
 
+// ================================================================= ragged last block
+//
+// A tensor whose size is not a multiple of the block size ends in a shorter block.  It is handled
+// by one CTA with plain loops (fewer than 4096 weights): the same arithmetic as the streaming
+// kernels, written out element by element.  The block is its own unit: its own maximum, its own
+// mean and deviation over its own length; the two tree sums pad it with zeros to the next power
+// of two (neighbours first, as everywhere); a code byte with a single weight has a zero low nibble.
+
+constexpr int kTailThreads = 256;
+
+template <class DT>
+__device__ __forceinline__ float tail_load(const void* w, int64_t k);
+template <>
+__device__ __forceinline__ float tail_load<F32>(const void* w, int64_t k)
+{
+    return static_cast<const float*>(w)[k];
+}
+template <>
+__device__ __forceinline__ float tail_load<BF16>(const void* w, int64_t k)
+{
+    return __uint_as_float((uint32_t)static_cast<const uint16_t*>(w)[k] << 16);
+}
+template <class DT>
+__device__ __forceinline__ void tail_store(void* w, int64_t k, float v);  // v is exact in DT
+template <>
+__device__ __forceinline__ void tail_store<F32>(void* w, int64_t k, float v)
+{
+    static_cast<float*>(w)[k] = v;
+}
+template <>
+__device__ __forceinline__ void tail_store<BF16>(void* w, int64_t k, float v)
+{
+    static_cast<uint16_t*>(w)[k] = (uint16_t)(__float_as_uint(v) >> 16);
+}
+
+// Balanced tree sum of s_t[0 .. P), P a power of two, neighbours first; result in s_t[0].
+__device__ __forceinline__ void tail_tree_sum(float* s_t, int P)
+{
+    for (int step = 1; step < P; step <<= 1) {
+        __syncthreads();
+        for (int i = threadIdx.x * 2 * step; i < P; i += kTailThreads * 2 * step)
+            s_t[i] = __fadd_rn(s_t[i], s_t[i + step]);
+    }
+    __syncthreads();
+}
+
+// OPQ: outlier split (Sec. 3.3) of the block, appended to the list after the whole blocks'
+// outliers; QUANT: block constant, codes and scale.  first = flat index of the block's first
+// weight (a multiple of the block size), len = its length.
+template <class DT, bool SIGNED, class ST, bool QUANT, bool OPQ>
+__global__ void __launch_bounds__(kTailThreads)
+tail_block_kernel(const void* __restrict__ w, int64_t first, int len, const float* __restrict__ levels,
+                  float tau, uint8_t* __restrict__ codes, void* __restrict__ scales, int64_t scale_index,
+                  void* __restrict__ w_clean, int32_t* __restrict__ out_idx, uint16_t* __restrict__ out_val,
+                  int64_t capacity, int64_t* __restrict__ n_out)
+{
+    __shared__ float s_w[4096], s_t[4096];
+    __shared__ unsigned char s_c[4096];
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ float s_val;
+    const int tid = threadIdx.x;
+    for (int i = tid; i < len; i += kTailThreads) s_w[i] = tail_load<DT>(w, first + i);
+    __syncthreads();
+    if (OPQ) {
+        int P = 1;
+        while (P < len) P <<= 1;
+        for (int i = tid; i < P; i += kTailThreads) s_t[i] = (i < len) ? s_w[i] : 0.0f;
+        tail_tree_sum(s_t, P);
+        if (tid == 0) s_val = __fdiv_rn(s_t[0], (float)len);
+        __syncthreads();
+        const float mean = s_val;
+        __syncthreads();
+        for (int i = tid; i < P; i += kTailThreads) {
+            const float d = (i < len) ? __fsub_rn(s_w[i], mean) : 0.0f;
+            s_t[i] = __fmul_rn(d, d);
+        }
+        tail_tree_sum(s_t, P);
+        if (tid == 0) {
+            // one weight: 0 / 0 = NaN, and nothing compares greater than NaN
+            const float thr = __fmul_rn(__fsqrt_rn(__fdiv_rn(s_t[0], (float)(len - 1))), tau);
+            int64_t k = *n_out;
+            for (int i = 0; i < len; ++i) {
+                if (fabsf(s_w[i]) > thr) {
+                    if (k < capacity) {
+                        out_idx[k] = (int32_t)(first + i);
+                        out_val[k] = (uint16_t)bf16_rne(s_w[i]);
+                    }
+                    ++k;
+                    s_w[i] = 0.0f;
+                }
+            }
+            *n_out = k;
+        }
+        __syncthreads();
+        if (w_clean)
+            for (int i = tid; i < len; i += kTailThreads) tail_store<DT>(w_clean, first + i, s_w[i]);
+    }
+    if (QUANT) {
+        make_thresholds(levels, s_xi, s_lv, tid);
+        if (tid == 0) {
+            float best = 0.0f, m = 0.0f;  // largest magnitude, lowest index on ties (Eq. 1 / Eq. 4)
+            for (int i = 0; i < len; ++i) {
+                const float a = fabsf(s_w[i]);
+                if (a > best) {
+                    best = a;
+                    m = SIGNED ? s_w[i] : a;
+                }
+            }
+            s_val = m;
+            store_scale<ST>(scales, scale_index, m);
+        }
+        __syncthreads();
+        const float m = s_val;
+        for (int i = tid; i < len; i += kTailThreads) s_c[i] = (unsigned char)region_of(normalise(s_w[i], m), s_xi);
+        __syncthreads();
+        for (int k = tid; k < (len + 1) / 2; k += kTailThreads)
+            codes[first / 2 + k] = (uint8_t)((s_c[2 * k] << 4) | ((2 * k + 1 < len) ? s_c[2 * k + 1] : 0));
+    }
+}
+
+template <class ST, class OT>
+__global__ void __launch_bounds__(kTailThreads)
+tail_dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t first, int len,
+                       int64_t scale_index, const float* __restrict__ levels, void* __restrict__ out)
+{
+    const float m = load_scale<ST>(scales, scale_index);
+    for (int i = threadIdx.x; i < len; i += kTailThreads) {
+        const int64_t k = first + i;
+        const uint32_t byte = codes[k >> 1];
+        const uint32_t c = (k & 1) ? (byte & 15u) : (byte >> 4);
+        const float v = __fmul_rn(m, levels[c]);
+        if (OT::code == BF16::code)
+            static_cast<uint16_t*>(out)[k] = (uint16_t)bf16_rne(v);
+        else
+            static_cast<float*>(out)[k] = v;
+    }
+}
+
+
 int grid_for(int64_t rows, int per_sm)
 {
     const int64_t cap = (int64_t)kSMs * per_sm;
     return (int)(rows < 1 ? 1 : (rows < cap ? rows : cap));
 }
 
-int check_common(const char* fn, int64_t n, int block_size)
+int check_common(const char* fn, int64_t n, int block_size, bool ragged_ok)
 {
     if (n < 0) {
         set_error("%s: n is negative", fn);
@@ -563,7 +702,7 @@ int check_common(const char* fn, int64_t n, int block_size)
         set_error("%s: block_size %d is not a power of two in 32 ... 4096", fn, block_size);
         return BOF4_ERR_SHAPE;
     }
-    if (n % block_size) {
+    if (!ragged_ok && n % block_size) {
         set_error("%s: n = %lld is not a multiple of block_size %d", fn, (long long)n, block_size);
         return BOF4_ERR_SHAPE;
     }
@@ -627,7 +766,7 @@ extern "C" int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_
                              const float* d_codebook, uint8_t* d_codes, void* d_scales,
                              int scale_dtype, void* stream)
 {
-    int rc = check_common("bof4_quantize", n, block_size);
+    int rc = check_common("bof4_quantize", n, block_size, true);
     if (rc) return rc;
     rc = check_quant_dtypes("bof4_quantize", w_dtype, scale_dtype, norm);
     if (rc) return rc;
@@ -639,15 +778,28 @@ extern "C" int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_
     if ((rc = check_aligned("bof4_quantize", "d_w", d_w)) || (rc = check_aligned("bof4_quantize", "d_codes", d_codes)))
         return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int64_t rows = (n + kQRow - 1) / kQRow;
-    const int grid = grid_for(rows, kQCtasPerSm);
-    BOF4_DISPATCH_WS(w_dtype, scale_dtype,
-        BOF4_DISPATCH_I(block_size,
+    const int tail = (int)(n % block_size);  // a ragged last block goes to its own small kernel
+    const int64_t n_whole = n - tail;
+    n = n_whole;
+    if (n > 0) {
+        const int64_t rows = (n + kQRow - 1) / kQRow;
+        const int grid = grid_for(rows, kQCtasPerSm);
+        BOF4_DISPATCH_WS(w_dtype, scale_dtype,
+            BOF4_DISPATCH_I(block_size,
+                BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                    { auto kern = quantize_kernel<DT, I_, SG, ST>;
+                      BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
+                      kern<<<grid, kQThreads, kLutBytes, st>>>(d_w, n, d_codebook, d_codes, d_scales); })));
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
+    if (tail) {
+        BOF4_DISPATCH_WS(w_dtype, scale_dtype,
             BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
-                { auto kern = quantize_kernel<DT, I_, SG, ST>;
-                  BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
-                  kern<<<grid, kQThreads, kLutBytes, st>>>(d_w, n, d_codebook, d_codes, d_scales); })));
-    BOF4_CUDA_TRY(cudaGetLastError());
+                (tail_block_kernel<DT, SG, ST, true, false><<<1, kTailThreads, 0, st>>>(
+                    d_w, n_whole, tail, d_codebook, 0.0f, d_codes, d_scales, n_whole / block_size, nullptr, nullptr,
+                    nullptr, 0, nullptr))));
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
     return BOF4_OK;
 }
 
@@ -657,7 +809,7 @@ extern "C" int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int
                                const int64_t* d_n_out, int64_t capacity, void* d_out,
                                int out_dtype, void* stream)
 {
-    int rc = check_common("bof4_dequantize", n, block_size);
+    int rc = check_common("bof4_dequantize", n, block_size, true);
     if (rc) return rc;
     if ((scale_dtype != BOF4_F32 && scale_dtype != BOF4_BF16) ||
         (out_dtype != BOF4_F32 && out_dtype != BOF4_BF16)) {
@@ -681,10 +833,19 @@ extern "C" int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int
     if ((rc = check_aligned("bof4_dequantize", "d_codes", d_codes)) || (rc = check_aligned("bof4_dequantize", "d_out", d_out)))
         return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int64_t rows = (n + kDRow - 1) / kDRow;
+    const int tail = (int)(n % block_size);  // a ragged last block goes to its own small kernel
+    const int64_t n_whole = n - tail;
+    const int64_t rows = (n_whole + kDRow - 1) / kDRow;
     const int grid = grid_for(rows, 8);
-#define BOF4_DEQ(ST_, OT_) \
-    BOF4_DISPATCH_I(block_size, (dequantize_kernel<ST_, OT_, I_><<<grid, kDThreads, 0, st>>>(d_codes, d_scales, n, d_codebook, d_out)))
+#define BOF4_DEQ(ST_, OT_)                                                                                   \
+    {                                                                                                        \
+        if (n_whole > 0)                                                                                     \
+            BOF4_DISPATCH_I(block_size, (dequantize_kernel<ST_, OT_, I_><<<grid, kDThreads, 0, st>>>(        \
+                                            d_codes, d_scales, n_whole, d_codebook, d_out)))                 \
+        if (tail)                                                                                            \
+            tail_dequantize_kernel<ST_, OT_><<<1, kTailThreads, 0, st>>>(d_codes, d_scales, n_whole, tail,   \
+                                                                         n_whole / block_size, d_codebook, d_out); \
+    }
     if (scale_dtype == BOF4_F32 && out_dtype == BOF4_F32) { BOF4_DEQ(F32, F32) }
     else if (scale_dtype == BOF4_F32) { BOF4_DEQ(F32, BF16) }
     else if (out_dtype == BOF4_F32) { BOF4_DEQ(BF16, F32) }
@@ -709,9 +870,9 @@ template <bool QUANT>
 int launch_opq(const char* fn, const void* d_w, int w_dtype, int64_t n, int block_size, int norm,
                const float* d_codebook, float tau, uint8_t* d_codes, void* d_scales, int scale_dtype,
                void* d_w_clean, int32_t* d_out_idx, void* d_out_val, int64_t capacity,
-               int64_t* d_n_out, void* d_ws, size_t ws_bytes, void* stream)
+               int64_t* d_n_out, void* d_ws, size_t ws_bytes, void* stream, bool ragged_ok = true)
 {
-    int rc = check_common(fn, n, block_size);
+    int rc = check_common(fn, n, block_size, ragged_ok);
     if (rc) return rc;
     rc = check_quant_dtypes(fn, w_dtype, scale_dtype, norm);
     if (rc) return rc;
@@ -754,26 +915,47 @@ int launch_opq(const char* fn, const void* d_w, int w_dtype, int64_t n, int bloc
     int32_t* stage_idx = reinterpret_cast<int32_t*>(ws + L.stage_idx);
     uint16_t* stage_val = reinterpret_cast<uint16_t*>(ws + L.stage_val);
     uint16_t* out_val = static_cast<uint16_t*>(d_out_val);
-    const int64_t rows = (n + kQRow - 1) / kQRow;
-    const int grid = grid_for(rows, kQCtasPerSm);
-    const int smem = QUANT ? kLutBytes : 0;
-    BOF4_CUDA_TRY(cudaMemsetAsync(chunk_sum, 0, (size_t)L.chunks * 8, st));
-    BOF4_DISPATCH_WS(w_dtype, scale_dtype,
-        BOF4_DISPATCH_I(block_size,
-            BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
-                { auto kern = opq_pass1_kernel<DT, I_, SG, ST, QUANT>;
-                  BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
-                  kern<<<grid, kQThreads, smem, st>>>(
-                      d_w, n, d_codebook, tau, d_codes, d_scales, d_w_clean, counts, chunk_sum, stage_idx, stage_val); })));
-    BOF4_CUDA_TRY(cudaGetLastError());
-    if (w_dtype == BOF4_F32) {
-        BOF4_DISPATCH_I(block_size, (opq_gather_kernel<F32, I_><<<(int)L.chunks, 256, 0, st>>>(
-            d_w, n, tau, counts, L.tiles, chunk_sum, stage_idx, stage_val, d_out_idx, out_val, capacity, d_n_out)));
+    const int tail = (int)(n % block_size);  // a ragged last block goes to its own small kernel
+    const int64_t n_whole = n - tail;
+    if (n_whole == 0) {
+        BOF4_CUDA_TRY(cudaMemsetAsync(d_n_out, 0, sizeof(int64_t), st));
     } else {
-        BOF4_DISPATCH_I(block_size, (opq_gather_kernel<BF16, I_><<<(int)L.chunks, 256, 0, st>>>(
-            d_w, n, tau, counts, L.tiles, chunk_sum, stage_idx, stage_val, d_out_idx, out_val, capacity, d_n_out)));
+        const OpqLayout Lw = opq_layout(n_whole);  // never larger than the layout of n
+        const int64_t rows = (n_whole + kQRow - 1) / kQRow;
+        const int grid = grid_for(rows, kQCtasPerSm);
+        const int smem = QUANT ? kLutBytes : 0;
+        counts = reinterpret_cast<int32_t*>(ws + Lw.counts);
+        chunk_sum = reinterpret_cast<unsigned long long*>(ws + Lw.chunk_off);
+        stage_idx = reinterpret_cast<int32_t*>(ws + Lw.stage_idx);
+        stage_val = reinterpret_cast<uint16_t*>(ws + Lw.stage_val);
+        BOF4_CUDA_TRY(cudaMemsetAsync(chunk_sum, 0, (size_t)Lw.chunks * 8, st));
+        BOF4_DISPATCH_WS(w_dtype, scale_dtype,
+            BOF4_DISPATCH_I(block_size,
+                BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                    { auto kern = opq_pass1_kernel<DT, I_, SG, ST, QUANT>;
+                      BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
+                      kern<<<grid, kQThreads, smem, st>>>(d_w, n_whole, d_codebook, tau, d_codes, d_scales, d_w_clean,
+                                                          counts, chunk_sum, stage_idx, stage_val); })));
+        BOF4_CUDA_TRY(cudaGetLastError());
+        if (w_dtype == BOF4_F32) {
+            BOF4_DISPATCH_I(block_size, (opq_gather_kernel<F32, I_><<<(int)Lw.chunks, 256, 0, st>>>(
+                d_w, n_whole, tau, counts, Lw.tiles, chunk_sum, stage_idx, stage_val, d_out_idx, out_val, capacity,
+                d_n_out)));
+        } else {
+            BOF4_DISPATCH_I(block_size, (opq_gather_kernel<BF16, I_><<<(int)Lw.chunks, 256, 0, st>>>(
+                d_w, n_whole, tau, counts, Lw.tiles, chunk_sum, stage_idx, stage_val, d_out_idx, out_val, capacity,
+                d_n_out)));
+        }
+        BOF4_CUDA_TRY(cudaGetLastError());
     }
-    BOF4_CUDA_TRY(cudaGetLastError());
+    if (tail) {  // after the gather kernel: its outliers follow those of the whole blocks
+        BOF4_DISPATCH_WS(w_dtype, scale_dtype,
+            BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                (tail_block_kernel<DT, SG, ST, QUANT, true><<<1, kTailThreads, 0, st>>>(
+                    d_w, n_whole, tail, d_codebook, tau, d_codes, d_scales, n_whole / block_size, d_w_clean, d_out_idx,
+                    out_val, capacity, d_n_out))));
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
     return BOF4_OK;
 }
 
@@ -856,5 +1038,5 @@ extern "C" int opq_split_static(const void* d_w, int w_dtype, int64_t n, int blo
     if (rc) return rc;
     return launch_opq<false>("opq_split_static", d_w, w_dtype, n, block_size, BOF4_NORM_ABS, nullptr, tau,
                              nullptr, nullptr, w_dtype, d_w_clean, d_out_idx, d_out_val, capacity,
-                             d_n_out, scratch, kStaticScratchBytes, stream);
+                             d_n_out, scratch, kStaticScratchBytes, stream, false);
 }

@@ -83,8 +83,7 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     fake = ctypes.c_void_p(0x1000)  # never dereferenced: validation fails first
     # block size and divisibility
     assert L.bof4_quantize(fake, b.BF16, 128, 48, 0, fake, fake, fake, b.BF16, None) == -2
-    assert L.bof4_quantize(fake, b.BF16, 100, 64, 0, fake, fake, fake, b.BF16, None) == -2
-    assert b"multiple" in L.bof4_last_error()
+    assert L.bof4_quantize(fake, b.BF16, 128, 8192, 0, fake, fake, fake, b.BF16, None) == -2
     assert L.bof4_quantize(fake, b.BF16, -64, 64, 0, fake, fake, fake, b.BF16, None) == -1
     # dtypes: unknown, and fp32 weights with bf16 scales
     assert L.bof4_quantize(fake, 3, 128, 64, 0, fake, fake, fake, b.BF16, None) == -3
@@ -92,7 +91,7 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     assert L.bof4_quantize(fake, b.BF16, 128, 64, 2, fake, fake, fake, b.BF16, None) == -1
     assert L.bof4_quantize(None, b.BF16, 128, 64, 0, fake, fake, fake, b.BF16, None) == -1
     # dequantise
-    assert L.bof4_dequantize(fake, fake, b.BF16, 96, 64, fake, None, None, None, 0, fake, b.BF16, None) == -2
+    assert L.bof4_dequantize(fake, fake, b.BF16, 96, 24, fake, None, None, None, 0, fake, b.BF16, None) == -2
     assert L.bof4_dequantize(fake, fake, 9, 128, 64, fake, None, None, None, 0, fake, b.BF16, None) == -3
     assert L.bof4_dequantize(fake, fake, b.BF16, 128, 64, fake, fake, None, None, 4, fake, b.BF16, None) == -1
     assert L.bof4_dequantize(fake, fake, b.BF16, 128, 64, fake, fake, fake, fake, -1, fake, b.BF16, None) == -5
@@ -108,6 +107,7 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     ptrs = (ctypes.c_void_p * 1)(0x1000)
     ns = (ctypes.c_int64 * 1)(100)
     assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, fake, ws, 1 << 40, None) == -2
+    assert b"multiple" in L.bof4_last_error()  # the fit needs whole blocks (quantise / OPQ take a ragged end)
     ns[0] = 128
     assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, fake, ws, 8, None) == -4
     assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 4, fake, fake, ws, 1 << 40, None) == -1

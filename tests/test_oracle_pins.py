@@ -601,3 +601,53 @@ def test_gemv_is_the_library_matvec_of_the_dequantised_matrix():
     # a transposed operand or a dropped outlier list is caught
     y_no, _ = oracle.gemv(codes, scales, rows, cols, I, lv, x)
     assert np.abs(y_no - ref).max() > 100 * 2.0 ** -23 * mag.max()
+
+
+# --------------------------------------------------------------------------- ragged last block
+
+
+def test_ragged_last_block_is_a_block_of_its_own():
+    """A tensor that does not end on a block boundary: the last block is quantised by its own
+    maximum.  Zero padding changes no maximum, so its codes must equal those of the zero-padded
+    block; only a half-filled last byte differs (zero low nibble instead of the code of 0)."""
+    rng = np.random.default_rng(11)
+    I, tail = 64, 37
+    lv = TAB6[:, 4].astype(np.float32)
+    w = (rng.standard_normal(3 * I + tail) * 0.02).astype(np.float32)
+    for norm in (ABS, SGN):
+        codes, scales = oracle.quantize(w, I, norm, lv)
+        assert codes.size == (w.size + 1) // 2 and scales.size == 4
+        head_c, head_s = oracle.quantize(w[:3 * I], I, norm, lv)
+        assert np.array_equal(codes[:3 * I // 2], head_c) and np.array_equal(scales[:3], head_s)
+        padded = np.concatenate([w[3 * I:], np.zeros(I - tail, np.float32)])
+        pc, ps = oracle.quantize(padded, I, norm, lv)
+        assert scales[3] == ps[0] == oracle.block_constants(w[3 * I:], tail, norm)[0]
+        assert np.array_equal(codes[96:96 + tail // 2], pc[:tail // 2])
+        assert codes[96 + tail // 2] == (pc[tail // 2] & 0xF0)          # element 36 high, nothing low
+        deq = oracle.dequantize(codes, scales, I, lv, n=w.size)
+        assert deq.size == w.size
+        assert np.array_equal(deq[3 * I:], oracle.dequantize(pc, ps, I, lv)[:tail])
+
+
+def test_ragged_last_block_sigma_and_outliers():
+    """sigma of the short block is the corrected sample deviation over ITS elements (numpy's
+    ddof = 1), not over a padded block; a one-weight block has no outliers."""
+    rng = np.random.default_rng(12)
+    I = 64
+    for tail in (1, 2, 3, 33, 63):
+        w = (rng.standard_normal(2 * I + tail) * 0.02).astype(np.float32)
+        w[2 * I] = 0.5                                   # would be an outlier in any longer block
+        sig = oracle.block_sigmas(w, I)
+        assert sig.size == 3
+        if tail == 1:
+            assert np.isnan(sig[2])
+        else:
+            ref = np.std(w[2 * I:].astype(np.float64), ddof=1)
+            assert abs(sig[2] - ref) <= 1e-6 * ref
+        clean, idx, val, k = oracle.opq_split(w, I, 1.2)
+        in_tail = idx[idx >= 2 * I]
+        expect = np.nonzero(np.abs(w[2 * I:]) > np.float32(sig[2]) * np.float32(1.2))[0] + 2 * I if tail > 1 else []
+        assert np.array_equal(in_tail, np.asarray(expect, dtype=np.int64))
+        assert np.all(clean[idx] == 0) and clean.size == w.size
+        if tail == 1:
+            assert clean[2 * I] == np.float32(0.5)
