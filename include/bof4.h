@@ -258,6 +258,19 @@ BOF4_API int bof4_theoretical_codebook(int block_size, int norm, int metric, flo
                               uint32_t fixed_mask, int iters, void* d_ws, size_t ws_bytes,
                               void* stream);
 
+/*
+ * The same for up to 128 problems at once (for instance every block size of a sweep under both
+ * normalisations and metrics): problem p has block size h_block_size[p], normalisation
+ * h_norm[p], metric h_metric[p], fixed levels h_fixed_mask[p] (host arrays, read before the call
+ * returns) and its levels in d_codebooks[16 p .. 16 p + 15] (device, in/out).  All problems
+ * advance together, one launch per iteration.  d_ws: 256 bytes per problem, 256-byte aligned.
+ * Results equal those of n_problems single calls bit for bit.
+ */
+BOF4_API int bof4_theoretical_codebook_batch(int n_problems, const int* h_block_size, const int* h_norm,
+                                    const int* h_metric, const uint32_t* h_fixed_mask,
+                                    float* d_codebooks, int iters, void* d_ws, size_t ws_bytes,
+                                    void* stream);
+
 /* ---- host helpers (no CUDA call) ---- */
 
 /* tau = F_M^{-1}(q) for unit-variance Gaussian weights, F_M(m) = (2 G(m) - 1)^I the CDF of the

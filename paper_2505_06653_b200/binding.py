@@ -31,7 +31,8 @@ MAE_LAUNCHES_PER_ITERATION = 7
 
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
-           "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_gemv")
+           "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_theoretical_codebook_batch",
+           "bof4_gemv")
 
 
 class Bof4Error(RuntimeError):
@@ -80,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.bof4_gemv.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, vp, vp, vp, i64, vp, vp]
         L.bof4_theoretical_codebook.restype = i32
         L.bof4_theoretical_codebook.argtypes = [i32, i32, i32, vp, ctypes.c_uint32, i32, vp, sz, vp]
+        L.bof4_theoretical_codebook_batch.restype = i32
+        L.bof4_theoretical_codebook_batch.argtypes = [i32, vp, vp, vp, vp, vp, i32, vp, sz, vp]
         L.bof4_opq_threshold.restype = ctypes.c_double
         L.bof4_opq_threshold.argtypes = [ctypes.c_double, i32]
         L.bof4_default_init.restype = i32
@@ -232,6 +235,29 @@ def bof4_theoretical_codebook(block_size: int, norm: int, metric: int, levels, f
     with torch.cuda.device(dev):
         _check(lib().bof4_theoretical_codebook(block_size, norm, metric, _ptr(cb), fixed_mask, iters,
                                                _ptr(ws), ws.numel(), _stream()))
+    return cb
+
+
+def bof4_theoretical_codebook_batch(block_sizes, norms, metrics, levels, fixed_masks, iters: int,
+                                    device="cuda") -> torch.Tensor:
+    """The same for several problems at once; `levels` is [n, 16] (or [16], used for every
+    problem).  -> levels fp32[n, 16] on the device."""
+    dev = torch.device(device)
+    n = len(block_sizes)
+    if not (len(norms) == len(metrics) == len(fixed_masks) == n):
+        raise ValueError("one block size, norm, metric and mask per problem")
+    lv = torch.as_tensor(np.asarray(levels.cpu() if isinstance(levels, torch.Tensor) else levels, dtype=np.float32))
+    if lv.dim() == 1:
+        lv = lv.expand(n, LEVELS)
+    if tuple(lv.shape) != (n, LEVELS):
+        raise ValueError("levels must be [n, 16] or [16]")
+    cb = lv.contiguous().to(dev).clone()
+    ws = torch.empty(256 * max(n, 1), dtype=torch.uint8, device=dev)
+    arr = lambda v, t: (t * max(n, 1))(*[int(x) for x in v])
+    with torch.cuda.device(dev):
+        _check(lib().bof4_theoretical_codebook_batch(
+            n, arr(block_sizes, ctypes.c_int), arr(norms, ctypes.c_int), arr(metrics, ctypes.c_int),
+            arr(fixed_masks, ctypes.c_uint32), _ptr(cb), iters, _ptr(ws), ws.numel(), _stream()))
     return cb
 
 

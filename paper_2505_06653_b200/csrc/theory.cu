@@ -50,13 +50,26 @@ __device__ __forceinline__ void node(int q, double& m, double& wq)
     wq = (q == 0 || q == kThIntervals) ? h / 3.0 : ((q & 1) ? 4.0 * h / 3.0 : 2.0 * h / 3.0);
 }
 
-// One Lloyd iteration: CTA l recomputes level l from the thresholds of levels_in.
+// Problems of one batched call: block size, metric and fixed levels of each (kernel parameter).
+constexpr int kThMaxBatch = 128;
+struct TheoryBatch {
+    int I[kThMaxBatch];
+    int metric[kThMaxBatch];
+    uint32_t fixed_mask[kThMaxBatch];
+};
+
+// One Lloyd iteration of every problem: CTA (l, p) recomputes level l of problem p from the
+// thresholds of its current levels.  Problem p keeps two sets of 16 fp64 levels in the workspace
+// (32 doubles); `flip` tells which of the two is current.
 __global__ void __launch_bounds__(kThThreads)
-theory_step_kernel(const double* __restrict__ levels_in, double* __restrict__ levels_out, int I, int metric,
-                   uint32_t fixed_mask)
+theory_step_kernel(double* __restrict__ state, int flip, const TheoryBatch B)
 {
     __shared__ double s_red[kThThreads / 32];
-    const int l = blockIdx.x;
+    const int l = blockIdx.x, p = blockIdx.y;
+    const double* levels_in = state + (size_t)p * 2 * kLevels + (flip ? kLevels : 0);
+    double* levels_out = state + (size_t)p * 2 * kLevels + (flip ? 0 : kLevels);
+    const int I = B.I[p], metric = B.metric[p];
+    const uint32_t fixed_mask = B.fixed_mask[p];
     const double cur = levels_in[l];
     if ((fixed_mask >> l) & 1u) {
         if (threadIdx.x == 0) levels_out[l] = cur;
@@ -109,13 +122,62 @@ theory_step_kernel(const double* __restrict__ levels_in, double* __restrict__ le
     }
 }
 
-__global__ void theory_load_kernel(const float* __restrict__ codebook, double* __restrict__ levels)
+// levels of problem p: codebooks[p][16] (fp32) <-> the current set of the fp64 state
+__global__ void theory_load_kernel(const float* __restrict__ codebooks, double* __restrict__ state)
 {
-    if (threadIdx.x < kLevels) levels[threadIdx.x] = (double)codebook[threadIdx.x];
+    const int p = blockIdx.x;
+    if (threadIdx.x < kLevels) state[(size_t)p * 2 * kLevels + threadIdx.x] = (double)codebooks[p * kLevels + threadIdx.x];
 }
-__global__ void theory_store_kernel(const double* __restrict__ levels, float* __restrict__ codebook)
+__global__ void theory_store_kernel(const double* __restrict__ state, int flip, float* __restrict__ codebooks)
 {
-    if (threadIdx.x < kLevels) codebook[threadIdx.x] = (float)levels[threadIdx.x];
+    const int p = blockIdx.x;
+    if (threadIdx.x < kLevels)
+        codebooks[p * kLevels + threadIdx.x] = (float)state[(size_t)p * 2 * kLevels + (flip ? kLevels : 0) + threadIdx.x];
+}
+
+static int check_theory_problem(const char* fn, int block_size, int norm, int metric, uint32_t fixed_mask)
+{
+    if (block_size < 2 || block_size > (1 << 20)) {
+        set_error("%s: block_size must be in 2 ... 2^20", fn);
+        return BOF4_ERR_SHAPE;
+    }
+    if ((norm != BOF4_NORM_ABS && norm != BOF4_NORM_SIGNED) ||
+        (metric != BOF4_METRIC_MSE && metric != BOF4_METRIC_MAE)) {
+        set_error("%s: bad norm or metric", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (!((fixed_mask >> 15) & 1u) || (norm == BOF4_NORM_ABS && !(fixed_mask & 1u))) {
+        set_error("%s: the outermost levels (1, and -1 for absolute normalisation) "
+                  "carry the point mass of the block maximum and must be fixed", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    return BOF4_OK;
+}
+
+static int run_theory(const char* fn, int n, const TheoryBatch& B, float* d_codebooks, int iters, void* d_ws,
+                      size_t ws_bytes, void* stream)
+{
+    if (iters < 0 || !d_codebooks) {
+        set_error("%s: negative iteration count or NULL codebook", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (!d_ws || ((uintptr_t)d_ws & 255u) || ws_bytes < (size_t)256 * n) {
+        set_error("%s: workspace NULL, not 256-byte aligned, or smaller than 256 bytes per problem", fn);
+        return BOF4_ERR_WORKSPACE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double* state = static_cast<double*>(d_ws);
+    theory_load_kernel<<<n, 32, 0, st>>>(d_codebooks, state);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    int flip = 0;
+    for (int t = 0; t < iters; ++t) {
+        theory_step_kernel<<<dim3(kLevels, n), kThThreads, 0, st>>>(state, flip, B);
+        BOF4_CUDA_TRY(cudaGetLastError());
+        flip ^= 1;
+    }
+    theory_store_kernel<<<n, 32, 0, st>>>(state, flip, d_codebooks);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
 }
 
 }  // namespace bof4
@@ -125,37 +187,38 @@ extern "C" int bof4_theoretical_codebook(int block_size, int norm, int metric, f
                                          void* stream)
 {
     using namespace bof4;
-    if (block_size < 2 || block_size > (1 << 20)) {
-        set_error("bof4_theoretical_codebook: block_size must be in 2 ... 2^20");
+    const int rc = check_theory_problem("bof4_theoretical_codebook", block_size, norm, metric, fixed_mask);
+    if (rc) return rc;
+    TheoryBatch B{};
+    B.I[0] = block_size;
+    B.metric[0] = metric;
+    B.fixed_mask[0] = fixed_mask;
+    return run_theory("bof4_theoretical_codebook", 1, B, d_codebook, iters, d_ws, ws_bytes, stream);
+}
+
+extern "C" int bof4_theoretical_codebook_batch(int n_problems, const int* h_block_size, const int* h_norm,
+                                               const int* h_metric, const uint32_t* h_fixed_mask,
+                                               float* d_codebooks, int iters, void* d_ws, size_t ws_bytes,
+                                               void* stream)
+{
+    using namespace bof4;
+    if (n_problems < 0 || n_problems > kThMaxBatch) {
+        set_error("bof4_theoretical_codebook_batch: n_problems must be in 0 ... %d", kThMaxBatch);
         return BOF4_ERR_SHAPE;
     }
-    if ((norm != BOF4_NORM_ABS && norm != BOF4_NORM_SIGNED) ||
-        (metric != BOF4_METRIC_MSE && metric != BOF4_METRIC_MAE) || iters < 0 || !d_codebook) {
-        set_error("bof4_theoretical_codebook: bad norm, metric, iteration count or NULL codebook");
+    if (n_problems == 0) return BOF4_OK;
+    if (!h_block_size || !h_norm || !h_metric || !h_fixed_mask) {
+        set_error("bof4_theoretical_codebook_batch: NULL parameter array");
         return BOF4_ERR_INVALID_ARG;
     }
-    if (!((fixed_mask >> 15) & 1u) || (norm == BOF4_NORM_ABS && !(fixed_mask & 1u))) {
-        set_error("bof4_theoretical_codebook: the outermost levels (1, and -1 for absolute normalisation) "
-                  "carry the point mass of the block maximum and must be fixed");
-        return BOF4_ERR_INVALID_ARG;
+    TheoryBatch B{};
+    for (int p = 0; p < n_problems; ++p) {
+        const int rc = check_theory_problem("bof4_theoretical_codebook_batch", h_block_size[p], h_norm[p],
+                                            h_metric[p], h_fixed_mask[p]);
+        if (rc) return rc;
+        B.I[p] = h_block_size[p];
+        B.metric[p] = h_metric[p];
+        B.fixed_mask[p] = h_fixed_mask[p];
     }
-    if (!d_ws || ((uintptr_t)d_ws & 255u) || ws_bytes < 256) {
-        set_error("bof4_theoretical_codebook: workspace NULL, not 256-byte aligned, or smaller than 256 bytes");
-        return BOF4_ERR_WORKSPACE;
-    }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    double* a = static_cast<double*>(d_ws);
-    double* b = a + kLevels;
-    theory_load_kernel<<<1, 32, 0, st>>>(d_codebook, a);
-    BOF4_CUDA_TRY(cudaGetLastError());
-    for (int t = 0; t < iters; ++t) {
-        theory_step_kernel<<<kLevels, kThThreads, 0, st>>>(a, b, block_size, metric, fixed_mask);
-        BOF4_CUDA_TRY(cudaGetLastError());
-        double* tmp = a;
-        a = b;
-        b = tmp;
-    }
-    theory_store_kernel<<<1, 32, 0, st>>>(a, d_codebook);
-    BOF4_CUDA_TRY(cudaGetLastError());
-    return BOF4_OK;
+    return run_theory("bof4_theoretical_codebook_batch", n_problems, B, d_codebooks, iters, d_ws, ws_bytes, stream);
 }

@@ -135,6 +135,13 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     assert L.bof4_theoretical_codebook(64, 0, 2, fake, full, 1, ws, 256, None) == -1
     assert L.bof4_theoretical_codebook(1, 0, 0, fake, full, 1, ws, 256, None) == -2
     assert L.bof4_theoretical_codebook(64, 0, 0, fake, full, 1, ws, 8, None) == -4
+    one = lambda v, t=ctypes.c_int: (t * 1)(v)
+    batch = L.bof4_theoretical_codebook_batch
+    assert batch(129, one(64), one(0), one(0), one(full, ctypes.c_uint32), fake, 1, ws, 1 << 20, None) == -2
+    assert batch(1, one(64), one(0), one(0), one(1 << 15, ctypes.c_uint32), fake, 1, ws, 256, None) == -1
+    assert batch(1, one(64), one(0), one(0), one(full, ctypes.c_uint32), fake, 1, ws, 128, None) == -4
+    assert batch(1, None, one(0), one(0), one(full, ctypes.c_uint32), fake, 1, ws, 256, None) == -1
+    assert batch(0, None, None, None, None, None, 1, None, 0, None) == 0
 
 
 def test_binding_refuses_cpu_tensors(L):

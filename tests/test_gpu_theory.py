@@ -60,3 +60,21 @@ def test_agrees_with_the_oracles_quadrature(bof4, I, signed, metric):
                                          start, mask, 3).cpu().numpy()
     assert np.abs(got - ref).max() < 2e-6
     assert np.all(np.diff(got) > 0)
+
+
+def test_batched_solver_equals_single_calls(bof4):
+    """Every block size of a sweep under both normalisations and metrics in one call: bit for bit
+    the results of the single calls."""
+    probs = [(I, norm, metric) for I in (32, 64, 100, 1024) for norm in (bof4.NORM_ABS, bof4.NORM_SIGNED)
+             for metric in (bof4.METRIC_MSE, bof4.METRIC_MAE)]
+    masks = [FIX4 if norm == bof4.NORM_ABS else FIX4S for _, norm, _ in probs]
+    start = workloads.init_levels_7_0_8()
+    got = bof4.bof4_theoretical_codebook_batch([p[0] for p in probs], [p[1] for p in probs], [p[2] for p in probs],
+                                               start, masks, 25).cpu().numpy()
+    assert got.shape == (len(probs), 16)
+    for row, (I, norm, metric), mask in zip(got, probs, masks):
+        one = bof4.bof4_theoretical_codebook(I, norm, metric, start, mask, 25).cpu().numpy()
+        assert np.array_equal(row, one), (I, norm, metric)
+    assert bof4.bof4_theoretical_codebook_batch([], [], [], start, [], 3).shape == (0, 16)
+    with pytest.raises(bof4.Bof4Error):
+        bof4.bof4_theoretical_codebook_batch([64] * 129, [0] * 129, [0] * 129, start, [FIX4] * 129, 1)
