@@ -54,7 +54,7 @@ extern "C" {
 #define BOF4_ERR_SHAPE (-2)       /* block size unsupported, n not a multiple where it must be, n too large */
 #define BOF4_ERR_DTYPE (-3)       /* dtype code unknown or combination not supported        */
 #define BOF4_ERR_WORKSPACE (-4)   /* workspace NULL, misaligned or smaller than required    */
-#define BOF4_ERR_CAPACITY (-5)    /* outlier list capacity is negative or too large         */
+#define BOF4_ERR_CAPACITY (-5)    /* outlier list capacity negative / too large, or (bof4_outlier_count) exceeded */
 #define BOF4_ERR_CUDA (-6)        /* a CUDA runtime call failed (message has the reason)    */
 
 /* ---- enums (plain ints in the signatures) ---- */
@@ -133,8 +133,6 @@ BOF4_API int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_tens
  *   d_err_log   [iters] fp64 or NULL: entry t = mean error (MSE or MAE over all weights,
  *               un-normalised domain) of the levels that ENTER iteration t
  * No host synchronisation happens inside; the whole loop is enqueued on `stream`.
- * (MAE only: the environment variable BOF4_MAE_COLLECT_PASS = 1 or 2 overrides which data pass
- * fills the candidate lists of the median selection; results do not depend on it.)
  */
 BOF4_API int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int n_tensors, int w_dtype,
                       int block_size, int norm, int metric, float* d_codebook,
@@ -161,11 +159,26 @@ BOF4_API int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_si
  *   d_out_val  out [capacity] bf16 outlier values (round-to-nearest-even from fp32 weights)
  *   d_n_out    out: the true number of outliers, also when it exceeds `capacity` (then only
  *              the first `capacity` entries are written)
- * n must be below 2^31.
+ * n must be below 2^31.  Check the count with bof4_outlier_count before relying on the list.
  */
 BOF4_API int opq_split(const void* d_w, int w_dtype, int64_t n, int block_size, float tau,
               void* d_w_clean, int32_t* d_out_idx, void* d_out_val, int64_t capacity,
               int64_t* d_n_out, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * Second half of the two-call pattern of the outlier lists (Sec. 3.3: outliers are PRESERVED, so
+ * a list that did not fit must not pass unnoticed).  opq_split, opq_split_static and
+ * bof4_quantize_opq are asynchronous and can only leave the true count in *d_n_out; this call
+ * waits for `stream`, copies the count to the host and compares it with the capacity that was
+ * passed to the producing call.
+ *   d_n_out   device: the count written by the producing call on the same stream
+ *   h_n_out   host, out (may be NULL): the true number of outliers
+ * Returns BOF4_OK when count <= capacity, BOF4_ERR_CAPACITY when outliers were dropped (the
+ * message names the capacity that would have sufficed; codes, scales and the stored part of the
+ * list are valid, so only the producing call has to be repeated with larger arrays).
+ * This is the one entry point that synchronises (the stream it is given, nothing else).
+ */
+BOF4_API int bof4_outlier_count(const int64_t* d_n_out, int64_t capacity, int64_t* h_n_out, void* stream);
 
 /*
  * opq_split without a workspace argument and without any allocation.  (The paper has no
@@ -179,12 +192,16 @@ BOF4_API int opq_split(const void* d_w, int w_dtype, int64_t n, int block_size, 
  * 4 MiB array inside the library image; every GPU that loads the library holds that array
  * until the process exits.
  *
- *   - Same arguments, outputs and bit-exact results as opq_split, minus d_ws / ws_bytes.
+ *   - Same arguments, outputs and bit-exact results as opq_split, minus d_ws / ws_bytes, for
+ *     tensors of whole blocks: n must be a multiple of block_size (BOF4_ERR_SHAPE otherwise; the
+ *     ragged last block of opq_split is not offered here).
  *   - n is limited to 2^24 weights per call (BOF4_ERR_SHAPE beyond; split larger tensors at
  *     multiples of block_size and add the chunk's first index to its outlier indices, or use
  *     opq_split).
  *   - The first call on each device looks up the array's device address (once per device,
- *     with that device current).  Make that first call outside any stream capture.
+ *     with that device current).  Make that first call outside any stream capture.  The address
+ *     is remembered per device ordinal for the life of the process: after a cudaDeviceReset of
+ *     that device the remembered address is stale and this entry point must not be used again.
  *   - All calls on one device share the one array.  Every call rewrites each cell before it
  *     reads it, so nothing has to be cleared between calls, but two calls whose kernels
  *     overlap on the GPU (different streams, no ordering between them) race on it: order them.

@@ -113,13 +113,3 @@ def region_probabilities(levels, I: int, signed: bool,
         p[0] += 0.5 / I
         p[15] += 0.5 / I
     return p
-
-
-def agreement_db(theo, emp, probs) -> float:
-    """Codebook agreement of App. C in dB: probability-weighted squared deviation over
-    probability-weighted squared theoretical levels."""
-    theo = np.asarray(theo, dtype=np.float64)
-    emp = np.asarray(emp, dtype=np.float64)
-    num = np.sum(probs * (theo - emp) ** 2)
-    den = np.sum(probs * theo ** 2)
-    return 10.0 * np.log10(num / den)

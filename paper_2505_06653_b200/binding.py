@@ -32,7 +32,7 @@ MAE_LAUNCHES_PER_ITERATION = 7
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_theoretical_codebook_batch",
-           "bof4_gemv")
+           "bof4_gemv", "bof4_outlier_count")
 
 
 class Bof4Error(RuntimeError):
@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.bof4_theoretical_codebook.argtypes = [i32, i32, i32, vp, ctypes.c_uint32, i32, vp, sz, vp]
         L.bof4_theoretical_codebook_batch.restype = i32
         L.bof4_theoretical_codebook_batch.argtypes = [i32, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+        L.bof4_outlier_count.restype = i32
+        L.bof4_outlier_count.argtypes = [vp, i64, vp, vp]
         L.bof4_opq_threshold.restype = ctypes.c_double
         L.bof4_opq_threshold.argtypes = [ctypes.c_double, i32]
         L.bof4_default_init.restype = i32
@@ -346,6 +348,18 @@ def opq_split(w: torch.Tensor, block_size: int, tau: float, capacity: int,
         _check(lib().opq_split(_ptr(w), dt, n, block_size, tau, _ptr(clean), _ptr(idx), _ptr(val),
                                capacity, _ptr(cnt), _ptr(wsp), wsp.numel(), _stream()))
     return clean, idx, val, cnt
+
+
+def bof4_outlier_count(n_out: torch.Tensor, capacity: int) -> int:
+    """Waits for the current stream and returns the true outlier count; raises Bof4Error
+    (BOF4_ERR_CAPACITY) when it exceeds `capacity`, i.e. when outliers were dropped."""
+    n_out = _dev(n_out, "n_out")
+    if n_out.dtype != torch.int64 or n_out.numel() != 1:
+        raise ValueError("n_out must be the int64[1] count tensor of an OPQ call")
+    host = ctypes.c_int64(0)
+    with torch.cuda.device(n_out.device):
+        _check(lib().bof4_outlier_count(_ptr(n_out), int(capacity), ctypes.byref(host), _stream()))
+    return int(host.value)
 
 
 def bof4_quantize_opq(w: torch.Tensor, block_size: int, norm: int, levels, tau: float,

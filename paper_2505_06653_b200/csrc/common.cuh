@@ -12,6 +12,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/bof4.h"
 
 namespace bof4 {
@@ -32,6 +34,22 @@ int cuda_fail(cudaError_t e, const char* what);
         cudaError_t e__ = (expr);                                   \
         if (e__ != cudaSuccess) return ::bof4::cuda_fail(e__, #expr); \
     } while (0)
+
+// Raises the dynamic shared-memory limit of kernel Kern to `bytes`, once per device and kernel
+// instantiation (the attribute belongs to the function on the current device), so that the
+// per-iteration launch path makes no attribute call.
+template <auto Kern>
+inline int ensure_dynamic_smem(int bytes)
+{
+    static std::atomic<unsigned long long> done{0ull};
+    int dev = 0;
+    BOF4_CUDA_TRY(cudaGetDevice(&dev));
+    const unsigned long long bit = (dev >= 0 && dev < 64) ? (1ull << dev) : 0ull;
+    if (bit && (done.load(std::memory_order_acquire) & bit)) return BOF4_OK;
+    BOF4_CUDA_TRY(cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    if (bit) done.fetch_or(bit, std::memory_order_release);
+    return BOF4_OK;
+}
 
 inline bool valid_block_size(int I) { return I >= 32 && I <= 4096 && (I & (I - 1)) == 0; }
 inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }

@@ -424,8 +424,8 @@ int launch_mse_chunk(const EmTensors& T, const float* d_codebook, double* partia
 {
     tail.enabled = T.last;
     using G = EmGeo<COUNT>;
-    auto kern = em_mse_kernel<DT, I, SG, COUNT>;
-    BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::smem));
+    constexpr auto kern = em_mse_kernel<DT, I, SG, COUNT>;
+    if (const int rc = ensure_dynamic_smem<kern>((int)G::smem)) return rc;
     kern<<<kEmGrid, G::threads, G::smem, st>>>(T, d_codebook, partials, tail);
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;

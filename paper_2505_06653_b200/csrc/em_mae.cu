@@ -20,8 +20,6 @@
 // the data (exact whenever |m| is within 2^-7 of it for fp32 input, 2^-23 for bf16 input), so
 // every sum is an integer sum: independent of the order of the atomics, bit-reproducible, and
 // equal to the exact real-number sums that define the median.
-#include <stdlib.h>
-
 #include "common.cuh"
 #include "em_common.cuh"
 #include "layout.h"
@@ -699,8 +697,8 @@ int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, int p
     const MaeFinal F = tail ? *tail : MaeFinal{};
 #define BOF4_MAE_GO(FIRST_, COUNT_, COLLECT_, TAIL_)                                                    \
     {                                                                                                   \
-        auto kern = mae_pass_kernel<DT, I, SG, FIRST_, COUNT_, COLLECT_, TAIL_>;                        \
-        BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaeSmem)); \
+        constexpr auto kern = mae_pass_kernel<DT, I, SG, FIRST_, COUNT_, COLLECT_, TAIL_>;              \
+        if (const int rc_ = ensure_dynamic_smem<kern>((int)kMaeSmem)) return rc_;                       \
         kern<<<kEmGrid, kMaeThreads, kMaeSmem, st>>>(T, d_levels, W, F);                                \
     }
     if (pass == 0 && count) BOF4_MAE_GO(true, true, false, false)
@@ -763,11 +761,7 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
     // The candidate lists are filled by the first pass after which a region's candidates
     // (about 1/512 of them survive each digit) are expected to fit: the second pass up to
     // 2^29 weights, the third beyond.
-    // BOF4_MAE_COLLECT_PASS=1|2 in the environment overrides the choice (tests, tuning).
-    int collect_pass = (a.n_total / kLevels / kMaeBins <= kMaeCand / 8) ? 1 : 2;
-    if (const char* env = getenv("BOF4_MAE_COLLECT_PASS")) {
-        if (env[0] == '1' || env[0] == '2') collect_pass = env[0] - '0';
-    }
+    const int collect_pass = (a.n_total / kLevels / kMaeBins <= kMaeCand / 8) ? 1 : 2;
     MaeFinal fin{};
     fin.n_records = kEmGrid;
     fin.n_total = a.n_total;

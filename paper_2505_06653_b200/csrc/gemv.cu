@@ -371,8 +371,8 @@ static int launch_gemv_kernel(const uint8_t* d_codes, const void* d_scales, int6
     while ((1 << block_shift) < block_size) ++block_shift;
     constexpr bool RING = MAXT > 512 || kGvRing512;
     constexpr int smem = RING ? gv_smem(MAXT) : kGvTabBytes;
-    auto kern = gemv_kernel<ST, XT, MAXT, RING>;
-    BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    constexpr auto kern = gemv_kernel<ST, XT, MAXT, RING>;
+    if (const int rc = ensure_dynamic_smem<kern>(smem)) return rc;
     kern<<<grid, 32 * stripes * groups, smem, st>>>(d_codes, d_scales, rows, cols, block_shift, d_codebook,
                                                              d_x, d_y, stripes, groups);
     BOF4_CUDA_TRY(cudaGetLastError());

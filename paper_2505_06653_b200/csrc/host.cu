@@ -41,6 +41,28 @@ size_t bof4_workspace_bytes(int op, int64_t n_max, int block_size, int metric)
     return 0;
 }
 
+// The synchronising half of the two-call pattern: the outlier-producing calls only leave the true
+// count on the device; this reads it back and turns an overflow into an error code.
+int bof4_outlier_count(const int64_t* d_n_out, int64_t capacity, int64_t* h_n_out, void* stream)
+{
+    if (!d_n_out || capacity < 0) {
+        bof4::set_error("bof4_outlier_count: NULL count pointer or negative capacity");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int64_t count = 0;
+    BOF4_CUDA_TRY(cudaMemcpyAsync(&count, d_n_out, sizeof(count), cudaMemcpyDeviceToHost, st));
+    BOF4_CUDA_TRY(cudaStreamSynchronize(st));
+    if (h_n_out) *h_n_out = count;
+    if (count > capacity) {
+        bof4::set_error("outlier list overflow: %lld outliers found, capacity %lld (only the first %lld were "
+                        "stored; call again with capacity >= %lld)",
+                        (long long)count, (long long)capacity, (long long)capacity, (long long)count);
+        return BOF4_ERR_CAPACITY;
+    }
+    return BOF4_OK;
+}
+
 // tau with G(tau) = (1 + q^(1/I)) / 2  <=>  erfc(tau / sqrt 2) = 1 - q^(1/I) = -expm1(ln q / I).
 // erfc is strictly decreasing, so bisection on [0, 40] converges to the last bit.
 double bof4_opq_threshold(double q, int block_size)

@@ -787,8 +787,8 @@ extern "C" int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_
         BOF4_DISPATCH_WS(w_dtype, scale_dtype,
             BOF4_DISPATCH_I(block_size,
                 BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
-                    { auto kern = quantize_kernel<DT, I_, SG, ST>;
-                      BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
+                    { constexpr auto kern = quantize_kernel<DT, I_, SG, ST>;
+                      if ((rc = ensure_dynamic_smem<kern>(kLutBytes))) return rc;
                       kern<<<grid, kQThreads, kLutBytes, st>>>(d_w, n, d_codebook, d_codes, d_scales); })));
         BOF4_CUDA_TRY(cudaGetLastError());
     }
@@ -932,8 +932,8 @@ int launch_opq(const char* fn, const void* d_w, int w_dtype, int64_t n, int bloc
         BOF4_DISPATCH_WS(w_dtype, scale_dtype,
             BOF4_DISPATCH_I(block_size,
                 BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
-                    { auto kern = opq_pass1_kernel<DT, I_, SG, ST, QUANT>;
-                      BOF4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes));
+                    { constexpr auto kern = opq_pass1_kernel<DT, I_, SG, ST, QUANT>;
+                      if ((rc = ensure_dynamic_smem<kern>(kLutBytes))) return rc;
                       kern<<<grid, kQThreads, smem, st>>>(d_w, n_whole, d_codebook, tau, d_codes, d_scales, d_w_clean,
                                                           counts, chunk_sum, stage_idx, stage_val); })));
         BOF4_CUDA_TRY(cudaGetLastError());
@@ -1019,6 +1019,8 @@ int static_scratch(void** out)
 
 }  // namespace
 
+// Whole blocks only (n % block_size == 0); the remembered scratch address does not survive a
+// cudaDeviceReset of its device.
 extern "C" int opq_split_static(const void* d_w, int w_dtype, int64_t n, int block_size, float tau,
                                 void* d_w_clean, int32_t* d_out_idx, void* d_out_val,
                                 int64_t capacity, int64_t* d_n_out, void* stream)

@@ -103,6 +103,9 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     assert L.opq_split(fake, b.BF16, 128, 64, 3.0, None, fake, fake, 8, fake, ws, 16, None) == -4
     assert L.opq_split(fake, b.BF16, 128, 64, 3.0, None, fake, fake, 8, fake, ctypes.c_void_p(0x10010), 1 << 40, None) == -4
     assert L.opq_split(fake, b.BF16, 128, 64, -1.0, None, fake, fake, 8, fake, ws, 1 << 40, None) == -1
+    # the synchronising count check rejects bad arguments before touching the device
+    assert L.bof4_outlier_count(None, 8, None, None) == -1
+    assert L.bof4_outlier_count(fake, -1, None, None) == -1
     # EM
     ptrs = (ctypes.c_void_p * 1)(0x1000)
     ns = (ctypes.c_int64 * 1)(100)

@@ -197,6 +197,16 @@ def test_opq_capacity_overflow_reports_true_count(bof4):
     assert int(cnt.item()) == rk
     assert np.array_equal(idx[:cap].cpu().numpy().astype(np.int64), ridx[:cap])
     assert np.all(idx[cap:].cpu().numpy() == -7)
+    # the two-call pattern: the synchronising count check turns the overflow into an error that
+    # names the capacity that would have sufficed; with that capacity the same check passes
+    host = ctypes.c_int64(-1)
+    rc = b.lib().bof4_outlier_count(cnt.data_ptr(), cap, ctypes.byref(host), None)
+    assert rc == -5 and host.value == rk
+    assert str(rk).encode() in b.lib().bof4_last_error()
+    with pytest.raises(b.Bof4Error) as ei:
+        b.bof4_outlier_count(cnt, cap)
+    assert ei.value.code == -5
+    assert b.bof4_outlier_count(cnt, rk) == rk
     # capacity 0: only the count
     cnt.zero_()
     rc = b.lib().bof4_quantize_opq(wd.data_ptr(), b.BF16, n, I, 1, cb.data_ptr(), tau, codes.data_ptr(),
@@ -420,24 +430,16 @@ def test_mae_candidate_list_overflow_takes_the_later_data_passes(bof4):
     assert lv.cpu().numpy()[11] == ref["median"][11]
 
 
-def test_mae_collecting_pass_choice_does_not_change_results(bof4):
-    """The pass that fills the candidate lists is chosen from the data size; forcing the other
-    choice (as for very large inputs) must give the same medians, bit for bit."""
-    import os
-    I, n = 64, 1 << 18
-    w = make_weights(n, torch.bfloat16, 301)
+def test_mae_above_2p26_weights_collects_candidates_one_pass_later(bof4):
+    """Up to 2^26 weights the second data pass fills the candidate lists; beyond that a level's
+    candidates would not fit after one digit, so the third pass collects.  Just above the limit
+    the medians must still be the oracle's, bit for bit (the smaller cases of this file cover the
+    other choice)."""
+    I, n = 64, (1 << 26) + (1 << 16)
+    w = workloads.gaussian_student_mixture(n, 0.02, 0.01, 4, 302, torch.bfloat16)
     ref = oracle.em_accumulate_mae(w, I, 1, LV_INIT)
-    old = os.environ.get("BOF4_MAE_COLLECT_PASS")
-    try:
-        for choice in ("1", "2"):
-            os.environ["BOF4_MAE_COLLECT_PASS"] = choice
-            got = bof4.bof4_em_step([w.cuda()], I, 1, bof4.METRIC_MAE, LV_INIT)
-            _check_mae_stats(got, ref, LV_INIT)
-    finally:
-        if old is None:
-            os.environ.pop("BOF4_MAE_COLLECT_PASS", None)
-        else:
-            os.environ["BOF4_MAE_COLLECT_PASS"] = old
+    got = bof4.bof4_em_step([w.cuda()], I, 1, bof4.METRIC_MAE, LV_INIT)
+    _check_mae_stats(got, ref, LV_INIT)
 
 
 # --------------------------------------------------------------------------- blocks wider than a warp

@@ -68,6 +68,21 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row(L):
         assert torch.equal(got[1][:k], ref[1][:k])              # outlier indices
         assert torch.equal(got[2][:k].view(torch.int16), ref[2][:k].view(torch.int16))
         assert bool((got[1][k:] == -1).all())                   # nothing written past the count
+        # the point of the entry point: with its outputs in place, a call takes no device memory,
+        # neither through torch's allocator nor behind its back
+        clean = torch.empty_like(wd)
+        idx = torch.empty(n, dtype=torch.int32, device="cuda")
+        val = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+        cnt = torch.zeros(1, dtype=torch.int64, device="cuda")
+        stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        free0, used0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+        rc = L.opq_split_static(wd.data_ptr(), b.BF16, n, I, tau, clean.data_ptr(), idx.data_ptr(),
+                                val.data_ptr(), n, cnt.data_ptr(), stream)
+        torch.cuda.synchronize()
+        assert rc == 0
+        assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == used0
+        assert int(cnt.item()) == k
 
 
 def test_static_entry_point_rejects_oversized_input(L):
@@ -76,3 +91,7 @@ def test_static_entry_point_rejects_oversized_input(L):
     rc = L.opq_split_static(fake, b.BF16, MAX_N + I, I, 3.0, None, fake, fake, 8, fake, None)
     assert rc == -2
     assert b"at most" in L.bof4_last_error()
+    # whole blocks only: the ragged last block of opq_split is not offered here
+    rc = L.opq_split_static(fake, b.BF16, 4 * I + 3, I, 3.0, None, fake, fake, 8, fake, None)
+    assert rc == -2
+    assert b"multiple" in L.bof4_last_error()
