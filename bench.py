@@ -1,16 +1,23 @@
 #!/usr/bin/env python
 """Benchmark of the BOF4 hot path on B200.
 
-One *step* is one pass of the whole path over one batch of synthetic weights (the BOF4-S
-workload: 2^26 bf16 weights, 99 % N(0, 0.02^2) + 1 % heavy-tailed, block size 64):
-    EM iteration (MSE)  ->  EM iteration (MAE)  ->  OPQ split + quantise  ->  dequantise with
-    outlier write-back,
-every component called through the C ABI with device-resident inputs.  L2 is flushed before
-every component (a 256 MiB write), so each one streams its inputs from HBM; the step time is
-the sum of the components' CUDA-event times.  Prints ONE JSON line.
+One *step* is one pass of the whole path over the largest single-GPU workloads, every component
+called through the C ABI (the ctypes binding) with device-resident inputs:
+
+    EM iteration, MSE        one bof4_fit_codebook(iters=1) over the 224 Llama-7B-shaped matrices
+    EM iteration, MAE        the same with the weighted-median centroid        (12.95 GB, bf16)
+    quantise                 bof4_quantize   of the 224 Llama-3-8B-shaped matrices (13.96 GB)
+    dequantise               bof4_dequantize of the same set, back to bf16
+    OPQ quantise             bof4_quantize_opq  of one Llama-70B-shaped layer      (1.71 GB)
+    OPQ dequantise           bof4_dequantize with outlier write-back of that layer
+
+Every component streams inputs far larger than L2 (126 MB), so no flush is needed between
+components.  Each component is captured once into a CUDA graph (the same binding calls, on the
+capturing stream) so that its several hundred launches are not limited by Python call overhead;
+the graphs are replayed and timed with CUDA events.  Prints ONE JSON line.
 
 `--impl reference` times the CPU oracle (test infrastructure, never tuned) on the host cores
-with the same metric, each step on a bounded sample of the same workload.
+with the same metric, each step on a bounded sample of the same workloads.
 """
 from __future__ import annotations
 
@@ -18,7 +25,6 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
 import threading
 import time
@@ -34,19 +40,27 @@ import workloads
 
 I = 64
 Q = 0.95
-N_WEIGHTS = workloads.C2_N
-WORKLOAD = "BOF4-S: 2^26 bf16 weights, 99% N(0,0.02^2) + 1% 0.02*t(nu=4), block 64, signed absmax"
-METRIC = ("hot-path step Gweights/s (EM iteration MSE + MAE, OPQ quantize, dequantize); "
-          "components: EM-iteration Gweights/s and quant/dequant HBM GB/s")
+WORKLOAD = ("EM iteration (MSE, MAE; BOF4-S, block 64) over 32 layers x {4 x 4096x4096, 3 x 4096x11008} bf16 "
+            "(sigma ~ U[0.01,0.04] per matrix); quantize + dequantize over 32 layers x {4096x4096, 1024x4096 x2, "
+            "4096x4096, 14336x4096 x2, 4096x14336} bf16 N(0,0.02^2); OPQ quantize + dequantize of one layer "
+            "{8192x8192, 1024x8192 x2, 8192x8192, 28672x8192 x2, 8192x28672} bf16 N(0,0.015^2) + 0.01% outliers")
+METRIC = ("hot-path Gweights/s (weights passed through a component per second, summed over the step's "
+          "components); components: EM-iteration Gweights/s and quant/dequant HBM GB/s")
 # algorithmic bytes per weight of each component (bf16 in, block 64)
 BYTES_EM = 2.0
 BYTES_QUANT = 2.0 + 0.5 + 2.0 / I
 BYTES_DEQUANT = 0.5 + 2.0 / I + 2.0
 BYTES_GEMV = 0.5 + 2.0 / I            # 4-bit codes + bf16 block constants; x and y are negligible
-# data passes of one MAE iteration that stream all weights on this workload: the max-|w| pass
-# and two selection passes (the rest of the selection runs on the candidate lists)
-MAE_DATA_PASSES = 3
+# data passes of one MAE iteration that carry the selection (the max-|w| pass of the call, which
+# exists only for the fixed-point sample weights, is not counted as algorithmic work)
+MAE_SELECTION_PASSES = 2
 FALLBACK_HBM_GBS = 6650.0
+OPQ_OUTLIER_FRACTION = 2.2e-3         # list capacity n / 64 leaves a 7x margin over the expected rate
+
+# dram__bytes_read.sum + dram__bytes_write.sum per weight of the dominant component's kernels,
+# from the committed ncu captures (profiles/), taken on a two-layer slice and scaled by the number
+# of weights (traffic is proportional to it); None once the kernels have changed since.
+TRAFFIC_PER_WEIGHT = {"em_mae": None, "em_mse": None}
 
 
 def measured_peak():
@@ -113,121 +127,139 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
-# --------------------------------------------------------------------------- GPU arm
+# --------------------------------------------------------------------------- workloads on the device
+
+
+def fit_set(dev, seed_offset=0, layers=32):
+    """The Llama-7B-shaped set of the fitting sweep (per-matrix sigma), generated on `dev`."""
+    sig = workloads.config3_sigmas()
+    out = []
+    for i, (r, c) in enumerate(workloads.llama7b_shapes()[: layers * 7]):
+        out.append(workloads.gaussian(r * c, sig[i], 2_000_000 + 1000 * seed_offset + i, torch.bfloat16, dev))
+    return out
+
+
+def quant_set(dev, seed_offset=0, layers=32):
+    """The Llama-3-8B-shaped set of the quantise / dequantise throughput run."""
+    return [workloads.gaussian(r * c, 0.02, 3_000_000 + 1000 * seed_offset + i, torch.bfloat16, dev)
+            for i, (r, c) in enumerate(workloads.llama3_8b_shapes()[: layers * 7])]
+
+
+def opq_layer(dev, seed_offset=0, layer=0):
+    """One Llama-70B-shaped layer with injected outliers."""
+    return workloads.config5_layer(layer + 80 * seed_offset, device=dev)
 
 
 class Step:
     """Device buffers and the component calls of one step."""
 
-    # kernels launched by each component (accumulate + finalise; selection passes; ...)
-    def __init__(self, bof4, dev, seed_offset: int = 0, w_host=None):
-        self.b = bof4
+    def __init__(self, bof4, dev, seed_offset: int = 0, layers: int = 32, sets=None):
+        b = self.b = bof4
         self.dev = dev
-        n = N_WEIGHTS
-        self.n = n
-        self.w_host = w_host if w_host is not None else workloads.gaussian_student_mixture(
-            n, 0.02, 0.01, 4, 1 + seed_offset, torch.bfloat16).pin_memory()
-        self.w = self.w_host.to(dev)
-        self.lv0, self.mask = bof4.bof4_default_init(bof4.NORM_SIGNED)
+        if sets is None:
+            sets = (fit_set(dev, seed_offset, layers), quant_set(dev, seed_offset, layers),
+                    opq_layer(dev, seed_offset))
+        self.w_fit, self.w_q, self.w_opq = sets
+        self.n_fit = sum(w.numel() for w in self.w_fit)
+        self.n_q = sum(w.numel() for w in self.w_q)
+        self.n_opq = sum(w.numel() for w in self.w_opq)
+        self.lv0, self.mask = b.bof4_default_init(b.NORM_SIGNED)
         self.cb0 = torch.tensor(self.lv0, device=dev)
-        self.tau = float(np.float32(bof4.bof4_opq_threshold(Q, I)))
-        self.cap = n // 64
-        self.ws_em = torch.empty(bof4.bof4_workspace_bytes(bof4.OP_EM, n, I, bof4.METRIC_MAE),
-                                 dtype=torch.uint8, device=dev)
-        self.ws_opq = torch.empty(bof4.bof4_workspace_bytes(bof4.OP_OPQ, n, I, 0), dtype=torch.uint8,
-                                  device=dev)
-        self.codes = torch.empty(n // 2, dtype=torch.uint8, device=dev)
-        self.scales = torch.empty(n // I, dtype=torch.bfloat16, device=dev)
-        self.idx = torch.empty(self.cap, dtype=torch.int32, device=dev)
-        self.val = torch.empty(self.cap, dtype=torch.bfloat16, device=dev)
-        self.cnt = torch.zeros(1, dtype=torch.int64, device=dev)
-        self.out = torch.empty(n, dtype=torch.bfloat16, device=dev)
-        self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-        self.flush_src = torch.zeros(64 << 20, dtype=torch.float32, device=dev)  # 256 MiB, only ever read
+        # levels the quantiser uses: the printed BOF4-S (MSE) codebook for block size 64 (Tab. 6)
+        self.cb_q = torch.tensor(np.array(workloads.BOF4S_MSE_I64, np.float32), device=dev)
+        self.tau = float(np.float32(b.bof4_opq_threshold(Q, I)))
+        nmax = max(max(w.numel() for w in s) for s in sets)
+        self.ws_em = torch.empty(b.bof4_workspace_bytes(b.OP_EM, nmax, I, b.METRIC_MAE), dtype=torch.uint8, device=dev)
+        self.ws_opq = torch.empty(b.bof4_workspace_bytes(b.OP_OPQ, nmax, I, 0), dtype=torch.uint8, device=dev)
+        u8, bf = torch.uint8, torch.bfloat16
+        self.q_out = [(torch.empty(w.numel() // 2, dtype=u8, device=dev),
+                       torch.empty(w.numel() // I, dtype=bf, device=dev)) for w in self.w_q]
+        self.q_deq = [torch.empty(w.numel(), dtype=bf, device=dev) for w in self.w_q]
+        self.o_out = []
+        for w in self.w_opq:
+            n, cap = w.numel(), w.numel() // 64
+            self.o_out.append((torch.empty(n // 2, dtype=u8, device=dev), torch.empty(n // I, dtype=bf, device=dev),
+                               torch.empty(cap, dtype=torch.int32, device=dev), torch.empty(cap, dtype=bf, device=dev),
+                               torch.zeros(1, dtype=torch.int64, device=dev)))
+        self.o_deq = [torch.empty(w.numel(), dtype=bf, device=dev) for w in self.w_opq]
         # result buffers of the two fits (levels, error log): no allocation inside the timed region
         self.fit_out = [(torch.empty(16, dtype=torch.float32, device=dev),
                          torch.zeros(1, dtype=torch.float64, device=dev)) for _ in range(2)]
-        self.cb_mse = self.cb_mae = self.cb0
-        self.log_mse = torch.zeros(1, dtype=torch.float64, device=dev)
-        self.have_mae = True
         self.only = None
-        # the decode-side product y = W_q x sees the same codes as a square matrix (profiling runs only)
-        self.gemv_rows = self.gemv_cols = int(round(n ** 0.5))
-        self.x = workloads.gaussian(self.gemv_cols, 1.0, 5 + seed_offset, torch.bfloat16).to(dev)
-        self.y = torch.empty(self.gemv_rows, dtype=torch.float32, device=dev)
+        self.graphs = {}
 
-    def flush_l2(self):
-        # a write larger than L2, then a read of another buffer of the same size: the read pushes
-        # the dirty lines of the write out, so that the timed kernel starts on a cold cache
-        # without having to write somebody else's lines back
-        self.flush_buf.zero_()
-        self.flush_sink = self.flush_src.sum()
-
+    # ---- the six components (binding calls only)
     def em_mse(self):
         b = self.b
-        self.cb_mse, self.log_mse = b.bof4_fit_codebook([self.w], I, b.NORM_SIGNED, b.METRIC_MSE, self.cb0,
-                                                        self.mask, 1, workspace=self.ws_em, sync=False,
-                                                        out=self.fit_out[0])
+        b.bof4_fit_codebook(self.w_fit, I, b.NORM_SIGNED, b.METRIC_MSE, self.cb0, self.mask, 1,
+                            workspace=self.ws_em, sync=False, out=self.fit_out[0])
 
     def em_mae(self):
         b = self.b
-        self.cb_mae, self.log_mae = b.bof4_fit_codebook([self.w], I, b.NORM_SIGNED, b.METRIC_MAE, self.cb0,
-                                                        self.mask, 1, workspace=self.ws_em, sync=False,
-                                                        out=self.fit_out[1])
+        b.bof4_fit_codebook(self.w_fit, I, b.NORM_SIGNED, b.METRIC_MAE, self.cb0, self.mask, 1,
+                            workspace=self.ws_em, sync=False, out=self.fit_out[1])
 
     def quant(self):
         b = self.b
-        b.bof4_quantize_opq(self.w, I, b.NORM_SIGNED, self.cb_mse, self.tau, self.cap,
-                            workspace=self.ws_opq,
-                            out=(self.codes, self.scales, self.idx, self.val, self.cnt))
-
-    def quant_plain(self):
-        b = self.b
-        b.bof4_quantize(self.w, I, b.NORM_SIGNED, self.cb_mse, out=(self.codes, self.scales))
+        for w, out in zip(self.w_q, self.q_out):
+            b.bof4_quantize(w, I, b.NORM_SIGNED, self.cb_q, out=out)
 
     def dequant(self):
         b = self.b
-        b.bof4_dequantize(self.codes, self.scales, I, self.cb_mse, b.BF16, (self.idx, self.val, self.cnt),
-                          out=self.out)
+        for (codes, scales), out in zip(self.q_out, self.q_deq):
+            b.bof4_dequantize(codes, scales, I, self.cb_q, b.BF16, out=out)
 
-    def gemv(self):
+    def opq_quant(self):
         b = self.b
-        b.bof4_gemv(self.codes, self.scales, self.gemv_rows, self.gemv_cols, I, self.cb_mse, self.x,
-                    (self.idx, self.val, self.cnt), out=self.y)
+        for w, out in zip(self.w_opq, self.o_out):
+            b.bof4_quantize_opq(w, I, b.NORM_SIGNED, self.cb_q, self.tau, out[2].numel(), workspace=self.ws_opq, out=out)
+
+    def opq_dequant(self):
+        b = self.b
+        for (codes, scales, idx, val, cnt), out in zip(self.o_out, self.o_deq):
+            b.bof4_dequantize(codes, scales, I, self.cb_q, b.BF16, (idx, val, cnt), out=out)
 
     def components(self):
-        comps = [("em_mse", self.em_mse, 2), ("em_mae", self.em_mae, None), ("quantize_opq", self.quant, 4),
-                 ("dequantize", self.dequant, 2)]
-        comps = [c for c in comps if c[0] != "em_mae" or self.have_mae]
+        """(name, call, weights per call, algorithmic bytes per weight, kernels launched per call)"""
+        b = self.b.binding
+        nt, nq, no = len(self.w_fit), len(self.w_q), len(self.w_opq)
+        comps = [("em_mse", self.em_mse, self.n_fit, BYTES_EM, b.mse_launches_per_iteration(nt)),
+                 ("em_mae", self.em_mae, self.n_fit, BYTES_EM * MAE_SELECTION_PASSES,
+                  b.mae_launches_per_call(nt, self.n_fit, 1)),
+                 ("quantize", self.quant, self.n_q, BYTES_QUANT, nq),
+                 ("dequantize", self.dequant, self.n_q, BYTES_DEQUANT, nq),
+                 ("opq_quantize", self.opq_quant, self.n_opq, BYTES_QUANT + 6 * OPQ_OUTLIER_FRACTION / 2.2, 2 * no),
+                 ("opq_dequantize", self.opq_dequant, self.n_opq, BYTES_DEQUANT + 6 * OPQ_OUTLIER_FRACTION / 2.2, 2 * no)]
         if self.only:
-            comps.append(("quantize", self.quant_plain, 1))  # profiling runs only
-            comps.append(("gemv", self.gemv, 2))
             comps = [c for c in comps if c[0] in self.only]
         return comps
 
+    def capture(self):
+        """Captures every component into its own CUDA graph (after it has run once eagerly, so that
+        one-time set-up such as shared-memory attributes is done before the capture)."""
+        for name, fn, *_ in self.components():
+            fn()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            self.graphs[name] = g
+
     def run_timed(self):
-        """One step; returns {component: ms} from CUDA events on the current stream."""
+        """One step; returns {component: (start, end)} CUDA events on the current stream."""
         times = {}
-        for name, fn, _ in self.components():
-            self.flush_l2()
+        for name, fn, *_ in self.components():
             s = torch.cuda.Event(enable_timing=True)
             e = torch.cuda.Event(enable_timing=True)
             s.record()
-            fn()
+            g = self.graphs.get(name)
+            if g is not None:
+                g.replay()
+            else:
+                fn()
             e.record()
             times[name] = (s, e)
         return times
-
-    def run_e2e(self, host_out):
-        """The same step from pinned host memory and back (copies inside the timed region)."""
-        self.w.copy_(self.w_host, non_blocking=True)
-        for _, fn, _ in self.components():
-            fn()
-        k = 0
-        for name in ("codes", "scales", "idx", "val", "cnt", "out"):
-            host_out[name].copy_(getattr(self, name), non_blocking=True)
-        host_out["cb_mse"].copy_(self.cb_mse, non_blocking=True)
-        host_out["log_mse"].copy_(self.log_mse, non_blocking=True)
 
 
 def rank_env():
@@ -256,8 +288,77 @@ def whole_job_gweights_per_s(world: int, n_per_rank: int, ms_per_step: float) ->
     return world * n_per_rank / ms_per_step / 1e6
 
 
-def mae_launches(bof4) -> int:
-    return getattr(bof4.binding, "MAE_LAUNCHES_PER_ITERATION", 0)
+# --------------------------------------------------------------------------- end to end (host buffers)
+
+
+class E2E:
+    """The same component calls fed from pinned host memory and read back to it, on a bounded slice
+    of the step's workloads (the first `layers` layers of the two 32-layer sets and the whole OPQ
+    layer), two slices in flight on two streams so that one upload overlaps the other download.
+    quantize_only: weights up, quantise / OPQ quantise, codes + scales + outlier lists down."""
+
+    def __init__(self, bof4, dev, full: Step, layers: int, quantize_only: bool):
+        self.quantize_only = quantize_only
+        k = layers * 7
+        sets = (full.w_fit[:k], full.w_q[:k], full.w_opq)
+        self.used = (1, 2) if quantize_only else (0, 1, 2)     # which sets travel
+        self.host_in = [[w.cpu().pin_memory() for w in s] if i in self.used else [] for i, s in enumerate(sets)]
+        self.slots = []
+        for _ in range(2):
+            dsets = tuple([torch.empty_like(w) for w in s] if i in self.used else s for i, s in enumerate(sets))
+            st = Step(bof4, dev, sets=dsets)
+            outs = [t for pair in st.q_out for t in pair] + [t for o in st.o_out for t in o]
+            if not quantize_only:
+                outs += [st.fit_out[0][0], st.fit_out[0][1], st.fit_out[1][0], st.fit_out[1][1]]
+                outs += st.q_deq + st.o_deq
+            host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in outs]
+            self.slots.append((st, dsets, outs, host_out))
+        st = self.slots[0][0]
+        self.weights_per_step = (st.n_q + st.n_opq) if quantize_only else 2 * (st.n_fit + st.n_q + st.n_opq)
+        self.h2d = sum(w.numel() * 2 for i in self.used for w in sets[i])
+        self.d2h = sum(t.numel() * t.element_size() for t in self.slots[0][3])
+
+    def one(self, slot):
+        st, dsets, outs, host_out = self.slots[slot]
+        for i in self.used:
+            for h, d in zip(self.host_in[i], dsets[i]):
+                d.copy_(h, non_blocking=True)
+        if self.quantize_only:
+            st.quant()
+            st.opq_quant()
+        else:
+            for _, fn, *_ in st.components():
+                fn()
+        for d, h in zip(outs, host_out):
+            h.copy_(d, non_blocking=True)
+
+    def run(self, count, streams):
+        main = torch.cuda.current_stream()
+        for sm in streams:
+            sm.wait_stream(main)
+        for i in range(count):
+            with torch.cuda.stream(streams[i & 1]):
+                self.one(i & 1)
+        for sm in streams:
+            main.wait_stream(sm)
+
+
+def time_e2e(e2e: E2E, steps: int, dist, dev):
+    streams = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    e2e.run(2, streams)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    s = torch.cuda.Event(enable_timing=True)
+    e = torch.cuda.Event(enable_timing=True)
+    s.record()
+    e2e.run(steps, streams)
+    e.record()
+    torch.cuda.synchronize()
+    return s.elapsed_time(e)
+
+
+# --------------------------------------------------------------------------- GPU arm
 
 
 def run_gpu(args):
@@ -278,15 +379,13 @@ def run_gpu(args):
     from paper_2505_06653_b200 import binding
     binding.lib()
 
-    st = Step(bof4, dev, seed_offset=workload_seed_offset(rank))  # no data-path collective
-    st.have_mae = hasattr(binding, "MAE_LAUNCHES_PER_ITERATION")
+    st = Step(bof4, dev, seed_offset=workload_seed_offset(rank), layers=args.layers)  # no data-path collective
     if args.only:
         st.only = set(args.only.split(","))
         args.no_e2e = args.no_cpu_baseline = True
-        if "gemv" in st.only:
-            assert st.gemv_rows * st.gemv_cols == st.n
-            st.quant()  # the matrix the product reads
     K, W = args.steps, args.warmup
+    if not args.no_graphs:
+        st.capture()
     for _ in range(W):
         st.run_timed()
     torch.cuda.synchronize()
@@ -301,176 +400,195 @@ def run_gpu(args):
         dist.barrier()
     comp_ms = {name: [s.elapsed_time(e) for s, e in (r[name] for r in recs)] for name in recs[0]}
     total_ms = sum(sum(v) for v in comp_ms.values())
-    # keep the device busy a little longer so that the clock sampler sees the loaded state
-    t_end = time.time() + 0.3
-    while time.time() < t_end:
-        st.run_timed()
-    torch.cuda.synchronize()
     clocks = sampler.stop()
 
-    # ---- end to end: pinned host buffers in and out, through the same calls.  Two steps are in
-    # flight on two streams with their own device and host buffers, so that one step's upload
-    # overlaps the previous step's download (the copy engines work in both directions at once);
-    # every step still uploads its weights and downloads all of its results inside the timed region.
-    def make_host_out(step):
-        h = {k: torch.empty_like(getattr(step, k), device="cpu").pin_memory()
-             for k in ("codes", "scales", "idx", "val", "cnt", "out")}
-        h["cb_mse"] = torch.empty(16, dtype=torch.float32).pin_memory()
-        h["log_mse"] = torch.empty(1, dtype=torch.float64).pin_memory()
-        return h
+    # one 30-iteration MAE and MSE fit per call, as the fitting sweep runs them: the per-call
+    # max-|w| pass of the MAE fit is then shared by 30 iterations (reported beside the step)
+    fit30 = {}
+    if not args.only:
+        b = bof4
+        for name, metric in (("mse", b.METRIC_MSE), ("mae", b.METRIC_MAE)):
+            log = torch.zeros(30, dtype=torch.float64, device=dev)
+            cb = torch.empty(16, dtype=torch.float32, device=dev)
+            s = torch.cuda.Event(enable_timing=True)
+            e = torch.cuda.Event(enable_timing=True)
+            s.record()
+            b.bof4_fit_codebook(st.w_fit, I, b.NORM_SIGNED, metric, st.cb0, st.mask, 30, workspace=st.ws_em,
+                                sync=False, out=(cb, log))
+            e.record()
+            torch.cuda.synchronize()
+            fit30[name] = s.elapsed_time(e) / 30.0
 
-    Ke = 0 if args.no_e2e else max(2, min(K, 10))
-    host_out = make_host_out(st)
-    e2e_ms = 0.0
+    # ---- end to end: pinned host buffers in and out, through the same calls
+    e2e_ms = e2eq_ms = 0.0
+    Ke = 0 if args.no_e2e else 3
+    e2e = e2eq = None
     if Ke:
-        st2 = Step(bof4, dev, seed_offset=workload_seed_offset(rank), w_host=st.w_host)
-        st2.have_mae = st.have_mae
-        sets, outs = [st, st2], [host_out, make_host_out(st2)]
-        streams = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+        el = min(args.e2e_layers, args.layers)
+        e2e = E2E(bof4, dev, st, el, quantize_only=False)
+        e2e_ms = time_e2e(e2e, Ke, dist, dev)
+        del e2e.slots
+        e2eq = E2E(bof4, dev, st, el, quantize_only=True)
+        e2eq_ms = time_e2e(e2eq, Ke, dist, dev)
+        del e2eq.slots
 
-        def e2e_steps(count):
-            main = torch.cuda.current_stream()
-            for sm in streams:
-                sm.wait_stream(main)
-            for i in range(count):
-                with torch.cuda.stream(streams[i & 1]):
-                    sets[i & 1].run_e2e(outs[i & 1])
-            for sm in streams:
-                main.wait_stream(sm)
-
-        e2e_steps(2)
-        torch.cuda.synchronize()
-        if dist:
-            dist.barrier()
-        s = torch.cuda.Event(enable_timing=True)
-        e = torch.cuda.Event(enable_timing=True)
-        s.record()
-        e2e_steps(Ke)
-        e.record()
-        torch.cuda.synchronize()
-        e2e_ms = s.elapsed_time(e)
-    h2d = st.w_host.numel() * 2
-    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
-
-    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, dev)
+    total_ms, e2e_ms, e2eq_ms = max_over_ranks([total_ms, e2e_ms, e2eq_ms], dist, dev)
     if rank != 0:
         if dist:
             dist.destroy_process_group()
         return
 
-    n = st.n
     ms_per_step = total_ms / K
     peak, peak_kind = measured_peak()
     avg = {k: sum(v) / len(v) for k, v in comp_ms.items()}
-    bytes_per_w = {"em_mse": BYTES_EM, "em_mae": None, "quantize_opq": BYTES_QUANT, "dequantize": BYTES_DEQUANT,
-                   "quantize": BYTES_QUANT, "gemv": BYTES_GEMV}
-    # em_mae: the iteration's kernels + the call's max-|w| pass
-    kernels = {"em_mse": 1, "em_mae": mae_launches(bof4) + 1, "quantize_opq": 2, "dequantize": 2, "quantize": 1,
-               "gemv": 2}
-    comp, launches = {}, 0
+    comp, launches, weights_per_step = {}, 0, 0
+    info = {c[0]: c for c in st.components()}
     for name, ms in avg.items():
+        _, _, n, bpw, nk = info[name]
         comp[name + "_ms"] = ms
-        if name.startswith("em_"):
-            comp[name + "_gweights_s"] = n / ms / 1e6
-        if bytes_per_w[name]:
-            comp[name + "_gbs"] = bytes_per_w[name] * n / ms / 1e6
-        launches += kernels[name]
-    for k in list(comp):
-        if k.endswith("_gbs"):
-            comp[k.replace("_gbs", "_frac_of_%s_hbm" % peak_kind)] = comp[k] / peak
+        comp[name + "_gweights_s"] = n / ms / 1e6
+        comp[name + "_gbs"] = bpw * n / ms / 1e6
+        comp[name + "_frac_of_%s_hbm" % peak_kind] = bpw * n / ms / 1e6 / peak
+        launches += nk
+        weights_per_step += n
+    if fit30:
+        comp["em_mse_ms_per_iteration_in_a_30_iteration_fit"] = fit30["mse"]
+        comp["em_mae_ms_per_iteration_in_a_30_iteration_fit"] = fit30["mae"]
+        comp["em_mae_gbs_in_a_30_iteration_fit"] = BYTES_EM * MAE_SELECTION_PASSES * st.n_fit / fit30["mae"] / 1e6
     # dominant component = the one with the largest share of the step
     dom = max(avg, key=avg.get)
-    dom_bytes = {"em_mse": BYTES_EM, "em_mae": BYTES_EM * MAE_DATA_PASSES, "quantize_opq": BYTES_QUANT,
-                 "dequantize": BYTES_DEQUANT, "quantize": BYTES_QUANT, "gemv": BYTES_GEMV}[dom] * n
-    achieved = dom_bytes / avg[dom] / 1e6
+    _, _, dn, dbpw, _ = info[dom]
+    achieved = dbpw * dn / avg[dom] / 1e6
+    tpw = TRAFFIC_PER_WEIGHT.get(dom)
     line = {
-        "metric": METRIC, "value": whole_job_gweights_per_s(world, n, ms_per_step), "unit": "Gweights/s",
-        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_per_step,
+        "metric": METRIC, "value": whole_job_gweights_per_s(world, weights_per_step, ms_per_step),
+        "unit": "Gweights/s", "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD, "n_weights_per_gpu": n, "block_size": I,
-                   "opq_q": Q, "l2": "flushed before every component (256 MiB write, then 256 MiB read: no dirty lines left)",
+        "config": {"workload": WORKLOAD, "layers": args.layers,
+                   "weights_per_gpu": {"fit_set": st.n_fit, "quantize_set": st.n_q, "opq_layer": st.n_opq},
+                   "weight_passes_per_step": weights_per_step, "block_size": I, "opq_q": Q,
+                   "l2": "inputs larger than L2 (12.95 GB / 13.96 GB / 1.71 GB per component): no flush",
+                   "launch": "one CUDA graph per component" if not args.no_graphs else "eager binding calls",
                    "multi_gpu": "independent problem per rank, no collective",
-                   "e2e": "two steps in flight on two streams (upload of one overlaps download of the other)"},
+                   "e2e": "first %d layers of the two 32-layer sets and the whole OPQ layer from pinned host memory, "
+                          "all results (incl. dequantised tensors) back; two slices in flight on two streams"
+                          % min(args.e2e_layers, args.layers)},
         "components": comp,
         "clocks": clocks,
-        "e2e": {"value": (world * n * Ke / e2e_ms / 1e6) if Ke else None, "unit": "Gweights/s",
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": Ke},
+        "e2e": {"value": (world * e2e.weights_per_step * Ke / e2e_ms / 1e6) if Ke else None, "unit": "Gweights/s",
+                "h2d_bytes_per_step": e2e.h2d if Ke else 0, "d2h_bytes_per_step": e2e.d2h if Ke else 0, "steps": Ke},
+        "e2e_quantize_only": {"value": (world * e2eq.weights_per_step * Ke / e2eq_ms / 1e6) if Ke else None,
+                              "unit": "Gweights/s", "h2d_bytes_per_step": e2eq.h2d if Ke else 0,
+                              "d2h_bytes_per_step": e2eq.d2h if Ke else 0, "steps": Ke,
+                              "what": "weights up, quantise / OPQ quantise, codes + scales + outlier lists down"},
         "gpu_launches": launches * K,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": TRAFFIC.get(dom)},
+                     "traffic": (tpw * dn) if tpw else None},
     }
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(st.w_host, have_mae=st.have_mae)
+        line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line), flush=True)
     if dist:
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the dominant component's data-carrying kernels
-# per step, from the committed ncu captures (profiles/); None for a component whose kernels have
-# changed since the counters were taken
-TRAFFIC = {"em_mae": 414.4e6,   # max-|w| pass 137.3 MB + first pass 138.8 MB + collecting pass 138.3 MB
-           "em_mse": 138.3e6}
-
-
 # --------------------------------------------------------------------------- CPU arm (oracle)
 
 
-def oracle_step(oracle, w32, lv0, mask, tau, have_mae=True):
-    """The same step computed by the CPU oracle on fp32-widened weights."""
-    cb, _ = oracle.fit(w32, I, oracle.NORM_SIGNED, oracle.METRIC_MSE, lv0, mask, 1)
-    if have_mae:
-        oracle.fit(w32, I, oracle.NORM_SIGNED, oracle.METRIC_MAE, lv0, mask, 1)
-    clean, idx, val, k = oracle.opq_split(w32, I, tau)
-    codes, scales = oracle.quantize(clean, I, oracle.NORM_SIGNED, cb)
-    out = oracle.dequantize(codes, scales, I, cb)
+def oracle_sample(rows: int = 256):
+    """A bounded sample of the step's workloads for the CPU legs: the first matrix of each set
+    cut to its first `rows` rows (CPU generator, same recipe)."""
+    sig = workloads.config3_sigmas()
+    r, c = workloads.llama7b_shapes()[0]
+    fit = workloads.gaussian(min(rows, r) * c, sig[0], 2_000_000, torch.bfloat16)
+    r, c = workloads.llama3_8b_shapes()[0]
+    qs = workloads.gaussian(min(rows, r) * c, 0.02, 3_000_000, torch.bfloat16)
+    r, c = workloads.llama70b_layer_shapes()[0]
+    op = workloads.inject_outliers(workloads.gaussian(min(rows // 2, r) * c, 0.015, 4_000_000, torch.bfloat16),
+                                   0.015, 1e-4, 10.0, 40.0, 4_000_008)
+    return fit, qs, op
+
+
+def oracle_step(oracle, sample, lv0, lvq, mask, tau):
+    """The same six components computed by the CPU oracle on fp32-widened weights; returns the
+    number of weight passes."""
+    fit, qs, op = sample
+    oracle.fit(fit, I, oracle.NORM_SIGNED, oracle.METRIC_MSE, lv0, mask, 1)
+    oracle.fit(fit, I, oracle.NORM_SIGNED, oracle.METRIC_MAE, lv0, mask, 1)
+    codes, scales = oracle.quantize(qs, I, oracle.NORM_SIGNED, lvq)
+    oracle.dequantize(codes, scales, I, lvq)
+    clean, idx, val, k = oracle.opq_split(op, I, tau)
+    codes, scales = oracle.quantize(clean, I, oracle.NORM_SIGNED, lvq)
+    out = oracle.dequantize(codes, scales, I, lvq)
     oracle.opq_restore(out, idx, val)
-    return out
+    return 2 * (fit.size + qs.size + op.size)
 
 
-def cpu_baseline(w_host, have_mae=True, sample=1 << 25, reps=2):
+def _oracle_setup(rows):
     import oracle
     oracle.build()
-    w32 = oracle.as_f32(w_host[:sample])
+    sample = tuple(oracle.as_f32(t) for t in oracle_sample(rows))
     lv0 = np.array(workloads.init_levels_7_0_8(), np.float32)
+    lvq = np.array(workloads.BOF4S_MSE_I64, np.float32)
     tau = float(np.float32(oracle.opq_threshold(Q, I)))
+    return oracle, sample, lv0, lvq, tau
+
+
+def omp_set_threads(n: int):
+    """Thread count of the OpenMP runtime the oracle's library is linked against (the oracle itself
+    is left as it stands)."""
+    import ctypes
+    ctypes.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
+
+
+def cpu_baseline(rows: int = 1024, reps: int = 2):
+    """The oracle on all host cores, and on one core, on a bounded sample of the step."""
+    oracle, sample, lv0, lvq, tau = _oracle_setup(rows)
     t0 = time.time()
     for _ in range(reps):
-        oracle_step(oracle, w32, lv0, workloads.FIXED_BOF4S, tau, have_mae)
+        passes = oracle_step(oracle, sample, lv0, lvq, workloads.FIXED_BOF4S, tau)
     dt = (time.time() - t0) / reps
-    return {"value": sample / dt / 1e9, "unit": "Gweights/s", "cores": oracle.n_threads(),
-            "kind": "oracle", "sample": "first 2^%d weights of the workload, %d steps" %
-            (int(np.log2(sample)), reps)}
+    out = {"value": passes / dt / 1e9, "unit": "Gweights/s", "cores": oracle.n_threads(), "kind": "oracle",
+           "sample": "first %d rows of the first matrix of each of the three sets (%.1e weight passes per step), "
+                     "%d steps" % (rows, passes, reps)}
+    # single-threaded, on a quarter of that sample
+    _, small, _, _, _ = _oracle_setup(rows // 4)
+    all_cores = oracle.n_threads()
+    omp_set_threads(1)
+    t0 = time.time()
+    p1 = oracle_step(oracle, small, lv0, lvq, workloads.FIXED_BOF4S, tau)
+    dt1 = time.time() - t0
+    omp_set_threads(all_cores)
+    out["single_thread"] = {"value": p1 / dt1 / 1e9, "unit": "Gweights/s", "cores": 1,
+                            "sample": "first %d rows, 1 step" % (rows // 4)}
+    return out
 
 
 def run_reference(args):
     rank = rank_env()[0]
     if rank != 0:
         return None
-    import oracle
-    oracle.build()
-    sample = 1 << 24
-    w = workloads.gaussian_student_mixture(sample, 0.02, 0.01, 4, 1, torch.bfloat16)
-    w32 = oracle.as_f32(w)
-    lv0 = np.array(workloads.init_levels_7_0_8(), np.float32)
-    tau = float(np.float32(oracle.opq_threshold(Q, I)))
+    rows = 512
+    oracle, sample, lv0, lvq, tau = _oracle_setup(rows)
     for _ in range(args.warmup):
-        oracle_step(oracle, w32, lv0, workloads.FIXED_BOF4S, tau)
+        oracle_step(oracle, sample, lv0, lvq, workloads.FIXED_BOF4S, tau)
     t0 = time.time()
+    passes = 0
     for _ in range(args.steps):
-        oracle_step(oracle, w32, lv0, workloads.FIXED_BOF4S, tau)
+        passes += oracle_step(oracle, sample, lv0, lvq, workloads.FIXED_BOF4S, tau)
     dt = time.time() - t0
-    val = sample * args.steps / dt / 1e9
-    desc = {"value": val, "unit": "Gweights/s", "cores": oracle.n_threads(), "kind": "oracle",
-            "sample": "2^24 weights of the workload per step"}
+    val = passes / dt / 1e9
+    what = "first %d rows of the first matrix of each of the three sets per step" % rows
+    desc = {"value": val, "unit": "Gweights/s", "cores": oracle.n_threads(), "kind": "oracle", "sample": what}
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "Gweights/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "ms_per_step": dt / max(args.steps, 1) * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "n_weights_per_step": sample, "block_size": I, "opq_q": Q},
+        "config": {"workload": WORKLOAD, "sample": what, "weight_passes_per_step": passes // max(args.steps, 1),
+                   "block_size": I, "opq_q": Q},
         "cpu_baseline": desc,
         "e2e": {"value": val, "unit": "Gweights/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }), flush=True)
@@ -483,7 +601,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer legs (profiling runs)")
+    ap.add_argument("--no-graphs", action="store_true", help="call the binding eagerly instead of replaying graphs")
+    ap.add_argument("--layers", type=int, default=32, help="layers of the two 32-layer sets (fewer: profiling "
+                    "runs on a slice; the JSON line is then not a bench result)")
+    ap.add_argument("--e2e-layers", type=int, default=4, help="layers of the 32-layer sets in the host-buffer legs")
     ap.add_argument("--only", default="", help="comma list of components to run (profiling runs only; "
                     "the JSON line is then not a bench result)")
     args = ap.parse_args()

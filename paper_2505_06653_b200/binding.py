@@ -29,6 +29,23 @@ LEVELS = 16
 # that carry their own selection and the level update
 MAE_LAUNCHES_PER_ITERATION = 7
 
+TENSORS_PER_LAUNCH = 64  # tensors of a multi-tensor fit that one accumulation launch covers
+
+
+def mse_launches_per_iteration(n_tensors: int) -> int:
+    """Kernels one MSE iteration enqueues (the M step rides in the last accumulation launch)."""
+    return max(1, -(-n_tensors // TENSORS_PER_LAUNCH))
+
+
+def mae_launches_per_call(n_tensors: int, n_total: int, iters: int) -> int:
+    """Kernels a MAE fit of `iters` iterations enqueues: the max-|w| pass of the call, then per
+    iteration the set-up, four data passes and the selection kernels of the passes that do not
+    carry their own selection (two up to 2^26 weights, three beyond)."""
+    chunks = max(1, -(-n_tensors // TENSORS_PER_LAUNCH))
+    small = n_total // LEVELS // 512 <= (1 << 16) // 8
+    return chunks + iters * (1 + 4 * chunks + (2 if small else 3))
+
+
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_theoretical_codebook_batch",

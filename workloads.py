@@ -167,5 +167,12 @@ def init_levels_linspace() -> List[float]:
     return lv
 
 
+# The printed BOF4-S (MSE) codebook for block size 64 (Tab. 6): the levels the quantise /
+# dequantise throughput runs use (an input, like the starting codebooks above).
+BOF4S_MSE_I64 = [-0.8568463921546936, -0.6692874431610107, -0.5235266089439392, -0.4004882574081421,
+                 -0.2910638153553009, -0.1900092959403992, -0.0938529595732689, 0.0,
+                 0.0887671709060669, 0.1794802695512772, 0.2743096053600311, 0.3760197460651398,
+                 0.4886530041694641, 0.6188603639602661, 0.7791395783424377, 1.0]
+
 FIXED_BOF4 = (1 << 0) | (1 << 7) | (1 << 15)   # levels -1, 0, 1 (absolute normalisation)
 FIXED_BOF4S = (1 << 7) | (1 << 15)             # levels 0, 1 (signed normalisation)
