@@ -10,6 +10,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "lane32.cuh"
 #include "layout.h"
 
 namespace bof4 {
@@ -140,6 +141,130 @@ quantize_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__
         quantize_row<DT, I, SIGNED, ST>(v, mx, mn, map.idx(r), map.ok(r), T, lut_base, lane, codes, scales,
                                         &s_wide);
         raw = next;
+    }
+}
+
+// ---------------------------------------------------------------- quantise, bf16 weights
+//
+// 32 weights per lane (lane32.cuh); two row buffers used in turn, so that the load of the row
+// after next is issued before a row is processed and no register is copied between iterations.
+
+constexpr int kQRow32 = kQThreads * kLW;  // weights per CTA row
+
+struct QuantShared32 {
+    float xi[kLevels], lv[kLevels];
+    int multi;
+    WideScratch wide;
+    FastInfo info;
+};
+
+// Block constant, codes and stores for the lane's 32 (cleaned) weights of one row.
+template <int I, bool SIGNED, class ST>
+__device__ __forceinline__ void quantize_row32(const uint32_t (&u)[16], float mx, float mn, int64_t idx, bool ok,
+                                               bool lut_ok, uint32_t lut_base, QuantShared32* S,
+                                               uint8_t* __restrict__ codes, void* __restrict__ scales)
+{
+    float g;
+    const float m = block_constant32<I, SIGNED>(u, mx, mn, g, &S->wide);
+    const int path = row_path(g, m, ok, lut_ok, &S->info);
+    const float md = ok ? m : 1.0f;  // divisor of the table paths: never zero
+    uint32_t cw[4];
+    if (path == kPathFast)
+        encode32_lut<false>(u, md, lut_base, cw);
+    else if (path == kPathExact)
+        encode32_lut<true>(u, md, lut_base, cw);
+    else
+        encode32_slow(u, m, S->xi, cw);
+    if (ok) {
+        st_stream128(codes + idx / 2, cw[0], cw[1], cw[2], cw[3]);
+        if ((idx & (I - 1)) == 0) store_scale<ST>(scales, idx / I, m);  // the block's first lane
+    }
+}
+
+// The same for one row outside the common case (a block constant that is zero, extreme, not
+// finite or of a "near" significand; a codebook the table cannot serve; the partial last row of
+// a tensor), kept out of line so that it costs the streaming loop no registers.  Blocks within
+// a warp only (the wide-block kernel below calls quantize_row32 itself).
+template <int I, bool SIGNED, class ST>
+__device__ __noinline__ void quantize_row32_generic(Raw32 raw, int64_t idx, bool ok, bool lut_ok, uint32_t lut_base,
+                                                    QuantShared32* S, uint8_t* __restrict__ codes,
+                                                    void* __restrict__ scales)
+{
+    uint32_t u[16];
+    words_of(raw, u);
+    float mx, mn;
+    lane_minmax32(u, mx, mn);
+    quantize_row32<I, SIGNED, ST>(u, mx, mn, idx, ok, lut_ok, lut_base, S, codes, scales);
+}
+
+template <int I, bool SIGNED, class ST>
+__global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
+quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels,
+                  uint8_t* __restrict__ codes, void* __restrict__ scales)
+{
+    extern __shared__ __align__(16) unsigned char s_lut[];
+    __shared__ QuantShared32 S;
+    const RowMap32 map(n, kQRow32, threadIdx.x);
+    const int G = gridDim.x;
+    int r = blockIdx.x;
+    if (r >= map.rows) return;
+    auto fetch = [&](int rr) { return map.ok(rr) ? load_raw32(w, map.idx(rr)) : zero_raw32(); };
+    const Raw32 first = fetch(r);  // on its way while the tables are built
+    QuantTables T{S.xi, s_lut, false};
+    T.lut_ok = build_tables32(levels, S.xi, S.lv, s_lut, &S.info, [](int base) { return (uint32_t)base; });
+    const uint32_t lut_base = lut_lane_base(s_lut, threadIdx.x & 31);
+    if constexpr (Geo32<I>::WPB > 1) {
+        // blocks of several warps: every thread of the CTA takes every step (barriers inside)
+        Raw32 a = first;
+        for (; r < map.rows; r += G) {
+            const Raw32 next = fetch(r + G);
+            uint32_t u[16];
+            words_of(a, u);
+            float mx, mn;
+            lane_minmax32(u, mx, mn);
+            quantize_row32<I, SIGNED, ST>(u, mx, mn, map.idx(r), map.ok(r), T.lut_ok, lut_base, &S, codes, scales);
+            a = next;
+        }
+    } else {
+        // Whole rows: unconditional loads into two buffers used in turn; a row all of whose block
+        // constants are ordinary is encoded here, any other goes to the out-of-line version.
+        const bool fast_ok = T.lut_ok && !S.info.tiny;
+        auto row = [&](const Raw32& raw, int rr) {
+            uint32_t u[16];
+            words_of(raw, u);
+            float mx, mn, g;
+            lane_minmax32(u, mx, mn);
+            const float m = block_constant32<I, SIGNED>(u, mx, mn, g, nullptr);
+            const int64_t idx = map.idx(rr);
+            if (fast_ok && __all_sync(kFull, div_safe(g) && !near_significand(m, &S.info))) {
+                uint32_t cw[4];
+                encode32_lut<false>(u, m, lut_base, cw);
+                st_stream128(codes + idx / 2, cw[0], cw[1], cw[2], cw[3]);
+                if ((idx & (I - 1)) == 0) store_scale<ST>(scales, idx / I, m);
+            } else {
+                quantize_row32_generic<I, SIGNED, ST>(raw, idx, true, T.lut_ok, lut_base, &S, codes, scales);
+            }
+        };
+        const int full = map.rows_full;
+        if (r < full) {
+            Raw32 a = first, b = first;
+            while (true) {
+                int rn = r + G;
+                if (rn < full) b = load_raw32(w, map.idx(rn));
+                row(a, r);
+                if (rn >= full) break;
+                r = rn;
+                rn = r + G;
+                if (rn < full) a = load_raw32(w, map.idx(rn));
+                row(b, r);
+                if (rn >= full) break;
+                r = rn;
+            }
+        }
+        // the partial last row of the tensor, by the CTA whose turn it is
+        if (map.rows > full && full % G == (int)blockIdx.x)
+            quantize_row32_generic<I, SIGNED, ST>(full == (int)blockIdx.x ? first : fetch(full), map.idx(full),
+                                                  map.ok(full), T.lut_ok, lut_base, &S, codes, scales);
     }
 }
 
@@ -754,6 +879,9 @@ int check_aligned(const char* fn, const char* what, const void* p)
 #define BOF4_DISPATCH_BOOL(FLAG, NAME, ...)                \
     if (FLAG) { constexpr bool NAME = true; __VA_ARGS__; } \
     else { constexpr bool NAME = false; __VA_ARGS__; }
+#define BOF4_DISPATCH_ST(SD, ...)                        \
+    if ((SD) == BOF4_BF16) { using ST = BF16; __VA_ARGS__; } \
+    else { using ST = F32; __VA_ARGS__; }
 // (weight dtype, scale dtype) in {(f32,f32), (bf16,bf16), (bf16,f32)}
 #define BOF4_DISPATCH_WS(WD, SD, ...)                                               \
     if ((WD) == BOF4_F32) { using DT = F32; using ST = F32; __VA_ARGS__; }          \
@@ -782,14 +910,22 @@ extern "C" int bof4_quantize(const void* d_w, int w_dtype, int64_t n, int block_
     const int64_t n_whole = n - tail;
     n = n_whole;
     if (n > 0) {
-        const int64_t rows = (n + kQRow - 1) / kQRow;
-        const int grid = grid_for(rows, kQCtasPerSm);
-        BOF4_DISPATCH_WS(w_dtype, scale_dtype,
+        if (w_dtype == BOF4_BF16) {
+            const int grid = grid_for((n + kQRow32 - 1) / kQRow32, kQCtasPerSm);
+            BOF4_DISPATCH_ST(scale_dtype,
+                BOF4_DISPATCH_I(block_size,
+                    BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                        { constexpr auto kern = quantize32_kernel<I_, SG, ST>;
+                          if ((rc = ensure_dynamic_smem<kern>(kLutBytes))) return rc;
+                          kern<<<grid, kQThreads, kLutBytes, st>>>(d_w, n, d_codebook, d_codes, d_scales); })));
+        } else {
+            const int grid = grid_for((n + kQRow - 1) / kQRow, kQCtasPerSm);
             BOF4_DISPATCH_I(block_size,
                 BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
-                    { constexpr auto kern = quantize_kernel<DT, I_, SG, ST>;
+                    { constexpr auto kern = quantize_kernel<F32, I_, SG, F32>;
                       if ((rc = ensure_dynamic_smem<kern>(kLutBytes))) return rc;
-                      kern<<<grid, kQThreads, kLutBytes, st>>>(d_w, n, d_codebook, d_codes, d_scales); })));
+                      kern<<<grid, kQThreads, kLutBytes, st>>>(d_w, n, d_codebook, d_codes, d_scales); }));
+        }
         BOF4_CUDA_TRY(cudaGetLastError());
     }
     if (tail) {
