@@ -183,20 +183,22 @@ class Step:
                                torch.zeros(1, dtype=torch.int64, device=dev)))
         self.o_deq = [torch.empty(w.numel(), dtype=bf, device=dev) for w in self.w_opq]
         # result buffers of the two fits (levels, error log): no allocation inside the timed region
-        self.fit_out = [(torch.empty(16, dtype=torch.float32, device=dev),
-                         torch.zeros(1, dtype=torch.float64, device=dev)) for _ in range(2)]
+        self.fit_out = [(self.cb0.clone(), torch.zeros(1, dtype=torch.float64, device=dev)) for _ in range(2)]
         self.only = None
         self.graphs = {}
 
-    # ---- the six components (binding calls only)
+    # ---- the six components (binding calls only).  The two fits continue from their own previous
+    # result (the levels buffer is both input and output), so that successive steps are successive
+    # Lloyd iterations of one fit, as in a 30-iteration run, rather than the first iteration over
+    # and over.
     def em_mse(self):
         b = self.b
-        b.bof4_fit_codebook(self.w_fit, I, b.NORM_SIGNED, b.METRIC_MSE, self.cb0, self.mask, 1,
+        b.bof4_fit_codebook(self.w_fit, I, b.NORM_SIGNED, b.METRIC_MSE, self.fit_out[0][0], self.mask, 1,
                             workspace=self.ws_em, sync=False, out=self.fit_out[0])
 
     def em_mae(self):
         b = self.b
-        b.bof4_fit_codebook(self.w_fit, I, b.NORM_SIGNED, b.METRIC_MAE, self.cb0, self.mask, 1,
+        b.bof4_fit_codebook(self.w_fit, I, b.NORM_SIGNED, b.METRIC_MAE, self.fit_out[1][0], self.mask, 1,
                             workspace=self.ws_em, sync=False, out=self.fit_out[1])
 
     def quant(self):

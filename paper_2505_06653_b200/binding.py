@@ -230,7 +230,9 @@ def bof4_fit_codebook(weights, block_size: int, norm: int, metric: int, levels, 
         cb, log = _dev(out[0], "out[0]"), _dev(out[1], "out[1]")
         if cb.dtype != torch.float32 or cb.numel() != LEVELS or log.dtype != torch.float64 or log.numel() < iters:
             raise ValueError("out must be (float32[16], float64[>= iters])")
-        cb.copy_(_codebook(levels, dev))
+        src = _codebook(levels, dev)
+        if src.data_ptr() != cb.data_ptr():  # levels may be the output buffer itself: continue in place
+            cb.copy_(src)
     else:
         cb = _codebook(levels, dev).clone()
         log = torch.zeros(max(iters, 1), dtype=torch.float64, device=dev)

@@ -12,6 +12,7 @@
 // bit-reproducible.  The COUNT variant also keeps the member count of every region.
 #include "common.cuh"
 #include "em_common.cuh"
+#include "lane32.cuh"
 #include "layout.h"
 
 namespace bof4 {
@@ -357,6 +358,257 @@ em_mse_kernel(const EmTensors T, const float* levels, double* partials, const Ms
     }
 }
 
+// ---------------------------------------------------------------- MSE pass, bf16 weights
+//
+// The same pass with the 64-byte-per-lane front end (lane32.cuh): 32 weights per lane, packed
+// min/max, the reciprocal FAST path (x~ = w RN(1/m); the region it falls into is the region of
+// the true quotient whenever the block constant's significand is not marked "near", so member
+// counts stay exact, and the sums only see the last-place difference of x~).  Rows outside the
+// common case go to an out-of-line version that divides exactly.
+
+template <bool COUNT>
+struct EmGeo32 {
+    static constexpr int threads = 1024;
+    static constexpr int row = threads * kLW;               // weights per CTA row
+    static constexpr uint32_t acc_row_bytes = threads * 8;  // one level's float2 columns
+    static constexpr int lut_rep = COUNT ? 16 : 32;
+    static constexpr int flush_rows = 32;                   // 1024 weights per thread between folds
+    static constexpr size_t smem =
+        (size_t)lut_bytes(lut_rep) + (size_t)kLevels * threads * (COUNT ? 10 : 8);
+};
+
+// s1[c] += mm x, s0[c] += mm in the thread's private column of level c (byte offset `off`).
+template <bool COUNT>
+__device__ __forceinline__ void em_add(unsigned char* s_acc, unsigned char* s_cnt, uint32_t off, float mm, float x)
+{
+    float2* pa = reinterpret_cast<float2*>(s_acc + off);
+    float2 a = *pa;
+    a.x = fmaf(mm, x, a.x);
+    a.y += mm;
+    *pa = a;
+    if (COUNT) *reinterpret_cast<uint16_t*>(s_cnt + (off >> 2)) += 1;
+}
+
+// One row of a lane the slow way (true quotients, binary search against the true thresholds).
+// Out of line.
+template <bool COUNT>
+__device__ __noinline__ float em_row32_slow(Raw32 raw, float m, float mm, bool unit, const float* s_xi,
+                                            unsigned char* s_acc, unsigned char* s_cnt, uint32_t tid_off,
+                                            uint32_t row_bytes)
+{
+    uint32_t u[16];
+    words_of(raw, u);
+    const bool recip = div_safe(fabsf(m));
+    const float r = recip ? __frcp_rn(m) : 0.0f;
+    float2 sq = make_float2(0.0f, 0.0f);
+#pragma unroll 4
+    for (int k = 0; k < 16; ++k) {
+        const float2 v = make_float2(bf_lo(u[k]), bf_hi(u[k]));
+        const float2 x = exact_quotient2(v, m, r, recip);
+        sq = unit ? __ffma2_rn(x, x, sq) : __ffma2_rn(v, v, sq);
+        em_add<COUNT>(s_acc, s_cnt, (uint32_t)region_of(x.x, s_xi) * row_bytes + tid_off, mm, x.x);
+        em_add<COUNT>(s_acc, s_cnt, (uint32_t)region_of(x.y, s_xi) * row_bytes + tid_off, mm, x.y);
+    }
+    return sq.x + sq.y;
+}
+
+template <int I, bool SIGNED, bool COUNT>
+__global__ void __launch_bounds__(EmGeo32<COUNT>::threads, 1)
+em_mse32_kernel(const EmTensors T, const float* levels, double* partials, const MseTail tail)
+{
+    using G = EmGeo32<COUNT>;
+    constexpr int NT = G::threads, NW = NT / 32, NSEG = NW / kLevels;
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    unsigned char* s_lut = s_raw;
+    unsigned char* s_acc = s_raw + lut_bytes(G::lut_rep);               // float2 [16][NT]
+    unsigned char* s_cnt = s_acc + (size_t)kLevels * G::acc_row_bytes;  // uint16 [16][NT] (COUNT)
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ FastInfo s_info;
+    __shared__ WideScratch s_wide;
+    __shared__ double s_part[NSEG][3][kLevels];
+    __shared__ double s_tot[3 * kLevels];  // s1, s0, count (as uint64 bits)
+    __shared__ double s_w2[NW];
+    __shared__ const void* s_ptr[kEmMaxTensors];
+    __shared__ int64_t s_n[kEmMaxTensors], s_row_end[kEmMaxTensors];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid < 3 * kLevels) s_tot[tid] = 0.0;  // all-zero bits are also uint64 zero
+    if (tid < T.count) {
+        s_ptr[tid] = T.ptr[tid];
+        s_n[tid] = T.n[tid];
+        s_row_end[tid] = T.row_end[tid];
+    }
+#pragma unroll
+    for (int l = 0; l < kLevels; ++l) {
+        *reinterpret_cast<float2*>(s_acc + l * G::acc_row_bytes + tid * 8) = make_float2(0.0f, 0.0f);
+        if (COUNT) *reinterpret_cast<uint16_t*>(s_cnt + l * (G::acc_row_bytes / 4) + tid * 2) = 0;
+    }
+    const bool lut_ok = build_tables32<G::lut_rep>(levels, s_xi, s_lv, s_lut, &s_info,
+                                                   [](int base) { return (uint32_t)base * G::acc_row_bytes; });
+    const bool fast_ok = lut_ok && !s_info.tiny;
+
+    const int64_t total_rows = T.row_end[T.count - 1];
+    const bool unit = T.unit != 0;
+    const uint32_t lut_base = lut_lane_base<G::lut_rep>(s_lut, lane), tid_off = tid * 8;
+    double w2sum = 0.0;
+    int t_cur = 0;
+    int since_flush = 0;
+
+    // Folds the private fp32 columns into the fp64 CTA totals (fixed order) and clears them.
+    auto flush = [&]() {
+        __syncthreads();
+        {
+            const int l = warp & (kLevels - 1), seg = warp >> 4;
+            double a1 = 0.0, a0 = 0.0;
+            unsigned long long ac = 0;
+            constexpr int PER = NT / NSEG / 32;  // columns per lane
+#pragma unroll 4
+            for (int k = 0; k < PER; ++k) {
+                const int col = seg * (NT / NSEG) + k * 32 + lane;
+                float2* pa = reinterpret_cast<float2*>(s_acc + l * G::acc_row_bytes + col * 8);
+                const float2 a = *pa;
+                a1 += (double)a.x;
+                a0 += (double)a.y;
+                *pa = make_float2(0.0f, 0.0f);
+                if (COUNT) {
+                    uint16_t* pc = reinterpret_cast<uint16_t*>(s_cnt + l * (G::acc_row_bytes / 4) + col * 2);
+                    ac += *pc;
+                    *pc = 0;
+                }
+            }
+#pragma unroll
+            for (int off = 16; off; off >>= 1) {
+                a1 += __shfl_xor_sync(kFull, a1, off);
+                a0 += __shfl_xor_sync(kFull, a0, off);
+                if (COUNT) ac += __shfl_xor_sync(kFull, ac, off);
+            }
+            if (lane == 0) {
+                s_part[seg][0][l] = a1;
+                s_part[seg][1][l] = a0;
+                s_part[seg][2][l] = __longlong_as_double((long long)ac);
+            }
+        }
+        __syncthreads();
+        if (tid < 3 * kLevels) {
+            const int q = tid / kLevels, l = tid % kLevels;
+            if (q < 2) {
+                double a = s_tot[tid];
+                for (int sg = 0; sg < NSEG; ++sg) a += s_part[sg][q][l];
+                s_tot[tid] = a;
+            } else {
+                unsigned long long a = (unsigned long long)__double_as_longlong(s_tot[tid]);
+                for (int sg = 0; sg < NSEG; ++sg)
+                    a += (unsigned long long)__double_as_longlong(s_part[sg][2][l]);
+                s_tot[tid] = __longlong_as_double((long long)a);
+            }
+        }
+        __syncthreads();
+    };
+
+    // Loads the lane's 32 weights of global row g (zeros beyond the end of the row's tensor or of
+    // the data); rows are fetched in ascending order.
+    auto fetch = [&](int64_t g, bool& ok) -> Raw32 {
+        ok = false;
+        if (g < total_rows) {
+            while (g >= s_row_end[t_cur]) ++t_cur;
+            const int64_t r = g - (t_cur ? s_row_end[t_cur - 1] : 0);
+            const int64_t idx = (r * NT + tid) * kLW;
+            ok = idx < s_n[t_cur];
+            if (ok) return load_raw32(s_ptr[t_cur], idx);
+        }
+        return zero_raw32();
+    };
+
+    auto row = [&](const Raw32& raw, bool ok) {
+        uint32_t u[16];
+        words_of(raw, u);
+        float mx, mn, g;
+        lane_minmax32(u, mx, mn);
+        const float m = block_constant32<I, SIGNED>(u, mx, mn, g, &s_wide);
+        const float mm = unit ? 1.0f : m * m;
+        float sq;
+        if (row_is_fast(g, m, ok, fast_ok, &s_info)) {
+            const float r = __frcp_rn(m);
+            const float2 rr = make_float2(r, r);
+            float2 sq2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const float2 v = make_float2(bf_lo(u[k]), bf_hi(u[k]));
+                const float2 x = __fmul2_rn(v, rr);
+                const float2 key = lut_key2(x);
+                sq2 = unit ? __ffma2_rn(x, x, sq2) : __ffma2_rn(v, v, sq2);
+                const uint2 e0 = lut_probe<G::lut_rep>(key.x, lut_base), e1 = lut_probe<G::lut_rep>(key.y, lut_base);
+                em_add<COUNT>(s_acc, s_cnt, e0.y + ((x.x >= __uint_as_float(e0.x)) ? G::acc_row_bytes : 0u) + tid_off, mm, x.x);
+                em_add<COUNT>(s_acc, s_cnt, e1.y + ((x.y >= __uint_as_float(e1.x)) ? G::acc_row_bytes : 0u) + tid_off, mm, x.y);
+            }
+            sq = sq2.x + sq2.y;
+        } else {
+            sq = ok ? em_row32_slow<COUNT>(raw, m, mm, unit, s_xi, s_acc, s_cnt, tid_off, G::acc_row_bytes) : 0.0f;
+        }
+        w2sum += (double)sq;
+        if (++since_flush == G::flush_rows) {
+            flush();
+            since_flush = 0;
+        }
+    };
+
+    bool ok_a, ok_b;
+    int64_t g = blockIdx.x;
+    const int64_t GS = gridDim.x;
+    Raw32 a = fetch(g, ok_a), b;
+    if (g < total_rows) {
+        while (true) {
+            b = fetch(g + GS, ok_b);
+            row(a, ok_a);
+            g += GS;
+            if (g >= total_rows) break;
+            a = fetch(g + GS, ok_a);
+            row(b, ok_b);
+            g += GS;
+            if (g >= total_rows) break;
+        }
+    }
+    flush();
+
+    // sum of squares: fixed-order fold over the CTA
+#pragma unroll
+    for (int off = 16; off; off >>= 1) w2sum += __shfl_xor_sync(kFull, w2sum, off);
+    if (lane == 0) s_w2[warp] = w2sum;
+    __syncthreads();
+    double* rec = partials + (size_t)blockIdx.x * kEmRecordDoubles;
+    if (tid < kLevels) {
+        unsigned long long* rc = reinterpret_cast<unsigned long long*>(rec);
+        const unsigned long long cnt = (unsigned long long)__double_as_longlong(s_tot[2 * kLevels + tid]);
+        if (T.accumulate) {
+            rec[kRecS1 + tid] += s_tot[tid];
+            rec[kRecS0 + tid] += s_tot[kLevels + tid];
+            rc[kRecCnt + tid] += cnt;
+        } else {
+            rec[kRecS1 + tid] = s_tot[tid];
+            rec[kRecS0 + tid] = s_tot[kLevels + tid];
+            rc[kRecCnt + tid] = cnt;
+        }
+    }
+    if (tid == 0) {
+        double e = 0.0;
+        for (int k = 0; k < NW; ++k) e += s_w2[k];
+        rec[kRecW2] = T.accumulate ? rec[kRecW2] + e : e;
+    }
+    if (tail.enabled) {
+        __shared__ int s_last;
+        __shared__ double s_q[kRecW2 + 1], s_corr[kLevels];
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = (atomicAdd(tail.ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            mse_combine(partials, tail, s_q, s_corr, reinterpret_cast<unsigned long long*>(s_acc));
+            if (tid == 0) *tail.ticket = 0u;
+        }
+    }
+}
+
 }  // namespace bof4
 
 // ================================================================= launchers (C ABI)
@@ -423,10 +675,17 @@ int launch_mse_chunk(const EmTensors& T, const float* d_codebook, double* partia
                      cudaStream_t st)
 {
     tail.enabled = T.last;
-    using G = EmGeo<COUNT>;
-    constexpr auto kern = em_mse_kernel<DT, I, SG, COUNT>;
-    if (const int rc = ensure_dynamic_smem<kern>((int)G::smem)) return rc;
-    kern<<<kEmGrid, G::threads, G::smem, st>>>(T, d_codebook, partials, tail);
+    if constexpr (DT::code == BOF4_BF16) {
+        using G = EmGeo32<COUNT>;
+        constexpr auto kern = em_mse32_kernel<I, SG, COUNT>;
+        if (const int rc = ensure_dynamic_smem<kern>((int)G::smem)) return rc;
+        kern<<<kEmGrid, G::threads, G::smem, st>>>(T, d_codebook, partials, tail);
+    } else {
+        using G = EmGeo<COUNT>;
+        constexpr auto kern = em_mse_kernel<DT, I, SG, COUNT>;
+        if (const int rc = ensure_dynamic_smem<kern>((int)G::smem)) return rc;
+        kern<<<kEmGrid, G::threads, G::smem, st>>>(T, d_codebook, partials, tail);
+    }
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }
@@ -459,7 +718,8 @@ int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials,
 #undef BOF4_EM_GO
     };
     int calls = 0;
-    const int rc = for_each_tensor_chunk(a, EmGeo<COUNT>::row, fire, &calls);
+    const int rc = for_each_tensor_chunk(a, a.w_dtype == BOF4_BF16 ? EmGeo32<COUNT>::row : EmGeo<COUNT>::row, fire,
+                                         &calls);
     if (rc) return rc;
     if (calls == 0) {
         BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));

@@ -6,21 +6,28 @@
 // the weights per lane halve everything that is paid per lane and row (block reduction,
 // reciprocal, row bookkeeping, stores), which is what bounds these kernels.
 //
-// Three ways to the region of a weight (Sec. 2.1 Eq. 2 + Sec. 3.2), chosen per warp row:
+// Two ways to the region of a weight (Sec. 2.1 Eq. 2 + Sec. 3.2), chosen per warp row:
 //   FAST   x~ = RN(w * RN(1/m)), one packed multiplication per two weights, then the one-probe
-//          table search.  x~ differs from the true quotient RN(w/m) by at most a few units in
-//          the last place, which only matters if a decision threshold lies that close to a
-//          quotient the data can take.  Both operands have 8-bit significands, so for a given
-//          significand of m the possible quotients are a small set that can be enumerated: at
-//          table-build time every (threshold, significand of m) pair is checked, and a block
-//          whose constant has a significand marked "near" does not take this path
-//          (near_mask).  Thresholds of magnitude below 2^-90 (zero included) switch the path off for the
-//          whole launch, because then the rounding of subnormal quotients would matter.
-//   EXACT  the reciprocal sequence of normalise16 (the IEEE quotient for every normal result),
-//          its guard for tiny quotients, and the table search.
-//   SLOW   IEEE division and binary search: rows with a zero, non-finite or extreme block
-//          constant, and codebooks the table cannot serve.
-// All three give the same codes: the code of RN(w/m) against the fp32 thresholds.
+//          table search against thresholds LOWERED by three floating-point steps (xi' = the third
+//          fp32 number below xi).  With q = w/m: x~ lies within 2.01 * 2^-24 (relative) of q, and
+//          RN(q) >= xi  <=>  q >= xi up to rounding in the last place, so
+//              q >= xi                   =>  x~ >= xi'      (x~ > xi (1 - 2.01 * 2^-24) > xi'),
+//              q <  xi - 9 * 2^-24 |xi|  =>  x~ <  xi'  and  RN(q) < xi,
+//          i.e. the comparison x~ >= xi' decides exactly like RN(w/m) >= xi unless q falls into
+//          the narrow window just below xi (and a quotient less than half a step below xi rounds
+//          to xi and has x~ >= xi' as well).  Both operands have 8-bit significands, so for a
+//          given significand of m the quotients are a small set: at table-build time every
+//          (threshold, significand of m) pair is checked, and a block whose constant has a
+//          significand with a quotient in some window ("near") takes the other way.  A quotient
+//          that equals a threshold, or whose fp32 rounding does (codebooks with dyadic or other
+//          simple rational levels), is decided correctly here.
+//          Thresholds of magnitude below 2^-90 (zero included) switch the path off for the whole
+//          launch: the rounding of subnormal quotients would matter.
+//   SLOW   the true quotient RN(w/m) (reciprocal sequence with its guard where it is proven,
+//          IEEE division elsewhere) against the true thresholds by binary search: "near" rows,
+//          rows with a zero, non-finite or extreme block constant, partial rows, and codebooks
+//          the table cannot serve.
+// Both give the same codes: the code of RN(w/m) against the fp32 thresholds.
 #pragma once
 
 #include "common.cuh"
@@ -164,11 +171,17 @@ __device__ __forceinline__ float block_constant32(const uint32_t (&u)[16], float
 // ---------------------------------------------------------------- which significands of m are "near"
 //
 // bf16 values are a * 2^e with an integer a < 256, so for a block constant with significand
-// b (128..255) every quotient is (a / b) * 2^j.  A threshold xi is "near" for b when some a in
-// 128..255 (any j) has | a / b - |xi| 2^-j | <= 2^-20 |xi| 2^-j: with X the 24-bit significand
-// of |xi|, a 2^s = X b up to that tolerance, s being the shift that brings X b into [128, 256).
-// x~ and RN(w/m) are both within 2^-23 (relative) of the true quotient, so outside this set no
-// threshold separates them.  near_mask: bit (b - 128) of a 128-bit mask, four words.
+// b (128..255) every quotient has magnitude (a / b) * 2^j.  With X the 24-bit significand of
+// |xi|, P = X b = a_real * 2^s for the s that brings a_real into [128, 256); one unit of P is
+// 1 / b of a unit in the last place of xi.  The quotient with numerator a = floor(a_real)
+// (xi > 0: slightly smaller magnitude) or ceil(a_real) (xi < 0: slightly larger) lies
+// dist = frac(P) resp. 2^s - frac(P) units of P below xi.  FAST decides like the true quotient
+//   * for dist < b / 4: the quotient is less than a quarter step below xi, RN(q) = xi and
+//     x~ > xi' (this is the case of codebooks with rational levels, whose thresholds are fp32
+//     roundings of quotients the data takes);
+//   * for dist > 9 * 2^-24 P: the quotient is more than 9 * 2^-24 |xi| below xi.
+// In between the significand is marked (upper bound rounded up to 16 * 2^-24 P).
+// near_mask: bit (b - 128) of a 128-bit mask.
 struct FastInfo {
     uint32_t near_mask[4];
     int tiny;  // some threshold has magnitude below 2^-90 (zero included): FAST is off
@@ -177,18 +190,28 @@ struct FastInfo {
 // One bin of the near-significand test: threshold index j, significand b.
 __device__ __forceinline__ void mark_if_near(const float* s_xi, int j, int b, FastInfo* s_info)
 {
-    const uint32_t xb = __float_as_uint(s_xi[j]) & 0x7fffffffu;
+    const uint32_t bits = __float_as_uint(s_xi[j]), xb = bits & 0x7fffffffu;
     if (xb >= 0x7f800000u || xb < 0x12800000u) return;  // not finite, or below 2^-90 (see tiny)
     const uint32_t X = (xb & 0x7fffffu) | 0x800000u;       // 24-bit significand
     const uint32_t P = X * (uint32_t)b;                    // < 2^32, >= 2^30
     const int s = (P >> 31) ? 24 : 23;                     // P >> s in [128, 256)
-    const uint32_t frac = P & ((1u << s) - 1u), tol = 1u << (s - 12);   // 2^-20 relative, rounded up
-    if (frac <= tol || frac >= (1u << s) - tol) atomicOr(&s_info->near_mask[(b - 128) >> 5], 1u << ((b - 128) & 31));
+    const uint32_t frac = P & ((1u << s) - 1u);
+    const uint32_t dist = (bits >> 31) ? ((1u << s) - frac) & ((1u << s) - 1u) : frac;  // distance into the window side
+    const bool near = 4u * dist >= (uint32_t)b && dist <= (P >> 20);
+    if (near) atomicOr(&s_info->near_mask[(b - 128) >> 5], 1u << ((b - 128) & 31));
 }
 
-// Everything a quantising kernel derives from the codebook, in two barriers: thresholds and
-// levels (s_xi, s_lv), the one-probe region table (s_lut, [bin][lane] replicated REP times;
-// payload(base) beside every threshold) and the FAST-path information.  Every thread derives
+// The third fp32 number below x (finite, |x| >= 2^-90: no zero crossing).
+__device__ __forceinline__ float three_steps_down(float x)
+{
+    const uint32_t u = __float_as_uint(x);
+    return __uint_as_float((u >> 31) ? u + 3u : u - 3u);
+}
+
+// Everything a quantising kernel derives from the codebook, in two barriers: the true thresholds
+// and the levels (s_xi, s_lv), the one-probe region table of the FAST path over the LOWERED
+// thresholds (s_lut, [bin][lane] replicated REP times; payload(base) beside every threshold) and
+// the FAST-path information.  Every thread derives
 // the thresholds and their table bins itself from the 16 levels, so that the table entries, the
 // "two thresholds in one bin" test and the "tiny threshold" test need no exchange.  Returns
 // whether the table can serve the codebook.  Call with all threads of the CTA (>= 257).
@@ -207,24 +230,27 @@ __device__ __forceinline__ bool build_tables32(const float* __restrict__ levels,
         lv[4 * q + 2] = t.z;
         lv[4 * q + 3] = t.w;
     }
+    float lo[kLevels];  // lowered thresholds (table side)
     int bin[kLevels - 1];
     bool multi = false, tiny = false;
 #pragma unroll
     for (int j = 0; j < kLevels - 1; ++j) {
         xi[j] = __fmul_rn(__fadd_rn(lv[j], lv[j + 1]), 0.5f);
-        const int bj = (int)(__float_as_uint(lut_key(xi[j])) - kLutMagicBits);
+        const bool usable = fabsf(xi[j]) >= 0x1p-90f && fabsf(xi[j]) < __int_as_float(0x7f800000);
+        tiny = tiny || !(fabsf(xi[j]) >= 0x1p-90f);
+        lo[j] = usable ? three_steps_down(xi[j]) : xi[j];
+        const int bj = (int)(__float_as_uint(lut_key(lo[j])) - kLutMagicBits);
         bin[j] = bj < 0 ? 0 : (bj > kLutBins - 1 ? kLutBins - 1 : bj);
-        tiny = tiny || fabsf(xi[j]) < 0x1p-90f;
         if (j > 0) multi = multi || bin[j] == bin[j - 1];   // ascending thresholds: equal bins are adjacent
     }
-    xi[kLevels - 1] = __int_as_float(0x7f800000);
+    xi[kLevels - 1] = lo[kLevels - 1] = __int_as_float(0x7f800000);
     if (tid < kLutBins) {
         int base = 0;
 #pragma unroll
         for (int j = 0; j < kLevels - 1; ++j) base += (bin[j] < tid) ? 1 : 0;
-        float thr = xi[kLevels - 1];
+        float thr = lo[kLevels - 1];
 #pragma unroll
-        for (int j = kLevels - 2; j >= 0; --j) thr = (base == j) ? xi[j] : thr;
+        for (int j = kLevels - 2; j >= 0; --j) thr = (base == j) ? lo[j] : thr;
         s_ent[tid] = make_uint2(__float_as_uint(thr), payload(base));
     }
     if (tid < kLevels) {
@@ -271,26 +297,18 @@ __device__ __forceinline__ uint32_t horner_code(uint32_t wd, float x, uint2 entr
     return wd;
 }
 
-template <bool REFINE>
-__device__ __forceinline__ void encode32_lut(const uint32_t (&u)[16], float m, uint32_t lut_base, uint32_t (&cw)[4])
+// FAST path: m != 0, every |w| <= |m|, so every x~ is a finite number in [-1, 1].
+__device__ __forceinline__ void encode32_fast(const uint32_t (&u)[16], float m, uint32_t lut_base, uint32_t (&cw)[4])
 {
-    const float r = __frcp_rn(m);  // m != 0: the caller passes 1 for lanes without data
-    const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
+    const float r = __frcp_rn(m);
+    const float2 rr = make_float2(r, r);
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
         uint32_t wd = 0u;
 #pragma unroll
         for (int j = 3; j >= 0; --j) {
             const uint32_t uu = u[4 * h + j];
-            const float2 v = make_float2(bf_lo(uu), bf_hi(uu));
-            float2 x = __fmul2_rn(v, rr);
-            if (REFINE) {
-                const float2 e = __ffma2_rn(x, nm, v);
-                x = __ffma2_rn(e, rr, x);
-                // quotients below 2^-100: one rounding of the subnormal result
-                if (fabsf(x.x) < 0x1p-100f && v.x != 0.0f) x.x = __fdiv_rn(v.x, m);
-                if (fabsf(x.y) < 0x1p-100f && v.y != 0.0f) x.y = __fdiv_rn(v.y, m);
-            }
+            const float2 x = __fmul2_rn(make_float2(bf_lo(uu), bf_hi(uu)), rr);
             const float2 key = lut_key2(x);
             const uint2 e0 = lut_probe(key.x, lut_base), e1 = lut_probe(key.y, lut_base);
             wd = horner_code(wd, x.x, e0);
@@ -300,12 +318,30 @@ __device__ __forceinline__ void encode32_lut(const uint32_t (&u)[16], float m, u
     }
 }
 
-// IEEE division and binary search; any input.  Kept out of line (the words travel by value) so
-// that the rare path costs the common ones neither registers nor code size.
-__device__ __noinline__ uint4 encode32_slow_words(uint4 q0, uint4 q1, uint4 q2, uint4 q3, float m, const float* s_xi)
+// The quotients RN(v / m) of two weights for the SLOW path: the reciprocal sequence of
+// normalise16 with its guard where it is proven (recip: |m| in [2^-60, 2^60], r = RN(1/m)),
+// IEEE division otherwise (x = 0 when m = 0).
+__device__ __forceinline__ float2 exact_quotient2(float2 v, float m, float r, bool recip)
+{
+    if (!recip) return make_float2(normalise(v.x, m), normalise(v.y, m));
+    const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
+    float2 x = __fmul2_rn(v, rr);
+    const float2 e = __ffma2_rn(x, nm, v);
+    x = __ffma2_rn(e, rr, x);
+    if (fabsf(x.x) < 0x1p-100f && v.x != 0.0f) x.x = __fdiv_rn(v.x, m);  // subnormal results: one rounding
+    if (fabsf(x.y) < 0x1p-100f && v.y != 0.0f) x.y = __fdiv_rn(v.y, m);
+    return x;
+}
+
+// SLOW path: true quotients against the true thresholds by binary search; any input.  Kept out
+// of line (the words travel by value) so that it costs the common path neither registers nor
+// code size.
+static __device__ __noinline__ uint4 encode32_slow_words(uint4 q0, uint4 q1, uint4 q2, uint4 q3, float m, const float* s_xi)
 {
     const uint32_t u[16] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w,
                             q2.x, q2.y, q2.z, q2.w, q3.x, q3.y, q3.z, q3.w};
+    const bool recip = div_safe(fabsf(m));
+    const float r = recip ? __frcp_rn(m) : 0.0f;
     uint32_t cw[4];
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
@@ -313,8 +349,9 @@ __device__ __noinline__ uint4 encode32_slow_words(uint4 q0, uint4 q1, uint4 q2, 
 #pragma unroll
         for (int j = 3; j >= 0; --j) {
             const uint32_t uu = u[4 * h + j];
-            wd = wd * 16u + (uint32_t)region_of(normalise(bf_lo(uu), m), s_xi);
-            wd = wd * 16u + (uint32_t)region_of(normalise(bf_hi(uu), m), s_xi);
+            const float2 x = exact_quotient2(make_float2(bf_lo(uu), bf_hi(uu)), m, r, recip);
+            wd = wd * 16u + (uint32_t)region_of(x.x, s_xi);
+            wd = wd * 16u + (uint32_t)region_of(x.y, s_xi);
         }
         cw[h] = wd;
     }
@@ -331,17 +368,13 @@ __device__ __forceinline__ void encode32_slow(const uint32_t (&u)[16], float m, 
     cw[3] = c.w;
 }
 
-// Which way a warp row takes (warp-uniform).  g: the lane's block maximum (or NaN); ok: the lane
-// holds data (a lane without data must hold zeros and is encoded with m = 1); lut_ok: the
-// codebook fits the one-probe table.  An all-zero block sends its row the slow way.
-enum RowPath { kPathFast = 0, kPathExact = 1, kPathSlow = 2 };
-
-__device__ __forceinline__ int row_path(float g, float m, bool ok, bool lut_ok, const FastInfo* s_info)
+// Warp-uniform: the row takes the FAST path.  g: the lane's block maximum (or NaN), m its block
+// constant; ok: the lane holds data; fast_ok: the table serves the codebook and no threshold is
+// tiny.  A zero, extreme or non-finite block constant, a "near" significand or a lane without
+// data send the row the slow way.
+__device__ __forceinline__ bool row_is_fast(float g, float m, bool ok, bool fast_ok, const FastInfo* s_info)
 {
-    const bool safe = div_safe(g) || !ok;
-    if (!lut_ok || !__all_sync(kFull, safe)) return kPathSlow;
-    if (s_info->tiny) return kPathExact;
-    return __any_sync(kFull, ok && near_significand(m, s_info)) ? kPathExact : kPathFast;
+    return fast_ok && __all_sync(kFull, ok && div_safe(g) && !near_significand(m, s_info));
 }
 
 // Rows of `row` consecutive weights over a tensor of n weights (n a multiple of 32); the calling

@@ -161,18 +161,14 @@ struct QuantShared32 {
 // Block constant, codes and stores for the lane's 32 (cleaned) weights of one row.
 template <int I, bool SIGNED, class ST>
 __device__ __forceinline__ void quantize_row32(const uint32_t (&u)[16], float mx, float mn, int64_t idx, bool ok,
-                                               bool lut_ok, uint32_t lut_base, QuantShared32* S,
+                                               bool fast_ok, uint32_t lut_base, QuantShared32* S,
                                                uint8_t* __restrict__ codes, void* __restrict__ scales)
 {
     float g;
     const float m = block_constant32<I, SIGNED>(u, mx, mn, g, &S->wide);
-    const int path = row_path(g, m, ok, lut_ok, &S->info);
-    const float md = ok ? m : 1.0f;  // divisor of the table paths: never zero
     uint32_t cw[4];
-    if (path == kPathFast)
-        encode32_lut<false>(u, md, lut_base, cw);
-    else if (path == kPathExact)
-        encode32_lut<true>(u, md, lut_base, cw);
+    if (row_is_fast(g, m, ok, fast_ok, &S->info))
+        encode32_fast(u, m, lut_base, cw);
     else
         encode32_slow(u, m, S->xi, cw);
     if (ok) {
@@ -186,7 +182,7 @@ __device__ __forceinline__ void quantize_row32(const uint32_t (&u)[16], float mx
 // a tensor), kept out of line so that it costs the streaming loop no registers.  Blocks within
 // a warp only (the wide-block kernel below calls quantize_row32 itself).
 template <int I, bool SIGNED, class ST>
-__device__ __noinline__ void quantize_row32_generic(Raw32 raw, int64_t idx, bool ok, bool lut_ok, uint32_t lut_base,
+__device__ __noinline__ void quantize_row32_generic(Raw32 raw, int64_t idx, bool ok, bool fast_ok, uint32_t lut_base,
                                                     QuantShared32* S, uint8_t* __restrict__ codes,
                                                     void* __restrict__ scales)
 {
@@ -194,7 +190,7 @@ __device__ __noinline__ void quantize_row32_generic(Raw32 raw, int64_t idx, bool
     words_of(raw, u);
     float mx, mn;
     lane_minmax32(u, mx, mn);
-    quantize_row32<I, SIGNED, ST>(u, mx, mn, idx, ok, lut_ok, lut_base, S, codes, scales);
+    quantize_row32<I, SIGNED, ST>(u, mx, mn, idx, ok, fast_ok, lut_base, S, codes, scales);
 }
 
 template <int I, bool SIGNED, class ST>
@@ -210,8 +206,8 @@ quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict
     if (r >= map.rows) return;
     auto fetch = [&](int rr) { return map.ok(rr) ? load_raw32(w, map.idx(rr)) : zero_raw32(); };
     const Raw32 first = fetch(r);  // on its way while the tables are built
-    QuantTables T{S.xi, s_lut, false};
-    T.lut_ok = build_tables32(levels, S.xi, S.lv, s_lut, &S.info, [](int base) { return (uint32_t)base; });
+    const bool lut_ok = build_tables32(levels, S.xi, S.lv, s_lut, &S.info, [](int base) { return (uint32_t)base; });
+    const bool fast_ok = lut_ok && !S.info.tiny;
     const uint32_t lut_base = lut_lane_base(s_lut, threadIdx.x & 31);
     if constexpr (Geo32<I>::WPB > 1) {
         // blocks of several warps: every thread of the CTA takes every step (barriers inside)
@@ -222,13 +218,12 @@ quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict
             words_of(a, u);
             float mx, mn;
             lane_minmax32(u, mx, mn);
-            quantize_row32<I, SIGNED, ST>(u, mx, mn, map.idx(r), map.ok(r), T.lut_ok, lut_base, &S, codes, scales);
+            quantize_row32<I, SIGNED, ST>(u, mx, mn, map.idx(r), map.ok(r), fast_ok, lut_base, &S, codes, scales);
             a = next;
         }
     } else {
         // Whole rows: unconditional loads into two buffers used in turn; a row all of whose block
         // constants are ordinary is encoded here, any other goes to the out-of-line version.
-        const bool fast_ok = T.lut_ok && !S.info.tiny;
         auto row = [&](const Raw32& raw, int rr) {
             uint32_t u[16];
             words_of(raw, u);
@@ -236,13 +231,13 @@ quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict
             lane_minmax32(u, mx, mn);
             const float m = block_constant32<I, SIGNED>(u, mx, mn, g, nullptr);
             const int64_t idx = map.idx(rr);
-            if (fast_ok && __all_sync(kFull, div_safe(g) && !near_significand(m, &S.info))) {
+            if (row_is_fast(g, m, true, fast_ok, &S.info)) {
                 uint32_t cw[4];
-                encode32_lut<false>(u, m, lut_base, cw);
+                encode32_fast(u, m, lut_base, cw);
                 st_stream128(codes + idx / 2, cw[0], cw[1], cw[2], cw[3]);
                 if ((idx & (I - 1)) == 0) store_scale<ST>(scales, idx / I, m);
             } else {
-                quantize_row32_generic<I, SIGNED, ST>(raw, idx, true, T.lut_ok, lut_base, &S, codes, scales);
+                quantize_row32_generic<I, SIGNED, ST>(raw, idx, true, fast_ok, lut_base, &S, codes, scales);
             }
         };
         const int full = map.rows_full;
@@ -264,7 +259,7 @@ quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict
         // the partial last row of the tensor, by the CTA whose turn it is
         if (map.rows > full && full % G == (int)blockIdx.x)
             quantize_row32_generic<I, SIGNED, ST>(full == (int)blockIdx.x ? first : fetch(full), map.idx(full),
-                                                  map.ok(full), T.lut_ok, lut_base, &S, codes, scales);
+                                                  map.ok(full), fast_ok, lut_base, &S, codes, scales);
     }
 }
 
