@@ -22,6 +22,7 @@
 // equal to the exact real-number sums that define the median.
 #include "common.cuh"
 #include "em_common.cuh"
+#include "lane32.cuh"
 #include "layout.h"
 
 namespace bof4 {
@@ -39,6 +40,7 @@ struct MaeState {
     uint32_t base[kLevels];              // key of the region's lower edge
     uint32_t prefix[kLevels];            // digits chosen so far
     int top[kLevels];                    // key bits still unresolved (0: done)
+    uint32_t limit[kLevels];             // largest relative key that can still take part (bound of the range)
     uint32_t cand_count[kLevels];        // samples offered to the candidate list of level l
     uint32_t active;                     // bit l: level l takes part in the selection
     uint32_t max_bits;                   // bits of the largest |w| of the data
@@ -143,9 +145,10 @@ mae_init_kernel(const float* __restrict__ levels, uint32_t skip_mask, MaeWs W)
         W.state->total[l] = 0ull;
         W.state->count[l] = 0ull;
         W.state->cand_count[l] = 0u;
+        W.state->limit[l] = 0xffffffffu;
     }
     if (threadIdx.x == 0) W.state->active = ~skip_mask & 0xffffu;
-    for (int k = threadIdx.x; k < kLevels * kMaeBins; k += blockDim.x) {
+    for (int k = threadIdx.x; k < kFineSlots; k += blockDim.x) {  // covers the 16 x kMaeBins digit bins as well
         W.hist[k] = 0ull;
         W.chist[k] = 0ull;
     }
@@ -571,6 +574,320 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W, co
     }
 }
 
+// ---------------------------------------------------------------- later passes, bf16 weights
+//
+// The passes after the first on the 64-byte-per-lane front end: the same set-up, queue, digit
+// histogram, candidate lists and fused selection as mae_pass_kernel without its first-pass
+// parts; only the streaming loop differs (32 weights per lane, packed min/max, two row buffers
+// used in turn).
+
+// What a participating sample of a later pass does (digit histogram, candidate list), out of
+// line: the streaming loop only queues samples, and its thirty-two unrolled copies must stay small
+// enough for the instruction cache.
+struct LaterCtx {
+    const float* xi;
+    const uint4* lvl;
+    const uint32_t* limit;
+    uint32_t *lo, *hi, *ncand;
+    uint2* cand;
+    volatile uint32_t* over;
+    MaeState* state;
+    uint2* gcand;
+};
+template <bool COLLECT>
+__device__ __noinline__ void later_sample_fn(const LaterCtx* C, float xk, uint32_t a)
+{
+    const uint32_t c = (uint32_t)region_of(xk, C->xi);
+    const uint4 L = C->lvl[c];
+    const uint32_t rel = order_key(xk) - L.x;
+    const uint32_t top = L.z & 0xffu, sh = (L.z >> 8) & 0xffu, mask = L.z >> 16;
+    if (!(L.w && (uint32_t)((unsigned long long)rel >> top) == L.y && rel <= C->limit[c])) return;
+    const uint32_t bin = c * kMaeBins + ((rel >> sh) & mask);
+    const uint32_t old = atomicAdd(&C->lo[bin], a);
+    if (old + a < old) atomicAdd(&C->hi[bin], 1u);
+    if (COLLECT) {
+        // staged per CTA and level; the rare overflow of a slot goes straight to the
+        // global list (whose count only needs to stay above the capacity once full)
+        const uint32_t slot = atomicAdd(&C->ncand[c], 1u);
+        if (slot < (uint32_t)kMaeStage) {
+            C->cand[c * kMaeStage + slot] = make_uint2(rel, a);
+        } else if (!C->over[c]) {
+            uint32_t* cnt = &C->state->cand_count[c];
+            if (*reinterpret_cast<volatile uint32_t*>(cnt) <= (uint32_t)kMaeCand) {
+                const uint32_t gslot = atomicAdd(cnt, 1u);
+                if (gslot < (uint32_t)kMaeCand) C->gcand[c * kMaeCand + gslot] = make_uint2(rel, a);
+            } else {
+                C->over[c] = 1u;  // remembered per CTA: later samples of this level skip the look-up
+            }
+        }
+    }
+}
+
+template <int I, bool SIGNED, bool COLLECT, bool TAIL>
+__global__ void __launch_bounds__(kMaeThreads, 1)
+mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W, const MaeFinal F)
+{
+    constexpr bool FIRST = false, COUNT = false;
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    unsigned char* s_lut = s_raw;
+    uint32_t* s_lo = reinterpret_cast<uint32_t*>(s_raw + kLutBytes);
+    uint32_t* s_hi = s_lo + kLevels * kMaeBins;
+    uint32_t* s_cn = s_hi + kLevels * kMaeBins;
+    uint2* s_queue = reinterpret_cast<uint2*>(s_cn);  // later passes (which keep no counts)
+    uint2* s_cand = reinterpret_cast<uint2*>(s_cn + kLevels * kMaeBins);  // [16][kMaeStage] (COLLECT)
+    __shared__ uint32_t s_ncand[kLevels], s_gbase[kLevels];
+    __shared__ volatile uint32_t s_over[kLevels];  // level's global list is known to have overflowed
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ int s_multi;
+    __shared__ WideScratch s_wide;
+    __shared__ uint4 s_lvl[kLevels];  // {base, prefix, top | shift << 8 | mask << 16, on}
+    __shared__ uint32_t s_limit[kLevels];  // largest relative key of the level's range
+    // first pass: {base, shift | on << 31, level, -}, one column per lane of a quarter warp (the unit
+    // a 16-byte shared-memory read is served in), so that the read never meets a bank conflict
+    __shared__ uint4 s_lvl1[kLevels * 8];
+    __shared__ uint2 s_iv[kLutBins];  // later passes: bits of {lo, hi} per table bin (lo > hi: nothing)
+    __shared__ float2 s_span[kLevels];
+    __shared__ uint32_t s_qn;
+    __shared__ double s_err[kMaeThreads / 32];
+    __shared__ const void* s_ptr[kEmMaxTensors];
+    __shared__ int64_t s_n[kEmMaxTensors], s_row_end[kEmMaxTensors];
+
+    __shared__ unsigned long long s_wsum[kMaeThreads / 32];
+    __shared__ PickResult s_res;
+    __shared__ int s_last;
+    if (!FIRST) {  // nothing left to resolve: uniform over the grid
+        int any = 0;
+        for (int l = 0; l < kLevels; ++l) any |= W.state->top[l];
+        if (any <= 0) {
+            if (TAIL && F.enabled && T.last && blockIdx.x == 0) finalize_body(W, F, s_err);
+            return;
+        }
+    }
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    make_thresholds(levels, s_xi, s_lv, tid);
+    if (tid < kLevels) {
+        const int top = W.state->top[tid];
+        const int sh = max(top - kMaeDigitBits, 0);
+        const uint32_t mask = (1u << (top - sh)) - 1u;
+        s_lvl[tid] = make_uint4(W.state->base[tid], W.state->prefix[tid],
+                                (uint32_t)top | ((uint32_t)sh << 8) | (mask << 16), top > 0 ? 1u : 0u);
+        s_limit[tid] = W.state->limit[tid];
+        for (int q = 0; q < 8; ++q)
+            s_lvl1[tid * 8 + q] = make_uint4(W.state->base[tid], (uint32_t)sh | (top > 0 ? 0x80000000u : 0u),
+                                             __float_as_uint(levels[tid]), 0u);
+    }
+    if (tid < T.count) {
+        s_ptr[tid] = T.ptr[tid];
+        s_n[tid] = T.n[tid];
+        s_row_end[tid] = T.row_end[tid];
+    }
+    for (int k = tid; k < (FIRST ? 3 : 2) * kLevels * kMaeBins; k += kMaeThreads) s_lo[k] = 0u;
+    if (tid < kLevels) {
+        s_ncand[tid] = 0u;
+        s_over[tid] = 0u;
+    }
+    if (tid == 0) s_qn = 0u;
+    const uint32_t max_bits = W.state->max_bits;
+    __syncthreads();
+    bool lut_ok = true;
+    if (FIRST) {
+        build_lut(s_xi, s_lut, &s_multi, [](int base) { return (uint32_t)base; });
+        __syncthreads();
+        lut_ok = s_multi == 0;
+    } else {
+        // Participants of level l have keys in [base + (prefix << top), base + ((prefix + 1) << top));
+        // keys and normalised weights are ordered alike, so they lie between the weights of the
+        // two end keys (clipped to [-1, 1]), and so do their table bins.
+        if (tid < kLevels) {
+            const uint4 L = s_lvl[tid];
+            const int top = (int)(L.z & 0xffu);
+            float2 span = make_float2(2.0f, -2.0f);
+            if (L.w) {
+                const uint32_t kmin = order_key(-1.0f), kmax = order_key(1.0f);
+                const unsigned long long lo64 = (unsigned long long)L.x + ((unsigned long long)L.y << top);
+                unsigned long long hi64 = lo64 + ((1ull << top) - 1ull);
+                const unsigned long long cap64 = (unsigned long long)L.x + W.state->limit[tid];
+                if (hi64 > cap64) hi64 = cap64;
+                const uint32_t klo = max(lo64 > kmax ? kmax : (uint32_t)lo64, kmin);
+                const uint32_t khi = max(hi64 > kmax ? kmax : (uint32_t)hi64, kmin);
+                span = make_float2(key_to_float(klo), key_to_float(khi));
+            }
+            s_span[tid] = span;
+        }
+        __syncthreads();
+        for (int b = tid; b < kLutBins; b += kMaeThreads) {
+            float2 iv = make_float2(2.0f, -2.0f);
+            for (int l = 0; l < kLevels; ++l) {
+                const float2 sp = s_span[l];
+                if (sp.x > sp.y) continue;
+                const int blo = (int)(__float_as_uint(lut_key(sp.x)) - kLutMagicBits);
+                const int bhi = (int)(__float_as_uint(lut_key(sp.y)) - kLutMagicBits);
+                if (b >= blo && b <= bhi) iv = make_float2(fminf(iv.x, sp.x), fmaxf(iv.y, sp.y));
+            }
+            s_iv[b] = make_uint2(__float_as_uint(iv.x), __float_as_uint(iv.y));
+        }
+        __syncthreads();
+        for (int k = tid; k < kLutBins * 32; k += kMaeThreads)  // one column per lane, as in the region table
+            *reinterpret_cast<uint2*>(s_lut + k * 8) = s_iv[k >> 5];
+        __syncthreads();
+    }
+
+    // One participating sample of a later pass: digit histogram and (COLLECT) candidate list.
+    __shared__ LaterCtx s_ctx;
+    if (tid == 0)
+        s_ctx = LaterCtx{s_xi, s_lvl, s_limit, s_lo, s_hi, s_ncand, s_cand, s_over, W.state, W.cand};
+    __syncthreads();
+    auto later_sample = [&](float xk, uint32_t a) { later_sample_fn<COLLECT>(&s_ctx, xk, a); };
+
+    const int64_t total_rows = T.row_end[T.count - 1];
+    const uint32_t lut_base = lut_lane_base(s_lut, lane);
+    double err = 0.0;
+    int t_cur = 0;
+    // row g of the concatenated tensors: this thread's 32 weights, or zeros past the end (ok = false);
+    // src: where they came from (a participating weight is read again by its index)
+    auto fetch = [&](int64_t g, bool& ok, const uint16_t*& src) -> Raw32 {
+        ok = false;
+        if (g < total_rows) {
+            while (g >= s_row_end[t_cur]) ++t_cur;
+            const int64_t r = g - (t_cur ? s_row_end[t_cur - 1] : 0);
+            const int64_t idx = (r * kMaeThreads + tid) * kLW;
+            ok = idx < s_n[t_cur];
+            if (ok) {
+                src = static_cast<const uint16_t*>(s_ptr[t_cur]) + idx;
+                return load_raw32(s_ptr[t_cur], idx);
+            }
+        }
+        return zero_raw32();
+    };
+    // A sample that may take part is queued (and handled on the spot when the queue is full).
+    auto offer = [&](float xk, uint32_t a) {
+        const uint32_t slot = atomicAdd(&s_qn, 1u);
+        if (slot < (uint32_t)kMaeQueue)
+            s_queue[slot] = make_uint2(__float_as_uint(xk), a);
+        else
+            later_sample(xk, a);
+    };
+    // A weight inside its table bin's hull may take part.  The streaming loop only marks such
+    // weights in a bit mask (two comparisons and one predicated OR per weight); the few marked ones
+    // (about one in 200) are then read again by index, divided again and queued.  A row that cannot
+    // use the table (a zero, non-finite or extreme block constant) offers all its weights.
+    auto row = [&](const Raw32& raw, bool ok, const uint16_t* src) {
+        uint32_t u[16];
+        words_of(raw, u);
+        float mx, mn, g;
+        lane_minmax32(u, mx, mn);
+        const float m = block_constant32<I, SIGNED>(u, mx, mn, g, &s_wide);
+        const uint32_t a = T.unit ? 1u : fixed_weight(m, max_bits);
+        const bool table = __all_sync(kFull, ok && div_safe(g));
+        const bool recip = div_safe(fabsf(m));
+        const float r = recip ? __frcp_rn(m) : 0.0f;
+        const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
+        uint32_t marked = ok ? 0xffffffffu : 0u;
+        if (table) {
+            marked = 0u;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const float2 v = make_float2(bf_lo(u[k]), bf_hi(u[k]));
+                const float2 q0 = __fmul2_rn(v, rr);
+                const float2 x = __ffma2_rn(__ffma2_rn(q0, nm, v), rr, q0);  // the true quotients
+                const float2 key = lut_key2(x);
+                const uint2 i0 = lut_probe(key.x, lut_base), i1 = lut_probe(key.y, lut_base);
+                if (x.x >= __uint_as_float(i0.x) && x.x <= __uint_as_float(i0.y)) marked |= 1u << (2 * k);
+                if (x.y >= __uint_as_float(i1.x) && x.y <= __uint_as_float(i1.y)) marked |= 2u << (2 * k);
+            }
+        }
+        while (marked) {
+            const int j = __ffs(marked) - 1;
+            marked &= marked - 1u;
+            const float v = __uint_as_float((uint32_t)__ldg(src + j) << 16);
+            float x;
+            if (recip) {  // the same sequence as above, one weight
+                const float q0 = __fmul_rn(v, r);
+                x = fmaf(fmaf(q0, -m, v), r, q0);
+            } else {
+                x = normalise(v, m);
+            }
+            offer(x, a);
+        }
+    };
+    {
+        bool ok_a, ok_b;
+        const uint16_t *src_a = nullptr, *src_b = nullptr;
+        int64_t g = blockIdx.x;
+        const int64_t GS = gridDim.x;
+        Raw32 ra = fetch(g, ok_a, src_a), rb;
+        if (g < total_rows) {
+            while (true) {
+                rb = fetch(g + GS, ok_b, src_b);
+                row(ra, ok_a, src_a);
+                g += GS;
+                if (g >= total_rows) break;
+                ra = fetch(g + GS, ok_a, src_a);
+                row(rb, ok_b, src_b);
+                g += GS;
+                if (g >= total_rows) break;
+            }
+        }
+    }
+    __syncthreads();
+    if (!FIRST) {
+        const uint32_t q = min(s_qn, (uint32_t)kMaeQueue);
+        for (uint32_t i = tid; i < q; i += kMaeThreads) {
+            const uint2 ent = s_queue[i];
+            later_sample(__uint_as_float(ent.x), ent.y);
+        }
+        __syncthreads();
+    }
+    for (int k = tid; k < kLevels * kMaeBins; k += kMaeThreads) {
+        const unsigned long long wsum = ((unsigned long long)s_hi[k] << 32) + s_lo[k];
+        if (wsum) atomicAdd(&W.hist[k], wsum);
+        if (FIRST && COUNT && s_cn[k]) atomicAdd(&W.chist[k], (unsigned long long)s_cn[k]);
+    }
+    if (COLLECT) {
+        // one reservation per CTA and level, then a plain copy of the staged samples
+        if (tid < kLevels) {
+            const uint32_t k = min(s_ncand[tid], (uint32_t)kMaeStage);
+            s_gbase[tid] = k ? atomicAdd(&W.state->cand_count[tid], k) : 0u;
+        }
+        __syncthreads();
+        for (int k = tid; k < kLevels * kMaeStage; k += kMaeThreads) {
+            const int l = k / kMaeStage, i = k % kMaeStage;
+            const uint32_t dst = s_gbase[l] + (uint32_t)i;
+            if ((uint32_t)i < min(s_ncand[l], (uint32_t)kMaeStage) && dst < (uint32_t)kMaeCand)
+                W.cand[l * kMaeCand + dst] = s_cand[k];
+        }
+    }
+    if (FIRST) {
+#pragma unroll
+        for (int off = 16; off; off >>= 1) err += __shfl_xor_sync(kFull, err, off);
+        if (lane == 0) s_err[warp] = err;
+        __syncthreads();
+        if (tid == 0) {
+            double t = 0.0;
+            for (int k = 0; k < kMaeThreads / 32; ++k) t += s_err[k];
+            double* rec = W.partials + (size_t)blockIdx.x * kEmRecordDoubles;
+            rec[0] = T.accumulate ? rec[0] + t : t;
+        }
+    }
+    if (TAIL && T.last) {
+        // every thread's histogram atomics are ordered before the ticket of its CTA
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = (atomicAdd(&W.state->ticket, 1u) == gridDim.x - 1) ? 1 : 0;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            for (int l = 0; l < kLevels; ++l) select_body<kMaeThreads>(W, l, s_wsum, &s_res);
+            if (tid == 0) W.state->ticket = 0u;
+            if (F.enabled) {
+                __threadfence();
+                __syncthreads();  // the state written by thread 0 is read by the update
+                finalize_body(W, F, s_err);
+            }
+        }
+    }
+}
+
 // One CTA per level, one thread per bin.  For a level with bits left: the bin in which the
 // cumulative weight first reaches half of the total becomes the next digit.  After the first
 // pass the totals (and counts) are those of the whole region.
@@ -677,6 +994,385 @@ mae_resolve_kernel(MaeWs W)
     }
 }
 
+// ---------------------------------------------------------------- first pass, bf16 weights
+//
+// With the 64-byte-per-lane front end the first data pass bins every normalised weight on ONE
+// uniform grid instead of on a grid per region: fine bin f = RN(2048 x) + 2048 (a single packed
+// multiply-add for two weights), and the slot of a sample of region c is (f, c & 1).  Regions are
+// intervals of x, so a fine bin holds samples of consecutive regions; as long as no fine bin holds
+// two thresholds, these are at most two regions of different parity and every slot belongs to one
+// region.  Inside a region slots follow the order of x, so the selection walks the region's fine
+// bins in ascending order; no per-region key arithmetic is needed per weight (the former first
+// pass spent a third of its instructions on it).  The selected fine bin becomes the key range
+// [base, base + 2^top) that the later passes refine digit by digit, exactly as after a first
+// digit.  A codebook with two thresholds in one fine bin (levels closer than 1/2048) is
+// "degenerate": the pass then bins per region on the first nine bits of the region-relative
+// key, like the generic first pass, and the selection kernel does that pass's selection.
+
+constexpr float kFineMagic = 12582912.0f + (float)kFineScale;  // 1.5 * 2^23 + 2048
+__device__ __forceinline__ float2 fine_key2(float2 x)
+{
+    return __ffma2_rn(x, make_float2((float)kFineScale, (float)kFineScale), make_float2(kFineMagic, kFineMagic));
+}
+// Fine bin of x, clamped to the grid (x outside [-1, 1] only occurs for non-finite input).
+__device__ __forceinline__ int fine_bin(float x)
+{
+    const float c = fminf(fmaxf(x, -1.0f), 1.0f);
+    return (int)(__float_as_uint(fmaf(c, (float)kFineScale, kFineMagic)) - kLutMagicBits);
+}
+// Two thresholds share a fine bin.
+__device__ __forceinline__ bool degenerate_codebook(const float* s_xi)
+{
+    bool d = false;
+    for (int j = 0; j + 1 < kLevels - 1; ++j) d = d || fine_bin(s_xi[j]) == fine_bin(s_xi[j + 1]);
+    return d;
+}
+
+// Slot sums in shared memory: 64-bit bins kept as two words (native 32-bit atomics with carry;
+// addresses fall on random banks, so every atomic costs several wavefronts and a scheme with more,
+// carry-free partial words per slot measured slower).
+constexpr int kMae1Words = 2;
+constexpr size_t kMae1Smem(bool count) { return (size_t)kLutBytes + (size_t)kFineSlots * 4u * (kMae1Words + (count ? 1u : 0u)); }
+static_assert(kFineSlots >= kLevels * kMaeBins, "the per-region bins of the degenerate case fit the slot arrays");
+
+struct Mae1Shared {
+    float xi[kLevels], lv[kLevels];
+    uint2 lvrep[kLevels * 32];  // {level l, byte offset of its parity half of the slots} for lane q at [l * 32 + q]
+    uint32_t base[kLevels];     // degenerate case: key of each region's lower edge and digit shift
+    int shift[kLevels];
+    int multi, degenerate;
+    WideScratch wide;
+    double err[kMaeThreads / 32];
+    const void* ptr[kEmMaxTensors];
+    int64_t n[kEmMaxTensors], row_end[kEmMaxTensors];
+};
+
+// One sample into its slot.  The streaming loop addresses the slot arrays and the level table
+// through explicit shared-window addresses (32-bit), like the table probe.
+__device__ __forceinline__ void red_shared_add(uint32_t addr, uint32_t v)
+{
+    asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+template <int OFF>
+__device__ __forceinline__ void red_shared_add_off(uint32_t addr, uint32_t v)
+{
+    asm volatile("red.shared.add.u32 [%0+%2], %1;" ::"r"(addr), "r"(v), "n"(OFF) : "memory");
+}
+__device__ __forceinline__ uint2 ld_shared_v2(uint32_t addr)
+{
+    uint2 v;
+    asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t atom_shared_add(uint32_t addr, uint32_t v)
+{
+    uint32_t old;
+    asm volatile("atom.shared.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
+    return old;
+}
+// addr: shared-window address of the slot's low word (word arrays are kFineSlots * 4 bytes apart).
+template <bool COUNT>
+__device__ __forceinline__ void slot_add_at(uint32_t addr, uint32_t a)
+{
+    const uint32_t old = atom_shared_add(addr, a);
+    if (old + a < old) red_shared_add_off<kFineSlots * 4>(addr, 1u);
+    if (COUNT) red_shared_add_off<2 * kFineSlots * 4>(addr, 1u);
+}
+template <bool COUNT>
+__device__ __forceinline__ void slot_add(uint32_t* s_lo, int slot, uint32_t a)
+{
+    slot_add_at<COUNT>((uint32_t)__cvta_generic_to_shared(s_lo) + (uint32_t)slot * 4u, a);
+}
+
+// A row outside the common case (a zero, extreme or non-finite block constant, a codebook the
+// region table cannot serve, a degenerate codebook): true quotients, binary search.  Out of
+// line.  Returns the row's error sum.
+template <bool COUNT>
+__device__ __noinline__ float mae1_row_slow(Raw32 raw, float m, uint32_t a, bool unit, const Mae1Shared* S, uint32_t* s_lo)
+{
+    uint32_t u[16];
+    words_of(raw, u);
+    const bool recip = div_safe(fabsf(m));
+    const float r = recip ? __frcp_rn(m) : 0.0f;
+    float e = 0.0f;
+#pragma unroll 1
+    for (int k = 0; k < 16; ++k) {
+        const float2 v = make_float2(bf_lo(u[k]), bf_hi(u[k]));
+        float2 x;
+        if (recip) {  // the same quotient as the common path (reciprocal sequence, no guard)
+            const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
+            const float2 q0 = __fmul2_rn(v, rr);
+            x = __ffma2_rn(__ffma2_rn(q0, nm, v), rr, q0);
+        } else {
+            x = make_float2(normalise(v.x, m), normalise(v.y, m));
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const float xh = h ? x.y : x.x, vh = h ? v.y : v.x;
+            const int c = region_of(xh, S->xi);
+            e += unit ? fabsf(xh - S->lv[c]) : fabsf(fmaf(-m, S->lv[c], vh));
+            if (S->degenerate) {
+                const uint32_t rel = order_key(xh) - S->base[c];
+                slot_add<COUNT>(s_lo, c * kMaeBins + (int)((rel >> S->shift[c]) & (uint32_t)(kMaeBins - 1)), a);
+            } else if (xh == xh) {  // a NaN has no place on the grid
+                slot_add<COUNT>(s_lo, fine_bin(xh) + (c & 1) * kFineStride, a);
+            }
+        }
+    }
+    return e;
+}
+
+template <int I, bool SIGNED, bool COUNT>
+__global__ void __launch_bounds__(kMaeThreads, 1)
+mae_pass1_32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W)
+{
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    unsigned char* s_lut = s_raw;
+    uint32_t* s_lo = reinterpret_cast<uint32_t*>(s_raw + kLutBytes);  // lo [kFineSlots], hi, (count)
+    __shared__ Mae1Shared S;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    make_thresholds(levels, S.xi, S.lv, tid);
+    if (tid < T.count) {
+        S.ptr[tid] = T.ptr[tid];
+        S.n[tid] = T.n[tid];
+        S.row_end[tid] = T.row_end[tid];
+    }
+    if (tid < kLevels) {
+        const int top = W.state->top[tid];
+        S.base[tid] = W.state->base[tid];
+        S.shift[tid] = max(top - kMaeDigitBits, 0);
+    }
+    for (int k = tid; k < kFineSlots * (kMae1Words + (COUNT ? 1 : 0)); k += kMaeThreads) s_lo[k] = 0u;
+    if (tid < kLevels * 32)
+        S.lvrep[tid] = make_uint2(__float_as_uint(levels[tid >> 5]), (uint32_t)((tid >> 5) & 1) * (uint32_t)(kFineStride * 4));
+    const uint32_t max_bits = W.state->max_bits;
+    __syncthreads();
+    if (tid == 0) S.degenerate = degenerate_codebook(S.xi) ? 1 : 0;
+    // table payload: byte offset of the region's row in the level table
+    build_lut(S.xi, s_lut, &S.multi, [](int base) { return (uint32_t)base * 256u; });
+    __syncthreads();
+    const bool table_ok = S.multi == 0 && S.degenerate == 0;
+    const bool unit = T.unit != 0;
+
+    const int64_t total_rows = T.row_end[T.count - 1];
+    double err = 0.0;
+    int t_cur = 0;
+    auto fetch = [&](int64_t g, bool& ok) -> Raw32 {
+        ok = false;
+        if (g < total_rows) {
+            while (g >= S.row_end[t_cur]) ++t_cur;
+            const int64_t r = g - (t_cur ? S.row_end[t_cur - 1] : 0);
+            const int64_t idx = (r * kMaeThreads + tid) * kLW;
+            ok = idx < S.n[t_cur];
+            if (ok) return load_raw32(S.ptr[t_cur], idx);
+        }
+        return zero_raw32();
+    };
+    const uint32_t lut_base = lut_lane_base(s_lut, lane);
+    const uint32_t lv_base = (uint32_t)__cvta_generic_to_shared(S.lvrep) + (uint32_t)lane * 8u;
+    // slot address of a sample from the bits of its fine key: (bits - magic) * 4 + start of the slot array
+    const uint32_t slot_base = (uint32_t)__cvta_generic_to_shared(s_lo) - kLutMagicBits * 4u;
+
+    auto row = [&](const Raw32& raw, bool ok) {
+        uint32_t u[16];
+        words_of(raw, u);
+        float mx, mn, g;
+        lane_minmax32(u, mx, mn);
+        const float m = block_constant32<I, SIGNED>(u, mx, mn, g, &S.wide);
+        const uint32_t a = unit ? 1u : fixed_weight(m, max_bits);
+        float e = 0.0f;
+        if (table_ok && __all_sync(kFull, ok && div_safe(g))) {
+            // true quotients (reciprocal sequence), region by the one-probe table, fine bin
+            const float r = __frcp_rn(m), scale = unit ? 1.0f : m;
+            const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const float2 v = make_float2(bf_lo(u[k]), bf_hi(u[k]));
+                const float2 q0 = __fmul2_rn(v, rr);
+                const float2 x = __ffma2_rn(__ffma2_rn(q0, nm, v), rr, q0);
+                const float2 key = lut_key2(x), fk = fine_key2(x);
+                const float2 vv = unit ? x : v;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float xh = h ? x.y : x.x, vh = h ? vv.y : vv.x;
+                    const uint2 ent = lut_probe(h ? key.y : key.x, lut_base);
+                    const uint2 lv = ld_shared_v2(ent.y + ((xh >= __uint_as_float(ent.x)) ? 256u : 0u) + lv_base);
+                    e += fabsf(fmaf(-scale, __uint_as_float(lv.x), vh));
+                    slot_add_at<COUNT>(__float_as_uint(h ? fk.y : fk.x) * 4u + slot_base + lv.y, a);
+                }
+            }
+        } else if (ok) {
+            e = mae1_row_slow<COUNT>(raw, m, a, unit, &S, s_lo);
+        }
+        err += (double)e;
+    };
+
+    bool ok_a, ok_b;
+    int64_t g = blockIdx.x;
+    const int64_t GS = gridDim.x;
+    Raw32 ra = fetch(g, ok_a), rb;
+    if (g < total_rows) {
+        while (true) {
+            rb = fetch(g + GS, ok_b);
+            row(ra, ok_a);
+            g += GS;
+            if (g >= total_rows) break;
+            ra = fetch(g + GS, ok_a);
+            row(rb, ok_b);
+            g += GS;
+            if (g >= total_rows) break;
+        }
+    }
+    __syncthreads();
+    for (int k = tid; k < kFineSlots; k += kMaeThreads) {
+        const unsigned long long wsum = ((unsigned long long)s_lo[kFineSlots + k] << 32) + s_lo[k];
+        if (wsum) atomicAdd(&W.hist[k], wsum);
+        if (COUNT && s_lo[2 * kFineSlots + k]) atomicAdd(&W.chist[k], (unsigned long long)s_lo[2 * kFineSlots + k]);
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) err += __shfl_xor_sync(kFull, err, off);
+    if (lane == 0) S.err[warp] = err;
+    __syncthreads();
+    if (tid == 0) {
+        double t = 0.0;
+        for (int k = 0; k < kMaeThreads / 32; ++k) t += S.err[k];
+        double* rec = W.partials + (size_t)blockIdx.x * kEmRecordDoubles;
+        rec[0] = T.accumulate ? rec[0] + t : t;
+    }
+}
+
+// Selection after the bf16 first pass: one CTA per level walks the level's slots in ascending
+// order of x (thread t owns a run of consecutive fine bins), finds the fine bin in which the
+// cumulative weight reaches half of the region's total, and turns it into the key range of the
+// later passes: base = key of the smallest candidate, top = bits of the range.  Also records the
+// region's total weight and member count and clears the slots it read.  For a degenerate
+// codebook it performs the generic first selection on the per-region bins instead.
+__global__ void __launch_bounds__(1024)
+mae_select1_kernel(const float* __restrict__ levels, MaeWs W)
+{
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ unsigned long long s_wsum[32], s_csum[32];
+    __shared__ PickResult s_res;
+    __shared__ int s_pick;
+    __shared__ unsigned long long s_excl;
+    MaeState* S = W.state;
+    const int l = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    make_thresholds(levels, s_xi, s_lv, tid);
+    if (tid == 0) s_pick = -1;
+    __syncthreads();
+    const int top0 = S->top[l];  // from the set-up kernel: bits of the region's key range, 0 for a level that does not take part
+    if (degenerate_codebook(s_xi)) {
+        unsigned long long mine = 0ull, c = 0ull;
+        if (tid < kMaeBins) {
+            mine = __ldcg(&W.hist[l * kMaeBins + tid]);
+            W.hist[l * kMaeBins + tid] = 0ull;
+            c = __ldcg(&W.chist[l * kMaeBins + tid]);
+            W.chist[l * kMaeBins + tid] = 0ull;
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) c += __shfl_xor_sync(kFull, c, off);
+        if (lane == 0) s_csum[warp] = c;
+        unsigned long long all;
+        const PickResult r = pick_bin<1024>(mine, 0ull, 0ull, true, s_wsum, &s_res, &all);
+        if (tid == 0) {
+            unsigned long long count = 0ull;
+            for (int k = 0; k < 32; ++k) count += s_csum[k];
+            S->total[l] = all;
+            S->count[l] = count;
+            if (top0 > 0) {
+                const int sh = max(top0 - kMaeDigitBits, 0);
+                S->before[l] = r.excl;
+                S->prefix[l] = (uint32_t)r.bin;
+                S->top[l] = sh;
+            }
+        }
+        return;
+    }
+    // the region's closed range of fine bins
+    const float lo_x = (l == 0) ? -1.0f : fminf(fmaxf(s_xi[l - 1], -1.0f), 1.0f);
+    const float hi_x = (l == kLevels - 1) ? 1.0f : fminf(fmaxf(s_xi[l], -1.0f), 1.0f);
+    const int f_lo = fine_bin(lo_x), f_hi = fine_bin(hi_x);
+    const int span = f_hi - f_lo + 1, per = (span + 1023) / 1024;  // at most 5 bins per thread
+    const int half = (l & 1) * kFineStride;
+    unsigned long long mine = 0ull, cmine = 0ull;
+    unsigned long long vals[5];
+#pragma unroll
+    for (int q = 0; q < 5; ++q) {
+        const int f = f_lo + tid * per + q;
+        unsigned long long v = 0ull;
+        if (q < per && f <= f_hi) {
+            v = __ldcg(&W.hist[half + f]);
+            W.hist[half + f] = 0ull;
+            cmine += __ldcg(&W.chist[half + f]);
+            W.chist[half + f] = 0ull;
+        }
+        vals[q] = v;
+        mine += v;
+    }
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long t = __shfl_up_sync(kFull, incl, off);
+        if (lane >= off) incl += t;
+    }
+    unsigned long long csum = cmine;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) csum += __shfl_xor_sync(kFull, csum, off);
+    if (lane == 31) s_wsum[warp] = incl;
+    if (lane == 0) s_csum[warp] = csum;
+    __syncthreads();
+    unsigned long long carry = 0ull, total = 0ull, count = 0ull;
+    for (int k = 0; k < 32; ++k) {
+        if (k < warp) carry += s_wsum[k];
+        total += s_wsum[k];
+        count += s_csum[k];
+    }
+    incl += carry;
+    const unsigned long long excl = incl - mine;
+    if (top0 > 0 && total > 0ull && 2ull * incl >= total && 2ull * excl < total) {
+        unsigned long long run = excl;  // the crossing lies in this thread's run of bins
+#pragma unroll
+        for (int q = 0; q < 5; ++q) {
+            if (2ull * (run + vals[q]) >= total) {
+                s_pick = f_lo + tid * per + q;
+                s_excl = run;
+                break;
+            }
+            run += vals[q];
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        S->total[l] = total;
+        S->count[l] = count;
+        S->prefix[l] = 0u;
+        S->before[l] = 0ull;
+        S->top[l] = 0;
+        S->base[l] = order_key(lo_x);
+        if (s_pick >= 0) {
+            const int f = s_pick;
+            const uint32_t kmin = order_key(-1.0f), kmax = order_key(1.0f);
+            // smallest x of fine bin f: start a few steps below its lower edge and walk up
+            uint32_t kl = order_key(((float)(f - kFineScale) - 0.5f) * (1.0f / (float)kFineScale));
+            kl = (f == 0 || kl < kmin + 4u) ? kmin : kl - 4u;
+            while (kl < kmax && fine_bin(key_to_float(kl)) < f) ++kl;
+            // largest x of the bin, generously (keys above it only add samples beyond the median)
+            uint32_t kh = order_key(((float)(f - kFineScale) + 0.5f) * (1.0f / (float)kFineScale));
+            kh = (kh > kmax - 4u) ? kmax : kh + 4u;
+            // inside the region
+            const uint32_t rl = order_key(lo_x), rh = order_key(hi_x);
+            if (kl < rl) kl = rl;
+            if (kh > rh) kh = rh;
+            if (kh < kl) kh = kl;
+            const uint32_t range = kh - kl;
+            S->base[l] = kl;
+            S->limit[l] = range;
+            S->before[l] = s_excl;
+            S->top[l] = range ? 32 - __clz(range) : 0;  // key bits still unresolved
+        }
+    }
+}
+
 // ---------------------------------------------------------------- level update
 
 __global__ void __launch_bounds__(256)
@@ -709,6 +1405,79 @@ int launch_pass(const EmTensors& T, const float* d_levels, const MaeWs& W, int p
 #undef BOF4_MAE_GO
     BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
+}
+
+template <int I, bool SG>
+int launch_pass1_32(const EmTensors& T, const float* d_levels, const MaeWs& W, bool count, cudaStream_t st)
+{
+    if (count) {
+        constexpr auto kern = mae_pass1_32_kernel<I, SG, true>;
+        if (const int rc = ensure_dynamic_smem<kern>((int)kMae1Smem(true))) return rc;
+        kern<<<kEmGrid, kMaeThreads, kMae1Smem(true), st>>>(T, d_levels, W);
+    } else {
+        constexpr auto kern = mae_pass1_32_kernel<I, SG, false>;
+        if (const int rc = ensure_dynamic_smem<kern>((int)kMae1Smem(false))) return rc;
+        kern<<<kEmGrid, kMaeThreads, kMae1Smem(false), st>>>(T, d_levels, W);
+    }
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
+}
+
+template <int I, bool SG>
+int launch_later32(const EmTensors& T, const float* d_levels, const MaeWs& W, bool collect, const MaeFinal* tail,
+                   cudaStream_t st)
+{
+    const MaeFinal F = tail ? *tail : MaeFinal{};
+#define BOF4_MAE_L32(COLLECT_, TAIL_)                                                           \
+    {                                                                                           \
+        constexpr auto kern = mae_later32_kernel<I, SG, COLLECT_, TAIL_>;                       \
+        if (const int rc_ = ensure_dynamic_smem<kern>((int)kMaeSmem)) return rc_;               \
+        kern<<<kEmGrid, kMaeThreads, kMaeSmem, st>>>(T, d_levels, W, F);                        \
+    }
+    if (collect) BOF4_MAE_L32(true, false)
+    else if (tail) BOF4_MAE_L32(false, true)
+    else BOF4_MAE_L32(false, false)
+#undef BOF4_MAE_L32
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
+}
+
+int dispatch_later32(const EmArgs& a, const EmTensors& T, const float* d_levels, const MaeWs& W, bool collect,
+                     const MaeFinal* tail, cudaStream_t st)
+{
+    const bool sg = a.norm == BOF4_NORM_SIGNED;
+#define BOF4_MAEL_I(I_) return sg ? launch_later32<I_, true>(T, d_levels, W, collect, tail, st) \
+                                  : launch_later32<I_, false>(T, d_levels, W, collect, tail, st);
+    switch (a.block_size) {
+        case 32: BOF4_MAEL_I(32)
+        case 64: BOF4_MAEL_I(64)
+        case 128: BOF4_MAEL_I(128)
+        case 256: BOF4_MAEL_I(256)
+        case 512: BOF4_MAEL_I(512)
+        case 1024: BOF4_MAEL_I(1024)
+        case 2048: BOF4_MAEL_I(2048)
+        default: BOF4_MAEL_I(4096)
+    }
+#undef BOF4_MAEL_I
+}
+
+int dispatch_pass1_32(const EmArgs& a, const EmTensors& T, const float* d_levels, const MaeWs& W, bool count,
+                      cudaStream_t st)
+{
+    const bool sg = a.norm == BOF4_NORM_SIGNED;
+#define BOF4_MAE1_I(I_) return sg ? launch_pass1_32<I_, true>(T, d_levels, W, count, st) \
+                                  : launch_pass1_32<I_, false>(T, d_levels, W, count, st);
+    switch (a.block_size) {
+        case 32: BOF4_MAE1_I(32)
+        case 64: BOF4_MAE1_I(64)
+        case 128: BOF4_MAE1_I(128)
+        case 256: BOF4_MAE1_I(256)
+        case 512: BOF4_MAE1_I(512)
+        case 1024: BOF4_MAE1_I(1024)
+        case 2048: BOF4_MAE1_I(2048)
+        default: BOF4_MAE1_I(4096)
+    }
+#undef BOF4_MAE1_I
 }
 
 int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, const MaeWs& W, int pass,
@@ -761,6 +1530,9 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
     // The candidate lists are filled by the first pass after which a region's candidates
     // (about 1/512 of them survive each digit) are expected to fit: the second pass up to
     // 2^29 weights, the third beyond.
+    // (The bf16 first pass narrows a region to one of its 140 ... 400 fine bins rather than to one
+    // of 512 digit bins; a list that overflows all the same is finished by the later passes.)
+    const bool bf16 = a.w_dtype == BOF4_BF16;
     const int collect_pass = (a.n_total / kLevels / kMaeBins <= kMaeCand / 8) ? 1 : 2;
     MaeFinal fin{};
     fin.n_records = kEmGrid;
@@ -778,14 +1550,22 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
         // last pass, the level update ride in the pass kernel itself.
         const bool fused = p >= 2 && p != collect_pass;
         fin.enabled = (fused && p == kMaeMaxPasses - 1) ? 1 : 0;
+        const bool first32 = first && bf16;  // bf16 weights: first pass on the uniform grid
         auto fire = [&](const EmTensors& T) -> int {
+            if (first32) return dispatch_pass1_32(a, T, d_levels_in, W, d_stats != nullptr, st);
+            if (bf16) return dispatch_later32(a, T, d_levels_in, W, p == collect_pass, fused ? &fin : nullptr, st);
             return dispatch_pass(a, T, d_levels_in, W, p, p == collect_pass, first && d_stats != nullptr,
                                  fused ? &fin : nullptr, st);
         };
         int calls = 0;
-        const int rc = for_each_tensor_chunk(a, kMaeRow, fire, &calls);
+        const int rc = for_each_tensor_chunk(a, bf16 ? kMaeThreads * kLW : kMaeRow, fire, &calls);
         if (rc) return rc;
         if (first && calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(W.partials, 0, kEmPartialBytes, st));
+        if (first32) {
+            mae_select1_kernel<<<kLevels, 1024, 0, st>>>(d_levels_in, W);
+            BOF4_CUDA_TRY(cudaGetLastError());
+            continue;
+        }
         if (fused && calls > 0) {
             updated = fin.enabled != 0;
             continue;

@@ -20,7 +20,13 @@ constexpr int kMaeBins = 1 << kMaeDigitBits;  // bins per level and selection pa
 constexpr int kMaeMaxPasses = 4;          // 31 key bits / 9 bits per pass
 constexpr size_t kEmMaeOffset = 512 * 1024;
 constexpr size_t kEmMaeStateBytes = 4096;  // selection state (struct MaeState)
-constexpr size_t kEmMaeHistBytes = (size_t)16 * kMaeBins * 8;  // weight histogram, then count histogram
+// bf16 first pass: 2 x kFineStride slots (see em_mae.cu); later passes: 16 x kMaeBins digit bins
+constexpr int kFineScale = 2048;                 // fine bins per unit of the normalised weight
+constexpr int kFineBins = 2 * kFineScale + 1;    // fine bin of x in [-1, 1]: RN(2048 x) + 2048
+constexpr int kFineStride = 4112;                // slots per half (below / not below the bin's threshold)
+constexpr int kFineSlots = 2 * kFineStride;
+constexpr size_t kEmMaeHistBytes = 66048;        // weight histogram, then count histogram (>= 8 * kFineSlots)
+static_assert(kEmMaeHistBytes >= (size_t)kFineSlots * 8 && kEmMaeHistBytes >= (size_t)16 * kMaeBins * 8, "histogram space");
 constexpr int kMaeCand = 1 << 16;          // candidate samples kept per level by the second pass
 constexpr size_t kEmMaeCandBytes = (size_t)16 * kMaeCand * 8;
 constexpr size_t kEmMaeBytes = kEmMaeStateBytes + 2 * kEmMaeHistBytes + kEmMaeCandBytes;
