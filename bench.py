@@ -169,7 +169,7 @@ class Step:
         self.cb_q = torch.tensor(np.array(workloads.BOF4S_MSE_I64, np.float32), device=dev)
         self.tau = float(np.float32(b.bof4_opq_threshold(Q, I)))
         nmax = max(max(w.numel() for w in s) for s in sets)
-        self.ws_em = torch.empty(b.bof4_workspace_bytes(b.OP_EM, nmax, I, b.METRIC_MAE), dtype=torch.uint8, device=dev)
+        self.ws_em = torch.empty(b.bof4_workspace_bytes(b.OP_EM, self.n_fit, I, b.METRIC_MAE), dtype=torch.uint8, device=dev)
         self.ws_opq = torch.empty(b.bof4_workspace_bytes(b.OP_OPQ, nmax, I, 0), dtype=torch.uint8, device=dev)
         u8, bf = torch.uint8, torch.bfloat16
         self.q_out = [(torch.empty(w.numel() // 2, dtype=u8, device=dev),

@@ -100,11 +100,15 @@ typedef struct bof4_em_stats {
 } bof4_em_stats;
 
 /*
- * Bytes of device workspace an operation needs for tensors of at most n_max elements
- * (for the EM operations: n_max = the largest single tensor of the list).  Host function, no
- * CUDA call.  The workspace must be 256-byte aligned.  Returns 0 for invalid arguments.
+ * Bytes of device workspace an operation needs for tensors of at most n_max elements.  Host
+ * function, no CUDA call.  The workspace must be 256-byte aligned.  Returns 0 for invalid arguments.
  *   op = BOF4_OP_EM : partial records of the deterministic two-stage reduction and, for
- *                     metric = MAE, the per-level selection histograms.
+ *                     metric = MAE, the per-level selection histograms and candidate lists.
+ *                     n_max = the TOTAL number of weights of the tensor list.  The candidate lists
+ *                     grow with it (16 * 8 * n_max / 512 bytes, between 8 and 16 MiB); any workspace of at
+ *                     least bof4_workspace_bytes(BOF4_OP_EM, 0, ...) is accepted, a smaller one
+ *                     than asked for here only costs the MAE fit one more pass over the data per
+ *                     iteration.  Results do not depend on the workspace size.
  *   op = BOF4_OP_OPQ: per-tile outlier staging and tile offsets of the ordered compaction.
  */
 BOF4_API size_t bof4_workspace_bytes(int op, int64_t n_max, int block_size, int metric);

@@ -42,7 +42,8 @@ def mae_launches_per_call(n_tensors: int, n_total: int, iters: int) -> int:
     iteration the set-up, four data passes and the selection kernels of the passes that do not
     carry their own selection (two up to 2^26 weights, three beyond)."""
     chunks = max(1, -(-n_tensors // TENSORS_PER_LAUNCH))
-    small = n_total // LEVELS // 512 <= (1 << 16) // 8
+    cap = min(max(n_total // 512, 1 << 16), 1 << 17)       # candidate entries per level of the default workspace
+    small = n_total // 1024 <= cap
     return chunks + iters * (1 + 4 * chunks + (2 if small else 3))
 
 
@@ -208,7 +209,7 @@ def bof4_em_step(weights, block_size: int, norm: int, metric: int, levels,
     dev = ws[0].device
     cb = _codebook(levels, dev)
     wsp = workspace if workspace is not None else _workspace(
-        OP_EM, max(w.numel() for w in ws), block_size, metric, dev)
+        OP_EM, sum(w.numel() for w in ws), block_size, metric, dev)
     stats = torch.zeros(ctypes.sizeof(EmStats), dtype=torch.uint8, device=dev)
     with torch.cuda.device(dev):
         _check(lib().bof4_em_step(ptrs, sizes, len(ws), dt, block_size, norm, metric, _ptr(cb),
@@ -237,7 +238,7 @@ def bof4_fit_codebook(weights, block_size: int, norm: int, metric: int, levels, 
         cb = _codebook(levels, dev).clone()
         log = torch.zeros(max(iters, 1), dtype=torch.float64, device=dev)
     wsp = workspace if workspace is not None else _workspace(
-        OP_EM, max(w.numel() for w in ws), block_size, metric, dev)
+        OP_EM, sum(w.numel() for w in ws), block_size, metric, dev)
     with torch.cuda.device(dev):
         _check(lib().bof4_fit_codebook(ptrs, sizes, len(ws), dt, block_size, norm, metric, _ptr(cb),
                                        fixed_mask, iters, _ptr(log), _ptr(wsp), wsp.numel(), _stream()))

@@ -758,9 +758,9 @@ extern "C" int bof4_em_step(const void* const* h_w, const int64_t* h_n, int n_te
         tail.stats = d_stats;
         return enqueue_mse_pass<true>(a, d_codebook, partials, tail, st);
     }
-    rc = mae_prepare(a, d_ws, st);
+    rc = mae_prepare(a, d_ws, ws_bytes, st);
     if (rc) return rc;
-    return mae_iteration(a, d_codebook, nullptr, 0u, d_stats, nullptr, d_ws, st);
+    return mae_iteration(a, d_codebook, nullptr, 0u, d_stats, nullptr, d_ws, ws_bytes, st);
 }
 
 extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int n_tensors,
@@ -790,12 +790,12 @@ extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int
         return BOF4_OK;
     }
     if (iters > 0) {
-        rc = mae_prepare(a, d_ws, st);
+        rc = mae_prepare(a, d_ws, ws_bytes, st);
         if (rc) return rc;
     }
     for (int t = 0; t < iters; ++t) {
         rc = mae_iteration(a, d_codebook, d_codebook, fixed_mask, nullptr,
-                           d_err_log ? d_err_log + t : nullptr, d_ws, st);
+                           d_err_log ? d_err_log + t : nullptr, d_ws, ws_bytes, st);
         if (rc) return rc;
     }
     return BOF4_OK;

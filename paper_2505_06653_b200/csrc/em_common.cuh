@@ -69,8 +69,8 @@ int for_each_tensor_chunk(const EmArgs& a, int row, Fire fire, int* n_calls)
 // MAE (Eq. 8) side, implemented in em_mae.cu.  mae_prepare runs once per call (largest
 // |w| of the data, needed for the fixed-point weights); mae_iteration enqueues one
 // iteration: selection passes, then the level update / statistics.
-int mae_prepare(const EmArgs& a, void* d_ws, cudaStream_t st);
+int mae_prepare(const EmArgs& a, void* d_ws, size_t ws_bytes, cudaStream_t st);
 int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out, uint32_t skip_mask,
-                  bof4_em_stats* d_stats, double* d_err_slot, void* d_ws, cudaStream_t st);
+                  bof4_em_stats* d_stats, double* d_err_slot, void* d_ws, size_t ws_bytes, cudaStream_t st);
 
 }  // namespace bof4

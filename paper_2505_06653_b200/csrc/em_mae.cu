@@ -53,16 +53,17 @@ struct MaeWs {
     MaeState* state;
     unsigned long long* hist;   // [16][kMaeBins] weight
     unsigned long long* chist;  // [16][kMaeBins] count
-    uint2* cand;                // [16][kMaeCand] {rel key, fixed-point weight}
+    uint2* cand;                // [16][cand_cap] {rel key, fixed-point weight}
+    uint32_t cand_cap;          // entries per level (from the workspace size)
 };
 
-__host__ __device__ inline MaeWs mae_ws(void* d_ws)
+__host__ __device__ inline MaeWs mae_ws(void* d_ws, size_t ws_bytes)
 {
     char* p = static_cast<char*>(d_ws) + kEmMaeOffset;
     return MaeWs{static_cast<double*>(d_ws), reinterpret_cast<MaeState*>(p),
                  reinterpret_cast<unsigned long long*>(p + kEmMaeStateBytes),
                  reinterpret_cast<unsigned long long*>(p + kEmMaeStateBytes + kEmMaeHistBytes),
-                 reinterpret_cast<uint2*>(p + kEmMaeStateBytes + 2 * kEmMaeHistBytes)};
+                 reinterpret_cast<uint2*>(p + kEmMaeStateBytes + 2 * kEmMaeHistBytes), mae_cand_capacity(ws_bytes)};
 }
 
 // Order-preserving key: x <= y  <=>  key(x) <= key(y); -0 and +0 share a key.
@@ -412,9 +413,9 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W, co
                 s_cand[c * kMaeStage + slot] = make_uint2(rel, a);
             } else if (!s_over[c]) {
                 uint32_t* cnt = &W.state->cand_count[c];
-                if (*reinterpret_cast<volatile uint32_t*>(cnt) <= (uint32_t)kMaeCand) {
+                if (*reinterpret_cast<volatile uint32_t*>(cnt) <= W.cand_cap) {
                     const uint32_t gslot = atomicAdd(cnt, 1u);
-                    if (gslot < (uint32_t)kMaeCand) W.cand[c * kMaeCand + gslot] = make_uint2(rel, a);
+                    if (gslot < W.cand_cap) W.cand[(size_t)c * W.cand_cap + gslot] = make_uint2(rel, a);
                 } else {
                     s_over[c] = 1u;  // remembered per CTA: later samples of this level skip the look-up
                 }
@@ -539,8 +540,8 @@ mae_pass_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W, co
         for (int k = tid; k < kLevels * kMaeStage; k += kMaeThreads) {
             const int l = k / kMaeStage, i = k % kMaeStage;
             const uint32_t dst = s_gbase[l] + (uint32_t)i;
-            if ((uint32_t)i < min(s_ncand[l], (uint32_t)kMaeStage) && dst < (uint32_t)kMaeCand)
-                W.cand[l * kMaeCand + dst] = s_cand[k];
+            if ((uint32_t)i < min(s_ncand[l], (uint32_t)kMaeStage) && dst < W.cand_cap)
+                W.cand[(size_t)l * W.cand_cap + dst] = s_cand[k];
         }
     }
     if (FIRST) {
@@ -593,6 +594,7 @@ struct LaterCtx {
     volatile uint32_t* over;
     MaeState* state;
     uint2* gcand;
+    uint32_t cap;
 };
 template <bool COLLECT>
 __device__ __noinline__ void later_sample_fn(const LaterCtx* C, float xk, uint32_t a)
@@ -613,9 +615,9 @@ __device__ __noinline__ void later_sample_fn(const LaterCtx* C, float xk, uint32
             C->cand[c * kMaeStage + slot] = make_uint2(rel, a);
         } else if (!C->over[c]) {
             uint32_t* cnt = &C->state->cand_count[c];
-            if (*reinterpret_cast<volatile uint32_t*>(cnt) <= (uint32_t)kMaeCand) {
+            if (*reinterpret_cast<volatile uint32_t*>(cnt) <= C->cap) {
                 const uint32_t gslot = atomicAdd(cnt, 1u);
-                if (gslot < (uint32_t)kMaeCand) C->gcand[c * kMaeCand + gslot] = make_uint2(rel, a);
+                if (gslot < C->cap) C->gcand[(size_t)c * C->cap + gslot] = make_uint2(rel, a);
             } else {
                 C->over[c] = 1u;  // remembered per CTA: later samples of this level skip the look-up
             }
@@ -735,7 +737,7 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
     // One participating sample of a later pass: digit histogram and (COLLECT) candidate list.
     __shared__ LaterCtx s_ctx;
     if (tid == 0)
-        s_ctx = LaterCtx{s_xi, s_lvl, s_limit, s_lo, s_hi, s_ncand, s_cand, s_over, W.state, W.cand};
+        s_ctx = LaterCtx{s_xi, s_lvl, s_limit, s_lo, s_hi, s_ncand, s_cand, s_over, W.state, W.cand, W.cand_cap};
     __syncthreads();
     auto later_sample = [&](float xk, uint32_t a) { later_sample_fn<COLLECT>(&s_ctx, xk, a); };
 
@@ -853,8 +855,8 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
         for (int k = tid; k < kLevels * kMaeStage; k += kMaeThreads) {
             const int l = k / kMaeStage, i = k % kMaeStage;
             const uint32_t dst = s_gbase[l] + (uint32_t)i;
-            if ((uint32_t)i < min(s_ncand[l], (uint32_t)kMaeStage) && dst < (uint32_t)kMaeCand)
-                W.cand[l * kMaeCand + dst] = s_cand[k];
+            if ((uint32_t)i < min(s_ncand[l], (uint32_t)kMaeStage) && dst < W.cand_cap)
+                W.cand[(size_t)l * W.cand_cap + dst] = s_cand[k];
         }
     }
     if (FIRST) {
@@ -956,8 +958,8 @@ mae_resolve_kernel(MaeWs W)
         prefix = (prefix << (top - sh)) | (uint32_t)r.bin;
         top = sh;
     }
-    if (m <= (uint32_t)kMaeCand) {
-        const uint2* cand = W.cand + (size_t)l * kMaeCand;
+    if (m <= W.cand_cap) {
+        const uint2* cand = W.cand + (size_t)l * W.cand_cap;
         while (top > 0) {
             const int sh = max(top - kMaeDigitBits, 0);
             const uint32_t mask = (1u << (top - sh)) - 1u;
@@ -1505,9 +1507,9 @@ int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, co
 
 }  // namespace
 
-int mae_prepare(const EmArgs& a, void* d_ws, cudaStream_t st)
+int mae_prepare(const EmArgs& a, void* d_ws, size_t ws_bytes, cudaStream_t st)
 {
-    const MaeWs W = mae_ws(d_ws);
+    const MaeWs W = mae_ws(d_ws, ws_bytes);
     BOF4_CUDA_TRY(cudaMemsetAsync(W.state, 0, sizeof(MaeState), st));
     auto fire = [&](const EmTensors& T) -> int {
         if (a.w_dtype == BOF4_F32)
@@ -1522,9 +1524,9 @@ int mae_prepare(const EmArgs& a, void* d_ws, cudaStream_t st)
 }
 
 int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out, uint32_t skip_mask,
-                  bof4_em_stats* d_stats, double* d_err_slot, void* d_ws, cudaStream_t st)
+                  bof4_em_stats* d_stats, double* d_err_slot, void* d_ws, size_t ws_bytes, cudaStream_t st)
 {
-    const MaeWs W = mae_ws(d_ws);
+    const MaeWs W = mae_ws(d_ws, ws_bytes);
     mae_init_kernel<<<1, kMaeBins, 0, st>>>(d_levels_in, skip_mask, W);
     BOF4_CUDA_TRY(cudaGetLastError());
     // The candidate lists are filled by the first pass after which a region's candidates
@@ -1533,7 +1535,9 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
     // (The bf16 first pass narrows a region to one of its 140 ... 400 fine bins rather than to one
     // of 512 digit bins; a list that overflows all the same is finished by the later passes.)
     const bool bf16 = a.w_dtype == BOF4_BF16;
-    const int collect_pass = (a.n_total / kLevels / kMaeBins <= kMaeCand / 8) ? 1 : 2;
+    // fp32 first pass: one of 512 digit bins per region; bf16: one of its 140 ... 400 fine bins.
+    const int64_t expected = bf16 ? a.n_total / 1024 : a.n_total / kLevels / kMaeBins * 8;
+    const int collect_pass = (expected <= (int64_t)W.cand_cap) ? 1 : 2;
     MaeFinal fin{};
     fin.n_records = kEmGrid;
     fin.n_total = a.n_total;

@@ -35,7 +35,7 @@ size_t bof4_workspace_bytes(int op, int64_t n_max, int block_size, int metric)
     if (n_max < 0 || !bof4::valid_block_size(block_size)) return 0;
     if (op == BOF4_OP_EM) {
         if (metric < BOF4_METRIC_MSE || metric > BOF4_METRIC_MAE_NORMALIZED) return 0;
-        return bof4::em_workspace_bytes();
+        return bof4::em_workspace_bytes_for(n_max);
     }
     if (op == BOF4_OP_OPQ) return bof4::opq_layout(n_max).total;
     return 0;

@@ -27,11 +27,29 @@ constexpr int kFineStride = 4112;                // slots per half (below / not 
 constexpr int kFineSlots = 2 * kFineStride;
 constexpr size_t kEmMaeHistBytes = 66048;        // weight histogram, then count histogram (>= 8 * kFineSlots)
 static_assert(kEmMaeHistBytes >= (size_t)kFineSlots * 8 && kEmMaeHistBytes >= (size_t)16 * kMaeBins * 8, "histogram space");
-constexpr int kMaeCand = 1 << 16;          // candidate samples kept per level by the second pass
+constexpr int kMaeCand = 1 << 16;          // smallest candidate list per level (entries of 8 bytes)
+constexpr int kMaeCandMax = 1 << 17;       // largest one a workspace is sized for (entries are appended one by one)
 constexpr size_t kEmMaeCandBytes = (size_t)16 * kMaeCand * 8;
 constexpr size_t kEmMaeBytes = kEmMaeStateBytes + 2 * kEmMaeHistBytes + kEmMaeCandBytes;
 
+// Smallest workspace of the fit (any input size).
 inline size_t em_workspace_bytes() { return kEmMaeOffset + align_up(kEmMaeBytes, 256); }
+// Workspace for n_max weights in total: the candidate lists of the median selection grow with the
+// data (n_max / 512 entries per level, within [kMaeCand, kMaeCandMax]) so that the pass after the
+// first can collect a region's remaining candidates; with smaller lists one more data pass runs.
+inline size_t em_workspace_bytes_for(int64_t n_max)
+{
+    int64_t cand = n_max / 512;
+    cand = cand < kMaeCand ? kMaeCand : (cand > kMaeCandMax ? kMaeCandMax : cand);
+    return kEmMaeOffset + align_up(kEmMaeStateBytes + 2 * kEmMaeHistBytes + (size_t)16 * (size_t)cand * 8, 256);
+}
+// Entries per level that the candidate lists of a workspace of ws_bytes hold.
+inline uint32_t mae_cand_capacity(size_t ws_bytes)
+{
+    const size_t fixed = kEmMaeOffset + kEmMaeStateBytes + 2 * kEmMaeHistBytes;
+    const size_t cap = ws_bytes > fixed ? (ws_bytes - fixed) / (16 * 8) : 0;
+    return (uint32_t)(cap > (size_t)kMaeCandMax ? (size_t)kMaeCandMax : cap);
+}
 
 // ---------------------------------------------------------------- OPQ workspace
 // The weights are cut into tiles of kOpqTile elements (one warp iteration).  Each tile has a

@@ -571,6 +571,143 @@ opq_pass1_kernel(const void* __restrict__ w, int64_t n, const float* __restrict_
     }
 }
 
+// ---------------------------------------------------------------- OPQ pass 1, bf16 weights
+//
+// The same pass on the 64-byte-per-lane front end.  A warp iteration covers two tiles of
+// kOpqTile weights (lanes 0-15 and lanes 16-31), so the tile counts, staging slots and the gather
+// kernel are those of the generic pass.  The two tree sums of the block statistics (App. E) keep
+// the balanced-tree order: neighbours first inside the lane (32 weights, five levels, the upper
+// four on packed pairs), then the lane butterfly, then the warps of a wide block.
+
+// Balanced tree sum of the lane's 32 values given as 16 pairs {even, odd}: every addition is a
+// separate fp32 RN operation; levels two to five add two independent partial sums per instruction.
+__device__ __forceinline__ float lane_tree_sum32(const float2 (&t)[16])
+{
+    float a[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) a[k] = __fadd_rn(t[k].x, t[k].y);
+    float2 b[4], c[2];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)  // (a0 + a1, a2 + a3), (a4 + a5, a6 + a7), ...
+        b[k] = __fadd2_rn(make_float2(a[4 * k], a[4 * k + 2]), make_float2(a[4 * k + 1], a[4 * k + 3]));
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+        c[k] = __fadd2_rn(make_float2(b[2 * k].x, b[2 * k + 1].x), make_float2(b[2 * k].y, b[2 * k + 1].y));
+    const float2 d = __fadd2_rn(make_float2(c[0].x, c[1].x), make_float2(c[0].y, c[1].y));
+    return __fadd_rn(d.x, d.y);
+}
+
+template <int I>
+__device__ __forceinline__ float block_tree_sum32(float s, float* slot)
+{
+    constexpr int LPB = Geo32<I>::LPB, WPB = Geo32<I>::WPB;
+#pragma unroll
+    for (int off = 1; off < LPB; off <<= 1) s = __fadd_rn(s, __shfl_xor_sync(kFull, s, off));
+    if constexpr (WPB > 1) s = across_warps<WPB>(s, slot, [](float p, float q) { return __fadd_rn(p, q); });
+    return s;
+}
+
+// sigma_b * tau of the lane's block (two-pass formula in fp32, tree-ordered sums).
+template <int I>
+__device__ __forceinline__ float outlier_threshold32(const uint32_t (&u)[16], float tau, WideScratch* ws)
+{
+    float2 v[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) v[k] = make_float2(bf_lo(u[k]), bf_hi(u[k]));
+    const float mean = __fmul_rn(block_tree_sum32<I>(lane_tree_sum32(v), ws->a), 1.0f / (float)I);  // exact: I = 2^k
+    const float2 nm = make_float2(-mean, -mean);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        const float2 d = __fadd2_rn(v[k], nm);
+        v[k] = __fmul2_rn(d, d);
+    }
+    const float sigma = __fsqrt_rn(__fdiv_rn(block_tree_sum32<I>(lane_tree_sum32(v), ws->b), (float)(I - 1)));
+    return __fmul_rn(sigma, tau);
+}
+
+template <int I, bool SIGNED, class ST, bool QUANT>
+__global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
+opq_pass1_32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels, float tau,
+                    uint8_t* __restrict__ codes, void* __restrict__ scales, void* __restrict__ w_clean,
+                    int32_t* __restrict__ counts, unsigned long long* __restrict__ chunk_sum,
+                    int32_t* __restrict__ stage_idx, uint16_t* __restrict__ stage_val)
+{
+    static_assert(2 * kOpqTile == kWarpW32, "two tiles per warp iteration");
+    extern __shared__ __align__(16) unsigned char s_lut[];
+    __shared__ QuantShared32 S;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const RowMap32 map(n, kQRow32, threadIdx.x);
+    const int G = gridDim.x;
+    int r = blockIdx.x;
+    if (r >= map.rows) return;
+    auto fetch = [&](int rr) { return map.ok(rr) ? load_raw32(w, map.idx(rr)) : zero_raw32(); };
+    Raw32 a = fetch(r);
+    bool fast_ok = false;
+    uint32_t lut_base = 0u;
+    if (QUANT) {
+        const bool lut_ok = build_tables32(levels, S.xi, S.lv, s_lut, &S.info, [](int base) { return (uint32_t)base; });
+        fast_ok = lut_ok && !S.info.tiny;
+        lut_base = lut_lane_base(s_lut, lane);
+    }
+    for (; r < map.rows; r += G) {
+        const Raw32 next = fetch(r + G);
+        const int64_t idx = map.idx(r);
+        const bool ok = map.ok(r);
+        // this lane's tile: lanes 0-15 the first, lanes 16-31 the second tile of the warp row
+        const int64_t tile = ((int64_t)r * (kQThreads / 32) + warp) * 2 + (lane >> 4);
+        const bool tile_ok = tile * kOpqTile < n;  // uniform over the half warp
+        uint32_t u[16];
+        words_of(a, u);
+        float mx, mn;
+        lane_minmax32(u, mx, mn);
+        const float thr = outlier_threshold32<I>(u, tau, &S.wide);
+        // A lane can only hold an outlier if its largest magnitude exceeds the threshold, so the
+        // per-element test runs only in warps where some lane does (a NaN maximum also enters).
+        const bool maybe = !(fmaxf(mx, -mn) <= thr);
+        int total_half = 0;
+        if (__any_sync(kFull, maybe)) {
+            unsigned o = 0u;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                o |= (fabsf(bf_lo(u[k])) > thr) ? (1u << (2 * k)) : 0u;
+                o |= (fabsf(bf_hi(u[k])) > thr) ? (2u << (2 * k)) : 0u;
+            }
+            if (__any_sync(kFull, o != 0u)) {
+                int total;
+                int pos = warp_excl_scan(__popc(o), lane, total);
+                const int lower = __shfl_sync(kFull, pos, 16);  // outliers of lanes 0-15
+                total_half = (lane >> 4) ? total - lower : lower;
+                if (lane >> 4) pos -= lower;
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        if ((o >> (2 * k + h)) & 1u) {
+                            if (pos < kOpqStage) {
+                                stage_idx[tile * kOpqStage + pos] = (int32_t)(idx + 2 * k + h);
+                                stage_val[tile * kOpqStage + pos] = (uint16_t)(h ? (u[k] >> 16) : (u[k] & 0xffffu));
+                            }
+                            ++pos;
+                            u[k] &= h ? 0x0000ffffu : 0xffff0000u;  // the outlier becomes +0
+                        }
+                }
+                if ((lane & 15) == 0 && total_half > 0)
+                    atomicAdd(&chunk_sum[tile / kOpqChunk], (unsigned long long)total_half);  // integer: order-free
+                lane_minmax32(u, mx, mn);  // of the cleaned weights
+            }
+        }
+        if ((lane & 15) == 0 && tile_ok) counts[tile] = total_half;
+        if (QUANT) {
+            quantize_row32<I, SIGNED, ST>(u, mx, mn, idx, ok, fast_ok, lut_base, &S, codes, scales);
+        } else if (w_clean != nullptr && ok) {
+            uint16_t* dst = static_cast<uint16_t*>(w_clean) + idx;
+            st_stream256(dst, Raw8{{u[0], u[1], u[2], u[3], u[4], u[5], u[6], u[7]}});
+            st_stream256(dst + 16, Raw8{{u[8], u[9], u[10], u[11], u[12], u[13], u[14], u[15]}});
+        }
+        a = next;
+    }
+}
+
 // Pass 2: every tile's staged outliers are copied to their final, globally ascending position;
 // a tile with more than kOpqStage outliers is re-derived from the weights by one warp.  Each
 // CTA owns one chunk of tiles; its first output position is the sum of the earlier chunks'
@@ -1060,13 +1197,23 @@ int launch_opq(const char* fn, const void* d_w, int w_dtype, int64_t n, int bloc
         stage_idx = reinterpret_cast<int32_t*>(ws + Lw.stage_idx);
         stage_val = reinterpret_cast<uint16_t*>(ws + Lw.stage_val);
         BOF4_CUDA_TRY(cudaMemsetAsync(chunk_sum, 0, (size_t)Lw.chunks * 8, st));
-        BOF4_DISPATCH_WS(w_dtype, scale_dtype,
+        if (w_dtype == BOF4_BF16) {
+            const int grid32 = grid_for((n_whole + kQRow32 - 1) / kQRow32, kQCtasPerSm);
+            BOF4_DISPATCH_ST(scale_dtype,
+                BOF4_DISPATCH_I(block_size,
+                    BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                        { constexpr auto kern = opq_pass1_32_kernel<I_, SG, ST, QUANT>;
+                          if ((rc = ensure_dynamic_smem<kern>(kLutBytes))) return rc;
+                          kern<<<grid32, kQThreads, smem, st>>>(d_w, n_whole, d_codebook, tau, d_codes, d_scales,
+                                                                d_w_clean, counts, chunk_sum, stage_idx, stage_val); })));
+        } else {
             BOF4_DISPATCH_I(block_size,
                 BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
-                    { constexpr auto kern = opq_pass1_kernel<DT, I_, SG, ST, QUANT>;
+                    { constexpr auto kern = opq_pass1_kernel<F32, I_, SG, F32, QUANT>;
                       if ((rc = ensure_dynamic_smem<kern>(kLutBytes))) return rc;
                       kern<<<grid, kQThreads, smem, st>>>(d_w, n_whole, d_codebook, tau, d_codes, d_scales, d_w_clean,
-                                                          counts, chunk_sum, stage_idx, stage_val); })));
+                                                          counts, chunk_sum, stage_idx, stage_val); }));
+        }
         BOF4_CUDA_TRY(cudaGetLastError());
         if (w_dtype == BOF4_F32) {
             BOF4_DISPATCH_I(block_size, (opq_gather_kernel<F32, I_><<<(int)Lw.chunks, 256, 0, st>>>(

@@ -430,16 +430,22 @@ def test_mae_candidate_list_overflow_takes_the_later_data_passes(bof4):
     assert lv.cpu().numpy()[11] == ref["median"][11]
 
 
-def test_mae_above_2p26_weights_collects_candidates_one_pass_later(bof4):
-    """Up to 2^26 weights the second data pass fills the candidate lists; beyond that a level's
-    candidates would not fit after one digit, so the third pass collects.  Just above the limit
-    the medians must still be the oracle's, bit for bit (the smaller cases of this file cover the
-    other choice)."""
+def test_mae_with_the_smallest_workspace_collects_candidates_one_pass_later(bof4):
+    """The candidate lists of the median selection live in the workspace and grow with the size
+    asked for; with the smallest workspace the library accepts, a region's candidates do not fit
+    after the first pass of 2^26 weights, one more data pass runs before they are collected, and
+    the medians must still be the oracle's, bit for bit (the other tests use the default size)."""
+    from paper_2505_06653_b200 import binding as b
     I, n = 64, (1 << 26) + (1 << 16)
     w = workloads.gaussian_student_mixture(n, 0.02, 0.01, 4, 302, torch.bfloat16)
     ref = oracle.em_accumulate_mae(w, I, 1, LV_INIT)
-    got = bof4.bof4_em_step([w.cuda()], I, 1, bof4.METRIC_MAE, LV_INIT)
-    _check_mae_stats(got, ref, LV_INIT)
+    small = b.bof4_workspace_bytes(b.OP_EM, 0, I, b.METRIC_MAE)
+    assert small < b.bof4_workspace_bytes(b.OP_EM, n, I, b.METRIC_MAE)
+    wd = w.cuda()
+    for nbytes in (small, None):
+        ws = None if nbytes is None else torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        got = bof4.bof4_em_step([wd], I, 1, bof4.METRIC_MAE, LV_INIT, workspace=ws)
+        _check_mae_stats(got, ref, LV_INIT)
 
 
 # --------------------------------------------------------------------------- blocks wider than a warp
