@@ -12,9 +12,9 @@
  *    enqueued on that stream and the call returns without synchronising; outputs are valid once
  *    the stream has reached the end of the enqueued work.
  *  - Weights are a flattened tensor of n elements cut into B = n / block_size contiguous blocks
- *    (Sec. 2.1).  block_size is a power of two from 32 to 4096.  The EM entry points and
- *    opq_split_static need n to be a multiple of it.  bof4_quantize, bof4_dequantize, opq_split
- *    and bof4_quantize_opq also take a ragged tensor: its last block is simply shorter (its own
+ *    (Sec. 2.1).  block_size is a power of two from 32 to 4096.  opq_split_static and the gemv
+ *    need n (cols) to be a multiple of it.  Every other entry point, the codebook fit
+ *    included, also takes a ragged tensor: its last block is simply shorter (its own
  *    maximum; its own mean and deviation over its own length, the two tree sums padded with
  *    zeros to the next power of two; a one-weight block has no outliers), there are
  *    ceil(n / block_size) block constants and (n + 1) / 2 code bytes, and a code byte that holds a
@@ -117,7 +117,9 @@ BOF4_API size_t bof4_workspace_bytes(int op, int64_t n_max, int block_size, int 
  * One E+M accumulation pass with the codebook held fixed (Sec. 3.2; Eq. 6 or Eq. 8 with the
  * error of App. B.3 in the un-normalised weight domain) over the union of n_tensors tensors.
  *   h_w       host array of n_tensors DEVICE pointers to the tensors (dtype w_dtype each)
- *   h_n       host array of n_tensors element counts, each a multiple of block_size
+ *   h_n       host array of n_tensors element counts (any length; every tensor is cut into blocks
+ *             from its own start, and a length that is not a multiple of block_size ends in a
+ *             shorter block with its own constant: blocks never run across two tensors)
  *   d_codebook  [16] fp32 levels, read only
  *   d_stats   out: one bof4_em_stats record
  *   d_ws      workspace of at least bof4_workspace_bytes(BOF4_OP_EM, max_t h_n[t], ...)

@@ -154,42 +154,54 @@ def bf16_bits_to_f32(h: np.ndarray) -> np.ndarray:
     return out.reshape(h.shape)
 
 
+def _segments(w):
+    """A tensor or a list of tensors -> (concatenated fp32 data, int64 lengths).  Every tensor is
+    cut into blocks from its own start; a length that is not a multiple of the block size ends
+    in a shorter block."""
+    ws = list(w) if isinstance(w, (list, tuple)) else [w]
+    parts = [as_f32(t) for t in ws]
+    seg = np.array([p.size for p in parts], np.int64)
+    data = np.ascontiguousarray(np.concatenate(parts)) if len(parts) != 1 else parts[0]
+    return data, seg
+
+
 def em_accumulate_mse(w, I: int, norm: int, xhat, normdom: bool = False):
-    """-> dict(s1[16] f64, s0[16] f64, count[16] u64, err_sum f64, n).  normdom: App. D variant."""
-    a = as_f32(w)
-    _check(a.size, I)
+    """-> dict(s1[16] f64, s0[16] f64, count[16] u64, err_sum f64, n).  normdom: App. D variant.
+    `w`: a tensor or a list of tensors (ragged lengths allowed)."""
+    a, seg = _segments(w)
+    _check(a.size, I, ragged=True)
     lv = _levels(xhat)
     s1 = np.zeros(16, np.float64)
     s0 = np.zeros(16, np.float64)
     cnt = np.zeros(16, np.uint64)
     err = ctypes.c_double(0.0)
-    fn = _load().orc_em_accumulate_mse_normdom if normdom else _load().orc_em_accumulate_mse
-    fn(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv), _p(s1), _p(s0), _p(cnt), ctypes.byref(err))
+    _load().orc_em_accumulate_mse_seg(_p(a), _p(seg), int(seg.size), I, norm, _p(lv), int(bool(normdom)), _p(s1),
+                                      _p(s0), _p(cnt), ctypes.byref(err))
     return dict(s1=s1, s0=s0, count=cnt, err_sum=err.value, n=a.size)
 
 
 def em_accumulate_mae(w, I: int, norm: int, xhat, normdom: bool = False):
     """-> dict(median[16] f32, wsum[16] f64, count[16] u64, err_sum f64, n).  normdom: App. D variant."""
-    a = as_f32(w)
-    _check(a.size, I)
+    a, seg = _segments(w)
+    _check(a.size, I, ragged=True)
     lv = _levels(xhat)
     med = np.zeros(16, np.float32)
     ws = np.zeros(16, np.float64)
     cnt = np.zeros(16, np.uint64)
     err = ctypes.c_double(0.0)
-    fn = _load().orc_em_accumulate_mae_normdom if normdom else _load().orc_em_accumulate_mae
-    fn(_p(a), ctypes.c_int64(a.size), I, norm, _p(lv), _p(med), _p(ws), _p(cnt), ctypes.byref(err))
+    _load().orc_em_accumulate_mae_seg(_p(a), _p(seg), int(seg.size), I, norm, _p(lv), int(bool(normdom)), _p(med),
+                                      _p(ws), _p(cnt), ctypes.byref(err))
     return dict(median=med, wsum=ws, count=cnt, err_sum=err.value, n=a.size)
 
 
 def fit(w, I: int, norm: int, metric: int, xhat, fixed_mask: int, iters: int):
     """-> (levels fp32[16], err_log f64[iters])."""
-    a = as_f32(w)
-    _check(a.size, I)
+    a, seg = _segments(w)
+    _check(a.size, I, ragged=True)
     lv = _levels(xhat)
     log = np.zeros(max(iters, 1), np.float64)
-    _load().orc_fit(_p(a), ctypes.c_int64(a.size), I, norm, metric, _p(lv),
-                    ctypes.c_uint32(fixed_mask), iters, _p(log))
+    _load().orc_fit_seg(_p(a), _p(seg), int(seg.size), I, norm, metric, _p(lv),
+                        ctypes.c_uint32(fixed_mask), iters, _p(log))
     return lv, log[:iters]
 
 

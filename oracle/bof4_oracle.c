@@ -129,6 +129,29 @@ static int block_len(int64_t n, int I, int64_t b)
     return (int)(left < I ? left : I);
 }
 
+/* The blocks of a list of tensors laid out one after the other: every tensor is cut into blocks
+ * of I weights from its own start, its last block being shorter when its length is not a multiple
+ * of I (a block never spans two tensors).  Returns the number of blocks; off[b] is the position
+ * of block b in the concatenated data, len[b] its length. */
+static int64_t build_blocks(const int64_t *seg, int n_seg, int I, int64_t **off, int **len)
+{
+    int64_t B = 0;
+    for (int s = 0; s < n_seg; ++s)
+        B += (seg[s] + I - 1) / I;
+    *off = malloc(sizeof(int64_t) * (size_t)(B > 0 ? B : 1));
+    *len = malloc(sizeof(int) * (size_t)(B > 0 ? B : 1));
+    int64_t b = 0, pos = 0;
+    for (int s = 0; s < n_seg; ++s) {
+        int64_t nb = (seg[s] + I - 1) / I;
+        for (int64_t k = 0; k < nb; ++k, ++b) {
+            (*off)[b] = pos + k * I;
+            (*len)[b] = block_len(seg[s], I, k);
+        }
+        pos += seg[s];
+    }
+    return B;
+}
+
 void orc_block_constants(const float *w, int64_t n, int I, int norm, float *m_out)
 {
     int64_t B = (n + I - 1) / I;
@@ -184,13 +207,22 @@ void orc_dequantize(const uint8_t *codes, const float *scales, int64_t n, int I,
 /* One expectation + accumulation pass with the levels held fixed (Eq. 6 and the first line
  * of the un-normalised-domain error, App. B.3):
  *   s1[l] = sum m^2 x,  s0[l] = sum m^2,  cnt[l] = K_l,  err = sum (w - m xhat(l))^2. */
-static void em_accumulate_mse_impl(const float *w, int64_t n, int I, int norm, const float *xhat,
-                                   int unit, double *s1, double *s0, uint64_t *cnt, double *err);
+static void em_accumulate_mse_impl(const float *w, const int64_t *seg, int n_seg, int I, int norm,
+                                   const float *xhat, int unit, double *s1, double *s0, uint64_t *cnt,
+                                   double *err);
 
 void orc_em_accumulate_mse(const float *w, int64_t n, int I, int norm, const float *xhat,
                            double *s1, double *s0, uint64_t *cnt, double *err)
 {
-    em_accumulate_mse_impl(w, n, I, norm, xhat, 0, s1, s0, cnt, err);
+    em_accumulate_mse_impl(w, &n, 1, I, norm, xhat, 0, s1, s0, cnt, err);
+}
+
+/* The same over a list of n_seg tensors of seg[] weights each, stored one after the other. */
+void orc_em_accumulate_mse_seg(const float *w, const int64_t *seg, int n_seg, int I, int norm,
+                               const float *xhat, int unit, double *s1, double *s0, uint64_t *cnt,
+                               double *err)
+{
+    em_accumulate_mse_impl(w, seg, n_seg, I, norm, xhat, unit, s1, s0, cnt, err);
 }
 
 /* The same pass for the quantisation error of the NORMALISED weights (App. D, the plain-mean
@@ -198,15 +230,18 @@ void orc_em_accumulate_mse(const float *w, int64_t n, int I, int norm, const flo
 void orc_em_accumulate_mse_normdom(const float *w, int64_t n, int I, int norm, const float *xhat,
                                    double *s1, double *s0, uint64_t *cnt, double *err)
 {
-    em_accumulate_mse_impl(w, n, I, norm, xhat, 1, s1, s0, cnt, err);
+    em_accumulate_mse_impl(w, &n, 1, I, norm, xhat, 1, s1, s0, cnt, err);
 }
 
-static void em_accumulate_mse_impl(const float *w, int64_t n, int I, int norm, const float *xhat,
-                                   int unit, double *s1, double *s0, uint64_t *cnt, double *err)
+static void em_accumulate_mse_impl(const float *w, const int64_t *seg, int n_seg, int I, int norm,
+                                   const float *xhat, int unit, double *s1, double *s0, uint64_t *cnt,
+                                   double *err)
 {
     float xi[L - 1];
     orc_thresholds(xhat, xi);
-    int64_t B = n / I;
+    int64_t *boff;
+    int *blen;
+    int64_t B = build_blocks(seg, n_seg, I, &boff, &blen);
     int64_t nchunk = (B + ORC_CHUNK - 1) / ORC_CHUNK;
     double *p1 = calloc((size_t)nchunk * L, sizeof(double));
     double *p0 = calloc((size_t)nchunk * L, sizeof(double));
@@ -221,10 +256,11 @@ static void em_accumulate_mse_impl(const float *w, int64_t n, int I, int norm, c
         uint64_t *ac = pc + ch * L;
         double e = 0.0;
         for (int64_t b = b0; b < b1; ++b) {
-            const float *wb = w + b * I;
-            float m = block_constant(wb, I, norm);
+            const float *wb = w + boff[b];
+            const int Ib = blen[b];
+            float m = block_constant(wb, Ib, norm);
             double md = (double)m;
-            for (int i = 0; i < I; ++i) {
+            for (int i = 0; i < Ib; ++i) {
                 float x = normalise(wb[i], m);
                 int c = region_of(x, xi);
                 if (unit) {
@@ -262,6 +298,8 @@ static void em_accumulate_mse_impl(const float *w, int64_t n, int I, int norm, c
     free(p0);
     free(pc);
     free(pe);
+    free(boff);
+    free(blen);
 }
 
 /* ---------------------------------------------------------------- EM, MAE ------------- */
@@ -282,43 +320,59 @@ static int cmp_member(const void *p, const void *q)
  * the minimiser of f(xh) = sum a_k |x_k - xh| (objective of App. B.3, "MAE Optimization").
  *   med[l]  = that sample (unchanged input level when the region's total weight is 0),
  *   wsum[l] = total weight of the region, cnt[l] = K_l, err = sum |w - m xhat(l)|. */
-static void em_accumulate_mae_impl(const float *w, int64_t n, int I, int norm, const float *xhat,
-                                   int unit, float *med, double *wsum, uint64_t *cnt, double *err);
+static void em_accumulate_mae_impl(const float *w, const int64_t *seg, int n_seg, int I, int norm,
+                                   const float *xhat, int unit, float *med, double *wsum, uint64_t *cnt,
+                                   double *err);
 
 void orc_em_accumulate_mae(const float *w, int64_t n, int I, int norm, const float *xhat,
                            float *med, double *wsum, uint64_t *cnt, double *err)
 {
-    em_accumulate_mae_impl(w, n, I, norm, xhat, 0, med, wsum, cnt, err);
+    em_accumulate_mae_impl(w, &n, 1, I, norm, xhat, 0, med, wsum, cnt, err);
+}
+
+/* The same over a list of n_seg tensors of seg[] weights each, stored one after the other. */
+void orc_em_accumulate_mae_seg(const float *w, const int64_t *seg, int n_seg, int I, int norm,
+                               const float *xhat, int unit, float *med, double *wsum, uint64_t *cnt,
+                               double *err)
+{
+    em_accumulate_mae_impl(w, seg, n_seg, I, norm, xhat, unit, med, wsum, cnt, err);
 }
 
 /* Normalised-domain variant (App. D, the plain median): all weights 1, err = sum |x - xhat(l)|. */
 void orc_em_accumulate_mae_normdom(const float *w, int64_t n, int I, int norm, const float *xhat,
                                    float *med, double *wsum, uint64_t *cnt, double *err)
 {
-    em_accumulate_mae_impl(w, n, I, norm, xhat, 1, med, wsum, cnt, err);
+    em_accumulate_mae_impl(w, &n, 1, I, norm, xhat, 1, med, wsum, cnt, err);
 }
 
-static void em_accumulate_mae_impl(const float *w, int64_t n, int I, int norm, const float *xhat,
-                                   int unit, float *med, double *wsum, uint64_t *cnt, double *err)
+static void em_accumulate_mae_impl(const float *w, const int64_t *seg, int n_seg, int I, int norm,
+                                   const float *xhat, int unit, float *med, double *wsum, uint64_t *cnt,
+                                   double *err)
 {
     float xi[L - 1];
     orc_thresholds(xhat, xi);
-    int64_t B = n / I;
+    int64_t n = 0;
+    for (int s = 0; s < n_seg; ++s)
+        n += seg[s];
+    int64_t *boff;
+    int *blen;
+    int64_t B = build_blocks(seg, n_seg, I, &boff, &blen);
     uint8_t *code = malloc((size_t)(n > 0 ? n : 1));
     float *xs = malloc(sizeof(float) * (size_t)(n > 0 ? n : 1));
-    float *ms = malloc(sizeof(float) * (size_t)(B > 0 ? B : 1));
+    float *ms = malloc(sizeof(float) * (size_t)(n > 0 ? n : 1)); /* |m| of the block of every weight */
     double e = 0.0;
     for (int l = 0; l < L; ++l)
         cnt[l] = 0;
     for (int64_t b = 0; b < B; ++b) {
-        const float *wb = w + b * I;
-        float m = block_constant(wb, I, norm);
-        ms[b] = m;
-        for (int i = 0; i < I; ++i) {
+        const float *wb = w + boff[b];
+        const int Ib = blen[b];
+        float m = block_constant(wb, Ib, norm);
+        for (int i = 0; i < Ib; ++i) {
             float x = normalise(wb[i], m);
             int c = region_of(x, xi);
-            xs[b * I + i] = x;
-            code[b * I + i] = (uint8_t)c;
+            xs[boff[b] + i] = x;
+            ms[boff[b] + i] = fabsf(m);
+            code[boff[b] + i] = (uint8_t)c;
             cnt[c] += 1;
             e += unit ? fabs((double)x - (double)xhat[c])
                       : fabs((double)wb[i] - (double)m * (double)xhat[c]);
@@ -336,7 +390,7 @@ static void em_accumulate_mae_impl(const float *w, int64_t n, int I, int norm, c
         for (int64_t j = 0; j < n; ++j)
             if (code[j] == l) {
                 mem[k].x = xs[j];
-                mem[k].a = unit ? 1.0f : fabsf(ms[j / I]);
+                mem[k].a = unit ? 1.0f : ms[j];
                 ++k;
             }
         qsort(mem, (size_t)k, sizeof(member_t), cmp_member);
@@ -359,6 +413,8 @@ static void em_accumulate_mae_impl(const float *w, int64_t n, int I, int norm, c
     free(code);
     free(xs);
     free(ms);
+    free(boff);
+    free(blen);
 }
 
 /* ---------------------------------------------------------------- EM loop ------------- */
@@ -368,22 +424,36 @@ static void em_accumulate_mae_impl(const float *w, int64_t n, int I, int norm, c
  * error (MSE or MAE over all n weights, un-normalised domain) of the levels that ENTER
  * iteration t.  metric: 0 = MSE (Eq. 6), 1 = MAE (Eq. 8); 2 / 3 = the same criteria on the
  * normalised weights (App. D: plain mean / plain median, error measured on x). */
+void orc_fit_seg(const float *w, const int64_t *seg, int n_seg, int I, int norm, int metric,
+                 float *xhat, uint32_t fixed_mask, int iters, double *err_log);
+
 void orc_fit(const float *w, int64_t n, int I, int norm, int metric, float *xhat,
              uint32_t fixed_mask, int iters, double *err_log)
 {
+    orc_fit_seg(w, &n, 1, I, norm, metric, xhat, fixed_mask, iters, err_log);
+}
+
+/* The same over a list of tensors (every tensor cut into blocks from its own start; a tensor
+ * whose length is not a multiple of I ends in a shorter block with its own constant). */
+void orc_fit_seg(const float *w, const int64_t *seg, int n_seg, int I, int norm, int metric,
+                 float *xhat, uint32_t fixed_mask, int iters, double *err_log)
+{
+    int64_t n = 0;
+    for (int s = 0; s < n_seg; ++s)
+        n += seg[s];
     for (int t = 0; t < iters; ++t) {
         uint64_t cnt[L];
         double err;
         if (metric == 0 || metric == 2) {
             double s1[L], s0[L];
-            em_accumulate_mse_impl(w, n, I, norm, xhat, metric == 2, s1, s0, cnt, &err);
+            em_accumulate_mse_impl(w, seg, n_seg, I, norm, xhat, metric == 2, s1, s0, cnt, &err);
             for (int l = 0; l < L; ++l)
                 if (!((fixed_mask >> l) & 1u) && s0[l] > 0.0)
                     xhat[l] = (float)(s1[l] / s0[l]);
         } else {
             float med[L];
             double ws[L];
-            em_accumulate_mae_impl(w, n, I, norm, xhat, metric == 3, med, ws, cnt, &err);
+            em_accumulate_mae_impl(w, seg, n_seg, I, norm, xhat, metric == 3, med, ws, cnt, &err);
             for (int l = 0; l < L; ++l)
                 if (!((fixed_mask >> l) & 1u) && ws[l] > 0.0)
                     xhat[l] = med[l];

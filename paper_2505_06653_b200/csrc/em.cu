@@ -60,7 +60,7 @@ __device__ __forceinline__ void mse_combine(const double* partials, const MseTai
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     constexpr int NQ = kRecW2 + 1;            // quantities per record
-    constexpr int PER = (kEmGrid + 31) / 32;  // records per lane
+    constexpr int PER = (kEmRecords + 31) / 32;  // records per lane
     // Stage all records in shared memory first: coalesced, independent loads (every thread has
     // several in flight), instead of a chain of dependent L2 round trips per quantity.
     const int total = t.n_records * NQ;
@@ -142,6 +142,77 @@ em_mse_finalize_kernel(const double* partials, const MseTail t)
     __shared__ double s_q[kRecW2 + 1], s_corr[kLevels];
     __shared__ unsigned long long s_stage[kRecW2 + 1];  // the launcher passes a single (zero) record
     mse_combine(partials, t, s_q, s_corr, s_stage);
+}
+
+// The short last blocks of ragged tensors: one CTA, block after block.  Warp l sums the members
+// of region l (lane-strided, then the butterfly: a fixed order), in fp64 throughout, and the
+// result goes to a record of its own.
+template <class DT, bool SIGNED>
+__global__ void __launch_bounds__(kEmTailThreads)
+em_mse_tail_kernel(const EmTails Q, const float* __restrict__ levels, double* __restrict__ rec)
+{
+    __shared__ float s_w[4096], s_x[4096];
+    __shared__ unsigned char s_c[4096];
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ unsigned long long s_red[kEmTailThreads / 32];
+    __shared__ double s_w2[kLevels];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    static_assert(kEmTailThreads / 32 == kLevels, "one warp per level");
+    make_thresholds(levels, s_xi, s_lv, tid);
+    double a1 = 0.0, a0 = 0.0, aw = 0.0;
+    unsigned long long cnt = 0ull;
+    for (int q = 0; q < Q.count; ++q) {
+        const int len = Q.len[q];
+        const float m = load_short_block<DT, SIGNED>(Q.ptr[q], len, s_w, s_red);  // orders s_xi as well
+        for (int i = tid; i < len; i += kEmTailThreads) {
+            const float x = normalise(s_w[i], m);
+            s_x[i] = x;
+            s_c[i] = (unsigned char)region_of(x, s_xi);
+        }
+        __syncthreads();
+        const double md = (double)m, m2 = md * md;
+        for (int i = lane; i < len; i += 32) {
+            if (s_c[i] != warp) continue;
+            const double x = (double)s_x[i], w = (double)s_w[i];
+            if (Q.unit) {  // normalised-domain variant (App. D): unit weights, error on x
+                a1 += x;
+                a0 += 1.0;
+                aw += x * x;
+            } else {
+                a1 += m2 * x;
+                a0 += m2;
+                aw += w * w;
+            }
+            ++cnt;
+        }
+        __syncthreads();  // before the next block overwrites the arrays
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+        a1 += __shfl_xor_sync(kFull, a1, off);
+        a0 += __shfl_xor_sync(kFull, a0, off);
+        aw += __shfl_xor_sync(kFull, aw, off);
+        cnt += __shfl_xor_sync(kFull, cnt, off);
+    }
+    if (lane == 0) {
+        unsigned long long* rc = reinterpret_cast<unsigned long long*>(rec);
+        if (Q.accumulate) {
+            rec[kRecS1 + warp] += a1;
+            rec[kRecS0 + warp] += a0;
+            rc[kRecCnt + warp] += cnt;
+        } else {
+            rec[kRecS1 + warp] = a1;
+            rec[kRecS0 + warp] = a0;
+            rc[kRecCnt + warp] = cnt;
+        }
+        s_w2[warp] = aw;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        double e = 0.0;
+        for (int l = 0; l < kLevels; ++l) e += s_w2[l];
+        rec[kRecW2] = Q.accumulate ? rec[kRecW2] + e : e;
+    }
 }
 
 template <class DT, int I, bool SIGNED, bool COUNT>
@@ -644,11 +715,6 @@ int check_em(const char* fn, EmArgs& a, const void* d_codebook, void* d_ws, size
             set_error("%s: tensor %d is not 32-byte aligned", fn, t);
             return BOF4_ERR_INVALID_ARG;
         }
-        if (a.h_n[t] % a.block_size) {
-            set_error("%s: tensor %d has %lld elements, not a multiple of block_size %d", fn, t,
-                      (long long)a.h_n[t], a.block_size);
-            return BOF4_ERR_SHAPE;
-        }
         tot += a.h_n[t];
     }
     if (!d_codebook) {
@@ -697,7 +763,27 @@ template <bool COUNT>
 int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials, MseTail tail,
                      cudaStream_t st)
 {
-    tail.n_records = kEmGrid;
+    // Short last blocks first, into a record of their own (the only record when no tensor holds a
+    // whole block).
+    const bool tails = has_tails(a), whole = has_whole_blocks(a);
+    if (!whole) BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));
+    if (tails) {
+        double* rec = partials + (size_t)(whole ? kEmGrid : 0) * kEmRecordDoubles;
+        const bool sgn = a.norm == BOF4_NORM_SIGNED;
+        const int rc = for_each_tail_chunk(a, [&](const EmTails& Q) -> int {
+            if (a.w_dtype == BOF4_F32) {
+                if (sgn) em_mse_tail_kernel<F32, true><<<1, kEmTailThreads, 0, st>>>(Q, d_codebook, rec);
+                else em_mse_tail_kernel<F32, false><<<1, kEmTailThreads, 0, st>>>(Q, d_codebook, rec);
+            } else {
+                if (sgn) em_mse_tail_kernel<BF16, true><<<1, kEmTailThreads, 0, st>>>(Q, d_codebook, rec);
+                else em_mse_tail_kernel<BF16, false><<<1, kEmTailThreads, 0, st>>>(Q, d_codebook, rec);
+            }
+            BOF4_CUDA_TRY(cudaGetLastError());
+            return BOF4_OK;
+        });
+        if (rc) return rc;
+    }
+    tail.n_records = kEmGrid + (tails ? 1 : 0);
     tail.n_total = a.n_total;
     tail.levels_in = d_codebook;
     tail.ticket = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(partials) + kEmTicketOffset);
@@ -721,8 +807,7 @@ int enqueue_mse_pass(const EmArgs& a, const float* d_codebook, double* partials,
     const int rc = for_each_tensor_chunk(a, a.w_dtype == BOF4_BF16 ? EmGeo32<COUNT>::row : EmGeo<COUNT>::row, fire,
                                          &calls);
     if (rc) return rc;
-    if (calls == 0) {
-        BOF4_CUDA_TRY(cudaMemsetAsync(partials, 0, kEmPartialBytes, st));
+    if (calls == 0) {  // records zeroed above; record 0 holds the short blocks' sums, if any
         tail.enabled = 0;
         tail.n_records = 1;
         em_mse_finalize_kernel<<<1, 1024, 0, st>>>(partials, tail);

@@ -1375,6 +1375,97 @@ mae_select1_kernel(const float* __restrict__ levels, MaeWs W)
     }
 }
 
+// ---------------------------------------------------------------- short last blocks
+//
+// The short last blocks of ragged tensors take part in every data pass through one small CTA
+// that is enqueued before the pass's streaming kernel and adds to the same global histograms,
+// candidate lists and error records (integer sums: the order of the additions does not
+// matter).  mode selects what the pass needs of them.
+enum : int {
+    kTailAbsmax = 0,     // largest |w| (fixed-point reference of the weights)
+    kTailFirst = 1,      // first pass, per-region digit bins (fp32 weights)
+    kTailFirstFine = 2,  // first pass, uniform fine grid (bf16 weights)
+    kTailLater = 3       // later passes
+};
+
+template <class DT, bool SIGNED>
+__global__ void __launch_bounds__(kEmTailThreads)
+mae_tail_kernel(const EmTails Q, const float* __restrict__ levels, MaeWs W, int mode, int count, int collect,
+                int record)
+{
+    __shared__ float s_w[4096];
+    __shared__ float s_xi[kLevels], s_lv[kLevels];
+    __shared__ unsigned long long s_red[kEmTailThreads / 32];
+    __shared__ double s_err[kEmTailThreads / 32];
+    MaeState* S = W.state;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (mode == kTailAbsmax) {
+        uint32_t b = 0u;
+        for (int q = 0; q < Q.count; ++q)
+            for (int i = tid; i < Q.len[q]; i += kEmTailThreads)
+                b = max(b, __float_as_uint(fmaxf(0.0f, fabsf(short_block_elem<DT>(Q.ptr[q], i)))));  // fmaxf drops a NaN
+#pragma unroll
+        for (int off = 16; off; off >>= 1) b = max(b, __shfl_xor_sync(kFull, b, off));
+        if (lane == 0 && b) atomicMax(&S->max_bits, b);
+        return;
+    }
+    if (mode == kTailLater) {  // nothing left to resolve: uniform over the CTA
+        int any = 0;
+        for (int l = 0; l < kLevels; ++l) any |= S->top[l];
+        if (any <= 0) return;
+    }
+    make_thresholds(levels, s_xi, s_lv, tid);
+    __syncthreads();
+    const bool fine = mode == kTailFirstFine && !degenerate_codebook(s_xi);
+    const uint32_t max_bits = S->max_bits;
+    double err = 0.0;
+    for (int q = 0; q < Q.count; ++q) {
+        const int len = Q.len[q];
+        const float m = load_short_block<DT, SIGNED>(Q.ptr[q], len, s_w, s_red);
+        const uint32_t a = Q.unit ? 1u : fixed_weight(m, max_bits);
+        for (int i = tid; i < len; i += kEmTailThreads) {
+            const float w = s_w[i], x = normalise(w, m);
+            const int c = region_of(x, s_xi);
+            const uint32_t rel = order_key(x) - S->base[c];
+            const int top = S->top[c];
+            const int sh = max(top - kMaeDigitBits, 0);
+            if (mode == kTailLater) {
+                const uint32_t mask = (1u << (top - sh)) - 1u;
+                if (!(top > 0 && (uint32_t)((unsigned long long)rel >> top) == S->prefix[c] && rel <= S->limit[c])) continue;
+                atomicAdd(&W.hist[c * kMaeBins + ((rel >> sh) & mask)], (unsigned long long)a);
+                if (collect) {
+                    const uint32_t gslot = atomicAdd(&S->cand_count[c], 1u);
+                    if (gslot < W.cand_cap) W.cand[(size_t)c * W.cand_cap + gslot] = make_uint2(rel, a);
+                }
+                continue;
+            }
+            err += (double)(Q.unit ? fabsf(x - s_lv[c]) : fabsf(fmaf(-m, s_lv[c], w)));
+            int slot = -1;
+            if (fine) {
+                if (x == x) slot = fine_bin(x) + (c & 1) * kFineStride;  // a NaN has no place on the grid
+            } else if (mode == kTailFirstFine || top > 0) {  // per-region digit bins (degenerate codebook, fp32 weights)
+                slot = c * kMaeBins + (int)((rel >> sh) & (uint32_t)(kMaeBins - 1));
+            }
+            if (slot >= 0) {
+                atomicAdd(&W.hist[slot], (unsigned long long)a);
+                if (count) atomicAdd(&W.chist[slot], 1ull);
+            }
+        }
+        __syncthreads();  // before the next block overwrites s_w
+    }
+    if (mode == kTailLater) return;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) err += __shfl_xor_sync(kFull, err, off);
+    if (lane == 0) s_err[warp] = err;
+    __syncthreads();
+    if (tid == 0) {
+        double t = 0.0;
+        for (int k = 0; k < kEmTailThreads / 32; ++k) t += s_err[k];
+        double* rec = W.partials + (size_t)record * kEmRecordDoubles;
+        rec[0] = Q.accumulate ? rec[0] + t : t;
+    }
+}
+
 // ---------------------------------------------------------------- level update
 
 __global__ void __launch_bounds__(256)
@@ -1507,10 +1598,31 @@ int dispatch_pass(const EmArgs& a, const EmTensors& T, const float* d_levels, co
 
 }  // namespace
 
+namespace {
+// The short last blocks' part of a pass (see mae_tail_kernel).
+int enqueue_tails(const EmArgs& a, const float* d_levels, const MaeWs& W, int mode, bool count, bool collect,
+                  cudaStream_t st)
+{
+    const bool sg = a.norm == BOF4_NORM_SIGNED;
+    return for_each_tail_chunk(a, [&](const EmTails& Q) -> int {
+        if (a.w_dtype == BOF4_F32) {
+            if (sg) mae_tail_kernel<F32, true><<<1, kEmTailThreads, 0, st>>>(Q, d_levels, W, mode, count, collect, kEmGrid);
+            else mae_tail_kernel<F32, false><<<1, kEmTailThreads, 0, st>>>(Q, d_levels, W, mode, count, collect, kEmGrid);
+        } else {
+            if (sg) mae_tail_kernel<BF16, true><<<1, kEmTailThreads, 0, st>>>(Q, d_levels, W, mode, count, collect, kEmGrid);
+            else mae_tail_kernel<BF16, false><<<1, kEmTailThreads, 0, st>>>(Q, d_levels, W, mode, count, collect, kEmGrid);
+        }
+        BOF4_CUDA_TRY(cudaGetLastError());
+        return BOF4_OK;
+    });
+}
+}  // namespace
+
 int mae_prepare(const EmArgs& a, void* d_ws, size_t ws_bytes, cudaStream_t st)
 {
     const MaeWs W = mae_ws(d_ws, ws_bytes);
     BOF4_CUDA_TRY(cudaMemsetAsync(W.state, 0, sizeof(MaeState), st));
+    if (const int rc = enqueue_tails(a, nullptr, W, kTailAbsmax, false, false, st)) return rc;
     auto fire = [&](const EmTensors& T) -> int {
         if (a.w_dtype == BOF4_F32)
             mae_absmax_kernel<F32><<<kEmGrid, kMaeThreads, 0, st>>>(T, W.state);
@@ -1539,7 +1651,8 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
     const int64_t expected = bf16 ? a.n_total / 1024 : a.n_total / kLevels / kMaeBins * 8;
     const int collect_pass = (expected <= (int64_t)W.cand_cap) ? 1 : 2;
     MaeFinal fin{};
-    fin.n_records = kEmGrid;
+    const bool tails = has_tails(a);
+    fin.n_records = kEmGrid + (tails ? 1 : 0);
     fin.n_total = a.n_total;
     fin.levels_in = d_levels_in;
     fin.levels_out = d_levels_out;
@@ -1561,10 +1674,15 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
             return dispatch_pass(a, T, d_levels_in, W, p, p == collect_pass, first && d_stats != nullptr,
                                  fused ? &fin : nullptr, st);
         };
+        if (first && !has_whole_blocks(a)) BOF4_CUDA_TRY(cudaMemsetAsync(W.partials, 0, kEmPartialBytes, st));
+        if (tails) {
+            const int mode = first ? (bf16 ? kTailFirstFine : kTailFirst) : kTailLater;
+            if (const int rc = enqueue_tails(a, d_levels_in, W, mode, first && d_stats != nullptr, p == collect_pass, st))
+                return rc;
+        }
         int calls = 0;
         const int rc = for_each_tensor_chunk(a, bf16 ? kMaeThreads * kLW : kMaeRow, fire, &calls);
         if (rc) return rc;
-        if (first && calls == 0) BOF4_CUDA_TRY(cudaMemsetAsync(W.partials, 0, kEmPartialBytes, st));
         if (first32) {
             mae_select1_kernel<<<kLevels, 1024, 0, st>>>(d_levels_in, W);
             BOF4_CUDA_TRY(cudaGetLastError());

@@ -13,7 +13,8 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // [kEmMaeOffset, +kEmMaeBytes)    weighted-median selection state and histograms (MAE)
 constexpr int kEmGrid = 148;              // CTAs of the accumulation kernels (1 per SM)
 constexpr int kEmRecordDoubles = 64;      // 16 s1 + 16 s0 + 16 count + sum w^2, padded to 512 B
-constexpr size_t kEmPartialBytes = (size_t)kEmGrid * kEmRecordDoubles * 8;
+constexpr int kEmRecords = kEmGrid + 1;    // one per CTA, and one for the short last blocks of ragged tensors
+constexpr size_t kEmPartialBytes = (size_t)kEmRecords * kEmRecordDoubles * 8;
 constexpr size_t kEmTicketOffset = kEmPartialBytes;  // arrival counter of the accumulation CTAs (4 bytes)
 constexpr int kMaeDigitBits = 9;          // key bits resolved per selection pass
 constexpr int kMaeBins = 1 << kMaeDigitBits;  // bins per level and selection pass

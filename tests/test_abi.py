@@ -109,9 +109,10 @@ def test_argument_validation_happens_before_any_cuda_call(L):
     # EM
     ptrs = (ctypes.c_void_p * 1)(0x1000)
     ns = (ctypes.c_int64 * 1)(100)
-    assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, fake, ws, 1 << 40, None) == -2
-    assert b"multiple" in L.bof4_last_error()  # the fit needs whole blocks (quantise / OPQ take a ragged end)
-    ns[0] = 128
+    assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 48, 0, 0, fake, fake, ws, 1 << 40, None) == -2   # block size
+    ns[0] = -1
+    assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, fake, ws, 1 << 40, None) == -1
+    ns[0] = 100                      # a ragged length is accepted; the small workspace is refused next
     assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 0, fake, fake, ws, 8, None) == -4
     assert L.bof4_em_step(ptrs, ns, 1, b.BF16, 64, 0, 4, fake, fake, ws, 1 << 40, None) == -1
     assert L.bof4_em_step(ptrs, ns, 1, 7, 64, 0, 0, fake, fake, ws, 1 << 40, None) == -3

@@ -1,5 +1,5 @@
-"""Tensors that do not end on a block boundary: bof4_quantize, bof4_dequantize, opq_split and
-bof4_quantize_opq treat the last, shorter block as a block of its own (the paper only uses whole
+"""Tensors that do not end on a block boundary: bof4_quantize, bof4_dequantize, opq_split,
+bof4_quantize_opq and the codebook fit treat the last, shorter block as a block of its own (the paper only uses whole
 blocks; the reading is stated in the header and pinned in the oracle).  Bit-exact as everywhere."""
 import numpy as np
 import pytest
@@ -104,8 +104,92 @@ def test_ragged_outlier_list_capacity(bof4):
     assert np.array_equal(_bits(val), rval[:cap])
 
 
-def test_fit_still_needs_whole_blocks(bof4):
-    w = torch.zeros(100, dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(bof4.Bof4Error) as e:
-        bof4.bof4_em_step([w], 64, 0, bof4.METRIC_MSE, LV)
-    assert e.value.code == -2
+# --------------------------------------------------------------------------- ragged tensors in the fit
+
+RTOL = 1e-5
+
+
+def _ragged_list(I, dtype, seed, lens):
+    out = []
+    for k, n in enumerate(lens):
+        w = workloads.gaussian_student_mixture(max(n, 1), 0.02 * (1 + k % 3), 0.02, 3, seed + k, dtype)[:n].clone()
+        if n % I >= 2:
+            w[n - 1] = -0.5 if k % 2 else 0.5            # the short block's maximum is its own
+        out.append(w.contiguous())
+    return out
+
+
+def _check_stats(got, ref_mse, ref_mae, metric, lv):
+    if metric in (0, 2):
+        assert np.array_equal(got["count"], ref_mse["count"])
+        np.testing.assert_allclose(got["s1"], ref_mse["s1"], rtol=RTOL, atol=1e-6 * np.abs(ref_mse["s1"]).max())
+        np.testing.assert_allclose(got["s0"], ref_mse["s0"], rtol=RTOL)
+        np.testing.assert_allclose(got["err_sum"], ref_mse["err_sum"], rtol=RTOL)
+        assert got["n"] == ref_mse["n"]
+    else:
+        assert np.array_equal(got["count"], ref_mae["count"])
+        assert np.array_equal(got["median"], ref_mae["median"])
+        np.testing.assert_allclose(got["s0"], ref_mae["wsum"], rtol=RTOL)
+        np.testing.assert_allclose(got["err_sum"], ref_mae["err_sum"], rtol=RTOL)
+
+
+EM_LENS = [
+    lambda I: [5 * I + 7],
+    lambda I: [I - 1],
+    lambda I: [1, 2],                                   # no whole block anywhere
+    lambda I: [3 * I, 2 * I + 1, 0, I // 2, 4 * I + I - 1, 1],
+    lambda I: [40 * I + 3 + k for k in range(70)],      # more short blocks than one launch's table holds
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("norm", [0, 1])
+@pytest.mark.parametrize("metric", [0, 1, 2, 3])
+def test_em_step_on_ragged_tensor_lists(bof4, dtype, norm, metric):
+    """bof4_em_step over tensors whose lengths are not multiples of the block size: the short last
+    block of every tensor is a block of its own, in the sums (MSE) as in the weighted medians
+    (MAE), for both weight-domain and normalised-domain variants."""
+    for I in (32, 64, 1024, 4096):
+        for make in EM_LENS:
+            ws = _ragged_list(I, dtype, 40 + I, make(I))
+            got = bof4.bof4_em_step([w.cuda() for w in ws], I, norm, metric, LV)
+            ref_mse = oracle.em_accumulate_mse(ws, I, norm, LV, normdom=metric == 2) if metric in (0, 2) else None
+            ref_mae = oracle.em_accumulate_mae(ws, I, norm, LV, normdom=metric == 3) if metric in (1, 3) else None
+            _check_stats(got, ref_mse, ref_mae, metric, LV)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("metric", [0, 1])
+def test_em_step_ragged_over_many_rows(bof4, dtype, metric):
+    """Several rows per CTA of whole blocks plus short blocks: both kernels' contributions land
+    in the same statistics."""
+    I = 64
+    ws = _ragged_list(I, dtype, 77, [148 * 32768 * 2 + 64 * 11 + 37, (1 << 20) + 5, 63])
+    got = bof4.bof4_em_step([w.cuda() for w in ws], I, 1, metric, LV)
+    ref_mse = oracle.em_accumulate_mse(ws, I, 1, LV) if metric == 0 else None
+    ref_mae = oracle.em_accumulate_mae(ws, I, 1, LV) if metric == 1 else None
+    _check_stats(got, ref_mse, ref_mae, metric, LV)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("norm,mask", [(0, workloads.FIXED_BOF4), (1, workloads.FIXED_BOF4S)])
+@pytest.mark.parametrize("metric", [0, 1])
+def test_fit_on_ragged_tensor_lists(bof4, dtype, norm, mask, metric):
+    I = 64
+    ws = _ragged_list(I, dtype, 91, [3000 * I + 17, 41, 2000 * I, 555 * I + 63])
+    cb, log = bof4.bof4_fit_codebook([w.cuda() for w in ws], I, norm, metric, LV, mask, 8)
+    rcb, rlog = oracle.fit(ws, I, norm, metric, LV, mask, 8)
+    np.testing.assert_allclose(cb.cpu().numpy(), rcb, rtol=RTOL, atol=1e-7)
+    np.testing.assert_allclose(log.cpu().numpy(), rlog, rtol=RTOL)
+
+
+def test_mae_ragged_with_late_candidate_collection(bof4):
+    """The smallest workspace moves the candidate collection of a 2^26-weight fit one pass back;
+    the short blocks' samples must reach the lists in that pass too."""
+    from paper_2505_06653_b200 import binding as b
+    I = 64
+    ws = _ragged_list(I, torch.bfloat16, 303, [(1 << 26) + (1 << 16) + 33, 31])
+    ref = oracle.em_accumulate_mae(ws, I, 1, LV)
+    small = torch.empty(b.bof4_workspace_bytes(b.OP_EM, 0, I, b.METRIC_MAE), dtype=torch.uint8, device="cuda")
+    got = bof4.bof4_em_step([w.cuda() for w in ws], I, 1, bof4.METRIC_MAE, LV, workspace=small)
+    _check_stats(got, None, ref, 1, LV)

@@ -663,3 +663,86 @@ def test_ragged_last_block_sigma_and_outliers():
         assert np.all(clean[idx] == 0) and clean.size == w.size
         if tail == 1:
             assert clean[2 * I] == np.float32(0.5)
+
+
+# --------------------------------------------------------------------------- ragged tensors in the fit
+
+
+def _by_hand_stats(w, I, norm, lv):
+    """E-step statistics written out with numpy from the definitions (Eq. 1/4 block constant,
+    Eq. 2 regions, Sec. 3.1 sums), block by block, every tensor cut from its own start."""
+    lv = np.asarray(lv, np.float32)
+    xi = ((lv[:-1] + lv[1:]) * np.float32(0.5)).astype(np.float32)
+    s1, s0, cnt = np.zeros(16), np.zeros(16), np.zeros(16, np.uint64)
+    xs, aw, cs = [], [], []
+    err2 = err1 = 0.0
+    for t in w:
+        for o in range(0, t.size, I):
+            blk = t[o:o + I]
+            k = int(np.argmax(np.abs(blk)))               # first of the largest magnitudes
+            m = np.float32(blk[k] if norm == SGN else abs(blk[k]))
+            x = (blk / m).astype(np.float32) if m != 0 else np.zeros_like(blk)
+            c = (xi[None, :] <= x[:, None]).sum(1)
+            md = float(m)
+            np.add.at(s1, c, md * md * x.astype(np.float64))
+            np.add.at(s0, c, md * md)
+            np.add.at(cnt, c, 1)
+            d = blk.astype(np.float64) - md * lv[c].astype(np.float64)     # w - m xhat (App. B.3)
+            err2 += float(np.sum(d ** 2))
+            err1 += float(np.sum(np.abs(d)))
+            xs.append(x), aw.append(np.full(blk.size, abs(md))), cs.append(c)
+    return s1, s0, cnt, err2, err1, np.concatenate(xs), np.concatenate(aw), np.concatenate(cs)
+
+
+@pytest.mark.parametrize("norm", [ABS, SGN])
+def test_fit_statistics_of_ragged_tensor_lists_by_hand(norm):
+    """Tensors whose lengths are not multiples of the block size: the last block of every tensor
+    is a block of its own (its own maximum), and blocks never run across two tensors.  Sums,
+    counts, errors and weighted medians against the definitions written out in numpy."""
+    rng = np.random.default_rng(21)
+    I = 32
+    lens = [3 * I + 5, 1, 2 * I, I - 1, 4 * I + 17]
+    w = [(rng.standard_normal(n) * rng.uniform(0.01, 0.1)).astype(np.float32) for n in lens]
+    lv = np.array(workloads.init_levels_7_0_8(), np.float32)
+    s1, s0, cnt, err2, err1, x, a, c = _by_hand_stats(w, I, norm, lv)
+    st = oracle.em_accumulate_mse(w, I, norm, lv)
+    assert np.array_equal(st["count"], cnt) and st["n"] == sum(lens)
+    np.testing.assert_allclose(st["s1"], s1, rtol=1e-12, atol=1e-18)
+    np.testing.assert_allclose(st["s0"], s0, rtol=1e-12)
+    np.testing.assert_allclose(st["err_sum"], err2, rtol=1e-12)
+    sa = oracle.em_accumulate_mae(w, I, norm, lv)
+    assert np.array_equal(sa["count"], cnt)
+    np.testing.assert_allclose(sa["err_sum"], err1, rtol=1e-12)
+    for l in range(16):
+        xs, ws = x[c == l].astype(np.float64), a[c == l]
+        if xs.size == 0:
+            assert sa["median"][l] == lv[l]
+            continue
+        np.testing.assert_allclose(sa["wsum"][l], ws.sum(), rtol=1e-12)
+        f = lambda v: np.sum(ws * np.abs(xs - v))
+        assert f(float(sa["median"][l])) <= min(f(v) for v in xs) * (1 + 1e-12)
+        assert sa["median"][l] in x[c == l]
+
+
+def test_ragged_fit_is_not_the_fit_of_the_concatenation():
+    """The planted mistake: cutting the CONCATENATED data into blocks (blocks running across
+    tensor boundaries) gives other block constants; and a ragged tensor equals its whole blocks
+    plus the short block fitted as a tensor of its own."""
+    rng = np.random.default_rng(22)
+    I = 64
+    a = (rng.standard_normal(5 * I + 9) * 0.02).astype(np.float32)
+    b = (rng.standard_normal(3 * I) * 0.05).astype(np.float32)
+    lv = TAB6[:, 4].astype(np.float32)
+    both = oracle.em_accumulate_mse([a, b], I, SGN, lv)
+    parts = [oracle.em_accumulate_mse(t, I, SGN, lv) for t in (a[:5 * I], a[5 * I:], b)]
+    assert np.array_equal(both["count"], sum(p["count"] for p in parts))
+    np.testing.assert_allclose(both["s1"], sum(p["s1"] for p in parts), rtol=1e-12, atol=1e-18)
+    np.testing.assert_allclose(both["s0"], sum(p["s0"] for p in parts), rtol=1e-12)
+    cat = np.concatenate([a, b])
+    pad = np.concatenate([cat, np.zeros(-cat.size % I, np.float32)])
+    wrong = oracle.em_accumulate_mse(pad, I, SGN, lv)
+    assert abs(wrong["s0"].sum() - both["s0"].sum()) > 1e-6 * both["s0"].sum()
+    # a whole fit over the list runs and never increases the error
+    for metric in (MSE, MAE):
+        cb, log = oracle.fit([a, b], I, SGN, metric, workloads.init_levels_7_0_8(), FIX4S, 6)
+        assert np.all(np.diff(log) <= 1e-15) and np.all(np.diff(cb) > 0)
