@@ -240,6 +240,32 @@ BOF4_API int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int s
                     void* d_out, int out_dtype, void* stream);
 
 /*
+ * Double quantisation of the block constants (Limitations; App. F).  The paper names the technique
+ * and the extra sign bit per block that signed normalisation needs; it fixes no format.  Here, in
+ * fp32: the constants of 256 consecutive blocks (fewer in the last group) share the group constant
+ * g = max |m|; with t = g / 255, block b keeps q_b = min(255, round-half-even(|m_b| / t)) (0 when
+ * t = 0) and, for norm = BOF4_NORM_SIGNED, its sign in bit (b mod 8) of byte (b div 8) of d_sign.
+ * The decoder's constant is m^_b = +-(t * q_b); |m^ - m| <= g / 510 up to fp32 rounding.  The 4-bit
+ * codes stay those formed with the exact constants, so the element of largest magnitude of a block
+ * is no longer reconstructed exactly.  Storage: 8 (+1) bits per block and 32 bits per group.
+ *   d_scales   device, n_blocks constants of scale_dtype, as written by the quantising calls
+ *   d_q        out, device, n_blocks bytes
+ *   d_group    out, device, ceil(n_blocks / 256) fp32
+ *   d_sign     out, device, ceil(n_blocks / 8) bytes; ignored (may be NULL) for BOF4_NORM_ABS
+ * One launch on `stream`, no workspace.  BOF4_ERR_INVALID_ARG / BOF4_ERR_DTYPE on bad arguments.
+ */
+BOF4_API int bof4_scales_compress(const void* d_scales, int scale_dtype, int64_t n_blocks, int norm,
+                         uint8_t* d_q, float* d_group, uint8_t* d_sign, void* stream);
+
+/*
+ * The decoding side of the double quantisation: d_scales_out[b] = m^_b (fp32, n_blocks values),
+ * to be passed to bof4_dequantize or bof4_gemv with scale_dtype = BOF4_F32.  d_sign = NULL:
+ * all constants positive (absolute normalisation).  One launch on `stream`.
+ */
+BOF4_API int bof4_scales_expand(const uint8_t* d_q, const float* d_group, const uint8_t* d_sign,
+                       int64_t n_blocks, float* d_scales_out, void* stream);
+
+/*
  * Matrix-vector product with the 4-bit matrix decoded on the fly: Eq. 3 fused into its consumer,
  * the operation behind the paper's token-generation timings (App. E.2), with the OPQ outliers
  * applied as a sparse correction (Sec. 3.3, decoding side).  W is rows x cols, row-major, quantised

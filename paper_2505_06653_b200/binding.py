@@ -50,7 +50,7 @@ def mae_launches_per_call(n_tensors: int, n_total: int, iters: int) -> int:
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_theoretical_codebook_batch",
-           "bof4_gemv", "bof4_outlier_count")
+           "bof4_gemv", "bof4_outlier_count", "bof4_scales_compress", "bof4_scales_expand")
 
 
 class Bof4Error(RuntimeError):
@@ -103,6 +103,10 @@ def lib() -> ctypes.CDLL:
         L.bof4_theoretical_codebook_batch.argtypes = [i32, vp, vp, vp, vp, vp, i32, vp, sz, vp]
         L.bof4_outlier_count.restype = i32
         L.bof4_outlier_count.argtypes = [vp, i64, vp, vp]
+        L.bof4_scales_compress.restype = i32
+        L.bof4_scales_compress.argtypes = [vp, i32, i64, i32, vp, vp, vp, vp]
+        L.bof4_scales_expand.restype = i32
+        L.bof4_scales_expand.argtypes = [vp, vp, vp, i64, vp, vp]
         L.bof4_opq_threshold.restype = ctypes.c_double
         L.bof4_opq_threshold.argtypes = [ctypes.c_double, i32]
         L.bof4_default_init.restype = i32
@@ -380,6 +384,31 @@ def bof4_outlier_count(n_out: torch.Tensor, capacity: int) -> int:
     with torch.cuda.device(n_out.device):
         _check(lib().bof4_outlier_count(_ptr(n_out), int(capacity), ctypes.byref(host), _stream()))
     return int(host.value)
+
+
+def bof4_scales_compress(scales: torch.Tensor, norm: int):
+    """Double quantisation of block constants -> (q uint8[B], group fp32[ceil(B/256)], sign uint8[ceil(B/8)] or None)."""
+    scales = _dev(scales, "scales")
+    B = scales.numel()
+    dev = scales.device
+    q = torch.empty(B, dtype=torch.uint8, device=dev)
+    g = torch.empty((B + 255) // 256, dtype=torch.float32, device=dev)
+    sign = torch.empty((B + 7) // 8, dtype=torch.uint8, device=dev) if norm == NORM_SIGNED else None
+    with torch.cuda.device(dev):
+        _check(lib().bof4_scales_compress(_ptr(scales), _dt(scales), B, norm, _ptr(q), _ptr(g),
+                                          _ptr(sign) if sign is not None else None, _stream()))
+    return q, g, sign
+
+
+def bof4_scales_expand(q: torch.Tensor, group: torch.Tensor, sign: Optional[torch.Tensor]) -> torch.Tensor:
+    """The decoder's fp32 block constants from their double-quantised form."""
+    q = _dev(q, "q")
+    out = torch.empty(q.numel(), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        _check(lib().bof4_scales_expand(_ptr(q), _ptr(_dev(group, "group")),
+                                        _ptr(_dev(sign, "sign")) if sign is not None else None, q.numel(),
+                                        _ptr(out), _stream()))
+    return out
 
 
 def bof4_quantize_opq(w: torch.Tensor, block_size: int, norm: int, levels, tau: float,

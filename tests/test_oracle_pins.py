@@ -746,3 +746,68 @@ def test_ragged_fit_is_not_the_fit_of_the_concatenation():
     for metric in (MSE, MAE):
         cb, log = oracle.fit([a, b], I, SGN, metric, workloads.init_levels_7_0_8(), FIX4S, 6)
         assert np.all(np.diff(log) <= 1e-15) and np.all(np.diff(cb) > 0)
+
+
+# --------------------------------------------------------------------------- double quantisation
+
+
+def test_double_quantisation_by_hand_and_bounds():
+    """8-bit uniform quantisation of |m| against the maximum of its group of 256 (the reading
+    stated in oracle/double_quant.py), with the sign bit the paper asks for under signed
+    normalisation (Limitations)."""
+    from oracle import double_quant as dq
+    # exact arithmetic: g = 255 -> t = 1, q = |m|
+    m = np.array([0.0, 1.0, -2.0, 255.0, -17.0, 100.0, 254.0, -3.0, 7.0], np.float32)
+    q, g, sign = dq.compress(m, True)
+    assert np.array_equal(q, [0, 1, 2, 255, 17, 100, 254, 3, 7]) and g.tolist() == [255.0]
+    assert sign.tolist() == [0b10010100, 0b0]                       # blocks 2, 4, 7 negative; block 8 positive
+    assert np.array_equal(dq.expand(q, g, sign, m.size), m)
+    # halves round to even: a / t = 0.5 -> 0, 1.5 -> 2, 2.5 -> 2
+    m = np.array([255.0, 0.5, 1.5, 2.5], np.float32)
+    assert dq.compress(m, False)[0].tolist() == [255, 0, 2, 2]
+    # random constants over three groups and a ragged fourth: error bound, signs, group maxima
+    rng = np.random.default_rng(31)
+    B = 3 * 256 + 57
+    m = (np.abs(rng.standard_normal(B)) * 0.05 + 0.01).astype(np.float32) * rng.choice([-1.0, 1.0], B).astype(np.float32)
+    m[256:512] *= np.float32(40.0)                                   # a group on another scale
+    q, g, sign = dq.compress(m, True)
+    assert g.size == 4 and sign.size == (B + 7) // 8
+    for k in range(4):
+        assert g[k] == np.abs(m[k * 256:(k + 1) * 256]).max()        # own maximum, not the neighbour's
+    mh = dq.expand(q, g, sign, B)
+    assert np.array_equal(np.signbit(mh), np.signbit(m))             # signs exactly
+    bound = np.repeat(g, 256)[:B].astype(np.float64) / 510.0
+    assert np.all(np.abs(mh.astype(np.float64) - m) <= bound * (1 + 1e-5))
+    assert np.abs(mh.astype(np.float64) - m).max() > 0.3 * bound.max()   # and it is a real quantiser
+    # fp64 formula round(255 a / g): identical except where fp32 rounding moves a tie
+    ref = np.rint(255.0 * np.abs(m).astype(np.float64) / np.repeat(g, 256)[:B])
+    assert np.abs(q.astype(np.int64) - ref).max() <= 1 and (q != ref).mean() < 1e-3
+    # unsigned: no sign array, magnitudes only; a zero group stays zero
+    q0, g0, s0 = dq.compress(np.zeros(300, np.float32), False)
+    assert s0 is None and not q0.any() and not g0.any()
+    assert not dq.expand(q0, g0, None, 300).any()
+
+
+def test_double_quantisation_changes_the_block_maximum():
+    """With exact constants the element of largest magnitude of a block is reconstructed exactly
+    (Sec. 3.1); after double quantisation only the LARGEST constant of a group comes back within
+    an fp32 rounding of itself, every other one moves by up to g/510, and with it the block's
+    maximum.  The codes stay those formed with the exact constant."""
+    from oracle import double_quant as dq
+    rng = np.random.default_rng(32)
+    I, B = 64, 512
+    w = (rng.standard_normal(B * I) * 0.02).astype(np.float32)
+    lv = TAB6[:, 4].astype(np.float32)
+    codes, m = oracle.quantize(w, I, SGN, lv)
+    q, g, sign = dq.compress(m, True)
+    mh = dq.expand(q, g, sign, B)
+    for k in range(2):
+        top = np.argmax(np.abs(m[k * 256:(k + 1) * 256])) + k * 256
+        assert q[top] == 255 and abs(float(mh[top]) - float(m[top])) <= 2.0 ** -22 * abs(float(m[top]))
+    assert (mh != m).mean() > 0.9
+    exact = oracle.dequantize(codes, m, I, lv)
+    dq_out = oracle.dequantize(codes, mh, I, lv)
+    peak = np.abs(w.reshape(B, I)).argmax(1) + np.arange(B) * I
+    assert np.array_equal(exact[peak], w[peak])                      # the property with exact constants
+    assert (dq_out[peak] != w[peak]).mean() > 0.9                    # and what double quantisation gives up
+    assert np.abs(dq_out - exact).max() <= np.abs(mh - m).max() * (1 + 1e-6)   # |xhat| <= 1
