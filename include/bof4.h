@@ -320,6 +320,24 @@ BOF4_API int bof4_theoretical_codebook_batch(int n_problems, const int* h_block_
                                     float* d_codebooks, int iters, void* d_ws, size_t ws_bytes,
                                     void* stream);
 
+/*
+ * Data-free codebook for ANY symmetric zero-mean weight density (Sec. 3.2 Eq. 5 / Eq. 7 before the
+ * Gaussian simplification; App. B.1 for the cdf of the normalised weights given the block maximum
+ * and the density of the maximum, App. B.2 for the centroid integrals).  p_W is passed as samples:
+ *   d_pdf    device, n_grid fp64 values p_W(w_j) at w_j = j * w_max / (n_grid - 1), j = 0 .. n_grid-1
+ *            (w >= 0 only; any positive scale: the samples are normalised to total mass 1 on
+ *            [-w_max, w_max]); w_max must cover the range of the block maximum
+ *   n_grid   3 ... 2^20
+ * The integrals INT_0^w p_W and INT_0^w u p_W(u) du are cumulative trapezoid sums on the grid,
+ * read between nodes by linear interpolation; the integrals over the block maximum are trapezoid
+ * sums on the same grid, all in fp64.  Other arguments as for bof4_theoretical_codebook.
+ *   d_ws     256 + 24 * n_grid bytes, 256-byte aligned
+ * One set-up launch and one small launch per iteration on `stream`; no host synchronisation.
+ */
+BOF4_API int bof4_theoretical_codebook_general(int block_size, int norm, int metric, const double* d_pdf,
+                                      int n_grid, double w_max, float* d_codebook, uint32_t fixed_mask,
+                                      int iters, void* d_ws, size_t ws_bytes, void* stream);
+
 /* ---- host helpers (no CUDA call) ---- */
 
 /* tau = F_M^{-1}(q) for unit-variance Gaussian weights, F_M(m) = (2 G(m) - 1)^I the CDF of the

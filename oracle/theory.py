@@ -1,4 +1,5 @@
-"""Theoretical (data-free) centroid rules for unit-variance Gaussian weights, by quadrature.
+"""Theoretical (data-free) centroid rules, by quadrature: unit-variance Gaussian weights
+(GaussianBlockModel) and any tabulated symmetric density (TabulatedBlockModel).
 
 TEST INFRASTRUCTURE ONLY.  Used to pin the data-driven oracle against the paper's claim that
 the Monte-Carlo centroid and the analytical centroid are equivalent (Sec. 3.2, App. B.2, App. C).
@@ -71,8 +72,65 @@ class GaussianBlockModel:
         return 2.0 * self.I * self._int((ndtr(m * hi) - ndtr(m * lo)) * self.core)
 
 
+class TabulatedBlockModel:
+    """The same centroid rules for ANY symmetric zero-mean weight density (Sec. 3.2 Eq. 5 and
+    Eq. 7 with App. B.1 / B.2: the cdf of X given M = m, the density of M, the conditional
+    expectation of X for fixed m), the density given as samples p_W(w_j) on the uniform grid
+    w_j = j * w_max / (len(pdf) - 1), j >= 0.
+
+    With F_W(w) = 1/2 + Fc(w), Fc(w) = INT_0^w p_W (odd), and H(w) = INT_0^w u p_W(u) du (even), the
+    density of M is 2I (2 Fc(m))^(I-1) p_W(m), the cdf of X given m on (-1, 1) is
+    (F_W(m x) - F_W(-m)) / (2 Fc(m)), and INT_R m x p_W(m x) dx = [H(m x)]_R / m, so that
+        MSE centroid = INT m [H(m x)]_lo^hi c(m) dm / INT m^2 [Fc(m x)]_lo^hi c(m) dm,
+        MAE centroid = the x with INT m [Fc(m x)]_lo^x c(m) dm = 1/2 INT m [Fc(m x)]_lo^hi c(m) dm,
+    c(m) = (2 Fc(m))^(I-2) p_W(m): the Gaussian formulas with G -> F_W and -g -> H.
+
+    Numerics: the samples are scaled to total mass 1 on [-w_max, w_max]; Fc and H are cumulative
+    trapezoid sums on the grid, evaluated between nodes by linear interpolation; the integrals
+    over m use the trapezoid rule on the same grid (w_max must cover the block maximum's range).
+    """
+
+    def __init__(self, I: int, w_max: float, pdf):
+        p = np.asarray(pdf, dtype=np.float64)
+        self.I = I
+        self.m = np.linspace(0.0, w_max, p.size)
+        self.dm = self.m[1] - self.m[0]
+        half = (p.sum() - 0.5 * (p[0] + p[-1])) * self.dm
+        p = p / (2.0 * half)
+        self.p = p
+        self.Fc = np.concatenate(([0.0], np.cumsum(0.5 * (p[1:] + p[:-1]) * self.dm)))
+        up = self.m * p
+        self.H = np.concatenate(([0.0], np.cumsum(0.5 * (up[1:] + up[:-1]) * self.dm)))
+        self.core = np.power(2.0 * self.Fc, I - 2) * p
+
+    def _Fc(self, w):
+        return np.sign(w) * np.interp(np.abs(w), self.m, self.Fc)
+
+    def _H(self, w):
+        return np.interp(np.abs(w), self.m, self.H)
+
+    def _int(self, f):
+        return (f.sum() - 0.5 * (f[0] + f[-1])) * self.dm
+
+    def mse_centroid(self, lo: float, hi: float) -> float:
+        m = self.m
+        num = self._int(m * (self._H(m * hi) - self._H(m * lo)) * self.core)
+        den = self._int(m * m * (self._Fc(m * hi) - self._Fc(m * lo)) * self.core)
+        return num / den
+
+    def _mae_mass(self, lo: float, x: float) -> float:
+        m = self.m
+        return self._int(m * (self._Fc(m * x) - self._Fc(m * lo)) * self.core)
+
+    mae_centroid = GaussianBlockModel.mae_centroid
+
+    def cont_prob(self, lo: float, hi: float) -> float:
+        m = self.m
+        return 2.0 * self.I * self._int((self._Fc(m * hi) - self._Fc(m * lo)) * self.core)
+
+
 def lloyd(I: int, signed: bool, metric: str, levels0, fixed_mask: int, iters: int,
-          model: GaussianBlockModel | None = None) -> np.ndarray:
+          model=None) -> np.ndarray:
     """Lloyd iteration with the theoretical centroid for every free level.
 
     Thresholds are midpoints.  Free levels must own a region inside [-1, 1): the outermost

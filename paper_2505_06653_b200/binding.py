@@ -50,7 +50,8 @@ def mae_launches_per_call(n_tensors: int, n_total: int, iters: int) -> int:
 EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_quantize",
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_theoretical_codebook_batch",
-           "bof4_gemv", "bof4_outlier_count", "bof4_scales_compress", "bof4_scales_expand")
+           "bof4_gemv", "bof4_outlier_count", "bof4_scales_compress", "bof4_scales_expand",
+           "bof4_theoretical_codebook_general")
 
 
 class Bof4Error(RuntimeError):
@@ -101,6 +102,9 @@ def lib() -> ctypes.CDLL:
         L.bof4_theoretical_codebook.argtypes = [i32, i32, i32, vp, ctypes.c_uint32, i32, vp, sz, vp]
         L.bof4_theoretical_codebook_batch.restype = i32
         L.bof4_theoretical_codebook_batch.argtypes = [i32, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+        L.bof4_theoretical_codebook_general.restype = i32
+        L.bof4_theoretical_codebook_general.argtypes = [i32, i32, i32, vp, i32, ctypes.c_double, vp, ctypes.c_uint32,
+                                                        i32, vp, sz, vp]
         L.bof4_outlier_count.restype = i32
         L.bof4_outlier_count.argtypes = [vp, i64, vp, vp]
         L.bof4_scales_compress.restype = i32
@@ -261,6 +265,23 @@ def bof4_theoretical_codebook(block_size: int, norm: int, metric: int, levels, f
     with torch.cuda.device(dev):
         _check(lib().bof4_theoretical_codebook(block_size, norm, metric, _ptr(cb), fixed_mask, iters,
                                                _ptr(ws), ws.numel(), _stream()))
+    return cb
+
+
+def bof4_theoretical_codebook_general(block_size: int, norm: int, metric: int, pdf, w_max: float, levels,
+                                      fixed_mask: int, iters: int, device="cuda") -> torch.Tensor:
+    """Data-free codebook for a symmetric density given as samples pdf[j] = p_W(j * w_max / (len - 1)).
+    -> levels fp32[16] on the device."""
+    dev = torch.device(device)
+    cb = _codebook(levels, dev).clone()
+    tab = torch.as_tensor(np.ascontiguousarray(pdf, dtype=np.float64)).to(dev) if not isinstance(pdf, torch.Tensor) \
+        else _dev(pdf.to(torch.float64), "pdf")
+    n = tab.numel()
+    ws = torch.empty(256 + 24 * n, dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().bof4_theoretical_codebook_general(block_size, norm, metric, _ptr(tab), n, float(w_max), _ptr(cb),
+                                                       fixed_mask, iters, _ptr(ws), ws.numel(), _stream()))
+        torch.cuda.current_stream(dev).synchronize()   # the table is a temporary of this call
     return cb
 
 

@@ -1,4 +1,5 @@
-// Data-free codebook design for Gaussian weights (Sec. 3.2 Eq. 5 and Eq. 7; App. B.2, "Simplified
+// Data-free codebook design (Sec. 3.2 Eq. 5 and Eq. 7), for Gaussian weights in closed form and,
+// further down, for any tabulated symmetric density.  Gaussian weights (Sec. 3.2 Eq. 5 and Eq. 7; App. B.2, "Simplified
 // Solution for Gaussian Network Weights" and "MAE Optimization"): Lloyd iterations whose
 // centroids are ratios (MSE) or roots (MAE) of one-dimensional integrals over the absolute
 // block maximum m, evaluated by Simpson quadrature in fp64.
@@ -122,6 +123,120 @@ theory_step_kernel(double* __restrict__ state, int flip, const TheoryBatch B)
     }
 }
 
+// ---------------------------------------------------------------- any symmetric weight density
+//
+// Eq. 5 and Eq. 7 before the Gaussian simplification (App. B.1: cdf of X given M = m, density of
+// M; App. B.2: centroid as a ratio of integrals over m, conditional expectation of X for fixed m).
+// The density p_W is given as samples on the uniform grid w_j = j h, j = 0 .. n-1 (w >= 0; p_W is
+// symmetric).  With Fc(w) = INT_0^w p_W (so F_W = 1/2 + Fc, odd) and H(w) = INT_0^w u p_W(u) du
+// (even), M has density 2I (2 Fc(m))^(I-1) p_W(m), INT_R m x p_W(m x) dx = [H(m x)]_R / m, and
+//   MSE centroid = INT m [H(m x)]_lo^hi c(m) dm / INT m^2 [Fc(m x)]_lo^hi c(m) dm,
+//   MAE centroid = the x with INT m [Fc(m x)]_lo^x c(m) dm = 1/2 INT m [Fc(m x)]_lo^hi c(m) dm,
+// c(m) = (2 Fc(m))^(I-2) p_W(m).  Fc and H are cumulative trapezoid sums on the grid (after
+// scaling the samples to total mass 1), read between nodes by linear interpolation; the
+// integrals over m are trapezoid sums on the same grid.
+
+struct DensityTable {
+    const double* fc;    // [n] Fc(w_j)
+    const double* hh;    // [n] H(w_j)
+    const double* core;  // [n] c(w_j) times the trapezoid weight of node j
+    int n;
+    double h, inv_h;
+};
+
+// Tables from the samples: one CTA.  ws: [n] fc, [n] hh, [n] core.
+__global__ void __launch_bounds__(kThThreads)
+theory_table_kernel(const double* __restrict__ pdf, int n, double h, int I, double* __restrict__ fc,
+                    double* __restrict__ hh, double* __restrict__ core)
+{
+    __shared__ double s_red[kThThreads / 32];
+    double part = 0.0;
+    for (int j = threadIdx.x; j < n; j += kThThreads) part += ((j == 0 || j == n - 1) ? 0.5 : 1.0) * pdf[j];
+    const double half_mass = cta_sum(part, s_red) * h;  // INT_0^wmax p
+    const double scale = (half_mass > 0.0) ? 0.5 / half_mass : 0.0;
+    if (threadIdx.x == 0) {  // cumulative sums in grid order
+        double a = 0.0;
+        fc[0] = 0.0;
+        for (int j = 1; j < n; ++j) {
+            a += 0.5 * (pdf[j] + pdf[j - 1]) * scale * h;
+            fc[j] = a;
+        }
+    }
+    if (threadIdx.x == 32) {
+        double a = 0.0;
+        hh[0] = 0.0;
+        for (int j = 1; j < n; ++j) {
+            a += 0.5 * (j * h * pdf[j] + (j - 1) * h * pdf[j - 1]) * scale * h;
+            hh[j] = a;
+        }
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < n; j += kThThreads)
+        core[j] = pow(2.0 * fc[j], (double)(I - 2)) * pdf[j] * scale * ((j == 0 || j == n - 1) ? 0.5 * h : h);
+}
+
+__device__ __forceinline__ double table_at(const double* __restrict__ t, const DensityTable& D, double w_abs)
+{
+    const double a = w_abs * D.inv_h;
+    int j = (int)a;
+    j = min(max(j, 0), D.n - 2);
+    const double lo = t[j];
+    return lo + (a - (double)j) * (t[j + 1] - lo);
+}
+__device__ __forceinline__ double fc_at(const DensityTable& D, double w)  // odd
+{
+    const double v = table_at(D.fc, D, fabs(w));
+    return w < 0.0 ? -v : v;
+}
+
+__global__ void __launch_bounds__(kThThreads)
+theory_general_step_kernel(double* __restrict__ state, int flip, int metric, uint32_t fixed_mask, const DensityTable D)
+{
+    __shared__ double s_red[kThThreads / 32];
+    const int l = blockIdx.x;
+    const double* levels_in = state + (flip ? kLevels : 0);
+    double* levels_out = state + (flip ? 0 : kLevels);
+    const double cur = levels_in[l];
+    if ((fixed_mask >> l) & 1u) {
+        if (threadIdx.x == 0) levels_out[l] = cur;
+        return;
+    }
+    double lo = (l > 0) ? 0.5 * (levels_in[l - 1] + cur) : -1.0;
+    double hi = (l < kLevels - 1) ? 0.5 * (cur + levels_in[l + 1]) : 1.0;
+    lo = fmin(fmax(lo, -1.0), 1.0);
+    hi = fmin(fmax(hi, -1.0), 1.0);
+    if (metric == BOF4_METRIC_MSE) {
+        double num = 0.0, den = 0.0;
+        for (int q = threadIdx.x; q < D.n; q += kThThreads) {
+            const double m = q * D.h, c = D.core[q];
+            num += m * (table_at(D.hh, D, fabs(m * hi)) - table_at(D.hh, D, fabs(m * lo))) * c;
+            den += m * m * (fc_at(D, m * hi) - fc_at(D, m * lo)) * c;
+        }
+        num = cta_sum(num, s_red);
+        den = cta_sum(den, s_red);
+        if (threadIdx.x == 0) levels_out[l] = (den > 0.0) ? num / den : cur;
+    } else {
+        auto mass = [&](double x) {
+            double part = 0.0;
+            for (int q = threadIdx.x; q < D.n; q += kThThreads) {
+                const double m = q * D.h;
+                part += m * (fc_at(D, m * x) - fc_at(D, m * lo)) * D.core[q];
+            }
+            return cta_sum(part, s_red);
+        };
+        const double half = 0.5 * mass(hi);
+        double a = lo, b = hi;
+        for (int it = 0; it < 60; ++it) {
+            const double x = 0.5 * (a + b);
+            if (mass(x) < half)
+                a = x;
+            else
+                b = x;
+        }
+        if (threadIdx.x == 0) levels_out[l] = (half > 0.0) ? 0.5 * (a + b) : cur;
+    }
+}
+
 // levels of problem p: codebooks[p][16] (fp32) <-> the current set of the fp64 state
 __global__ void theory_load_kernel(const float* __restrict__ codebooks, double* __restrict__ state)
 {
@@ -221,4 +336,44 @@ extern "C" int bof4_theoretical_codebook_batch(int n_problems, const int* h_bloc
         B.fixed_mask[p] = h_fixed_mask[p];
     }
     return run_theory("bof4_theoretical_codebook_batch", n_problems, B, d_codebooks, iters, d_ws, ws_bytes, stream);
+}
+
+extern "C" int bof4_theoretical_codebook_general(int block_size, int norm, int metric, const double* d_pdf,
+                                                 int n_grid, double w_max, float* d_codebook,
+                                                 uint32_t fixed_mask, int iters, void* d_ws, size_t ws_bytes,
+                                                 void* stream)
+{
+    using namespace bof4;
+    const char* fn = "bof4_theoretical_codebook_general";
+    const int rc = check_theory_problem(fn, block_size, norm, metric, fixed_mask);
+    if (rc) return rc;
+    if (!d_pdf || n_grid < 3 || n_grid > (1 << 20) || !(w_max > 0.0) || iters < 0 || !d_codebook) {
+        set_error("%s: NULL pointer, n_grid outside 3 ... 2^20, w_max <= 0 or negative iteration count", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    const size_t need = 256 + (size_t)3 * n_grid * sizeof(double);
+    if (!d_ws || ((uintptr_t)d_ws & 255u) || ws_bytes < need) {
+        set_error("%s: workspace NULL, not 256-byte aligned, or smaller than 256 + 24 * n_grid bytes", fn);
+        return BOF4_ERR_WORKSPACE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double* state = static_cast<double*>(d_ws);
+    double* fc = state + 32;
+    double* hh = fc + n_grid;
+    double* core = hh + n_grid;
+    const double h = w_max / (double)(n_grid - 1);
+    theory_table_kernel<<<1, kThThreads, 0, st>>>(d_pdf, n_grid, h, block_size, fc, hh, core);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    theory_load_kernel<<<1, 32, 0, st>>>(d_codebook, state);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    const DensityTable D{fc, hh, core, n_grid, h, 1.0 / h};
+    int flip = 0;
+    for (int t = 0; t < iters; ++t) {
+        theory_general_step_kernel<<<kLevels, kThThreads, 0, st>>>(state, flip, metric, fixed_mask, D);
+        BOF4_CUDA_TRY(cudaGetLastError());
+        flip ^= 1;
+    }
+    theory_store_kernel<<<1, 32, 0, st>>>(state, flip, d_codebook);
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
 }

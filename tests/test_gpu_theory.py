@@ -78,3 +78,55 @@ def test_batched_solver_equals_single_calls(bof4):
     assert bof4.bof4_theoretical_codebook_batch([], [], [], start, [], 3).shape == (0, 16)
     with pytest.raises(bof4.Bof4Error):
         bof4.bof4_theoretical_codebook_batch([64] * 129, [0] * 129, [0] * 129, start, [FIX4] * 129, 1)
+
+
+# --------------------------------------------------------------------------- tabulated densities
+
+
+def _density(name, n=20001):
+    if name == "gauss":
+        w = np.linspace(0.0, 12.0, n)
+        return 12.0, np.exp(-0.5 * w * w)
+    if name == "laplace":
+        w = np.linspace(0.0, 40.0, n)
+        return 40.0, 0.5 * np.exp(-w)
+    w = np.linspace(0.0, 400.0, n)                     # Student-t, 5 degrees of freedom (unnormalised)
+    return 400.0, (1.0 + w * w / 5.0) ** -3.0
+
+
+@pytest.mark.parametrize("name", ["gauss", "laplace", "student5"])
+@pytest.mark.parametrize("I", [32, 64, 500])
+@pytest.mark.parametrize("signed", [False, True])
+@pytest.mark.parametrize("metric", ["mse", "mae"])
+def test_general_density_solver_agrees_with_the_oracle(bof4, name, I, signed, metric):
+    """Eq. 5 / Eq. 7 for a tabulated p_W: the device solver against the oracle's tabulated model
+    on the same samples (both read the same table; levels within 1e-5 after three iterations)."""
+    w_max, pdf = _density(name, 20001 if name != "student5" else 80001)
+    mask = FIX4S if signed else FIX4
+    start = workloads.init_levels_7_0_8()
+    ref = theory.lloyd(I, signed, metric, start, mask, 3, theory.TabulatedBlockModel(I, w_max, pdf))
+    got = bof4.bof4_theoretical_codebook_general(I, bof4.NORM_SIGNED if signed else bof4.NORM_ABS,
+                                                 bof4.METRIC_MSE if metric == "mse" else bof4.METRIC_MAE,
+                                                 pdf, w_max, start, mask, 3).cpu().numpy()
+    assert np.abs(got - ref).max() < 1e-5
+    assert np.all(np.diff(got) > 0)
+
+
+def test_general_solver_with_a_gaussian_table_matches_the_gaussian_solver(bof4):
+    w_max, pdf = _density("gauss", 40001)
+    for norm, mask in ((bof4.NORM_ABS, FIX4), (bof4.NORM_SIGNED, FIX4S)):
+        for metric in (bof4.METRIC_MSE, bof4.METRIC_MAE):
+            a = bof4.bof4_theoretical_codebook_general(64, norm, metric, pdf, w_max, workloads.init_levels_7_0_8(),
+                                                       mask, 20).cpu().numpy()
+            b = bof4.bof4_theoretical_codebook(64, norm, metric, workloads.init_levels_7_0_8(), mask, 20).cpu().numpy()
+            assert np.abs(a - b).max() < 2e-6
+
+
+def test_general_solver_rejects_bad_arguments(bof4):
+    w_max, pdf = _density("gauss", 101)
+    with pytest.raises(bof4.Bof4Error):
+        bof4.bof4_theoretical_codebook_general(64, bof4.NORM_ABS, bof4.METRIC_MSE, pdf, -1.0, workloads.init_levels_7_0_8(),
+                                               FIX4, 1)
+    with pytest.raises(bof4.Bof4Error):          # the outermost levels must be fixed
+        bof4.bof4_theoretical_codebook_general(64, bof4.NORM_ABS, bof4.METRIC_MSE, pdf, w_max,
+                                               workloads.init_levels_7_0_8(), 0, 1)

@@ -811,3 +811,42 @@ def test_double_quantisation_changes_the_block_maximum():
     assert np.array_equal(exact[peak], w[peak])                      # the property with exact constants
     assert (dq_out[peak] != w[peak]).mean() > 0.9                    # and what double quantisation gives up
     assert np.abs(dq_out - exact).max() <= np.abs(mh - m).max() * (1 + 1e-6)   # |xhat| <= 1
+
+
+# --------------------------------------------------------------------------- general weight densities
+
+
+def test_tabulated_model_reproduces_the_gaussian_solver():
+    """Eq. 5 / Eq. 7 for a tabulated density, fed a Gaussian table, against the closed Gaussian
+    forms (boxed equations of App. B.2): centroids of single regions and a whole Lloyd run."""
+    w = np.linspace(0.0, 10.0, 20001)
+    tab = theory.TabulatedBlockModel(64, 10.0, np.exp(-0.5 * w * w))     # unnormalised on purpose
+    gau = theory.GaussianBlockModel(64)
+    for lo, hi in ((-1.0, -0.6), (-0.3, -0.1), (-0.04, 0.05), (0.2, 0.45), (0.6, 0.9)):
+        assert abs(tab.mse_centroid(lo, hi) - gau.mse_centroid(lo, hi)) < 2e-7
+        assert abs(tab.mae_centroid(lo, hi) - gau.mae_centroid(lo, hi)) < 2e-7
+        assert abs(tab.cont_prob(lo, hi) - gau.cont_prob(lo, hi)) < 2e-7
+    for signed, mask in ((False, FIX4), (True, FIX4S)):
+        for metric in ("mse", "mae"):
+            a = theory.lloyd(64, signed, metric, workloads.init_levels_7_0_8(), mask, 5, tab)
+            b = theory.lloyd(64, signed, metric, workloads.init_levels_7_0_8(), mask, 5, gau)
+            assert np.abs(a - b).max() < 5e-7
+
+
+@pytest.mark.parametrize("signed,norm,mask", [(False, ABS, FIX4), (True, SGN, FIX4S)])
+@pytest.mark.parametrize("metric", ["mse", "mae"])
+def test_tabulated_model_agrees_with_data_driven_fit_on_laplace_weights(signed, norm, mask, metric):
+    """A density that is not Gaussian: 2^24 Laplace samples.  One data-driven EM step (Eq. 6 /
+    Eq. 8) and one theoretical step (Eq. 5 / Eq. 7, p_W tabulated) from the same start agree
+    within Monte-Carlo noise, and the Gaussian model does NOT (the general formula is needed)."""
+    w = oracle.as_f32(workloads.laplace(1 << 24, 1.0, 321))
+    grid = np.linspace(0.0, 40.0, 40001)
+    tab = theory.TabulatedBlockModel(64, 40.0, 0.5 * np.exp(-grid))
+    start = workloads.init_levels_7_0_8()
+    theo = theory.lloyd(64, signed, metric, start, mask, 1, tab)
+    lv, _ = oracle.fit(w, 64, norm, MSE if metric == "mse" else MAE, start, mask, 1)
+    # the outer regions of the heavy-tailed density hold few samples: the median of region 1
+    # (some 1e4 members) moves by a few 1e-4 from sample to sample
+    assert np.abs(lv - theo).max() < (4e-4 if metric == "mse" else 1e-3)
+    gau = theory.lloyd(64, signed, metric, start, mask, 1, theory.GaussianBlockModel(64, points=4001))
+    assert np.abs(lv - gau).max() > 5e-3

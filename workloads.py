@@ -35,6 +35,13 @@ def gaussian(n: int, sigma: float, seed: int, dtype=torch.float32, device="cpu")
     return x.to(dtype)
 
 
+def laplace(n: int, b: float, seed: int, dtype=torch.float32, device="cpu") -> torch.Tensor:
+    """n samples of the Laplace density exp(-|w| / b) / (2 b) (inverse-cdf method)."""
+    u = torch.rand(n, generator=_gen(seed, device), dtype=torch.float64, device=device) - 0.5
+    w = -b * torch.sign(u) * torch.log1p(-2.0 * u.abs())
+    return w.to(dtype)
+
+
 def gaussian_student_mixture(n: int, sigma: float, frac_t: float, nu: int, seed: int,
                              dtype=torch.bfloat16, device="cpu") -> torch.Tensor:
     """(1-frac_t) N(0, sigma^2) + frac_t * sigma * Student-t(nu).
