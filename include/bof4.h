@@ -240,6 +240,23 @@ BOF4_API int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int s
                     void* d_out, int out_dtype, void* stream);
 
 /*
+ * bof4_quantize and bof4_dequantize (without an outlier list) over a list of tensors that share
+ * block size, normalisation, codebook and dtypes: the model-wide case, where a launch and a table
+ * set-up per matrix would cost as much as the matrix itself.  The rows of all tensors are dealt
+ * over one grid (64 tensors per launch); results are those of n_tensors single calls, bit for bit.
+ *   h_w / h_codes / h_scales / h_out   host arrays of n_tensors DEVICE pointers, one per tensor,
+ *                                      each with the size, alignment and meaning of the single call
+ *   h_n                                host array of n_tensors element counts (ragged lengths allowed)
+ * The host arrays are read before the call returns.
+ */
+BOF4_API int bof4_quantize_batch(const void* const* h_w, const int64_t* h_n, int n_tensors, int w_dtype,
+                        int block_size, int norm, const float* d_codebook, uint8_t* const* h_codes,
+                        void* const* h_scales, int scale_dtype, void* stream);
+BOF4_API int bof4_dequantize_batch(const uint8_t* const* h_codes, const void* const* h_scales, int scale_dtype,
+                          const int64_t* h_n, int n_tensors, int block_size, const float* d_codebook,
+                          void* const* h_out, int out_dtype, void* stream);
+
+/*
  * Double quantisation of the block constants (Limitations; App. F).  The paper names the technique
  * and the extra sign bit per block that signed normalisation needs; it fixes no format.  Here, in
  * fp32: the constants of 256 consecutive blocks (fewer in the last group) share the group constant

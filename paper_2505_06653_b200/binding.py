@@ -51,7 +51,7 @@ EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_qu
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_theoretical_codebook_batch",
            "bof4_gemv", "bof4_outlier_count", "bof4_scales_compress", "bof4_scales_expand",
-           "bof4_theoretical_codebook_general")
+           "bof4_theoretical_codebook_general", "bof4_quantize_batch", "bof4_dequantize_batch")
 
 
 class Bof4Error(RuntimeError):
@@ -107,6 +107,10 @@ def lib() -> ctypes.CDLL:
                                                         i32, vp, sz, vp]
         L.bof4_outlier_count.restype = i32
         L.bof4_outlier_count.argtypes = [vp, i64, vp, vp]
+        L.bof4_quantize_batch.restype = i32
+        L.bof4_quantize_batch.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
+        L.bof4_dequantize_batch.restype = i32
+        L.bof4_dequantize_batch.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, i32, vp]
         L.bof4_scales_compress.restype = i32
         L.bof4_scales_compress.argtypes = [vp, i32, i64, i32, vp, vp, vp, vp]
         L.bof4_scales_expand.restype = i32
@@ -146,6 +150,23 @@ def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
     return t
 
 
+_allocator = None
+
+
+def set_output_allocator(fn) -> None:
+    """Routes every buffer this binding allocates (outputs and workspaces) through
+    ``fn(numel, dtype, device, zero) -> tensor``; None restores plain torch allocation.  A test
+    harness uses it to surround each buffer with guard bands."""
+    global _allocator
+    _allocator = fn
+
+
+def _new(numel: int, dtype, device, zero: bool = False) -> torch.Tensor:
+    if _allocator is not None:
+        return _allocator(int(numel), dtype, torch.device(device), zero)
+    return (torch.zeros if zero else torch.empty)(int(numel), dtype=dtype, device=device)
+
+
 def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
@@ -168,7 +189,7 @@ def _workspace(op: int, n_max: int, block_size: int, metric: int, device) -> tor
     nbytes = lib().bof4_workspace_bytes(op, n_max, block_size, metric)
     if nbytes == 0:
         raise Bof4Error(-2, "bof4_workspace_bytes rejected the arguments")
-    return torch.empty(nbytes, dtype=torch.uint8, device=device)  # torch allocations are 512-B aligned
+    return _new(nbytes, torch.uint8, device)  # torch allocations are 512-B aligned
 
 
 # --------------------------------------------------------------------------- host helpers
@@ -218,7 +239,7 @@ def bof4_em_step(weights, block_size: int, norm: int, metric: int, levels,
     cb = _codebook(levels, dev)
     wsp = workspace if workspace is not None else _workspace(
         OP_EM, sum(w.numel() for w in ws), block_size, metric, dev)
-    stats = torch.zeros(ctypes.sizeof(EmStats), dtype=torch.uint8, device=dev)
+    stats = _new(ctypes.sizeof(EmStats), torch.uint8, dev, zero=True)
     with torch.cuda.device(dev):
         _check(lib().bof4_em_step(ptrs, sizes, len(ws), dt, block_size, norm, metric, _ptr(cb),
                                   _ptr(stats), _ptr(wsp), wsp.numel(), _stream()))
@@ -244,7 +265,7 @@ def bof4_fit_codebook(weights, block_size: int, norm: int, metric: int, levels, 
             cb.copy_(src)
     else:
         cb = _codebook(levels, dev).clone()
-        log = torch.zeros(max(iters, 1), dtype=torch.float64, device=dev)
+        log = _new(max(iters, 1), torch.float64, dev, zero=True)
     wsp = workspace if workspace is not None else _workspace(
         OP_EM, sum(w.numel() for w in ws), block_size, metric, dev)
     with torch.cuda.device(dev):
@@ -261,7 +282,7 @@ def bof4_theoretical_codebook(block_size: int, norm: int, metric: int, levels, f
     -> levels fp32[16] on the device."""
     dev = torch.device(device)
     cb = _codebook(levels, dev).clone()
-    ws = torch.empty(256, dtype=torch.uint8, device=dev)
+    ws = _new(256, torch.uint8, dev)
     with torch.cuda.device(dev):
         _check(lib().bof4_theoretical_codebook(block_size, norm, metric, _ptr(cb), fixed_mask, iters,
                                                _ptr(ws), ws.numel(), _stream()))
@@ -277,7 +298,7 @@ def bof4_theoretical_codebook_general(block_size: int, norm: int, metric: int, p
     tab = torch.as_tensor(np.ascontiguousarray(pdf, dtype=np.float64)).to(dev) if not isinstance(pdf, torch.Tensor) \
         else _dev(pdf.to(torch.float64), "pdf")
     n = tab.numel()
-    ws = torch.empty(256 + 24 * n, dtype=torch.uint8, device=dev)
+    ws = _new(256 + 24 * n, torch.uint8, dev)
     with torch.cuda.device(dev):
         _check(lib().bof4_theoretical_codebook_general(block_size, norm, metric, _ptr(tab), n, float(w_max), _ptr(cb),
                                                        fixed_mask, iters, _ptr(ws), ws.numel(), _stream()))
@@ -299,7 +320,7 @@ def bof4_theoretical_codebook_batch(block_sizes, norms, metrics, levels, fixed_m
     if tuple(lv.shape) != (n, LEVELS):
         raise ValueError("levels must be [n, 16] or [16]")
     cb = lv.contiguous().to(dev).clone()
-    ws = torch.empty(256 * max(n, 1), dtype=torch.uint8, device=dev)
+    ws = _new(256 * max(n, 1), torch.uint8, dev)
     arr = lambda v, t: (t * max(n, 1))(*[int(x) for x in v])
     with torch.cuda.device(dev):
         _check(lib().bof4_theoretical_codebook_batch(
@@ -320,8 +341,8 @@ def bof4_quantize(w: torch.Tensor, block_size: int, norm: int, levels,
     sd = dt if scale_dtype is None else scale_dtype
     cb = _codebook(levels, w.device)
     if out is None:
-        codes = torch.empty((n + 1) // 2, dtype=torch.uint8, device=w.device)
-        scales = torch.empty(-(-n // max(block_size, 1)), dtype=_torch_dt(sd), device=w.device)
+        codes = _new((n + 1) // 2, torch.uint8, w.device)
+        scales = _new(-(-n // max(block_size, 1)), _torch_dt(sd), w.device)
     else:
         codes, scales = out
     with torch.cuda.device(w.device):
@@ -342,7 +363,7 @@ def bof4_dequantize(codes: torch.Tensor, scales: torch.Tensor, block_size: int, 
         raise ValueError("codes must hold (n + 1) // 2 bytes")
     cb = _codebook(levels, codes.device)
     if out is None:
-        out = torch.empty(n, dtype=_torch_dt(out_dtype), device=codes.device)
+        out = _new(n, _torch_dt(out_dtype), codes.device)
     idx = val = cnt = None
     cap = 0
     if outliers is not None:
@@ -366,7 +387,7 @@ def bof4_gemv(codes: torch.Tensor, scales: torch.Tensor, rows: int, cols: int, b
         raise ValueError("codes must hold rows * cols weights and x cols values")
     cb = _codebook(levels, codes.device)
     if out is None:
-        out = torch.empty(rows, dtype=torch.float32, device=codes.device)
+        out = _new(rows, torch.float32, codes.device)
     idx = val = cnt = None
     cap = 0
     if outliers is not None:
@@ -385,10 +406,10 @@ def opq_split(w: torch.Tensor, block_size: int, tau: float, capacity: int,
     n, dt = w.numel(), _dt(w)
     dev = w.device
     wsp = workspace if workspace is not None else _workspace(OP_OPQ, n, block_size, 0, dev)
-    clean = torch.empty_like(w) if want_clean else None
-    idx = torch.empty(capacity, dtype=torch.int32, device=dev)
-    val = torch.empty(capacity, dtype=torch.bfloat16, device=dev)
-    cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+    clean = _new(w.numel(), w.dtype, w.device).view(w.shape) if want_clean else None
+    idx = _new(capacity, torch.int32, dev)
+    val = _new(capacity, torch.bfloat16, dev)
+    cnt = _new(1, torch.int64, dev, zero=True)
     with torch.cuda.device(dev):
         _check(lib().opq_split(_ptr(w), dt, n, block_size, tau, _ptr(clean), _ptr(idx), _ptr(val),
                                capacity, _ptr(cnt), _ptr(wsp), wsp.numel(), _stream()))
@@ -407,14 +428,57 @@ def bof4_outlier_count(n_out: torch.Tensor, capacity: int) -> int:
     return int(host.value)
 
 
+def _ptr_array(tensors):
+    return (ctypes.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+
+
+def bof4_quantize_batch(weights, block_size: int, norm: int, levels, scale_dtype: Optional[int] = None, out=None):
+    """bof4_quantize over a list of tensors in few launches -> (list of codes, list of scales).
+    `out` = (codes list, scales list) to write into instead of fresh allocations."""
+    ws, dt, ptrs, sizes = _tensor_list(weights)
+    dev = ws[0].device
+    cb = _codebook(levels, dev)
+    sd = dt if scale_dtype is None else scale_dtype
+    if out is not None:
+        codes, scales = [_dev(c, "codes") for c in out[0]], [_dev(s, "scales") for s in out[1]]
+    else:
+        codes = [_new((w.numel() + 1) // 2, torch.uint8, dev) for w in ws]
+        scales = [_new(-(-w.numel() // max(block_size, 1)), _torch_dt(sd), dev) for w in ws]
+    for w, c, sc in zip(ws, codes, scales):
+        if c.numel() != (w.numel() + 1) // 2 or sc.numel() != -(-w.numel() // max(block_size, 1)) or _dt(sc) != sd:
+            raise ValueError("out buffers do not match the tensors")
+    with torch.cuda.device(dev):
+        _check(lib().bof4_quantize_batch(ptrs, sizes, len(ws), dt, block_size, norm, _ptr(cb), _ptr_array(codes),
+                                         _ptr_array(scales), sd, _stream()))
+    return codes, scales
+
+
+def bof4_dequantize_batch(codes, scales, sizes, block_size: int, levels, out_dtype: int = BF16, out=None):
+    """bof4_dequantize (no outlier list) over a list of tensors in few launches -> list of outputs."""
+    codes = [_dev(c, "codes") for c in codes]
+    scales = [_dev(s, "scales") for s in scales]
+    dev = codes[0].device
+    cb = _codebook(levels, dev)
+    outs = [_dev(o, "out") for o in out] if out is not None else [_new(int(n), _torch_dt(out_dtype), dev) for n in sizes]
+    ns = (ctypes.c_int64 * len(codes))(*[int(n) for n in sizes])
+    for c, sc, o, n in zip(codes, scales, outs, sizes):
+        if c.numel() != (n + 1) // 2 or sc.numel() != -(-n // max(block_size, 1)) or o.numel() != n \
+                or _dt(o) != out_dtype or _dt(sc) != _dt(scales[0]):
+            raise ValueError("buffers do not match the sizes")
+    with torch.cuda.device(dev):
+        _check(lib().bof4_dequantize_batch(_ptr_array(codes), _ptr_array(scales), _dt(scales[0]), ns, len(codes),
+                                           block_size, _ptr(cb), _ptr_array(outs), out_dtype, _stream()))
+    return outs
+
+
 def bof4_scales_compress(scales: torch.Tensor, norm: int):
     """Double quantisation of block constants -> (q uint8[B], group fp32[ceil(B/256)], sign uint8[ceil(B/8)] or None)."""
     scales = _dev(scales, "scales")
     B = scales.numel()
     dev = scales.device
-    q = torch.empty(B, dtype=torch.uint8, device=dev)
-    g = torch.empty((B + 255) // 256, dtype=torch.float32, device=dev)
-    sign = torch.empty((B + 7) // 8, dtype=torch.uint8, device=dev) if norm == NORM_SIGNED else None
+    q = _new(B, torch.uint8, dev)
+    g = _new((B + 255) // 256, torch.float32, dev)
+    sign = _new((B + 7) // 8, torch.uint8, dev) if norm == NORM_SIGNED else None
     with torch.cuda.device(dev):
         _check(lib().bof4_scales_compress(_ptr(scales), _dt(scales), B, norm, _ptr(q), _ptr(g),
                                           _ptr(sign) if sign is not None else None, _stream()))
@@ -424,7 +488,7 @@ def bof4_scales_compress(scales: torch.Tensor, norm: int):
 def bof4_scales_expand(q: torch.Tensor, group: torch.Tensor, sign: Optional[torch.Tensor]) -> torch.Tensor:
     """The decoder's fp32 block constants from their double-quantised form."""
     q = _dev(q, "q")
-    out = torch.empty(q.numel(), dtype=torch.float32, device=q.device)
+    out = _new(q.numel(), torch.float32, q.device)
     with torch.cuda.device(q.device):
         _check(lib().bof4_scales_expand(_ptr(q), _ptr(_dev(group, "group")),
                                         _ptr(_dev(sign, "sign")) if sign is not None else None, q.numel(),
@@ -443,11 +507,11 @@ def bof4_quantize_opq(w: torch.Tensor, block_size: int, norm: int, levels, tau: 
     cb = _codebook(levels, dev)
     wsp = workspace if workspace is not None else _workspace(OP_OPQ, n, block_size, 0, dev)
     if out is None:
-        codes = torch.empty((n + 1) // 2, dtype=torch.uint8, device=dev)
-        scales = torch.empty(-(-n // max(block_size, 1)), dtype=_torch_dt(sd), device=dev)
-        idx = torch.empty(capacity, dtype=torch.int32, device=dev)
-        val = torch.empty(capacity, dtype=torch.bfloat16, device=dev)
-        cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+        codes = _new((n + 1) // 2, torch.uint8, dev)
+        scales = _new(-(-n // max(block_size, 1)), _torch_dt(sd), dev)
+        idx = _new(capacity, torch.int32, dev)
+        val = _new(capacity, torch.bfloat16, dev)
+        cnt = _new(1, torch.int64, dev, zero=True)
     else:
         codes, scales, idx, val, cnt = out
     with torch.cuda.device(dev):

@@ -193,22 +193,17 @@ __device__ __noinline__ void quantize_row32_generic(Raw32 raw, int64_t idx, bool
     quantize_row32<I, SIGNED, ST>(u, mx, mn, idx, ok, fast_ok, lut_base, S, codes, scales);
 }
 
+// The rows r, r + G, r + 2G, ... of one tensor (G = CTAs of the grid), `first` being row r already
+// on its way.  Called by all threads of the CTA with the tables in place.
 template <int I, bool SIGNED, class ST>
-__global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
-quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels,
-                  uint8_t* __restrict__ codes, void* __restrict__ scales)
+__device__ __forceinline__ void quantize32_rows(const void* __restrict__ w, int64_t n, uint8_t* __restrict__ codes,
+                                                void* __restrict__ scales, const int r0, const Raw32& first,
+                                                const bool fast_ok, const uint32_t lut_base, QuantShared32* S)
 {
-    extern __shared__ __align__(16) unsigned char s_lut[];
-    __shared__ QuantShared32 S;
     const RowMap32 map(n, kQRow32, threadIdx.x);
     const int G = gridDim.x;
-    int r = blockIdx.x;
-    if (r >= map.rows) return;
+    int r = r0;
     auto fetch = [&](int rr) { return map.ok(rr) ? load_raw32(w, map.idx(rr)) : zero_raw32(); };
-    const Raw32 first = fetch(r);  // on its way while the tables are built
-    const bool lut_ok = build_tables32(levels, S.xi, S.lv, s_lut, &S.info, [](int base) { return (uint32_t)base; });
-    const bool fast_ok = lut_ok && !S.info.tiny;
-    const uint32_t lut_base = lut_lane_base(s_lut, threadIdx.x & 31);
     if constexpr (Geo32<I>::WPB > 1) {
         // blocks of several warps: every thread of the CTA takes every step (barriers inside)
         Raw32 a = first;
@@ -218,7 +213,7 @@ quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict
             words_of(a, u);
             float mx, mn;
             lane_minmax32(u, mx, mn);
-            quantize_row32<I, SIGNED, ST>(u, mx, mn, map.idx(r), map.ok(r), fast_ok, lut_base, &S, codes, scales);
+            quantize_row32<I, SIGNED, ST>(u, mx, mn, map.idx(r), map.ok(r), fast_ok, lut_base, S, codes, scales);
             a = next;
         }
     } else {
@@ -231,13 +226,13 @@ quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict
             lane_minmax32(u, mx, mn);
             const float m = block_constant32<I, SIGNED>(u, mx, mn, g, nullptr);
             const int64_t idx = map.idx(rr);
-            if (row_is_fast(g, m, true, fast_ok, &S.info)) {
+            if (row_is_fast(g, m, true, fast_ok, &S->info)) {
                 uint32_t cw[4];
                 encode32_fast(u, m, lut_base, cw);
                 st_stream128(codes + idx / 2, cw[0], cw[1], cw[2], cw[3]);
                 if ((idx & (I - 1)) == 0) store_scale<ST>(scales, idx / I, m);
             } else {
-                quantize_row32_generic<I, SIGNED, ST>(raw, idx, true, fast_ok, lut_base, &S, codes, scales);
+                quantize_row32_generic<I, SIGNED, ST>(raw, idx, true, fast_ok, lut_base, S, codes, scales);
             }
         };
         const int full = map.rows_full;
@@ -257,9 +252,61 @@ quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict
             }
         }
         // the partial last row of the tensor, by the CTA whose turn it is
-        if (map.rows > full && full % G == (int)blockIdx.x)
-            quantize_row32_generic<I, SIGNED, ST>(full == (int)blockIdx.x ? first : fetch(full), map.idx(full),
-                                                  map.ok(full), fast_ok, lut_base, &S, codes, scales);
+        if (map.rows > full && full >= r0 && (full - r0) % G == 0)
+            quantize_row32_generic<I, SIGNED, ST>(full == r0 ? first : fetch(full), map.idx(full), map.ok(full),
+                                                  fast_ok, lut_base, S, codes, scales);
+    }
+}
+
+template <int I, bool SIGNED, class ST>
+__global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
+quantize32_kernel(const void* __restrict__ w, int64_t n, const float* __restrict__ levels,
+                  uint8_t* __restrict__ codes, void* __restrict__ scales)
+{
+    extern __shared__ __align__(16) unsigned char s_lut[];
+    __shared__ QuantShared32 S;
+    const RowMap32 map(n, kQRow32, threadIdx.x);
+    const int r = blockIdx.x;
+    if (r >= map.rows) return;
+    const Raw32 first = map.ok(r) ? load_raw32(w, map.idx(r)) : zero_raw32();  // on its way while the tables are built
+    const bool lut_ok = build_tables32(levels, S.xi, S.lv, s_lut, &S.info, [](int base) { return (uint32_t)base; });
+    const bool fast_ok = lut_ok && !S.info.tiny;
+    const uint32_t lut_base = lut_lane_base(s_lut, threadIdx.x & 31);
+    quantize32_rows<I, SIGNED, ST>(w, n, codes, scales, r, first, fast_ok, lut_base, &S);
+}
+
+// Several tensors in one launch: the tables are built once per CTA, and the rows of all tensors
+// are dealt round-robin over the CTAs as if they were one tensor (tensor t starts with the CTA
+// that follows the last row of tensor t - 1), so that small tensors neither pay for a launch and
+// a table build each nor leave part of the grid idle.
+constexpr int kQBatch = 64;  // tensors per launch (kernel parameter table)
+struct QuantBatch {
+    const void* w[kQBatch];
+    uint8_t* codes[kQBatch];
+    void* scales[kQBatch];
+    int64_t n[kQBatch];
+    int start[kQBatch];  // CTA that takes the tensor's first row
+    int count;
+};
+
+template <int I, bool SIGNED, class ST>
+__global__ void __launch_bounds__(kQThreads, kQCtasPerSm)
+quantize32_batch_kernel(const QuantBatch B, const float* __restrict__ levels)
+{
+    extern __shared__ __align__(16) unsigned char s_lut[];
+    __shared__ QuantShared32 S;
+    const int G = gridDim.x;
+    const bool lut_ok = build_tables32(levels, S.xi, S.lv, s_lut, &S.info, [](int base) { return (uint32_t)base; });
+    const bool fast_ok = lut_ok && !S.info.tiny;
+    const uint32_t lut_base = lut_lane_base(s_lut, threadIdx.x & 31);
+    for (int t = 0; t < B.count; ++t) {
+        const int64_t n = B.n[t];
+        const RowMap32 map(n, kQRow32, threadIdx.x);
+        const int r0 = ((int)blockIdx.x + G - B.start[t]) % G;
+        if (r0 >= map.rows) continue;  // uniform over the CTA
+        const void* w = B.w[t];
+        const Raw32 first = map.ok(r0) ? load_raw32(w, map.idx(r0)) : zero_raw32();
+        quantize32_rows<I, SIGNED, ST>(w, n, B.codes[t], B.scales[t], r0, first, fast_ok, lut_base, &S);
     }
 }
 
@@ -290,15 +337,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 // (xhat[b >> 4], xhat[b & 15]); one 8-byte shared-memory read and one packed multiplication by
 // the block constant give both products (Eq. 3).
 template <class ST, class OT, int I>
-__global__ void __launch_bounds__(kDThreads)
-dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t n,
-                  const float* __restrict__ levels, void* __restrict__ out)
+__device__ __forceinline__ void dequantize_rows(const uint8_t* __restrict__ codes, const void* __restrict__ scales,
+                                                int64_t n, void* __restrict__ out, const float2* s_pair, const int r0)
 {
-    __shared__ float2 s_pair[256];
-    s_pair[threadIdx.x] = make_float2(levels[threadIdx.x >> 4], levels[threadIdx.x & 15]);
-    __syncthreads();
     const int64_t rows = (n + kDRow - 1) / kDRow;
-    int64_t r = blockIdx.x;
+    int64_t r = r0;
     if (r >= rows) return;
     // n is a multiple of 32, so a lane's 32 outputs are all inside the tensor or all outside
     auto fetch = [&](int64_t row, int64_t& idx, uint4& cc, float& m) {
@@ -352,6 +395,41 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ sc
         cc = cc_next;
         m = m_next;
     }
+}
+
+template <class ST, class OT, int I>
+__global__ void __launch_bounds__(kDThreads)
+dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t n,
+                  const float* __restrict__ levels, void* __restrict__ out)
+{
+    __shared__ float2 s_pair[256];
+    s_pair[threadIdx.x] = make_float2(levels[threadIdx.x >> 4], levels[threadIdx.x & 15]);
+    __syncthreads();
+    dequantize_rows<ST, OT, I>(codes, scales, n, out, s_pair, (int)blockIdx.x);
+}
+
+// Several tensors in one launch, their rows dealt round-robin over the CTAs as in
+// quantize32_batch_kernel.
+struct DequantBatch {
+    const uint8_t* codes[kQBatch];
+    const void* scales[kQBatch];
+    void* out[kQBatch];
+    int64_t n[kQBatch];
+    int start[kQBatch];
+    int count;
+};
+
+template <class ST, class OT, int I>
+__global__ void __launch_bounds__(kDThreads)
+dequantize_batch_kernel(const DequantBatch B, const float* __restrict__ levels)
+{
+    __shared__ float2 s_pair[256];
+    s_pair[threadIdx.x] = make_float2(levels[threadIdx.x >> 4], levels[threadIdx.x & 15]);
+    __syncthreads();
+    const int G = gridDim.x;
+    for (int t = 0; t < B.count; ++t)
+        dequantize_rows<ST, OT, I>(B.codes[t], B.scales[t], B.n[t], B.out[t], s_pair,
+                                   ((int)blockIdx.x + G - B.start[t]) % G);
 }
 
 // Outliers written back over the dequantised tensor (Sec. 3.3, decoding side).
@@ -1126,6 +1204,156 @@ extern "C" int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int
             scatter_outliers_kernel<F32><<<kSMs, 256, 0, st>>>(d_out_idx, val, d_n_out, capacity, n, d_out);
         else
             scatter_outliers_kernel<BF16><<<kSMs, 256, 0, st>>>(d_out_idx, val, d_n_out, capacity, n, d_out);
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
+    return BOF4_OK;
+}
+
+// Many tensors per launch.  bf16 weights whose whole blocks go through the batch kernels, kQBatch
+// tensors per launch; fp32 weights and short last blocks take the single-tensor path.
+extern "C" int bof4_quantize_batch(const void* const* h_w, const int64_t* h_n, int n_tensors, int w_dtype,
+                                   int block_size, int norm, const float* d_codebook, uint8_t* const* h_codes,
+                                   void* const* h_scales, int scale_dtype, void* stream)
+{
+    const char* fn = "bof4_quantize_batch";
+    if (n_tensors < 0 || (n_tensors > 0 && (!h_w || !h_n || !h_codes || !h_scales))) {
+        set_error("%s: bad tensor list", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    int rc = check_quant_dtypes(fn, w_dtype, scale_dtype, norm);
+    if (rc) return rc;
+    if (!d_codebook) {
+        set_error("%s: NULL codebook", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    for (int t = 0; t < n_tensors; ++t) {
+        if ((rc = check_common(fn, h_n[t], block_size, true))) return rc;
+        if (h_n[t] == 0) continue;
+        if (!h_w[t] || !h_codes[t] || !h_scales[t]) {
+            set_error("%s: tensor %d has a NULL pointer", fn, t);
+            return BOF4_ERR_INVALID_ARG;
+        }
+        if ((rc = check_aligned(fn, "a weight tensor", h_w[t])) || (rc = check_aligned(fn, "a code array", h_codes[t])))
+            return rc;
+    }
+    if (w_dtype != BOF4_BF16) {
+        for (int t = 0; t < n_tensors; ++t)
+            if ((rc = bof4_quantize(h_w[t], w_dtype, h_n[t], block_size, norm, d_codebook, h_codes[t], h_scales[t],
+                                    scale_dtype, stream)))
+                return rc;
+        return BOF4_OK;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    QuantBatch B;
+    B.count = 0;
+    int64_t rows = 0;
+    const int G = kSMs * kQCtasPerSm;
+    for (int t = 0; t <= n_tensors; ++t) {
+        if (t < n_tensors) {
+            const int64_t n_whole = h_n[t] - h_n[t] % block_size;
+            if (n_whole > 0) {
+                B.w[B.count] = h_w[t];
+                B.codes[B.count] = h_codes[t];
+                B.scales[B.count] = h_scales[t];
+                B.n[B.count] = n_whole;
+                B.start[B.count] = (int)(rows % G);
+                rows += (n_whole + kQRow32 - 1) / kQRow32;
+                ++B.count;
+            }
+        }
+        if (B.count == kQBatch || (t == n_tensors && B.count > 0)) {
+            BOF4_DISPATCH_ST(scale_dtype,
+                BOF4_DISPATCH_I(block_size,
+                    BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                        { constexpr auto kern = quantize32_batch_kernel<I_, SG, ST>;
+                          if ((rc = ensure_dynamic_smem<kern>(kLutBytes))) return rc;
+                          kern<<<G, kQThreads, kLutBytes, st>>>(B, d_codebook); })));
+            BOF4_CUDA_TRY(cudaGetLastError());
+            B.count = 0;
+        }
+    }
+    for (int t = 0; t < n_tensors; ++t) {
+        const int tail = (int)(h_n[t] % block_size);
+        if (!tail) continue;
+        const int64_t n_whole = h_n[t] - tail;
+        BOF4_DISPATCH_ST(scale_dtype,
+            BOF4_DISPATCH_BOOL(norm == BOF4_NORM_SIGNED, SG,
+                (tail_block_kernel<BF16, SG, ST, true, false><<<1, kTailThreads, 0, st>>>(
+                    h_w[t], n_whole, tail, d_codebook, 0.0f, h_codes[t], h_scales[t], n_whole / block_size, nullptr,
+                    nullptr, nullptr, 0, nullptr))));
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
+    return BOF4_OK;
+}
+
+extern "C" int bof4_dequantize_batch(const uint8_t* const* h_codes, const void* const* h_scales, int scale_dtype,
+                                     const int64_t* h_n, int n_tensors, int block_size, const float* d_codebook,
+                                     void* const* h_out, int out_dtype, void* stream)
+{
+    const char* fn = "bof4_dequantize_batch";
+    if (n_tensors < 0 || (n_tensors > 0 && (!h_codes || !h_scales || !h_n || !h_out))) {
+        set_error("%s: bad tensor list", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if ((scale_dtype != BOF4_F32 && scale_dtype != BOF4_BF16) || (out_dtype != BOF4_F32 && out_dtype != BOF4_BF16)) {
+        set_error("%s: unknown dtype", fn);
+        return BOF4_ERR_DTYPE;
+    }
+    if (!d_codebook) {
+        set_error("%s: NULL codebook", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    int rc;
+    for (int t = 0; t < n_tensors; ++t) {
+        if ((rc = check_common(fn, h_n[t], block_size, true))) return rc;
+        if (h_n[t] == 0) continue;
+        if (!h_codes[t] || !h_scales[t] || !h_out[t]) {
+            set_error("%s: tensor %d has a NULL pointer", fn, t);
+            return BOF4_ERR_INVALID_ARG;
+        }
+        if ((rc = check_aligned(fn, "a code array", h_codes[t])) || (rc = check_aligned(fn, "an output tensor", h_out[t])))
+            return rc;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DequantBatch B;
+    B.count = 0;
+    int64_t rows = 0;
+    const int G = kSMs * 8;
+    for (int t = 0; t <= n_tensors; ++t) {
+        if (t < n_tensors) {
+            const int64_t n_whole = h_n[t] - h_n[t] % block_size;
+            if (n_whole > 0) {
+                B.codes[B.count] = h_codes[t];
+                B.scales[B.count] = h_scales[t];
+                B.out[B.count] = h_out[t];
+                B.n[B.count] = n_whole;
+                B.start[B.count] = (int)(rows % G);
+                rows += (n_whole + kDRow - 1) / kDRow;
+                ++B.count;
+            }
+        }
+        if (B.count == kQBatch || (t == n_tensors && B.count > 0)) {
+#define BOF4_DEQB(ST_, OT_) BOF4_DISPATCH_I(block_size, (dequantize_batch_kernel<ST_, OT_, I_><<<G, kDThreads, 0, st>>>(B, d_codebook)))
+            if (scale_dtype == BOF4_F32 && out_dtype == BOF4_F32) { BOF4_DEQB(F32, F32) }
+            else if (scale_dtype == BOF4_F32) { BOF4_DEQB(F32, BF16) }
+            else if (out_dtype == BOF4_F32) { BOF4_DEQB(BF16, F32) }
+            else { BOF4_DEQB(BF16, BF16) }
+#undef BOF4_DEQB
+            BOF4_CUDA_TRY(cudaGetLastError());
+            B.count = 0;
+        }
+    }
+    for (int t = 0; t < n_tensors; ++t) {
+        const int tail = (int)(h_n[t] % block_size);
+        if (!tail) continue;
+        const int64_t n_whole = h_n[t] - tail;
+#define BOF4_DEQT(ST_, OT_) tail_dequantize_kernel<ST_, OT_><<<1, kTailThreads, 0, st>>>( \
+        h_codes[t], h_scales[t], n_whole, tail, n_whole / block_size, d_codebook, h_out[t]);
+        if (scale_dtype == BOF4_F32 && out_dtype == BOF4_F32) { BOF4_DEQT(F32, F32) }
+        else if (scale_dtype == BOF4_F32) { BOF4_DEQT(F32, BF16) }
+        else if (out_dtype == BOF4_F32) { BOF4_DEQT(BF16, F32) }
+        else { BOF4_DEQT(BF16, BF16) }
+#undef BOF4_DEQT
         BOF4_CUDA_TRY(cudaGetLastError());
     }
     return BOF4_OK;
