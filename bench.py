@@ -6,8 +6,8 @@ called through the C ABI (the ctypes binding) with device-resident inputs:
 
     EM iteration, MSE        one bof4_fit_codebook(iters=1) over the 224 Llama-7B-shaped matrices
     EM iteration, MAE        the same with the weighted-median centroid        (12.95 GB, bf16)
-    quantise                 bof4_quantize   of the 224 Llama-3-8B-shaped matrices (13.96 GB)
-    dequantise               bof4_dequantize of the same set, back to bf16
+    quantise                 bof4_quantize_batch   of the 224 Llama-3-8B-shaped matrices (13.96 GB)
+    dequantise               bof4_dequantize_batch of the same set, back to bf16
     OPQ quantise             bof4_quantize_opq  of one Llama-70B-shaped layer      (1.71 GB)
     OPQ dequantise           bof4_dequantize with outlier write-back of that layer
 
@@ -203,13 +203,13 @@ class Step:
 
     def quant(self):
         b = self.b
-        for w, out in zip(self.w_q, self.q_out):
-            b.bof4_quantize(w, I, b.NORM_SIGNED, self.cb_q, out=out)
+        b.bof4_quantize_batch(self.w_q, I, b.NORM_SIGNED, self.cb_q,
+                              out=([c for c, _ in self.q_out], [s for _, s in self.q_out]))
 
     def dequant(self):
         b = self.b
-        for (codes, scales), out in zip(self.q_out, self.q_deq):
-            b.bof4_dequantize(codes, scales, I, self.cb_q, b.BF16, out=out)
+        b.bof4_dequantize_batch([c for c, _ in self.q_out], [s for _, s in self.q_out],
+                                [w.numel() for w in self.w_q], I, self.cb_q, b.BF16, out=self.q_deq)
 
     def opq_quant(self):
         b = self.b
@@ -228,8 +228,8 @@ class Step:
         comps = [("em_mse", self.em_mse, self.n_fit, BYTES_EM, b.mse_launches_per_iteration(nt)),
                  ("em_mae", self.em_mae, self.n_fit, BYTES_EM * MAE_SELECTION_PASSES,
                   b.mae_launches_per_call(nt, self.n_fit, 1)),
-                 ("quantize", self.quant, self.n_q, BYTES_QUANT, nq),
-                 ("dequantize", self.dequant, self.n_q, BYTES_DEQUANT, nq),
+                 ("quantize", self.quant, self.n_q, BYTES_QUANT, -(-nq // b.TENSORS_PER_LAUNCH)),
+                 ("dequantize", self.dequant, self.n_q, BYTES_DEQUANT, -(-nq // b.TENSORS_PER_LAUNCH)),
                  ("opq_quantize", self.opq_quant, self.n_opq, BYTES_QUANT + 6 * OPQ_OUTLIER_FRACTION / 2.2, 2 * no),
                  ("opq_dequantize", self.opq_dequant, self.n_opq, BYTES_DEQUANT + 6 * OPQ_OUTLIER_FRACTION / 2.2, 2 * no)]
         if self.only:
