@@ -812,14 +812,46 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
             offer(x, a);
         }
     };
+    // The queue is worked off by all threads: region search, digit, histogram; with COLLECT the
+    // candidates staged meanwhile go to the global lists (one reservation per level).  Called by
+    // the whole CTA every kDrainRows rows, so that neither the queue nor the staging slots fill up
+    // however many rows a CTA streams.
+    auto drain = [&]() {
+        __syncthreads();
+        const uint32_t q = min(s_qn, (uint32_t)kMaeQueue);
+        for (uint32_t i = tid; i < q; i += kMaeThreads) {
+            const uint2 ent = s_queue[i];
+            later_sample(__uint_as_float(ent.x), ent.y);
+        }
+        __syncthreads();
+        if (tid == 0) s_qn = 0u;
+        if (COLLECT) {
+            if (tid < kLevels) {
+                const uint32_t k = min(s_ncand[tid], (uint32_t)kMaeStage);
+                s_gbase[tid] = k ? atomicAdd(&W.state->cand_count[tid], k) : 0u;
+            }
+            __syncthreads();
+            for (int k = tid; k < kLevels * kMaeStage; k += kMaeThreads) {
+                const int l = k / kMaeStage, i = k % kMaeStage;
+                const uint32_t dst = s_gbase[l] + (uint32_t)i;
+                if ((uint32_t)i < min(s_ncand[l], (uint32_t)kMaeStage) && dst < W.cand_cap)
+                    W.cand[(size_t)l * W.cand_cap + dst] = s_cand[k];
+            }
+            __syncthreads();
+            if (tid < kLevels) s_ncand[tid] = 0u;
+        }
+        __syncthreads();
+    };
+    constexpr int kDrainRows = 16;  // about 2000 queued samples after a first pass on the fine grid
     {
         bool ok_a, ok_b;
         const uint16_t *src_a = nullptr, *src_b = nullptr;
         int64_t g = blockIdx.x;
         const int64_t GS = gridDim.x;
         Raw32 ra = fetch(g, ok_a, src_a), rb;
+        int since = 0;
         if (g < total_rows) {
-            while (true) {
+            while (true) {  // g and the trip count are the same for all threads of the CTA
                 rb = fetch(g + GS, ok_b, src_b);
                 row(ra, ok_a, src_a);
                 g += GS;
@@ -828,36 +860,19 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
                 row(rb, ok_b, src_b);
                 g += GS;
                 if (g >= total_rows) break;
+                since += 2;
+                if (since >= kDrainRows) {
+                    since = 0;
+                    drain();
+                }
             }
         }
     }
-    __syncthreads();
-    if (!FIRST) {
-        const uint32_t q = min(s_qn, (uint32_t)kMaeQueue);
-        for (uint32_t i = tid; i < q; i += kMaeThreads) {
-            const uint2 ent = s_queue[i];
-            later_sample(__uint_as_float(ent.x), ent.y);
-        }
-        __syncthreads();
-    }
+    drain();
     for (int k = tid; k < kLevels * kMaeBins; k += kMaeThreads) {
         const unsigned long long wsum = ((unsigned long long)s_hi[k] << 32) + s_lo[k];
         if (wsum) atomicAdd(&W.hist[k], wsum);
         if (FIRST && COUNT && s_cn[k]) atomicAdd(&W.chist[k], (unsigned long long)s_cn[k]);
-    }
-    if (COLLECT) {
-        // one reservation per CTA and level, then a plain copy of the staged samples
-        if (tid < kLevels) {
-            const uint32_t k = min(s_ncand[tid], (uint32_t)kMaeStage);
-            s_gbase[tid] = k ? atomicAdd(&W.state->cand_count[tid], k) : 0u;
-        }
-        __syncthreads();
-        for (int k = tid; k < kLevels * kMaeStage; k += kMaeThreads) {
-            const int l = k / kMaeStage, i = k % kMaeStage;
-            const uint32_t dst = s_gbase[l] + (uint32_t)i;
-            if ((uint32_t)i < min(s_ncand[l], (uint32_t)kMaeStage) && dst < W.cand_cap)
-                W.cand[(size_t)l * W.cand_cap + dst] = s_cand[k];
-        }
     }
     if (FIRST) {
 #pragma unroll
