@@ -105,7 +105,7 @@ typedef struct bof4_em_stats {
  *   op = BOF4_OP_EM : partial records of the deterministic two-stage reduction and, for
  *                     metric = MAE, the per-level selection histograms and candidate lists.
  *                     n_max = the TOTAL number of weights of the tensor list.  The candidate lists
- *                     grow with it (16 * 8 * n_max / 512 bytes, between 8 and 16 MiB); any workspace of at
+ *                     grow with it (n_max / 8 bytes, between 8 MiB and 1 GiB); any workspace of at
  *                     least bof4_workspace_bytes(BOF4_OP_EM, 0, ...) is accepted, a smaller one
  *                     than asked for here only costs the MAE fit one more pass over the data per
  *                     iteration.  Results do not depend on the workspace size.

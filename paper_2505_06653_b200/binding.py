@@ -42,7 +42,7 @@ def mae_launches_per_call(n_tensors: int, n_total: int, iters: int) -> int:
     iteration the set-up, four data passes and the selection kernels of the passes that do not
     carry their own selection (two up to 2^26 weights, three beyond)."""
     chunks = max(1, -(-n_tensors // TENSORS_PER_LAUNCH))
-    cap = min(max(n_total // 512, 1 << 16), 1 << 17)       # candidate entries per level of the default workspace
+    cap = min(max(n_total // 1024, 1 << 16), 1 << 23)      # candidate entries per level of the default workspace
     small = n_total // 1024 <= cap
     return chunks + iters * (1 + 4 * chunks + (2 if small else 3))
 

@@ -842,7 +842,9 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
         }
         __syncthreads();
     };
-    constexpr int kDrainRows = 16;  // about 2000 queued samples after a first pass on the fine grid
+    // after a first pass on the fine grid about 130 samples per row are queued, up to a sixth of
+    // them for one of the central levels (whose staging slot holds kMaeStage)
+    constexpr int kDrainRows = COLLECT ? 8 : 16;
     {
         bool ok_a, ok_b;
         const uint16_t *src_a = nullptr, *src_b = nullptr;

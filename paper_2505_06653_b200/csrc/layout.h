@@ -29,18 +29,19 @@ constexpr int kFineSlots = 2 * kFineStride;
 constexpr size_t kEmMaeHistBytes = 66048;        // weight histogram, then count histogram (>= 8 * kFineSlots)
 static_assert(kEmMaeHistBytes >= (size_t)kFineSlots * 8 && kEmMaeHistBytes >= (size_t)16 * kMaeBins * 8, "histogram space");
 constexpr int kMaeCand = 1 << 16;          // smallest candidate list per level (entries of 8 bytes)
-constexpr int kMaeCandMax = 1 << 17;       // largest one a workspace is sized for (entries are appended one by one)
+constexpr int kMaeCandMax = 1 << 23;       // largest one a workspace is sized for (1 GiB for the 16 lists)
 constexpr size_t kEmMaeCandBytes = (size_t)16 * kMaeCand * 8;
 constexpr size_t kEmMaeBytes = kEmMaeStateBytes + 2 * kEmMaeHistBytes + kEmMaeCandBytes;
 
 // Smallest workspace of the fit (any input size).
 inline size_t em_workspace_bytes() { return kEmMaeOffset + align_up(kEmMaeBytes, 256); }
 // Workspace for n_max weights in total: the candidate lists of the median selection grow with the
-// data (n_max / 512 entries per level, within [kMaeCand, kMaeCandMax]) so that the pass after the
-// first can collect a region's remaining candidates; with smaller lists one more data pass runs.
+// data (n_max / 1024 entries per level, within [kMaeCand, kMaeCandMax]: n_max / 8 bytes in all) so
+// that the pass after the first can collect a region's remaining candidates; with smaller lists
+// one more data pass runs.
 inline size_t em_workspace_bytes_for(int64_t n_max)
 {
-    int64_t cand = n_max / 512;
+    int64_t cand = n_max / 1024;
     cand = cand < kMaeCand ? kMaeCand : (cand > kMaeCandMax ? kMaeCandMax : cand);
     return kEmMaeOffset + align_up(kEmMaeStateBytes + 2 * kEmMaeHistBytes + (size_t)16 * (size_t)cand * 8, 256);
 }
