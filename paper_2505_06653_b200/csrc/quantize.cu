@@ -18,7 +18,9 @@ namespace bof4 {
 constexpr int kQThreads = 512;              // quantise / OPQ pass 1
 constexpr int kQRow = kQThreads * kLaneW;   // weights per CTA row
 constexpr int kQCtasPerSm = 2;              // two CTAs, each with its own region table
-constexpr int kDThreads = 256;              // dequantise
+constexpr int kDThreads = 512;              // dequantise
+constexpr int kDCtasPerSm = 3;              // each with its own 64 KiB level-pair table
+constexpr int kDTableBytes = 256 * 32 * 8;  // [code byte][lane] pairs of levels
 constexpr int kDLaneW = 32;                 // outputs per lane and row (16 code bytes in)
 constexpr int kDRow = kDThreads * kDLaneW;  // outputs per CTA row (dequantise)
 
@@ -335,14 +337,27 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 
 // One code byte holds two weights, so the levels are tabulated per byte: entry b is the pair
 // (xhat[b >> 4], xhat[b & 15]); one 8-byte shared-memory read and one packed multiplication by
-// the block constant give both products (Eq. 3).
+// the block constant give both products (Eq. 3).  The table is kept once per lane ([byte][lane],
+// 64 KiB): the code bytes of the 32 lanes are unrelated, and a shared table of 256 entries made
+// every read a three-fold bank conflict on average, which bound the kernel; with a column per
+// lane the bank only depends on the lane.
+__device__ __forceinline__ void build_pair_table(const float* __restrict__ levels, unsigned char* s_tab)
+{
+    for (int e = threadIdx.x; e < 256 * 32; e += blockDim.x) {
+        const int b = e >> 5;
+        *reinterpret_cast<float2*>(s_tab + (size_t)e * 8) = make_float2(levels[b >> 4], levels[b & 15]);
+    }
+    __syncthreads();
+}
+
 template <class ST, class OT, int I>
 __device__ __forceinline__ void dequantize_rows(const uint8_t* __restrict__ codes, const void* __restrict__ scales,
-                                                int64_t n, void* __restrict__ out, const float2* s_pair, const int r0)
+                                                int64_t n, void* __restrict__ out, const unsigned char* s_tab, const int r0)
 {
     const int64_t rows = (n + kDRow - 1) / kDRow;
     int64_t r = r0;
     if (r >= rows) return;
+    const uint32_t lane8 = (threadIdx.x & 31u) * 8u;
     // n is a multiple of 32, so a lane's 32 outputs are all inside the tensor or all outside
     auto fetch = [&](int64_t row, int64_t& idx, uint4& cc, float& m) {
         idx = (row * kDThreads + threadIdx.x) * kDLaneW;
@@ -369,8 +384,9 @@ __device__ __forceinline__ void dequantize_rows(const uint8_t* __restrict__ code
                 float2 o[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    const uint32_t byte = __byte_perm(word[2 * h + (k >> 2)], 0u, 0x4440u | (uint32_t)(k & 3));
-                    o[k] = __fmul2_rn(mm, s_pair[byte]);
+                    // byte offset of this lane's entry of the code byte: byte * 256 + lane * 8, one permute
+                    const uint32_t off = __byte_perm(word[2 * h + (k >> 2)], lane8, 0x5504u | ((uint32_t)(k & 3) << 4));
+                    o[k] = __fmul2_rn(mm, *reinterpret_cast<const float2*>(s_tab + off));
                 }
                 if (OT::code == BF16::code) {
                     Raw8 p;
@@ -398,14 +414,13 @@ __device__ __forceinline__ void dequantize_rows(const uint8_t* __restrict__ code
 }
 
 template <class ST, class OT, int I>
-__global__ void __launch_bounds__(kDThreads)
+__global__ void __launch_bounds__(kDThreads, kDCtasPerSm)
 dequantize_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t n,
                   const float* __restrict__ levels, void* __restrict__ out)
 {
-    __shared__ float2 s_pair[256];
-    s_pair[threadIdx.x] = make_float2(levels[threadIdx.x >> 4], levels[threadIdx.x & 15]);
-    __syncthreads();
-    dequantize_rows<ST, OT, I>(codes, scales, n, out, s_pair, (int)blockIdx.x);
+    extern __shared__ __align__(16) unsigned char s_tab[];
+    build_pair_table(levels, s_tab);
+    dequantize_rows<ST, OT, I>(codes, scales, n, out, s_tab, (int)blockIdx.x);
 }
 
 // Several tensors in one launch, their rows dealt round-robin over the CTAs as in
@@ -420,15 +435,14 @@ struct DequantBatch {
 };
 
 template <class ST, class OT, int I>
-__global__ void __launch_bounds__(kDThreads)
+__global__ void __launch_bounds__(kDThreads, kDCtasPerSm)
 dequantize_batch_kernel(const DequantBatch B, const float* __restrict__ levels)
 {
-    __shared__ float2 s_pair[256];
-    s_pair[threadIdx.x] = make_float2(levels[threadIdx.x >> 4], levels[threadIdx.x & 15]);
-    __syncthreads();
+    extern __shared__ __align__(16) unsigned char s_tab[];
+    build_pair_table(levels, s_tab);
     const int G = gridDim.x;
     for (int t = 0; t < B.count; ++t)
-        dequantize_rows<ST, OT, I>(B.codes[t], B.scales[t], B.n[t], B.out[t], s_pair,
+        dequantize_rows<ST, OT, I>(B.codes[t], B.scales[t], B.n[t], B.out[t], s_tab,
                                    ((int)blockIdx.x + G - B.start[t]) % G);
 }
 
@@ -1182,12 +1196,14 @@ extern "C" int bof4_dequantize(const uint8_t* d_codes, const void* d_scales, int
     const int tail = (int)(n % block_size);  // a ragged last block goes to its own small kernel
     const int64_t n_whole = n - tail;
     const int64_t rows = (n_whole + kDRow - 1) / kDRow;
-    const int grid = grid_for(rows, 8);
+    const int grid = grid_for(rows, kDCtasPerSm);
 #define BOF4_DEQ(ST_, OT_)                                                                                   \
     {                                                                                                        \
         if (n_whole > 0)                                                                                     \
-            BOF4_DISPATCH_I(block_size, (dequantize_kernel<ST_, OT_, I_><<<grid, kDThreads, 0, st>>>(        \
-                                            d_codes, d_scales, n_whole, d_codebook, d_out)))                 \
+            BOF4_DISPATCH_I(block_size, {                                                                    \
+                constexpr auto kern = dequantize_kernel<ST_, OT_, I_>;                                       \
+                if ((rc = ensure_dynamic_smem<kern>(kDTableBytes))) return rc;                               \
+                kern<<<grid, kDThreads, kDTableBytes, st>>>(d_codes, d_scales, n_whole, d_codebook, d_out); })  \
         if (tail)                                                                                            \
             tail_dequantize_kernel<ST_, OT_><<<1, kTailThreads, 0, st>>>(d_codes, d_scales, n_whole, tail,   \
                                                                          n_whole / block_size, d_codebook, d_out); \
@@ -1318,7 +1334,7 @@ extern "C" int bof4_dequantize_batch(const uint8_t* const* h_codes, const void* 
     DequantBatch B;
     B.count = 0;
     int64_t rows = 0;
-    const int G = kSMs * 8;
+    const int G = kSMs * kDCtasPerSm;
     for (int t = 0; t <= n_tensors; ++t) {
         if (t < n_tensors) {
             const int64_t n_whole = h_n[t] - h_n[t] % block_size;
@@ -1333,7 +1349,10 @@ extern "C" int bof4_dequantize_batch(const uint8_t* const* h_codes, const void* 
             }
         }
         if (B.count == kQBatch || (t == n_tensors && B.count > 0)) {
-#define BOF4_DEQB(ST_, OT_) BOF4_DISPATCH_I(block_size, (dequantize_batch_kernel<ST_, OT_, I_><<<G, kDThreads, 0, st>>>(B, d_codebook)))
+#define BOF4_DEQB(ST_, OT_) BOF4_DISPATCH_I(block_size, {                                  \
+        constexpr auto kern = dequantize_batch_kernel<ST_, OT_, I_>;                       \
+        if ((rc = ensure_dynamic_smem<kern>(kDTableBytes))) return rc;                     \
+        kern<<<G, kDThreads, kDTableBytes, st>>>(B, d_codebook); })
             if (scale_dtype == BOF4_F32 && out_dtype == BOF4_F32) { BOF4_DEQB(F32, F32) }
             else if (scale_dtype == BOF4_F32) { BOF4_DEQB(F32, BF16) }
             else if (out_dtype == BOF4_F32) { BOF4_DEQB(BF16, F32) }
