@@ -286,6 +286,7 @@ __device__ __forceinline__ void finalize_body(const MaeWs& W, const MaeFinal& F,
 // histogram, candidate list), so that the rare, long path does not run with one lane in 32.
 // COLLECT (second pass): every participating sample is also appended to its level's list.
 constexpr int kMaeQueue = kLevels * kMaeBins * 4 / 8;  // entries {x, weight} in the count histogram's space
+constexpr int kLaterQueue = kLevels * kMaeBins * 4 / 16;  // entries {address, block constant, weight} (bf16 later passes)
 
 // TAIL (a later pass without a candidate list): the CTA that finishes last, found by an atomic
 // ticket so that nobody waits, also selects the next digit of every level and, if F.enabled,
@@ -635,7 +636,7 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
     uint32_t* s_lo = reinterpret_cast<uint32_t*>(s_raw + kLutBytes);
     uint32_t* s_hi = s_lo + kLevels * kMaeBins;
     uint32_t* s_cn = s_hi + kLevels * kMaeBins;
-    uint2* s_queue = reinterpret_cast<uint2*>(s_cn);  // later passes (which keep no counts)
+    uint4* s_queue = reinterpret_cast<uint4*>(s_cn);  // kLaterQueue entries in the count histogram's space
     uint2* s_cand = reinterpret_cast<uint2*>(s_cn + kLevels * kMaeBins);  // [16][kMaeStage] (COLLECT)
     __shared__ uint32_t s_ncand[kLevels], s_gbase[kLevels];
     __shared__ volatile uint32_t s_over[kLevels];  // level's global list is known to have overflowed
@@ -761,18 +762,21 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
         }
         return zero_raw32();
     };
-    // A sample that may take part is queued (and handled on the spot when the queue is full).
-    auto offer = [&](float xk, uint32_t a) {
-        const uint32_t slot = atomicAdd(&s_qn, 1u);
-        if (slot < (uint32_t)kMaeQueue)
-            s_queue[slot] = make_uint2(__float_as_uint(xk), a);
-        else
-            later_sample(xk, a);
+    // A weight that may take part is queued as {address, block constant}: the streaming loop only
+    // notes where it is (a few instructions with one lane active); the division, the region search
+    // and the rest are done when the queue is worked off, with all lanes busy.  A full queue makes
+    // the lane handle its weight on the spot.
+    auto quotient = [&](float v, float m) {
+        if (div_safe(fabsf(m))) {  // the reciprocal sequence of the streaming loop, one weight
+            const float r = __frcp_rn(m), q0 = __fmul_rn(v, r);
+            return fmaf(fmaf(q0, -m, v), r, q0);
+        }
+        return normalise(v, m);
     };
     // A weight inside its table bin's hull may take part.  The streaming loop only marks such
     // weights in a bit mask (two comparisons and one predicated OR per weight); the few marked ones
-    // (about one in 200) are then read again by index, divided again and queued.  A row that cannot
-    // use the table (a zero, non-finite or extreme block constant) offers all its weights.
+    // (about one in 200) are queued by address.  A row that cannot use the table (a zero, non-finite
+    // or extreme block constant) offers all its weights.
     auto row = [&](const Raw32& raw, bool ok, const uint16_t* src) {
         uint32_t u[16];
         words_of(raw, u);
@@ -798,18 +802,20 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
                 if (x.y >= __uint_as_float(i1.x) && x.y <= __uint_as_float(i1.y)) marked |= 2u << (2 * k);
             }
         }
-        while (marked) {
-            const int j = __ffs(marked) - 1;
-            marked &= marked - 1u;
-            const float v = __uint_as_float((uint32_t)__ldg(src + j) << 16);
-            float x;
-            if (recip) {  // the same sequence as above, one weight
-                const float q0 = __fmul_rn(v, r);
-                x = fmaf(fmaf(q0, -m, v), r, q0);
-            } else {
-                x = normalise(v, m);
+        if (marked) {
+            const uint32_t cnt = (uint32_t)__popc(marked);
+            uint32_t slot = atomicAdd(&s_qn, cnt);
+            while (marked) {
+                const int j = __ffs(marked) - 1;
+                marked &= marked - 1u;
+                if (slot < (uint32_t)kLaterQueue) {
+                    const unsigned long long p = (unsigned long long)(src + j);
+                    s_queue[slot] = make_uint4((uint32_t)p, (uint32_t)(p >> 32), __float_as_uint(m), a);
+                } else {
+                    later_sample(quotient(__uint_as_float((uint32_t)__ldg(src + j) << 16), m), a);
+                }
+                ++slot;
             }
-            offer(x, a);
         }
     };
     // The queue is worked off by all threads: region search, digit, histogram; with COLLECT the
@@ -818,10 +824,12 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
     // however many rows a CTA streams.
     auto drain = [&]() {
         __syncthreads();
-        const uint32_t q = min(s_qn, (uint32_t)kMaeQueue);
+        const uint32_t q = min(s_qn, (uint32_t)kLaterQueue);
         for (uint32_t i = tid; i < q; i += kMaeThreads) {
-            const uint2 ent = s_queue[i];
-            later_sample(__uint_as_float(ent.x), ent.y);
+            const uint4 ent = s_queue[i];
+            const uint16_t* p = reinterpret_cast<const uint16_t*>(((unsigned long long)ent.y << 32) | ent.x);
+            const float m = __uint_as_float(ent.z);
+            later_sample(quotient(__uint_as_float((uint32_t)__ldg(p) << 16), m), ent.w);
         }
         __syncthreads();
         if (tid == 0) s_qn = 0u;
@@ -844,7 +852,7 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
     };
     // after a first pass on the fine grid about 130 samples per row are queued, up to a sixth of
     // them for one of the central levels (whose staging slot holds kMaeStage)
-    constexpr int kDrainRows = COLLECT ? 8 : 16;
+    constexpr int kDrainRows = 8;
     {
         bool ok_a, ok_b;
         const uint16_t *src_a = nullptr, *src_b = nullptr;
