@@ -597,6 +597,14 @@ struct LaterCtx {
     uint2* gcand;
     uint32_t cap;
 };
+// marked |= bit if lo <= x <= hi (iv = bits of {lo, hi}); two predicate operations and a predicated OR.
+__device__ __forceinline__ void mark_if_inside(uint32_t& marked, float x, uint2 iv, uint32_t bit)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.ge.f32 p, %1, %2;\n\tsetp.le.and.f32 p, %1, %3, p;\n\t@p or.b32 %0, %0, %4;\n\t}"
+        : "+r"(marked)
+        : "f"(x), "f"(__uint_as_float(iv.x)), "f"(__uint_as_float(iv.y)), "r"(bit));
+}
+
 template <bool COLLECT>
 __device__ __noinline__ void later_sample_fn(const LaterCtx* C, float xk, uint32_t a)
 {
@@ -714,6 +722,11 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
                 const uint32_t klo = max(lo64 > kmax ? kmax : (uint32_t)lo64, kmin);
                 const uint32_t khi = max(hi64 > kmax ? kmax : (uint32_t)hi64, kmin);
                 span = make_float2(key_to_float(klo), key_to_float(khi));
+                // The streaming loop tests the one-multiplication estimate x~ = RN(w RN(1/m)) of the
+                // quotient, which lies within 1.5 * 2^-23 (relative) of it: the span is widened by
+                // four times that, and what it lets through is tested again with the true quotient.
+                span.x -= fabsf(span.x) * 0x1p-21f + 1e-30f;
+                span.y += fabsf(span.y) * 0x1p-21f + 1e-30f;
             }
             s_span[tid] = span;
         }
@@ -787,19 +800,18 @@ mae_later32_kernel(const EmTensors T, const float* __restrict__ levels, MaeWs W,
         const bool table = __all_sync(kFull, ok && div_safe(g));
         const bool recip = div_safe(fabsf(m));
         const float r = recip ? __frcp_rn(m) : 0.0f;
-        const float2 rr = make_float2(r, r), nm = make_float2(-m, -m);
+        const float2 rr = make_float2(r, r);
         uint32_t marked = ok ? 0xffffffffu : 0u;
         if (table) {
             marked = 0u;
 #pragma unroll
             for (int k = 0; k < 16; ++k) {
                 const float2 v = make_float2(bf_lo(u[k]), bf_hi(u[k]));
-                const float2 q0 = __fmul2_rn(v, rr);
-                const float2 x = __ffma2_rn(__ffma2_rn(q0, nm, v), rr, q0);  // the true quotients
+                const float2 x = __fmul2_rn(v, rr);  // estimates of the quotients (see the widened spans)
                 const float2 key = lut_key2(x);
                 const uint2 i0 = lut_probe(key.x, lut_base), i1 = lut_probe(key.y, lut_base);
-                if (x.x >= __uint_as_float(i0.x) && x.x <= __uint_as_float(i0.y)) marked |= 1u << (2 * k);
-                if (x.y >= __uint_as_float(i1.x) && x.y <= __uint_as_float(i1.y)) marked |= 2u << (2 * k);
+                mark_if_inside(marked, x.x, i0, 1u << (2 * k));
+                mark_if_inside(marked, x.y, i1, 2u << (2 * k));
             }
         }
         if (marked) {
