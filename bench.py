@@ -60,7 +60,12 @@ OPQ_OUTLIER_FRACTION = 2.2e-3         # list capacity n / 64 leaves a 7x margin 
 # dram__bytes_read.sum + dram__bytes_write.sum per weight of the dominant component's kernels,
 # from the committed ncu captures (profiles/), taken on a two-layer slice and scaled by the number
 # of weights (traffic is proportional to it); None once the kernels have changed since.
-TRAFFIC_PER_WEIGHT = {"em_mae": None, "em_mse": None}
+TRAFFIC_PER_WEIGHT = {
+    # max-|w| pass 812.9 MB + first pass 813.9 MB + collecting pass 839.0 MB + two empty passes 0.14 MB
+    # over 404,750,336 weights (profiles/mae_*_c3_2layer_slice.md)
+    "em_mae": (812913664 + 813880064 + 839011328 + 140544) / 404750336.0,
+    "em_mse": (810906368 + 4438272) / 404750336.0,      # profiles/em_mse32_kernel_c3_2layer_slice.md
+}
 
 
 def measured_peak():
