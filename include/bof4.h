@@ -86,6 +86,12 @@ extern "C" {
  *     median[l] = weighted median of the members (the first sample, in ascending order, whose
  *     cumulative weight reaches half of s0[l]); the input level where s0[l] == 0,
  *     err_sum = sum over all weights of |w - m * xhat[code]|.
+ *     The weights |m| enter the selection as 31-bit fixed-point integers relative to the largest
+ *     |w| of the data (all sums are integer sums, hence independent of their order): exact for
+ *     |m| down to 2^-7 (fp32 weights) or 2^-23 (bf16 weights) of that magnitude, truncated below
+ *     and zero beyond 2^-31 of it.  The median is the exact weighted median unless the truncated
+ *     parts add up to more than the margin by which the cumulative weight passes half of s0[l]
+ *     at the selected sample; s0[l] is the sum of the fixed-point weights, rescaled.
  * For the normalised-domain metrics m^2 and |m| are replaced by 1 and w by x in these sums.
  * count[l] is the number of members of region l, n_total the number of weights seen.
  * For MSE median[l] is the centroid s1[l]/s0[l] rounded to fp32 (input level where s0[l] == 0).
