@@ -970,14 +970,15 @@ mae_select_kernel(MaeWs W, int first)
 // matched the first digit is finished here: the remaining digits are selected from the list.
 // A level whose list overflowed takes the ordinary histogram step and goes on to the later
 // passes.
-__global__ void __launch_bounds__(kMaeBins)
+__global__ void __launch_bounds__(kMaeThreads)
 mae_resolve_kernel(MaeWs W)
 {
-    __shared__ unsigned long long s_wsum[kMaeBins / 32];
+    __shared__ unsigned long long s_wsum[kMaeThreads / 32];
     __shared__ uint32_t s_lo[kMaeBins], s_hi[kMaeBins];  // 64-bit bins as two words: native 32-bit atomics
     __shared__ PickResult s_res;
     MaeState* S = W.state;
     const int l = blockIdx.x, j = threadIdx.x;
+    const bool has_bin = j < kMaeBins;  // one thread per bin; all threads read the list
     int top = S->top[l];
     if (top <= 0) return;  // uniform over the CTA
     const uint32_t m = S->cand_count[l];
@@ -987,9 +988,12 @@ mae_resolve_kernel(MaeWs W)
     unsigned long long all;
     // the digit of this pass, from the global histogram (also clears it)
     {
-        const unsigned long long mine = W.hist[l * kMaeBins + j];
-        W.hist[l * kMaeBins + j] = 0ull;
-        const PickResult r = pick_bin(mine, before, total, false, s_wsum, &s_res, &all);
+        unsigned long long mine = 0ull;
+        if (has_bin) {
+            mine = W.hist[l * kMaeBins + j];
+            W.hist[l * kMaeBins + j] = 0ull;
+        }
+        const PickResult r = pick_bin<kMaeThreads>(mine, before, total, false, s_wsum, &s_res, &all);
         const int sh = max(top - kMaeDigitBits, 0);
         before += r.excl;
         prefix = (prefix << (top - sh)) | (uint32_t)r.bin;
@@ -997,21 +1001,24 @@ mae_resolve_kernel(MaeWs W)
     }
     if (m <= W.cand_cap) {
         const uint2* cand = W.cand + (size_t)l * W.cand_cap;
+        constexpr int kInFlight = 16;  // independent loads per thread: the lists reach millions of entries
         while (top > 0) {
             const int sh = max(top - kMaeDigitBits, 0);
             const uint32_t mask = (1u << (top - sh)) - 1u;
-            s_lo[j] = 0u;
-            s_hi[j] = 0u;
+            if (has_bin) {
+                s_lo[j] = 0u;
+                s_hi[j] = 0u;
+            }
             __syncthreads();
-            for (uint32_t i0 = 0; i0 < m; i0 += 8 * kMaeBins) {  // 8 independent loads in flight per thread
-                uint2 c[8];
+            for (uint32_t i0 = 0; i0 < m; i0 += kInFlight * kMaeThreads) {
+                uint2 c[kInFlight];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint32_t i = i0 + u * kMaeBins + j;
-                    c[u] = (i < m) ? cand[i] : make_uint2(0xffffffffu, 0u);
+                for (int u = 0; u < kInFlight; ++u) {
+                    const uint32_t i = i0 + u * kMaeThreads + j;
+                    c[u] = (i < m) ? __ldcg(&cand[i]) : make_uint2(0xffffffffu, 0u);
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u)
+                for (int u = 0; u < kInFlight; ++u)
                     if (c[u].y != 0u && (c[u].x >> top) == prefix) {
                         const uint32_t bin = (c[u].x >> sh) & mask;
                         const uint32_t old = atomicAdd(&s_lo[bin], c[u].y);
@@ -1019,8 +1026,8 @@ mae_resolve_kernel(MaeWs W)
                     }
             }
             __syncthreads();
-            const PickResult r = pick_bin(((unsigned long long)s_hi[j] << 32) + s_lo[j], before, total, false,
-                                          s_wsum, &s_res, &all);
+            const unsigned long long mine = has_bin ? ((unsigned long long)s_hi[j] << 32) + s_lo[j] : 0ull;
+            const PickResult r = pick_bin<kMaeThreads>(mine, before, total, false, s_wsum, &s_res, &all);
             before += r.excl;
             prefix = (prefix << (top - sh)) | (uint32_t)r.bin;
             top = sh;
@@ -1730,7 +1737,7 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
             continue;
         }
         if (p == collect_pass)
-            mae_resolve_kernel<<<kLevels, kMaeBins, 0, st>>>(W);
+            mae_resolve_kernel<<<kLevels, kMaeThreads, 0, st>>>(W);
         else
             mae_select_kernel<<<kLevels, kMaeBins, 0, st>>>(W, first ? 1 : 0);
         BOF4_CUDA_TRY(cudaGetLastError());
