@@ -20,6 +20,8 @@
 // the data (exact whenever |m| is within 2^-7 of it for fp32 input, 2^-23 for bf16 input), so
 // every sum is an integer sum: independent of the order of the atomics, bit-reproducible, and
 // equal to the exact real-number sums that define the median.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "em_common.cuh"
 #include "lane32.cuh"
@@ -969,30 +971,35 @@ mae_select_kernel(MaeWs W, int first)
 // After the collecting (second) pass.  A level whose candidate list holds every sample that
 // matched the first digit is finished here: the remaining digits are selected from the list.
 // A level whose list overflowed takes the ordinary histogram step and goes on to the later
-// passes.
-__global__ void __launch_bounds__(kMaeThreads)
+// passes.  The lists reach millions of entries, so a cluster of kResolveCtas CTAs shares one
+// level: each reads its part of the list into its own histogram, the histograms are summed
+// through distributed shared memory, and every CTA takes the same (deterministic) decision.
+constexpr int kResolveCtas = 8;
+
+__global__ void __cluster_dims__(kResolveCtas, 1, 1) __launch_bounds__(kMaeThreads)
 mae_resolve_kernel(MaeWs W)
 {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned rank = cluster.block_rank();
     __shared__ unsigned long long s_wsum[kMaeThreads / 32];
     __shared__ uint32_t s_lo[kMaeBins], s_hi[kMaeBins];  // 64-bit bins as two words: native 32-bit atomics
     __shared__ PickResult s_res;
     MaeState* S = W.state;
-    const int l = blockIdx.x, j = threadIdx.x;
+    const int l = blockIdx.x / kResolveCtas, j = threadIdx.x;
     const bool has_bin = j < kMaeBins;  // one thread per bin; all threads read the list
     int top = S->top[l];
-    if (top <= 0) return;  // uniform over the CTA
+    if (top <= 0) return;  // the same for all CTAs of the cluster
     const uint32_t m = S->cand_count[l];
     unsigned long long before = S->before[l];
     const unsigned long long total = S->total[l];
     uint32_t prefix = S->prefix[l];
     unsigned long long all;
-    // the digit of this pass, from the global histogram (also clears it)
+    // the digit of this pass, from the global histogram (cleared once every CTA has read it)
     {
-        unsigned long long mine = 0ull;
-        if (has_bin) {
-            mine = W.hist[l * kMaeBins + j];
-            W.hist[l * kMaeBins + j] = 0ull;
-        }
+        const unsigned long long mine = has_bin ? __ldcg(&W.hist[l * kMaeBins + j]) : 0ull;
+        cluster.sync();  // also orders the reads of the state above before the write at the end
+        if (rank == 0 && has_bin) W.hist[l * kMaeBins + j] = 0ull;
         const PickResult r = pick_bin<kMaeThreads>(mine, before, total, false, s_wsum, &s_res, &all);
         const int sh = max(top - kMaeDigitBits, 0);
         before += r.excl;
@@ -1001,7 +1008,8 @@ mae_resolve_kernel(MaeWs W)
     }
     if (m <= W.cand_cap) {
         const uint2* cand = W.cand + (size_t)l * W.cand_cap;
-        constexpr int kInFlight = 16;  // independent loads per thread: the lists reach millions of entries
+        constexpr int kInFlight = 16;  // independent loads per thread
+        constexpr uint32_t kChunk = kInFlight * kMaeThreads;
         while (top > 0) {
             const int sh = max(top - kMaeDigitBits, 0);
             const uint32_t mask = (1u << (top - sh)) - 1u;
@@ -1010,7 +1018,7 @@ mae_resolve_kernel(MaeWs W)
                 s_hi[j] = 0u;
             }
             __syncthreads();
-            for (uint32_t i0 = 0; i0 < m; i0 += kInFlight * kMaeThreads) {
+            for (uint32_t i0 = rank * kChunk; i0 < m; i0 += kResolveCtas * kChunk) {
                 uint2 c[kInFlight];
 #pragma unroll
                 for (int u = 0; u < kInFlight; ++u) {
@@ -1025,15 +1033,23 @@ mae_resolve_kernel(MaeWs W)
                         if (old + c[u].y < old) atomicAdd(&s_hi[bin], 1u);
                     }
             }
-            __syncthreads();
-            const unsigned long long mine = has_bin ? ((unsigned long long)s_hi[j] << 32) + s_lo[j] : 0ull;
+            cluster.sync();  // every CTA's histogram is complete
+            unsigned long long mine = 0ull;
+            if (has_bin) {
+                for (unsigned r = 0; r < kResolveCtas; ++r) {  // fixed order; integer sums anyway
+                    const uint32_t* rlo = cluster.map_shared_rank(s_lo, r);
+                    const uint32_t* rhi = cluster.map_shared_rank(s_hi, r);
+                    mine += ((unsigned long long)rhi[j] << 32) + rlo[j];
+                }
+            }
+            cluster.sync();  // nobody clears its histogram while another CTA still reads it
             const PickResult r = pick_bin<kMaeThreads>(mine, before, total, false, s_wsum, &s_res, &all);
             before += r.excl;
             prefix = (prefix << (top - sh)) | (uint32_t)r.bin;
             top = sh;
         }
     }
-    if (j == 0) {
+    if (rank == 0 && j == 0) {
         S->before[l] = before;
         S->prefix[l] = prefix;
         S->top[l] = top;
@@ -1737,7 +1753,7 @@ int mae_iteration(const EmArgs& a, const float* d_levels_in, float* d_levels_out
             continue;
         }
         if (p == collect_pass)
-            mae_resolve_kernel<<<kLevels, kMaeThreads, 0, st>>>(W);
+            mae_resolve_kernel<<<kLevels * kResolveCtas, kMaeThreads, 0, st>>>(W);
         else
             mae_select_kernel<<<kLevels, kMaeBins, 0, st>>>(W, first ? 1 : 0);
         BOF4_CUDA_TRY(cudaGetLastError());
