@@ -152,6 +152,22 @@ BOF4_API int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int n
                       size_t ws_bytes, void* stream);
 
 /*
+ * M step of a fit whose E-step statistics come from several bof4_em_step calls - the joint fit
+ * over the shards of several GPUs: every GPU runs bof4_em_step on its shard, the records are
+ * gathered in rank order (432 bytes per GPU and iteration, the only exchange the path needs), and
+ * every GPU calls this with the same records, so that all hold the same levels (Sec. 3.2, Eq. 6:
+ * the centroid is a ratio of sums, and sums over shards add).  The records are summed in index
+ * order in fp64.  MSE metrics only: a weighted median of a union (Eq. 8) cannot be merged from
+ * per-shard medians (BOF4_ERR_INVALID_ARG).
+ *   d_stats     device, n_records records as written by bof4_em_step with the levels in d_codebook
+ *   d_codebook  in: the levels the records were computed with; out: free levels updated
+ *   d_err_slot  out or NULL: mean error of the incoming levels over all records' weights
+ *   d_total     out or NULL: the summed record
+ */
+BOF4_API int bof4_m_step(const bof4_em_stats* d_stats, int n_records, int metric, float* d_codebook,
+                uint32_t fixed_mask, double* d_err_slot, bof4_em_stats* d_total, void* stream);
+
+/*
  * Block-wise quantisation (Sec. 2.1 Eq. 1-3, Sec. 3.1 Eq. 4): per block the constant m,
  * x = w / m (x = 0 for an all-zero block), code = region of x.
  *   d_codes   out [(n+1)/2] bytes; byte k = (code[2k] << 4) | code[2k+1]

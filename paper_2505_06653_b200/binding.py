@@ -51,7 +51,7 @@ EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_qu
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_theoretical_codebook_batch",
            "bof4_gemv", "bof4_outlier_count", "bof4_scales_compress", "bof4_scales_expand",
-           "bof4_theoretical_codebook_general", "bof4_quantize_batch", "bof4_dequantize_batch")
+           "bof4_theoretical_codebook_general", "bof4_quantize_batch", "bof4_dequantize_batch", "bof4_m_step")
 
 
 class Bof4Error(RuntimeError):
@@ -111,6 +111,8 @@ def lib() -> ctypes.CDLL:
         L.bof4_quantize_batch.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
         L.bof4_dequantize_batch.restype = i32
         L.bof4_dequantize_batch.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, i32, vp]
+        L.bof4_m_step.restype = i32
+        L.bof4_m_step.argtypes = [vp, i32, i32, vp, ctypes.c_uint32, vp, vp, vp]
         L.bof4_scales_compress.restype = i32
         L.bof4_scales_compress.argtypes = [vp, i32, i64, i32, vp, vp, vp, vp]
         L.bof4_scales_expand.restype = i32
@@ -246,6 +248,66 @@ def bof4_em_step(weights, block_size: int, norm: int, metric: int, levels,
     rec = EmStats.from_buffer_copy(stats.cpu().numpy().tobytes())
     return dict(s1=np.array(rec.s1), s0=np.array(rec.s0), count=np.array(rec.count, dtype=np.uint64),
                 err_sum=float(rec.err_sum), n=int(rec.n_total), median=np.array(rec.median, dtype=np.float32))
+
+
+def em_step_record(weights, block_size: int, norm: int, metric: int, levels: torch.Tensor,
+                   workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """bof4_em_step with the record left on the device (uint8[sizeof(bof4_em_stats)]); `levels` is a
+    device tensor fp32[16].  Nothing waits for the stream."""
+    ws, dt, ptrs, sizes = _tensor_list(weights)
+    dev = ws[0].device
+    cb = _codebook(levels, dev)
+    wsp = workspace if workspace is not None else _workspace(
+        OP_EM, sum(w.numel() for w in ws), block_size, metric, dev)
+    stats = _new(ctypes.sizeof(EmStats), torch.uint8, dev, zero=True)
+    with torch.cuda.device(dev):
+        _check(lib().bof4_em_step(ptrs, sizes, len(ws), dt, block_size, norm, metric, _ptr(cb),
+                                  _ptr(stats), _ptr(wsp), wsp.numel(), _stream()))
+    return stats
+
+
+def gather_records(record: torch.Tensor, group=None) -> torch.Tensor:
+    """The records of all ranks of `group`, concatenated in rank order (the record itself without a
+    process group).  The one exchange of a joint fit: 432 bytes per rank and iteration."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return record
+    world = dist.get_world_size(group)
+    out = torch.empty(world * record.numel(), dtype=record.dtype, device=record.device)
+    dist.all_gather_into_tensor(out, record.contiguous(), group=group)
+    return out
+
+
+def bof4_m_step(records: torch.Tensor, metric: int, codebook: torch.Tensor, fixed_mask: int,
+                err_slot: Optional[torch.Tensor] = None) -> None:
+    """Sums the gathered records in rank order and updates `codebook` (device fp32[16]) in place."""
+    records = _dev(records, "records")
+    n = records.numel() // ctypes.sizeof(EmStats)
+    if records.dtype != torch.uint8 or n * ctypes.sizeof(EmStats) != records.numel():
+        raise ValueError("records must be whole bof4_em_stats records as uint8")
+    cb = _dev(codebook, "codebook")
+    if cb.dtype != torch.float32 or cb.numel() != LEVELS:
+        raise ValueError("codebook must be a device tensor float32[16]")
+    with torch.cuda.device(cb.device):
+        _check(lib().bof4_m_step(_ptr(records), n, metric, _ptr(cb), fixed_mask,
+                                 _ptr(err_slot) if err_slot is not None else None, None, _stream()))
+
+
+def bof4_fit_codebook_joint(weights, block_size: int, norm: int, metric: int, levels, fixed_mask: int,
+                            iters: int, group=None):
+    """Joint fit over the shards of all ranks of `group` (one process per GPU): every iteration is
+    one bof4_em_step on the local shard, one all-gather of the 432-byte records and one bof4_m_step,
+    so that every rank ends with the same levels.  MSE metrics.  -> (levels, err_log) on the device."""
+    ws, _, _, _ = _tensor_list(weights)
+    dev = ws[0].device
+    cb = _codebook(levels, dev).clone()
+    log = _new(max(iters, 1), torch.float64, dev, zero=True)
+    wsp = _workspace(OP_EM, sum(w.numel() for w in ws), block_size, metric, dev)
+    for t in range(iters):
+        rec = em_step_record(ws, block_size, norm, metric, cb, workspace=wsp)
+        bof4_m_step(gather_records(rec, group), metric, cb, fixed_mask, log[t:t + 1])
+    torch.cuda.current_stream(dev).synchronize()
+    return cb, log[:iters]
 
 
 def bof4_fit_codebook(weights, block_size: int, norm: int, metric: int, levels, fixed_mask: int,

@@ -144,6 +144,46 @@ em_mse_finalize_kernel(const double* partials, const MseTail t)
     mse_combine(partials, t, s_q, s_corr, s_stage);
 }
 
+// M step from E-step records that were produced by separate calls (one per GPU of a joint fit,
+// gathered in rank order): sums them in index order in fp64 and updates the free levels (Eq. 6).
+// One warp; lane l owns level l.
+__global__ void __launch_bounds__(32)
+m_step_kernel(const bof4_em_stats* __restrict__ stats, int n_records, float* __restrict__ codebook,
+              uint32_t fixed_mask, double* __restrict__ err_slot, bof4_em_stats* __restrict__ total)
+{
+    const int l = threadIdx.x;
+    double s1 = 0.0, s0 = 0.0, err = 0.0;
+    unsigned long long cnt = 0ull;
+    long long n = 0;
+    for (int r = 0; r < n_records; ++r) {
+        if (l < kLevels) {
+            s1 += stats[r].s1[l];
+            s0 += stats[r].s0[l];
+            cnt += stats[r].count[l];
+        }
+        err += stats[r].err_sum;
+        n += stats[r].n_total;
+    }
+    if (l < kLevels) {
+        const float old = codebook[l];
+        const float cen = (s0 > 0.0) ? (float)(s1 / s0) : old;
+        if (total) {
+            total->s1[l] = s1;
+            total->s0[l] = s0;
+            total->count[l] = cnt;
+            total->median[l] = cen;
+        }
+        if (!((fixed_mask >> l) & 1u)) codebook[l] = cen;
+    }
+    if (l == 0) {
+        if (total) {
+            total->err_sum = err;
+            total->n_total = n;
+        }
+        if (err_slot) *err_slot = (n > 0) ? err / (double)n : 0.0;
+    }
+}
+
 // The short last blocks of ragged tensors: one CTA, block after block.  Warp l sums the members
 // of region l (lane-strided, then the butterfly: a fixed order), in fp64 throughout, and the
 // result goes to a record of its own.
@@ -883,5 +923,23 @@ extern "C" int bof4_fit_codebook(const void* const* h_w, const int64_t* h_n, int
                            d_err_log ? d_err_log + t : nullptr, d_ws, ws_bytes, st);
         if (rc) return rc;
     }
+    return BOF4_OK;
+}
+
+extern "C" int bof4_m_step(const bof4_em_stats* d_stats, int n_records, int metric, float* d_codebook,
+                           uint32_t fixed_mask, double* d_err_slot, bof4_em_stats* d_total, void* stream)
+{
+    if (!d_stats || n_records < 1 || !d_codebook) {
+        set_error("bof4_m_step: NULL pointer or no records");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (metric != BOF4_METRIC_MSE && metric != BOF4_METRIC_MSE_NORMALIZED) {
+        set_error("bof4_m_step: only the MSE centroids are sums that can be merged from separate records "
+                  "(a weighted median of a union needs the histograms of every selection pass)");
+        return BOF4_ERR_INVALID_ARG;
+    }
+    m_step_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(d_stats, n_records, d_codebook, fixed_mask,
+                                                                   d_err_slot, d_total);
+    BOF4_CUDA_TRY(cudaGetLastError());
     return BOF4_OK;
 }
