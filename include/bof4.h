@@ -330,6 +330,28 @@ BOF4_API int bof4_gemv(const uint8_t* d_codes, const void* d_scales, int scale_d
               int64_t capacity, float* d_y, void* stream);
 
 /*
+ * The same product for a batch of right-hand sides on the tensor cores (App. E.2: the decode-side
+ * consumer with several tokens in flight): Y = W_q X^T with W rows x cols as for bof4_gemv and
+ * n_rhs = 16, 32, 48 or 64 right-hand sides.  Reading: the A operand is the dequantised weight
+ * rounded to bf16 - bit for bit the output of bof4_dequantize (Eq. 3, round to nearest even) - X is
+ * bf16, products are exact, sums are accumulated in fp32 by the tensor cores (tcgen05.mma into
+ * tensor memory), whose summation order and intermediate rounding are the hardware's: the result
+ * agrees with the fp64 sum of the same products within 2^-14 * sum |w x| (cols / 16 accumulation
+ * steps of at most 2^-23 each for cols <= 8192 * 16).  No outlier list: apply bof4_gemv's
+ * correction per right-hand side, or dequantise.
+ *   rows       multiple of 128;  cols multiple of 64 and of block_size
+ *   d_codes    device, rows * cols / 2 bytes, 16-byte aligned;  d_scales as for bof4_gemv
+ *   d_x        device, bf16 [n_rhs][cols] (each right-hand side contiguous), 16-byte aligned
+ *   d_y        device, fp32 [rows][n_rhs], written
+ *   d_status   device int, written: 0, or 1 when a bounded wait inside the kernel ran out (the result
+ *              is then undefined; the kernel has still released its tensor memory and returned)
+ * One launch on `stream` (preceded by a 4-byte clear of d_status); no workspace, no synchronisation.
+ */
+BOF4_API int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t rows,
+                 int64_t cols, int block_size, const float* d_codebook, const void* d_x, int n_rhs,
+                 float* d_y, int* d_status, void* stream);
+
+/*
  * Data-free codebook for unit-variance Gaussian weights (Sec. 3.2 Eq. 5 / Eq. 7; App. B.2): `iters`
  * Lloyd iterations in which every free level becomes the theoretical centroid of its region,
  * a ratio (MSE) or root (MAE) of integrals over the absolute block maximum, evaluated by

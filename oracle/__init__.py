@@ -7,7 +7,9 @@ to fp32 (exact) before they reach the C code.
 
 Parity pins: the C functions as listed in ``bof4_oracle.c``; ``gemv`` (fp64 numpy, the plain
 definition of the decoded matrix-vector product) by hand-built closed forms and numpy's matvec
-of the separately dequantised and restored matrix (tests/test_oracle_pins.py).
+of the separately dequantised and restored matrix; ``gemm_bf16`` by a hand-built case, by its
+columns equalling ``gemv`` wherever the products of Eq. 3 are exact in bf16, and by the size of
+the bf16 rounding where they are not (tests/test_oracle_pins.py).
 """
 from __future__ import annotations
 
@@ -275,3 +277,14 @@ def gemv(codes: np.ndarray, scales: np.ndarray, rows: int, cols: int, I: int, xh
     xv = np.asarray(x, dtype=np.float64).reshape(-1)
     assert xv.size == cols
     return W @ xv, np.abs(W) @ np.abs(xv)
+
+
+def gemm_bf16(codes: np.ndarray, scales: np.ndarray, rows: int, cols: int, I: int, xhat, X):
+    """Y = W X^T in fp64 for a batch of right-hand sides X [n_rhs, cols], the decoded weight being
+    the dequantised value ROUNDED TO bf16 (Eq. 3 followed by round-to-nearest-even, i.e. what
+    `dequantize` returns as bf16): the operand precision of the batched tensor-core consumer.
+    Also returns sum_c |W[r, c] X[b, c]|.  -> (Y fp64 [rows, n_rhs], mag fp64 [rows, n_rhs])."""
+    w32 = dequantize(codes, scales, I, xhat, n=rows * cols)              # fp32 products of Eq. 3
+    W = bf16_bits_to_f32(f32_to_bf16_bits(w32)).astype(np.float64).reshape(rows, cols)
+    Xd = np.asarray(X, dtype=np.float64).reshape(-1, cols)
+    return W @ Xd.T, np.abs(W) @ np.abs(Xd).T

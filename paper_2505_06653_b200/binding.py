@@ -51,7 +51,7 @@ EXPORTS = ("bof4_workspace_bytes", "bof4_em_step", "bof4_fit_codebook", "bof4_qu
            "opq_split", "opq_split_static", "bof4_quantize_opq", "bof4_dequantize", "bof4_opq_threshold",
            "bof4_default_init", "bof4_last_error", "bof4_theoretical_codebook", "bof4_theoretical_codebook_batch",
            "bof4_gemv", "bof4_outlier_count", "bof4_scales_compress", "bof4_scales_expand",
-           "bof4_theoretical_codebook_general", "bof4_quantize_batch", "bof4_dequantize_batch", "bof4_m_step")
+           "bof4_theoretical_codebook_general", "bof4_quantize_batch", "bof4_dequantize_batch", "bof4_m_step", "bof4_gemm_tc")
 
 
 class Bof4Error(RuntimeError):
@@ -111,6 +111,8 @@ def lib() -> ctypes.CDLL:
         L.bof4_quantize_batch.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
         L.bof4_dequantize_batch.restype = i32
         L.bof4_dequantize_batch.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, i32, vp]
+        L.bof4_gemm_tc.restype = i32
+        L.bof4_gemm_tc.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, vp, vp, vp]
         L.bof4_m_step.restype = i32
         L.bof4_m_step.argtypes = [vp, i32, i32, vp, ctypes.c_uint32, vp, vp, vp]
         L.bof4_scales_compress.restype = i32
@@ -476,6 +478,25 @@ def opq_split(w: torch.Tensor, block_size: int, tau: float, capacity: int,
         _check(lib().opq_split(_ptr(w), dt, n, block_size, tau, _ptr(clean), _ptr(idx), _ptr(val),
                                capacity, _ptr(cnt), _ptr(wsp), wsp.numel(), _stream()))
     return clean, idx, val, cnt
+
+
+def bof4_gemm_tc(codes: torch.Tensor, scales: torch.Tensor, rows: int, cols: int, block_size: int, levels,
+                 x: torch.Tensor):
+    """Y fp32 [rows, n_rhs] = W_q X^T on the tensor cores for x bf16 [n_rhs, cols].
+    -> (y, status int32[1]); status 0 unless a bounded wait inside the kernel ran out."""
+    codes = _dev(codes, "codes")
+    scales = _dev(scales, "scales")
+    x = _dev(x, "x")
+    if x.dtype != torch.bfloat16 or x.dim() != 2 or x.shape[1] != cols or codes.numel() * 2 != rows * cols:
+        raise ValueError("x must be bf16 [n_rhs, cols] and codes must hold rows * cols weights")
+    n_rhs = x.shape[0]
+    cb = _codebook(levels, codes.device)
+    y = _new(rows * n_rhs, torch.float32, codes.device).view(rows, n_rhs)
+    status = _new(1, torch.int32, codes.device, zero=True)
+    with torch.cuda.device(codes.device):
+        _check(lib().bof4_gemm_tc(_ptr(codes), _ptr(scales), _dt(scales), rows, cols, block_size, _ptr(cb), _ptr(x),
+                                  n_rhs, _ptr(y), _ptr(status), _stream()))
+    return y, status
 
 
 def bof4_outlier_count(n_out: torch.Tensor, capacity: int) -> int:

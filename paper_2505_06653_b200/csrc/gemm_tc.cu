@@ -1,0 +1,284 @@
+// Decode fused into a batched consumer on the tensor cores: Y = W_q X^T for 16 ... 64 right-hand
+// sides (App. E.2 times token generation; with several tokens or sequences in flight the
+// matrix-vector product of gemv.cu becomes this small-N matrix product, and the decode of Eq. 3
+// amortises over the batch).
+//
+// Reading (the paper gives no arithmetic for a fused consumer): the A operand is the dequantised
+// weight rounded to bf16, bit for bit what bof4_dequantize writes (Eq. 3, then round to nearest
+// even), X is bf16, products are exact and the sums are accumulated in fp32 by the tensor cores.
+//
+// One CTA owns 128 rows of W and all of K.  Per k-block of 64 weights the 256 threads decode the
+// 128 x 64 tile (4 KiB of codes) into shared memory as bf16 in the K-major 128-byte-swizzled
+// layout that the tcgen05 shared-memory descriptor names (8-row groups of 1024 bytes, 16-byte
+// chunk c of row r stored at chunk c ^ (r & 7)), copy the matching 64 columns of X the same way,
+// and one thread issues four tcgen05.mma (M = 128, N = batch, K = 16 each) that accumulate into
+// tensor memory.  Two shared-memory stages: a tcgen05.commit per k-block arrives on the stage's
+// mbarrier when the tensor cores have finished reading it, and the producers wait on that
+// barrier (bounded; a time-out sets the status word, the kernel still frees its tensor memory
+// and returns) before they overwrite the stage.  The epilogue reads the accumulator with
+// tcgen05.ld (one row per thread) and writes fp32.
+#include "common.cuh"
+
+namespace bof4 {
+
+constexpr int kTcThreads = 256;
+constexpr int kTcM = 128;         // rows per CTA = tensor-memory lanes
+constexpr int kTcK = 64;          // weights per k-block: one 128-byte swizzle row of bf16
+constexpr int kTcStages = 2;
+constexpr int kTcMaxN = 64;
+constexpr int kTcTmemCols = 64;   // power of two >= 32 and >= N
+constexpr int kTcABytes = kTcM * kTcK * 2;     // 16 KiB
+constexpr int kTcBBytes = kTcMaxN * kTcK * 2;  // 8 KiB
+constexpr int kTcSmem = kTcStages * (kTcABytes + kTcBBytes) + 1024;  // + slack to align to 1024 bytes
+constexpr uint32_t kTcSpinLimit = 1u << 16;    // try_wait calls before a wait gives up (a k-block takes microseconds)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Shared-memory matrix descriptor of a K-major tile in the 128-byte swizzled layout: start
+// address and offsets in units of 16 bytes, leading offset 1 (unused for swizzled K-major), stride
+// between 8-row groups 1024 bytes, descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, M = 128, N = n.
+__host__ __device__ inline uint32_t tc_instr_desc(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
+}
+
+__device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < kTcSpinLimit; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
+template <class ST>
+__device__ __forceinline__ float tc_scale(const void* scales, int64_t b);
+template <>
+__device__ __forceinline__ float tc_scale<F32>(const void* scales, int64_t b)
+{
+    return __ldg(static_cast<const float*>(scales) + b);
+}
+template <>
+__device__ __forceinline__ float tc_scale<BF16>(const void* scales, int64_t b)
+{
+    return __uint_as_float((uint32_t)__ldg(static_cast<const uint16_t*>(scales) + b) << 16);
+}
+
+template <class ST>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t cols, int block_size,
+               const float* __restrict__ levels, const uint16_t* __restrict__ x, int n_rhs, float* __restrict__ y,
+               int* __restrict__ status)
+{
+    extern __shared__ unsigned char s_dyn[];
+    __shared__ float s_lv[kLevels];
+    __shared__ __align__(8) unsigned long long s_bar[kTcStages + 1];  // one per stage, one for the end
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_fail;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t tiles = (smem_u32(s_dyn) + 1023u) & ~1023u;  // 1024-byte aligned: the swizzle atoms start here
+    unsigned char* tiles_ptr = s_dyn + (tiles - smem_u32(s_dyn));
+    const int64_t row0 = (int64_t)blockIdx.x * kTcM;
+    const int kblocks = (int)(cols / kTcK);
+
+    if (tid < kLevels) s_lv[tid] = levels[tid];
+    if (tid == 0) {
+        s_fail = 0;
+        for (int s = 0; s <= kTcStages; ++s)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_bar[s])), "r"(1) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {  // tensor memory for the 128 x N fp32 accumulator
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
+                     "r"(kTcTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s_tmem;
+    const uint32_t idesc = tc_instr_desc(n_rhs);
+
+    // this thread's part of the A tile: half a row (32 weights = 16 code bytes = four 16-byte chunks)
+    const int a_row = tid >> 1, a_half = tid & 1;
+    const uint8_t* a_codes = codes + ((row0 + a_row) * cols) / 2 + a_half * 16;
+    const int64_t a_first = (row0 + a_row) * cols + a_half * 32;  // flat index of its first weight in k-block 0
+    const uint32_t a_off = (uint32_t)((a_row >> 3) * 1024 + (a_row & 7) * 128);
+    bool failed = false, final_commit = false;
+    for (int kb = 0; kb < kblocks; ++kb) {
+        const int s = kb & 1;
+        unsigned char* sa = tiles_ptr + s * (kTcABytes + kTcBBytes);
+        unsigned char* sb = sa + kTcABytes;
+        if (kb >= kTcStages) {  // the tensor cores must have finished reading this stage (k-block kb - 2)
+            if (!tc_wait(smem_u32(&s_bar[s]), (uint32_t)(((kb >> 1) - 1) & 1))) s_fail = 1;
+        }
+        __syncthreads();
+        if (s_fail) {  // uniform: a wait ran out somewhere in the CTA
+            failed = true;
+            break;
+        }
+        // decode: 16 code bytes -> 32 bf16 values of Eq. 3, rounded to nearest even
+        const uint4 cc = *reinterpret_cast<const uint4*>(a_codes + (int64_t)kb * (kTcK / 2));
+        const float m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) / block_size);
+        const uint32_t word[4] = {cc.x, cc.y, cc.z, cc.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {  // chunk j of this half: weights 8j .. 8j+7 = code bytes 4j .. 4j+3
+            uint32_t p[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const uint32_t byte = (word[j] >> (8 * b)) & 0xffu;
+                const float hi = __fmul_rn(m, s_lv[byte >> 4]), lo = __fmul_rn(m, s_lv[byte & 15]);
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(p[b]) : "f"(lo), "f"(hi));  // even weight in the low half
+            }
+            const int chunk = a_half * 4 + j;
+            *reinterpret_cast<uint4*>(sa + a_off + ((chunk ^ (a_row & 7)) * 16)) = make_uint4(p[0], p[1], p[2], p[3]);
+        }
+        // the X tile: 16-byte chunk ch (8 values) of right-hand side n, same layout
+        for (int q = tid; q < n_rhs * 8; q += kTcThreads) {
+            const int n = q >> 3, ch = q & 7;
+            *reinterpret_cast<uint4*>(sb + (n >> 3) * 1024 + (n & 7) * 128 + ((ch ^ (n & 7)) * 16)) =
+                *reinterpret_cast<const uint4*>(x + (int64_t)n * cols + (int64_t)kb * kTcK + ch * 8);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t da = tc_smem_desc(smem_u32(sa)), db = tc_smem_desc(smem_u32(sb));
+#pragma unroll
+            for (int kk = 0; kk < kTcK / 16; ++kk) {  // 32 bytes of K per instruction: +2 in the address field
+                const uint32_t acc = (kb > 0 || kk > 0) ? 1u : 0u;
+                asm volatile(
+                    "{\n\t.reg .pred p;\n\t"
+                    "setp.ne.b32 p, %4, 0;\n\t"
+                    "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                    :
+                    : "r"(tmem), "l"(da + (uint64_t)(2 * kk)), "l"(db + (uint64_t)(2 * kk)), "r"(idesc), "r"(acc), "r"(0u)
+                    : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                             smem_u32(&s_bar[s]))
+                         : "memory");
+            if (kb == kblocks - 1) {
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                                 smem_u32(&s_bar[kTcStages]))
+                             : "memory");
+                final_commit = true;
+            }
+        }
+    }
+    // all instructions issued: wait for the accumulator, then read it back, one row per thread
+    if (!failed && kblocks > 0) {
+        if (!tc_wait(smem_u32(&s_bar[kTcStages]), 0u)) s_fail = 1;
+    }
+    __syncthreads();
+    failed = failed || s_fail != 0 || kblocks == 0;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (!failed && warp < 4) {
+        float* yrow = y + (row0 + warp * 32 + lane) * n_rhs;
+        for (int c0 = 0; c0 < n_rhs; c0 += 8) {
+            uint32_t v[8];
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                         : "r"(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int c = 0; c < 8; ++c) yrow[c0 + c] = __uint_as_float(v[c]);
+        }
+    }
+    if (failed && kblocks > 0) {
+        // A wait ran out.  The instructions already issued may still be running (their operands live in
+        // this CTA's shared memory, their result in its tensor memory): one more commit covers them
+        // all, and they get a bounded time to finish before the tensor memory goes back.
+        if (tid == 0) {
+            atomicExch(status, 1);
+            if (!final_commit)
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                                 smem_u32(&s_bar[kTcStages]))
+                             : "memory");
+        }
+        tc_wait(smem_u32(&s_bar[kTcStages]), 0u);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcTmemCols) : "memory");
+}
+
+}  // namespace bof4
+
+using namespace bof4;
+
+extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t rows, int64_t cols,
+                            int block_size, const float* d_codebook, const void* d_x, int n_rhs, float* d_y,
+                            int* d_status, void* stream)
+{
+    const char* fn = "bof4_gemm_tc";
+    if (!valid_block_size(block_size)) {
+        set_error("%s: block_size %d is not a power of two in 32 ... 4096", fn, block_size);
+        return BOF4_ERR_SHAPE;
+    }
+    if (scale_dtype != BOF4_F32 && scale_dtype != BOF4_BF16) {
+        set_error("%s: unknown scale dtype %d", fn, scale_dtype);
+        return BOF4_ERR_DTYPE;
+    }
+    if (rows < 0 || cols < 0 || rows % kTcM || cols % kTcK || cols % block_size || n_rhs < 16 || n_rhs > kTcMaxN ||
+        n_rhs % 16) {
+        set_error("%s: rows must be a multiple of 128, cols of 64 and of block_size, n_rhs one of 16, 32, 48, 64", fn);
+        return BOF4_ERR_SHAPE;
+    }
+    if (rows == 0) return BOF4_OK;
+    if (!d_codes || !d_scales || !d_codebook || !d_x || !d_y || !d_status) {
+        set_error("%s: NULL pointer", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (((uintptr_t)d_codes & 15u) || ((uintptr_t)d_x & 15u)) {
+        set_error("%s: d_codes and d_x must be 16-byte aligned", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (rows / kTcM > 0x7fffffff) {
+        set_error("%s: too many rows", fn);
+        return BOF4_ERR_SHAPE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    BOF4_CUDA_TRY(cudaMemsetAsync(d_status, 0, sizeof(int), st));
+    if (cols == 0) {
+        BOF4_CUDA_TRY(cudaMemsetAsync(d_y, 0, (size_t)rows * n_rhs * sizeof(float), st));
+        return BOF4_OK;
+    }
+    const int grid = (int)(rows / kTcM);
+    int rc;
+    if (scale_dtype == BOF4_F32) {
+        constexpr auto kern = gemm_tc_kernel<F32>;
+        if ((rc = ensure_dynamic_smem<kern>(kTcSmem))) return rc;
+        kern<<<grid, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_size, d_codebook,
+                                                static_cast<const uint16_t*>(d_x), n_rhs, d_y, d_status);
+    } else {
+        constexpr auto kern = gemm_tc_kernel<BF16>;
+        if ((rc = ensure_dynamic_smem<kern>(kTcSmem))) return rc;
+        kern<<<grid, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_size, d_codebook,
+                                                static_cast<const uint16_t*>(d_x), n_rhs, d_y, d_status);
+    }
+    BOF4_CUDA_TRY(cudaGetLastError());
+    return BOF4_OK;
+}

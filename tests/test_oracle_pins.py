@@ -850,3 +850,35 @@ def test_tabulated_model_agrees_with_data_driven_fit_on_laplace_weights(signed, 
     assert np.abs(lv - theo).max() < (4e-4 if metric == "mse" else 1e-3)
     gau = theory.lloyd(64, signed, metric, start, mask, 1, theory.GaussianBlockModel(64, points=4001))
     assert np.abs(lv - gau).max() > 5e-3
+
+
+# --------------------------------------------------------------------------- batched consumer
+
+
+def test_batched_product_with_bf16_weights_by_hand_and_against_gemv():
+    """gemm_bf16 = the decoded product for several right-hand sides with the dequantised weight
+    rounded to bf16.  (i) A 2 x 64 matrix by hand.  (ii) Where scale * level is exact in bf16
+    (power-of-two constants, levels with few significant bits) every column equals the pinned
+    matrix-vector product `gemv`.  (iii) With generic levels it differs from `gemv` by the bf16
+    rounding of the weights (relative 2^-9 at most, and not zero)."""
+    I, rows, cols = 32, 2, 64
+    lv = ((np.arange(16) - 7.5) / 8.0).astype(np.float32)                 # multiples of 1/16: 5 significant bits
+    rng = np.random.default_rng(41)
+    c = rng.integers(0, 16, rows * cols).astype(np.uint8)
+    codes = ((c[0::2] << 4) | c[1::2]).astype(np.uint8)
+    scales = np.array([0.5, -2.0, 1.0, 0.25], np.float32)                 # four blocks of 32
+    X = rng.integers(-3, 4, (3, cols)).astype(np.float32)
+    Y, mag = oracle.gemm_bf16(codes, scales, rows, cols, I, lv, X)
+    W = (lv[c].astype(np.float64) * np.repeat(scales.astype(np.float64), I)).reshape(rows, cols)
+    assert np.array_equal(Y, W @ X.astype(np.float64).T)                  # (i): exact small integers / 16
+    assert np.array_equal(mag, np.abs(W) @ np.abs(X.astype(np.float64)).T)
+    for b in range(3):                                                    # (ii)
+        y, m = oracle.gemv(codes, scales, rows, cols, I, lv, X[b])
+        assert np.array_equal(Y[:, b], y) and np.array_equal(mag[:, b], m)
+    lv2 = TAB6[:, 4].astype(np.float32)                                   # (iii)
+    scales2 = np.array([0.0131, -0.0207, 0.0179, 0.0093], np.float32)
+    Y2, mag2 = oracle.gemm_bf16(codes, scales2, rows, cols, I, lv2, X)
+    for b in range(3):
+        y, m = oracle.gemv(codes, scales2, rows, cols, I, lv2, X[b])
+        assert np.all(np.abs(Y2[:, b] - y) <= 2.0 ** -9 * m)
+        assert np.any(Y2[:, b] != y)
