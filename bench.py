@@ -226,10 +226,38 @@ class Step:
         for (codes, scales, idx, val, cnt), out in zip(self.o_out, self.o_deq):
             b.bof4_dequantize(codes, scales, I, self.cb_q, b.BF16, (idx, val, cnt), out=out)
 
+    # ---- consumers of the quantised matrix (profiling runs, `--only gemv,gemm_tc`): the two
+    # 28672 x 8192 matrices of the OPQ layer in turn (235 MB of codes, larger than L2)
+    def consumer_setup(self):
+        if hasattr(self, "cons"):
+            return
+        b = self.b
+        self.cons = []
+        for w in self.w_opq[4:6]:
+            codes, scales = b.bof4_quantize(w, I, b.NORM_SIGNED, self.cb_q)
+            self.cons.append((codes, scales, 28672, 8192))
+        self.cons_x = workloads.gaussian(64 * 8192, 1.0, 77, torch.bfloat16, self.dev).reshape(64, 8192)
+        self.cons_y = torch.empty(28672, dtype=torch.float32, device=self.dev)
+
+    def gemv(self):
+        b = self.b
+        for codes, scales, r, c in self.cons:
+            b.bof4_gemv(codes, scales, r, c, I, self.cb_q, self.cons_x[0], out=self.cons_y)
+
+    def gemm_tc(self):
+        b = self.b
+        for codes, scales, r, c in self.cons:
+            b.bof4_gemm_tc(codes, scales, r, c, I, self.cb_q, self.cons_x)
+
     def components(self):
         """(name, call, weights per call, algorithmic bytes per weight, kernels launched per call)"""
         b = self.b.binding
         nt, nq, no = len(self.w_fit), len(self.w_q), len(self.w_opq)
+        if self.only and (self.only & {"gemv", "gemm_tc"}):
+            self.consumer_setup()
+            nc = 2 * 28672 * 8192
+            extra = [("gemv", self.gemv, nc, BYTES_GEMV, 2), ("gemm_tc", self.gemm_tc, nc, BYTES_GEMV, 2)]
+            return [c for c in extra if c[0] in self.only]
         comps = [("em_mse", self.em_mse, self.n_fit, BYTES_EM, b.mse_launches_per_iteration(nt)),
                  ("em_mae", self.em_mae, self.n_fit, BYTES_EM * MAE_SELECTION_PASSES,
                   b.mae_launches_per_call(nt, self.n_fit, 1)),

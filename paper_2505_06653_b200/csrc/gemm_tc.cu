@@ -25,6 +25,7 @@ constexpr int kTcThreads = 256;
 constexpr int kTcM = 128;         // rows per CTA = tensor-memory lanes
 constexpr int kTcK = 64;          // weights per k-block: one 128-byte swizzle row of bf16
 constexpr int kTcStages = 2;
+constexpr int kTcCtasPerSm = 4;   // 50 KiB of shared memory and 64 tensor-memory columns each
 constexpr int kTcMaxN = 64;
 constexpr int kTcTmemCols = 64;   // power of two >= 32 and >= N
 constexpr int kTcABytes = kTcM * kTcK * 2;     // 16 KiB
@@ -84,13 +85,13 @@ __device__ __forceinline__ float tc_scale<BF16>(const void* scales, int64_t b)
 }
 
 template <class ST>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm)
 gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t cols, int block_size,
                const float* __restrict__ levels, const uint16_t* __restrict__ x, int n_rhs, float* __restrict__ y,
                int* __restrict__ status)
 {
     extern __shared__ unsigned char s_dyn[];
-    __shared__ float s_lv[kLevels];
+    __shared__ float s_lv[kLevels * 32];  // one column per lane: the bank only depends on the lane
     __shared__ __align__(8) unsigned long long s_bar[kTcStages + 1];  // one per stage, one for the end
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
@@ -100,7 +101,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     const int64_t row0 = (int64_t)blockIdx.x * kTcM;
     const int kblocks = (int)(cols / kTcK);
 
-    if (tid < kLevels) s_lv[tid] = levels[tid];
+    for (int e = tid; e < kLevels * 32; e += kTcThreads) s_lv[e] = levels[e >> 5];
     if (tid == 0) {
         s_fail = 0;
         for (int s = 0; s <= kTcStages; ++s)
@@ -125,6 +126,27 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     const int64_t a_first = (row0 + a_row) * cols + a_half * 32;  // flat index of its first weight in k-block 0
     const uint32_t a_off = (uint32_t)((a_row >> 3) * 1024 + (a_row & 7) * 128);
     bool failed = false, final_commit = false;
+    // what this thread reads from global memory for one k-block: 16 code bytes, their block constant,
+    // and up to two 16-byte chunks of X; the next k-block's are requested before the current is decoded
+    struct Fetched {
+        uint4 cc;
+        float m;
+        uint4 xq[2];
+    };
+    auto fetch = [&](int kb) {
+        Fetched f;
+        f.cc = __ldg(reinterpret_cast<const uint4*>(a_codes + (int64_t)kb * (kTcK / 2)));
+        f.m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) / block_size);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int q = tid + u * kTcThreads, n = q >> 3, ch = q & 7;
+            f.xq[u] = (q < n_rhs * 8)
+                          ? __ldg(reinterpret_cast<const uint4*>(x + (int64_t)n * cols + (int64_t)kb * kTcK + ch * 8))
+                          : make_uint4(0u, 0u, 0u, 0u);
+        }
+        return f;
+    };
+    Fetched cur = fetch(0);
     for (int kb = 0; kb < kblocks; ++kb) {
         const int s = kb & 1;
         unsigned char* sa = tiles_ptr + s * (kTcABytes + kTcBBytes);
@@ -137,28 +159,30 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
             failed = true;
             break;
         }
+        const Fetched next = (kb + 1 < kblocks) ? fetch(kb + 1) : cur;
         // decode: 16 code bytes -> 32 bf16 values of Eq. 3, rounded to nearest even
-        const uint4 cc = *reinterpret_cast<const uint4*>(a_codes + (int64_t)kb * (kTcK / 2));
-        const float m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) / block_size);
-        const uint32_t word[4] = {cc.x, cc.y, cc.z, cc.w};
+        const float m = cur.m;
+        const uint32_t word[4] = {cur.cc.x, cur.cc.y, cur.cc.z, cur.cc.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {  // chunk j of this half: weights 8j .. 8j+7 = code bytes 4j .. 4j+3
             uint32_t p[4];
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 const uint32_t byte = (word[j] >> (8 * b)) & 0xffu;
-                const float hi = __fmul_rn(m, s_lv[byte >> 4]), lo = __fmul_rn(m, s_lv[byte & 15]);
+                const float hi = __fmul_rn(m, s_lv[(byte >> 4) * 32 + lane]), lo = __fmul_rn(m, s_lv[(byte & 15) * 32 + lane]);
                 asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(p[b]) : "f"(lo), "f"(hi));  // even weight in the low half
             }
             const int chunk = a_half * 4 + j;
             *reinterpret_cast<uint4*>(sa + a_off + ((chunk ^ (a_row & 7)) * 16)) = make_uint4(p[0], p[1], p[2], p[3]);
         }
         // the X tile: 16-byte chunk ch (8 values) of right-hand side n, same layout
-        for (int q = tid; q < n_rhs * 8; q += kTcThreads) {
-            const int n = q >> 3, ch = q & 7;
-            *reinterpret_cast<uint4*>(sb + (n >> 3) * 1024 + (n & 7) * 128 + ((ch ^ (n & 7)) * 16)) =
-                *reinterpret_cast<const uint4*>(x + (int64_t)n * cols + (int64_t)kb * kTcK + ch * 8);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int q = tid + u * kTcThreads, n = q >> 3, ch = q & 7;
+            if (q < n_rhs * 8)
+                *reinterpret_cast<uint4*>(sb + (n >> 3) * 1024 + (n & 7) * 128 + ((ch ^ (n & 7)) * 16)) = cur.xq[u];
         }
+        cur = next;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
