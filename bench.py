@@ -238,6 +238,7 @@ class Step:
             self.cons.append((codes, scales, 28672, 8192))
         self.cons_x = workloads.gaussian(64 * 8192, 1.0, 77, torch.bfloat16, self.dev).reshape(64, 8192)
         self.cons_y = torch.empty(28672, dtype=torch.float32, device=self.dev)
+        self.cons_ws = torch.empty(8 * 28672 * 64 * 4, dtype=torch.uint8, device=self.dev)
 
     def gemv(self):
         b = self.b
@@ -247,7 +248,7 @@ class Step:
     def gemm_tc(self):
         b = self.b
         for codes, scales, r, c in self.cons:
-            b.bof4_gemm_tc(codes, scales, r, c, I, self.cb_q, self.cons_x)
+            b.bof4_gemm_tc(codes, scales, r, c, I, self.cb_q, self.cons_x, workspace=self.cons_ws)
 
     def components(self):
         """(name, call, weights per call, algorithmic bytes per weight, kernels launched per call)"""

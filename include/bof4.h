@@ -345,11 +345,14 @@ BOF4_API int bof4_gemv(const uint8_t* d_codes, const void* d_scales, int scale_d
  *   d_y        device, fp32 [rows][n_rhs], written
  *   d_status   device int, written: 0, or 1 when a bounded wait inside the kernel ran out (the result
  *              is then undefined; the kernel has still released its tensor memory and returned)
- * One launch on `stream` (preceded by a 4-byte clear of d_status); no workspace, no synchronisation.
+ *   d_ws       optional device workspace (16-byte aligned) of up to 8 * rows * n_rhs * 4 bytes, or NULL:
+ *              with it the product is split along K into up to 8 partial products (enough CTAs to fill
+ *              the GPU when rows / 128 is small) that a second launch sums in a fixed order
+ * One or two launches on `stream` (preceded by a 4-byte clear of d_status); no synchronisation.
  */
 BOF4_API int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t rows,
                  int64_t cols, int block_size, const float* d_codebook, const void* d_x, int n_rhs,
-                 float* d_y, int* d_status, void* stream);
+                 float* d_y, int* d_status, void* d_ws, size_t ws_bytes, void* stream);
 
 /*
  * Data-free codebook for unit-variance Gaussian weights (Sec. 3.2 Eq. 5 / Eq. 7; App. B.2): `iters`

@@ -86,9 +86,9 @@ __device__ __forceinline__ float tc_scale<BF16>(const void* scales, int64_t b)
 
 template <class ST>
 __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm)
-gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t cols, int block_size,
+gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t cols, int block_shift,
                const float* __restrict__ levels, const uint16_t* __restrict__ x, int n_rhs, float* __restrict__ y,
-               int* __restrict__ status)
+               int kb_per_split, int* __restrict__ status)
 {
     extern __shared__ unsigned char s_dyn[];
     __shared__ float s_lv[kLevels * 32];  // one column per lane: the bank only depends on the lane
@@ -99,7 +99,10 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     const uint32_t tiles = (smem_u32(s_dyn) + 1023u) & ~1023u;  // 1024-byte aligned: the swizzle atoms start here
     unsigned char* tiles_ptr = s_dyn + (tiles - smem_u32(s_dyn));
     const int64_t row0 = (int64_t)blockIdx.x * kTcM;
-    const int kblocks = (int)(cols / kTcK);
+    // blockIdx.y selects a range of k-blocks (split along K so that matrices with few row tiles still
+    // fill the machine); its partial product goes to slab blockIdx.y of y
+    const int kblocks = kb_per_split, kb0 = (int)blockIdx.y * kb_per_split;
+    y += (int64_t)blockIdx.y * ((int64_t)gridDim.x * kTcM) * n_rhs;
 
     for (int e = tid; e < kLevels * 32; e += kTcThreads) s_lv[e] = levels[e >> 5];
     if (tid == 0) {
@@ -135,8 +138,9 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     };
     auto fetch = [&](int kb) {
         Fetched f;
+        kb += kb0;
         f.cc = __ldg(reinterpret_cast<const uint4*>(a_codes + (int64_t)kb * (kTcK / 2)));
-        f.m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) / block_size);
+        f.m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) >> block_shift);
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const int q = tid + u * kTcThreads, n = q >> 3, ch = q & 7;
@@ -249,13 +253,23 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcTmemCols) : "memory");
 }
 
+// Sum of the K-split partial products in slab order (fixed: the result does not depend on scheduling).
+__global__ void gemm_tc_reduce_kernel(const float* __restrict__ part, int splits, int64_t total, float* __restrict__ y)
+{
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        float a = part[i];
+        for (int s = 1; s < splits; ++s) a += part[(int64_t)s * total + i];
+        y[i] = a;
+    }
+}
+
 }  // namespace bof4
 
 using namespace bof4;
 
 extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t rows, int64_t cols,
                             int block_size, const float* d_codebook, const void* d_x, int n_rhs, float* d_y,
-                            int* d_status, void* stream)
+                            int* d_status, void* d_ws, size_t ws_bytes, void* stream)
 {
     const char* fn = "bof4_gemm_tc";
     if (!valid_block_size(block_size)) {
@@ -291,18 +305,36 @@ extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int sc
         return BOF4_OK;
     }
     const int grid = (int)(rows / kTcM);
-    int rc;
+    // K split: enough CTAs for four per SM, a divisor of the number of k-blocks, partial products in
+    // the workspace (none: no split)
+    const int kblocks = (int)(cols / kTcK);
+    int splits = 1;
+    const size_t slab = (size_t)rows * n_rhs * sizeof(float);
+    if (d_ws && !((uintptr_t)d_ws & 15u)) {
+        for (int cand = 2; cand <= 8; ++cand)
+            if (kblocks % cand == 0 && (size_t)cand * slab <= ws_bytes && (int64_t)grid * (cand - 1) < kSMs * kTcCtasPerSm)
+                splits = cand;
+    }
+    float* out = splits > 1 ? static_cast<float*>(d_ws) : d_y;
+    const dim3 g(grid, splits);
+    const int per = kblocks / splits;
+    int rc, block_shift = 0;
+    while ((1 << block_shift) < block_size) ++block_shift;
     if (scale_dtype == BOF4_F32) {
         constexpr auto kern = gemm_tc_kernel<F32>;
         if ((rc = ensure_dynamic_smem<kern>(kTcSmem))) return rc;
-        kern<<<grid, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_size, d_codebook,
-                                                static_cast<const uint16_t*>(d_x), n_rhs, d_y, d_status);
+        kern<<<g, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_shift, d_codebook,
+                                             static_cast<const uint16_t*>(d_x), n_rhs, out, per, d_status);
     } else {
         constexpr auto kern = gemm_tc_kernel<BF16>;
         if ((rc = ensure_dynamic_smem<kern>(kTcSmem))) return rc;
-        kern<<<grid, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_size, d_codebook,
-                                                static_cast<const uint16_t*>(d_x), n_rhs, d_y, d_status);
+        kern<<<g, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_shift, d_codebook,
+                                             static_cast<const uint16_t*>(d_x), n_rhs, out, per, d_status);
     }
     BOF4_CUDA_TRY(cudaGetLastError());
+    if (splits > 1) {
+        gemm_tc_reduce_kernel<<<kSMs * 4, 256, 0, st>>>(out, splits, (int64_t)rows * n_rhs, d_y);
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
     return BOF4_OK;
 }

@@ -45,6 +45,10 @@ def test_integer_valued_products_are_exact(bof4, rows, cols, n_rhs, I, scale_dty
     assert int(status.item()) == 0
     ref, _ = oracle.gemm_bf16(codes, scales, rows, cols, I, lv, X)
     assert np.array_equal(y.cpu().numpy().astype(np.float64), ref)
+    # without the K split (one CTA per 128 rows) the same, bit for bit
+    y1, status1 = bof4.bof4_gemm_tc(torch.from_numpy(codes).cuda(), torch.from_numpy(scales).to(scale_dtype).cuda(),
+                                    rows, cols, I, lv, torch.from_numpy(X).to(torch.bfloat16).cuda(), split=False)
+    assert int(status1.item()) == 0 and torch.equal(y, y1)
 
 
 @pytest.mark.parametrize("rows,cols,n_rhs", [(256, 4096, 16), (512, 8192, 64), (128, 14336, 32)])
