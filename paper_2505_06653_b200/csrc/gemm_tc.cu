@@ -25,12 +25,13 @@ constexpr int kTcThreads = 256;
 constexpr int kTcM = 128;         // rows per CTA = tensor-memory lanes
 constexpr int kTcK = 64;          // weights per k-block: one 128-byte swizzle row of bf16
 constexpr int kTcStages = 2;
-constexpr int kTcCtasPerSm = 4;   // 50 KiB of shared memory and 64 tensor-memory columns each
+constexpr int kTcCtasPerSm = 2;   // 82 KiB of shared memory and 64 tensor-memory columns each
 constexpr int kTcMaxN = 64;
 constexpr int kTcTmemCols = 64;   // power of two >= 32 and >= N
 constexpr int kTcABytes = kTcM * kTcK * 2;     // 16 KiB
 constexpr int kTcBBytes = kTcMaxN * kTcK * 2;  // 8 KiB
-constexpr int kTcSmem = kTcStages * (kTcABytes + kTcBBytes) + 1024;  // + slack to align to 1024 bytes
+constexpr int kTcTableBytes = 256 * 16 * 8;    // level pairs per code byte, one column per lane pair (L, L + 16)
+constexpr int kTcSmem = kTcStages * (kTcABytes + kTcBBytes) + 1024 + kTcTableBytes;  // + slack to align to 1024 bytes
 constexpr uint32_t kTcSpinLimit = 1u << 16;    // try_wait calls before a wait gives up (a k-block takes microseconds)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -91,7 +92,6 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
                int kb_per_split, int* __restrict__ status)
 {
     extern __shared__ unsigned char s_dyn[];
-    __shared__ float s_lv[kLevels * 32];  // one column per lane: the bank only depends on the lane
     __shared__ __align__(8) unsigned long long s_bar[kTcStages + 1];  // one per stage, one for the end
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
@@ -104,7 +104,16 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     const int kblocks = kb_per_split, kb0 = (int)blockIdx.y * kb_per_split;
     y += (int64_t)blockIdx.y * ((int64_t)gridDim.x * kTcM) * n_rhs;
 
-    for (int e = tid; e < kLevels * 32; e += kTcThreads) s_lv[e] = levels[e >> 5];
+    // Level pairs of a code byte (Eq. 3's xhat for its two weights), one 8-byte column per pair of
+    // lanes L and L + 16: an 8-byte read is served half a warp at a time, so the 16 lanes of a half
+    // never share a bank whatever their code bytes are.
+    unsigned char* tab_ptr = tiles_ptr + kTcStages * (kTcABytes + kTcBBytes);
+    {
+        const float2 pr = make_float2(levels[tid >> 4], levels[tid & 15]);
+        static_assert(kTcThreads == 256, "one code byte per thread");
+        for (int c = 0; c < 16; ++c) reinterpret_cast<float2*>(tab_ptr)[tid * 16 + c] = pr;
+    }
+    const uint32_t tab = smem_u32(tab_ptr) + (uint32_t)(lane & 15) * 8u;
     if (tid == 0) {
         s_fail = 0;
         for (int s = 0; s <= kTcStages; ++s)
@@ -156,7 +165,8 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
         unsigned char* sa = tiles_ptr + s * (kTcABytes + kTcBBytes);
         unsigned char* sb = sa + kTcABytes;
         if (kb >= kTcStages) {  // the tensor cores must have finished reading this stage (k-block kb - 2)
-            if (!tc_wait(smem_u32(&s_bar[s]), (uint32_t)(((kb >> 1) - 1) & 1))) s_fail = 1;
+            // one thread polls; the others sleep at the barrier below instead of spending issue slots
+            if (tid == 0 && !tc_wait(smem_u32(&s_bar[s]), (uint32_t)(((kb >> 1) - 1) & 1))) s_fail = 1;
         }
         __syncthreads();
         if (s_fail) {  // uniform: a wait ran out somewhere in the CTA
@@ -165,16 +175,19 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
         }
         const Fetched next = (kb + 1 < kblocks) ? fetch(kb + 1) : cur;
         // decode: 16 code bytes -> 32 bf16 values of Eq. 3, rounded to nearest even
-        const float m = cur.m;
+        const float2 mm = make_float2(cur.m, cur.m);
         const uint32_t word[4] = {cur.cc.x, cur.cc.y, cur.cc.z, cur.cc.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {  // chunk j of this half: weights 8j .. 8j+7 = code bytes 4j .. 4j+3
             uint32_t p[4];
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
-                const uint32_t byte = (word[j] >> (8 * b)) & 0xffu;
-                const float hi = __fmul_rn(m, s_lv[(byte >> 4) * 32 + lane]), lo = __fmul_rn(m, s_lv[(byte & 15) * 32 + lane]);
-                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(p[b]) : "f"(lo), "f"(hi));  // even weight in the low half
+                // byte b of the word times 128 (the table's row size): one shift and one mask
+                const uint32_t off = ((b == 0) ? (word[j] << 7) : (word[j] >> (8 * b - 7))) & 0x7f80u;
+                float2 lv2;
+                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(lv2.x), "=f"(lv2.y) : "r"(tab + off));
+                const float2 w2 = __fmul2_rn(mm, lv2);  // (even, odd) weight of the byte
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(p[b]) : "f"(w2.y), "f"(w2.x));  // even weight in the low half
             }
             const int chunk = a_half * 4 + j;
             *reinterpret_cast<uint4*>(sa + a_off + ((chunk ^ (a_row & 7)) * 16)) = make_uint4(p[0], p[1], p[2], p[3]);
@@ -217,7 +230,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     }
     // all instructions issued: wait for the accumulator, then read it back, one row per thread
     if (!failed && kblocks > 0) {
-        if (!tc_wait(smem_u32(&s_bar[kTcStages]), 0u)) s_fail = 1;
+        if (tid == 0 && !tc_wait(smem_u32(&s_bar[kTcStages]), 0u)) s_fail = 1;
     }
     __syncthreads();
     failed = failed || s_fail != 0 || kblocks == 0;
@@ -245,7 +258,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
                                  smem_u32(&s_bar[kTcStages]))
                              : "memory");
         }
-        tc_wait(smem_u32(&s_bar[kTcStages]), 0u);
+        if (tid == 0) tc_wait(smem_u32(&s_bar[kTcStages]), 0u);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
