@@ -7,25 +7,29 @@
 // weight rounded to bf16, bit for bit what bof4_dequantize writes (Eq. 3, then round to nearest
 // even), X is bf16, products are exact and the sums are accumulated in fp32 by the tensor cores.
 //
-// One CTA owns 128 rows of W and all of K.  Per k-block of 64 weights the 256 threads decode the
-// 128 x 64 tile (4 KiB of codes) into shared memory as bf16 in the K-major 128-byte-swizzled
-// layout that the tcgen05 shared-memory descriptor names (8-row groups of 1024 bytes, 16-byte
-// chunk c of row r stored at chunk c ^ (r & 7)), copy the matching 64 columns of X the same way,
-// and one thread issues four tcgen05.mma (M = 128, N = batch, K = 16 each) that accumulate into
-// tensor memory.  Two shared-memory stages: a tcgen05.commit per k-block arrives on the stage's
-// mbarrier when the tensor cores have finished reading it, and the producers wait on that
-// barrier (bounded; a time-out sets the status word, the kernel still frees its tensor memory
-// and returns) before they overwrite the stage.  The epilogue reads the accumulator with
+// One CTA owns 128 rows of W and a range of K.  Eight producer warps decode, per k-block of 64
+// weights, the 128 x 64 tile (4 KiB of codes) into shared memory as bf16 in the K-major
+// 128-byte-swizzled layout that the tcgen05 shared-memory descriptor names (8-row groups of 1024
+// bytes, 16-byte chunk c of row r stored at chunk c ^ (r & 7)) and copy the matching 64 columns
+// of X the same way; each warp then arrives on the stage's "full" mbarrier.  One thread of a ninth
+// warp waits for a full stage and issues four tcgen05.mma (M = 128, N = batch, K = 16 each) that
+// accumulate into tensor memory; its tcgen05.commit arrives on the stage's "empty" mbarrier when
+// the tensor cores have read the stage, which the producers wait for before they overwrite it
+// (three stages).  No CTA-wide barrier inside the loop.  Every wait is bounded: a time-out sets
+// the status word, the issuing thread still commits and waits (bounded) for what it has issued,
+// and the kernel frees its tensor memory and returns.  The epilogue reads the accumulator with
 // tcgen05.ld (one row per thread) and writes fp32.
 #include "common.cuh"
 
 namespace bof4 {
 
-constexpr int kTcThreads = 256;
+constexpr int kTcProducerWarps = 8;
+constexpr int kTcProducers = kTcProducerWarps * 32;  // threads that decode
+constexpr int kTcThreads = 32 + kTcProducers;        // and one warp that issues the tensor-core instructions
 constexpr int kTcM = 128;         // rows per CTA = tensor-memory lanes
 constexpr int kTcK = 64;          // weights per k-block: one 128-byte swizzle row of bf16
-constexpr int kTcStages = 2;
-constexpr int kTcCtasPerSm = 2;   // 82 KiB of shared memory and 64 tensor-memory columns each
+constexpr int kTcStages = 3;
+constexpr int kTcCtasPerSm = 2;   // 106 KiB of shared memory and 64 tensor-memory columns each
 constexpr int kTcMaxN = 64;
 constexpr int kTcTmemCols = 64;   // power of two >= 32 and >= N
 constexpr int kTcABytes = kTcM * kTcK * 2;     // 16 KiB
@@ -92,7 +96,9 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
                int kb_per_split, int* __restrict__ status)
 {
     extern __shared__ unsigned char s_dyn[];
-    __shared__ __align__(8) unsigned long long s_bar[kTcStages + 1];  // one per stage, one for the end
+    // full[s]: the producers have filled stage s (one arrival per producer warp); empty[s]: the tensor
+    // cores have read it (tcgen05.commit); done: every instruction of the CTA has completed
+    __shared__ __align__(8) unsigned long long s_full[kTcStages], s_empty[kTcStages], s_done;
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -108,16 +114,16 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     // lanes L and L + 16: an 8-byte read is served half a warp at a time, so the 16 lanes of a half
     // never share a bank whatever their code bytes are.
     unsigned char* tab_ptr = tiles_ptr + kTcStages * (kTcABytes + kTcBBytes);
-    {
-        const float2 pr = make_float2(levels[tid >> 4], levels[tid & 15]);
-        static_assert(kTcThreads == 256, "one code byte per thread");
-        for (int c = 0; c < 16; ++c) reinterpret_cast<float2*>(tab_ptr)[tid * 16 + c] = pr;
-    }
+    for (int e = tid; e < 256 * 16; e += kTcThreads)
+        reinterpret_cast<float2*>(tab_ptr)[e] = make_float2(levels[e >> 8], levels[(e >> 4) & 15]);
     const uint32_t tab = smem_u32(tab_ptr) + (uint32_t)(lane & 15) * 8u;
     if (tid == 0) {
         s_fail = 0;
-        for (int s = 0; s <= kTcStages; ++s)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_bar[s])), "r"(1) : "memory");
+        for (int s = 0; s < kTcStages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_full[s])), "r"(kTcProducerWarps) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_empty[s])), "r"(1) : "memory");
+        }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_done)), "r"(1) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {  // tensor memory for the 128 x N fp32 accumulator
@@ -130,112 +136,123 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s_tmem;
-    const uint32_t idesc = tc_instr_desc(n_rhs);
 
-    // this thread's part of the A tile: half a row (32 weights = 16 code bytes = four 16-byte chunks)
-    const int a_row = tid >> 1, a_half = tid & 1;
-    const uint8_t* a_codes = codes + ((row0 + a_row) * cols) / 2 + a_half * 16;
-    const int64_t a_first = (row0 + a_row) * cols + a_half * 32;  // flat index of its first weight in k-block 0
-    const uint32_t a_off = (uint32_t)((a_row >> 3) * 1024 + (a_row & 7) * 128);
-    bool failed = false, final_commit = false;
-    // what this thread reads from global memory for one k-block: 16 code bytes, their block constant,
-    // and up to two 16-byte chunks of X; the next k-block's are requested before the current is decoded
-    struct Fetched {
-        uint4 cc;
-        float m;
-        uint4 xq[2];
-    };
-    auto fetch = [&](int kb) {
-        Fetched f;
-        kb += kb0;
-        f.cc = __ldg(reinterpret_cast<const uint4*>(a_codes + (int64_t)kb * (kTcK / 2)));
-        f.m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) >> block_shift);
+    if (warp == 0) {
+        // ---- the issuing warp: one thread waits for a full stage, issues its four instructions and
+        // lets tcgen05.commit hand the stage back
+        if (lane == 0) {
+            const uint32_t idesc = tc_instr_desc(n_rhs);
+            bool ok = true;
+            for (int kb = 0; kb < kblocks && ok; ++kb) {
+                const int s = kb % kTcStages;
+                if (!tc_wait(smem_u32(&s_full[s]), (uint32_t)((kb / kTcStages) & 1))) {
+                    ok = false;
+                    break;
+                }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = tiles + (uint32_t)s * (kTcABytes + kTcBBytes);
+                const uint64_t da = tc_smem_desc(sa), db = tc_smem_desc(sa + kTcABytes);
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int q = tid + u * kTcThreads, n = q >> 3, ch = q & 7;
-            f.xq[u] = (q < n_rhs * 8)
-                          ? __ldg(reinterpret_cast<const uint4*>(x + (int64_t)n * cols + (int64_t)kb * kTcK + ch * 8))
-                          : make_uint4(0u, 0u, 0u, 0u);
-        }
-        return f;
-    };
-    Fetched cur = fetch(0);
-    for (int kb = 0; kb < kblocks; ++kb) {
-        const int s = kb & 1;
-        unsigned char* sa = tiles_ptr + s * (kTcABytes + kTcBBytes);
-        unsigned char* sb = sa + kTcABytes;
-        if (kb >= kTcStages) {  // the tensor cores must have finished reading this stage (k-block kb - 2)
-            // one thread polls; the others sleep at the barrier below instead of spending issue slots
-            if (tid == 0 && !tc_wait(smem_u32(&s_bar[s]), (uint32_t)(((kb >> 1) - 1) & 1))) s_fail = 1;
-        }
-        __syncthreads();
-        if (s_fail) {  // uniform: a wait ran out somewhere in the CTA
-            failed = true;
-            break;
-        }
-        const Fetched next = (kb + 1 < kblocks) ? fetch(kb + 1) : cur;
-        // decode: 16 code bytes -> 32 bf16 values of Eq. 3, rounded to nearest even
-        const float2 mm = make_float2(cur.m, cur.m);
-        const uint32_t word[4] = {cur.cc.x, cur.cc.y, cur.cc.z, cur.cc.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {  // chunk j of this half: weights 8j .. 8j+7 = code bytes 4j .. 4j+3
-            uint32_t p[4];
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                // byte b of the word times 128 (the table's row size): one shift and one mask
-                const uint32_t off = ((b == 0) ? (word[j] << 7) : (word[j] >> (8 * b - 7))) & 0x7f80u;
-                float2 lv2;
-                asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(lv2.x), "=f"(lv2.y) : "r"(tab + off));
-                const float2 w2 = __fmul2_rn(mm, lv2);  // (even, odd) weight of the byte
-                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(p[b]) : "f"(w2.y), "f"(w2.x));  // even weight in the low half
-            }
-            const int chunk = a_half * 4 + j;
-            *reinterpret_cast<uint4*>(sa + a_off + ((chunk ^ (a_row & 7)) * 16)) = make_uint4(p[0], p[1], p[2], p[3]);
-        }
-        // the X tile: 16-byte chunk ch (8 values) of right-hand side n, same layout
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int q = tid + u * kTcThreads, n = q >> 3, ch = q & 7;
-            if (q < n_rhs * 8)
-                *reinterpret_cast<uint4*>(sb + (n >> 3) * 1024 + (n & 7) * 128 + ((ch ^ (n & 7)) * 16)) = cur.xq[u];
-        }
-        cur = next;
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        if (tid == 0) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint64_t da = tc_smem_desc(smem_u32(sa)), db = tc_smem_desc(smem_u32(sb));
-#pragma unroll
-            for (int kk = 0; kk < kTcK / 16; ++kk) {  // 32 bytes of K per instruction: +2 in the address field
-                const uint32_t acc = (kb > 0 || kk > 0) ? 1u : 0u;
-                asm volatile(
-                    "{\n\t.reg .pred p;\n\t"
-                    "setp.ne.b32 p, %4, 0;\n\t"
-                    "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-                    :
-                    : "r"(tmem), "l"(da + (uint64_t)(2 * kk)), "l"(db + (uint64_t)(2 * kk)), "r"(idesc), "r"(acc), "r"(0u)
-                    : "memory");
-            }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                             smem_u32(&s_bar[s]))
-                         : "memory");
-            if (kb == kblocks - 1) {
+                for (int kk = 0; kk < kTcK / 16; ++kk) {  // 32 bytes of K per instruction: +2 in the address field
+                    const uint32_t acc = (kb > 0 || kk > 0) ? 1u : 0u;
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t"
+                        "setp.ne.b32 p, %4, 0;\n\t"
+                        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                        :
+                        : "r"(tmem), "l"(da + (uint64_t)(2 * kk)), "l"(db + (uint64_t)(2 * kk)), "r"(idesc), "r"(acc), "r"(0u)
+                        : "memory");
+                }
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                                 smem_u32(&s_bar[kTcStages]))
+                                 smem_u32(&s_empty[s]))
                              : "memory");
-                final_commit = true;
             }
+            // whatever has been issued arrives on `done` when it has completed (also after a time-out)
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                             smem_u32(&s_done))
+                         : "memory");
+            if (!ok) s_fail = 1;
+            if (!tc_wait(smem_u32(&s_done), 0u)) s_fail = 1;
+        }
+    } else {
+        // ---- producer warps: thread t decodes half a row (32 weights = 16 code bytes = four 16-byte
+        // chunks) of the 128 x 64 tile and copies up to two 16-byte chunks of the X tile
+        const int t = tid - 32;
+        const int a_row = t >> 1, a_half = t & 1;
+        const uint8_t* a_codes = codes + ((row0 + a_row) * cols) / 2 + a_half * 16;
+        const int64_t a_first = (row0 + a_row) * cols + a_half * 32;  // flat index of its first weight in k-block 0
+        const uint32_t a_off = (uint32_t)((a_row >> 3) * 1024 + (a_row & 7) * 128);
+        struct Fetched {
+            uint4 cc;
+            float m;
+            uint4 xq[2];
+        };
+        auto fetch = [&](int kb) {  // what the thread reads from global memory for one k-block
+            Fetched f;
+            kb += kb0;
+            f.cc = __ldg(reinterpret_cast<const uint4*>(a_codes + (int64_t)kb * (kTcK / 2)));
+            f.m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) >> block_shift);
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int q = t + u * kTcProducers, n = q >> 3, ch = q & 7;
+                f.xq[u] = (q < n_rhs * 8)
+                              ? __ldg(reinterpret_cast<const uint4*>(x + (int64_t)n * cols + (int64_t)kb * kTcK + ch * 8))
+                              : make_uint4(0u, 0u, 0u, 0u);
+            }
+            return f;
+        };
+        Fetched cur = fetch(0);
+        for (int kb = 0; kb < kblocks; ++kb) {
+            const int s = kb % kTcStages;
+            unsigned char* sa = tiles_ptr + s * (kTcABytes + kTcBBytes);
+            unsigned char* sb = sa + kTcABytes;
+            const Fetched next = (kb + 1 < kblocks) ? fetch(kb + 1) : cur;  // on its way while this one is decoded
+            if (kb >= kTcStages) {  // the tensor cores must have read what the stage held (k-block kb - stages)
+                int ok = 1;
+                if (lane == 0) ok = tc_wait(smem_u32(&s_empty[s]), (uint32_t)(((kb / kTcStages) - 1) & 1)) ? 1 : 0;
+                ok = __shfl_sync(kFull, ok, 0);
+                if (!ok) {
+                    if (lane == 0) s_fail = 1;
+                    break;
+                }
+            }
+            const float2 mm = make_float2(cur.m, cur.m);
+            const uint32_t word[4] = {cur.cc.x, cur.cc.y, cur.cc.z, cur.cc.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {  // chunk j of this half: weights 8j .. 8j+7 = code bytes 4j .. 4j+3
+                uint32_t p[4];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    // byte b of the word times 128 (the table's row size): one shift and one mask
+                    const uint32_t off = ((b == 0) ? (word[j] << 7) : (word[j] >> (8 * b - 7))) & 0x7f80u;
+                    float2 lv2;
+                    asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(lv2.x), "=f"(lv2.y) : "r"(tab + off));
+                    const float2 w2 = __fmul2_rn(mm, lv2);  // Eq. 3 for the (even, odd) weight of the byte
+                    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(p[b]) : "f"(w2.y), "f"(w2.x));  // even weight in the low half
+                }
+                const int chunk = a_half * 4 + j;
+                *reinterpret_cast<uint4*>(sa + a_off + ((chunk ^ (a_row & 7)) * 16)) = make_uint4(p[0], p[1], p[2], p[3]);
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {  // the X tile, same layout
+                const int q = t + u * kTcProducers, n = q >> 3, ch = q & 7;
+                if (q < n_rhs * 8)
+                    *reinterpret_cast<uint4*>(sb + (n >> 3) * 1024 + (n & 7) * 128 + ((ch ^ (n & 7)) * 16)) = cur.xq[u];
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
+            __syncwarp();
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&s_full[s])) : "memory");
+            cur = next;
         }
     }
-    // all instructions issued: wait for the accumulator, then read it back, one row per thread
-    if (!failed && kblocks > 0) {
-        if (tid == 0 && !tc_wait(smem_u32(&s_bar[kTcStages]), 0u)) s_fail = 1;
-    }
+    // Every loop above is bounded, so every warp gets here.  After a time-out the issuing thread has
+    // still committed and waited (bounded) for what it issued.
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    failed = failed || s_fail != 0 || kblocks == 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (!failed && warp < 4) {
+    const bool failed = s_fail != 0;
+    if (!failed && warp < 4) {  // the accumulator, one row per thread (warp w reads lanes 32 w .. 32 w + 31)
         float* yrow = y + (row0 + warp * 32 + lane) * n_rhs;
         for (int c0 = 0; c0 < n_rhs; c0 += 8) {
             uint32_t v[8];
@@ -247,19 +264,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
             for (int c = 0; c < 8; ++c) yrow[c0 + c] = __uint_as_float(v[c]);
         }
     }
-    if (failed && kblocks > 0) {
-        // A wait ran out.  The instructions already issued may still be running (their operands live in
-        // this CTA's shared memory, their result in its tensor memory): one more commit covers them
-        // all, and they get a bounded time to finish before the tensor memory goes back.
-        if (tid == 0) {
-            atomicExch(status, 1);
-            if (!final_commit)
-                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                                 smem_u32(&s_bar[kTcStages]))
-                             : "memory");
-        }
-        if (tid == 0) tc_wait(smem_u32(&s_bar[kTcStages]), 0u);
-    }
+    if (failed && tid == 0) atomicExch(status, 1);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0)
