@@ -190,7 +190,11 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
         auto fetch = [&](int kb) {  // what the thread reads from global memory for one k-block
             Fetched f;
             kb += kb0;
-            f.cc = __ldg(reinterpret_cast<const uint4*>(a_codes + (int64_t)kb * (kTcK / 2)));
+            // a row's codes are read 32 bytes per k-block (two threads); the hint brings the whole 128-byte
+            // line into L2 at the first touch, so DRAM sees full lines instead of scattered sectors
+            asm volatile("ld.global.nc.L2::128B.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(f.cc.x), "=r"(f.cc.y), "=r"(f.cc.z), "=r"(f.cc.w)
+                         : "l"(a_codes + (int64_t)kb * (kTcK / 2)));
             f.m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) >> block_shift);
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
