@@ -337,21 +337,25 @@ BOF4_API int bof4_gemv(const uint8_t* d_codes, const void* d_scales, int scale_d
  * bf16, products are exact, sums are accumulated in fp32 by the tensor cores (tcgen05.mma into
  * tensor memory), whose summation order and intermediate rounding are the hardware's: the result
  * agrees with the fp64 sum of the same products within 2^-14 * sum |w x| (cols / 16 accumulation
- * steps of at most 2^-23 each for cols <= 8192 * 16).  No outlier list: apply bof4_gemv's
- * correction per right-hand side, or dequantise.
+ * steps of at most 2^-23 each for cols <= 8192 * 16).  With an outlier list (Sec. 3.3, decoding
+ * side) the stored bf16 value replaces the decoded weight: a second launch adds
+ * (val - decoded) * X[b][col] for every outlier, row by row in list order (fp32).
  *   rows       multiple of 128;  cols multiple of 64 and of block_size
  *   d_codes    device, rows * cols / 2 bytes, 16-byte aligned;  d_scales as for bof4_gemv
  *   d_x        device, bf16 [n_rhs][cols] (each right-hand side contiguous), 16-byte aligned
+ *   d_out_idx / d_out_val / d_n_out / capacity   outlier list as for bof4_dequantize (ascending
+ *              indices), or all NULL; with a list, rows * cols must fit 32-bit indices
  *   d_y        device, fp32 [rows][n_rhs], written
  *   d_status   device int, written: 0, or 1 when a bounded wait inside the kernel ran out (the result
  *              is then undefined; the kernel has still released its tensor memory and returned)
  *   d_ws       optional device workspace (16-byte aligned) of up to 8 * rows * n_rhs * 4 bytes, or NULL:
  *              with it the product is split along K into up to 8 partial products (enough CTAs to fill
  *              the GPU when rows / 128 is small) that a second launch sums in a fixed order
- * One or two launches on `stream` (preceded by a 4-byte clear of d_status); no synchronisation.
+ * One to three launches on `stream` (preceded by a 4-byte clear of d_status); no synchronisation.
  */
 BOF4_API int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t rows,
                  int64_t cols, int block_size, const float* d_codebook, const void* d_x, int n_rhs,
+                 const int32_t* d_out_idx, const void* d_out_val, const int64_t* d_n_out, int64_t capacity,
                  float* d_y, int* d_status, void* d_ws, size_t ws_bytes, void* stream);
 
 /*

@@ -279,12 +279,17 @@ def gemv(codes: np.ndarray, scales: np.ndarray, rows: int, cols: int, I: int, xh
     return W @ xv, np.abs(W) @ np.abs(xv)
 
 
-def gemm_bf16(codes: np.ndarray, scales: np.ndarray, rows: int, cols: int, I: int, xhat, X):
+def gemm_bf16(codes: np.ndarray, scales: np.ndarray, rows: int, cols: int, I: int, xhat, X,
+              idx: Optional[np.ndarray] = None, val: Optional[np.ndarray] = None):
     """Y = W X^T in fp64 for a batch of right-hand sides X [n_rhs, cols], the decoded weight being
     the dequantised value ROUNDED TO bf16 (Eq. 3 followed by round-to-nearest-even, i.e. what
-    `dequantize` returns as bf16): the operand precision of the batched tensor-core consumer.
+    `dequantize` returns as bf16): the operand precision of the batched tensor-core consumer.  With
+    OPQ the stored bf16 outlier values replace the decoded ones (W.flat[idx] = val).
     Also returns sum_c |W[r, c] X[b, c]|.  -> (Y fp64 [rows, n_rhs], mag fp64 [rows, n_rhs])."""
     w32 = dequantize(codes, scales, I, xhat, n=rows * cols)              # fp32 products of Eq. 3
-    W = bf16_bits_to_f32(f32_to_bf16_bits(w32)).astype(np.float64).reshape(rows, cols)
+    W = bf16_bits_to_f32(f32_to_bf16_bits(w32)).astype(np.float64)
+    if idx is not None and len(idx):                                    # OPQ: the stored values (Sec. 3.3)
+        W[np.asarray(idx, dtype=np.int64)] = bf16_bits_to_f32(np.asarray(val, dtype=np.uint16)).astype(np.float64)
+    W = W.reshape(rows, cols)
     Xd = np.asarray(X, dtype=np.float64).reshape(-1, cols)
     return W @ Xd.T, np.abs(W) @ np.abs(Xd).T

@@ -112,7 +112,7 @@ def lib() -> ctypes.CDLL:
         L.bof4_dequantize_batch.restype = i32
         L.bof4_dequantize_batch.argtypes = [vp, vp, i32, vp, i32, i32, vp, vp, i32, vp]
         L.bof4_gemm_tc.restype = i32
-        L.bof4_gemm_tc.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.bof4_gemm_tc.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, vp, vp, vp, i64, vp, vp, vp, sz, vp]
         L.bof4_m_step.restype = i32
         L.bof4_m_step.argtypes = [vp, i32, i32, vp, ctypes.c_uint32, vp, vp, vp]
         L.bof4_scales_compress.restype = i32
@@ -481,7 +481,8 @@ def opq_split(w: torch.Tensor, block_size: int, tau: float, capacity: int,
 
 
 def bof4_gemm_tc(codes: torch.Tensor, scales: torch.Tensor, rows: int, cols: int, block_size: int, levels,
-                 x: torch.Tensor, workspace: Optional[torch.Tensor] = None, split: bool = True):
+                 x: torch.Tensor, workspace: Optional[torch.Tensor] = None, split: bool = True,
+                 outliers: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None):
     """Y fp32 [rows, n_rhs] = W_q X^T on the tensor cores for x bf16 [n_rhs, cols].
     -> (y, status int32[1]); status 0 unless a bounded wait inside the kernel ran out."""
     codes = _dev(codes, "codes")
@@ -495,9 +496,14 @@ def bof4_gemm_tc(codes: torch.Tensor, scales: torch.Tensor, rows: int, cols: int
     status = _new(1, torch.int32, codes.device, zero=True)
     ws = workspace if workspace is not None else (_new(8 * rows * n_rhs * 4, torch.uint8, codes.device) if split else None)
     with torch.cuda.device(codes.device):
+        idx = val = cnt = None
+        cap = 0
+        if outliers is not None:
+            idx, val, cnt = (_dev(t, "outliers") for t in outliers)
+            cap = idx.numel()
         _check(lib().bof4_gemm_tc(_ptr(codes), _ptr(scales), _dt(scales), rows, cols, block_size, _ptr(cb), _ptr(x),
-                                  n_rhs, _ptr(y), _ptr(status), _ptr(ws), ws.numel() if ws is not None else 0,
-                                  _stream()))
+                                  n_rhs, _ptr(idx), _ptr(val), _ptr(cnt), cap, _ptr(y), _ptr(status), _ptr(ws),
+                                  ws.numel() if ws is not None else 0, _stream()))
     return y, status
 
 

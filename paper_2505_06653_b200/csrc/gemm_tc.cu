@@ -275,6 +275,51 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTcTmemCols) : "memory");
 }
 
+// OPQ (Sec. 3.3, decoding side): an outlier position holds its stored bf16 value instead of the
+// decoded weight, so Y[r][b] += (val - decoded) * X[b][c] for every outlier (r, c).  One warp per
+// row: the row's outliers are a contiguous run of the ascending index list (two binary searches),
+// each lane owns right-hand sides b = lane, lane + 32 and adds the row's terms in list order.
+template <class ST>
+__global__ void __launch_bounds__(256)
+gemm_tc_outlier_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t rows, int64_t cols,
+                       int block_shift, const float* __restrict__ levels, const uint16_t* __restrict__ x, int n_rhs,
+                       const int32_t* __restrict__ idx, const uint16_t* __restrict__ val,
+                       const int64_t* __restrict__ n_out, int64_t capacity, float* __restrict__ y)
+{
+    int64_t k_end = *n_out;
+    if (k_end > capacity) k_end = capacity;
+    if (k_end <= 0) return;
+    auto lower_bound = [&](int64_t key) {  // first k with idx[k] >= key
+        int64_t lo = 0, hi = k_end;
+        while (lo < hi) {
+            const int64_t mid = (lo + hi) >> 1;
+            if ((int64_t)idx[mid] < key) lo = mid + 1; else hi = mid;
+        }
+        return lo;
+    };
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < rows; r += warps) {
+        const int64_t lo = lower_bound(r * cols), hi = lower_bound((r + 1) * cols);
+        if (lo == hi) continue;
+        for (int b = lane; b < n_rhs; b += 32) {
+            float acc = y[r * n_rhs + b];
+            for (int64_t k = lo; k < hi; ++k) {
+                const int64_t i = idx[k];
+                const uint32_t byte = codes[i >> 1];
+                const uint32_t c = (i & 1) ? (byte & 15u) : (byte >> 4);
+                const float q32 = __fmul_rn(tc_scale<ST>(scales, i >> block_shift), __ldg(levels + c));
+                uint32_t qb;
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(qb) : "f"(0.0f), "f"(q32));  // the operand the tile held
+                const float delta = __uint_as_float((uint32_t)val[k] << 16) - __uint_as_float(qb << 16);
+                const float xv = __uint_as_float((uint32_t)x[(int64_t)b * cols + (i - r * cols)] << 16);
+                acc = __fadd_rn(acc, __fmul_rn(delta, xv));
+            }
+            y[r * n_rhs + b] = acc;
+        }
+    }
+}
+
 // Sum of the K-split partial products in slab order (fixed: the result does not depend on scheduling).
 __global__ void gemm_tc_reduce_kernel(const float* __restrict__ part, int splits, int64_t total, float* __restrict__ y)
 {
@@ -290,8 +335,9 @@ __global__ void gemm_tc_reduce_kernel(const float* __restrict__ part, int splits
 using namespace bof4;
 
 extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t rows, int64_t cols,
-                            int block_size, const float* d_codebook, const void* d_x, int n_rhs, float* d_y,
-                            int* d_status, void* d_ws, size_t ws_bytes, void* stream)
+                            int block_size, const float* d_codebook, const void* d_x, int n_rhs,
+                            const int32_t* d_out_idx, const void* d_out_val, const int64_t* d_n_out, int64_t capacity,
+                            float* d_y, int* d_status, void* d_ws, size_t ws_bytes, void* stream)
 {
     const char* fn = "bof4_gemm_tc";
     if (!valid_block_size(block_size)) {
@@ -305,6 +351,15 @@ extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int sc
     if (rows < 0 || cols < 0 || rows % kTcM || cols % kTcK || cols % block_size || n_rhs < 16 || n_rhs > kTcMaxN ||
         n_rhs % 16) {
         set_error("%s: rows must be a multiple of 128, cols of 64 and of block_size, n_rhs one of 16, 32, 48, 64", fn);
+        return BOF4_ERR_SHAPE;
+    }
+    const bool opq = d_out_idx != nullptr;
+    if (opq && (!d_out_val || !d_n_out || capacity < 0)) {
+        set_error("%s: outlier list needs d_out_idx, d_out_val and d_n_out together and a capacity >= 0", fn);
+        return BOF4_ERR_INVALID_ARG;
+    }
+    if (opq && rows * cols > 0x7fffffffLL) {
+        set_error("%s: outlier indices are 32-bit, rows * cols must not exceed 2^31 - 1", fn);
         return BOF4_ERR_SHAPE;
     }
     if (rows == 0) return BOF4_OK;
@@ -356,6 +411,17 @@ extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int sc
     BOF4_CUDA_TRY(cudaGetLastError());
     if (splits > 1) {
         gemm_tc_reduce_kernel<<<kSMs * 4, 256, 0, st>>>(out, splits, (int64_t)rows * n_rhs, d_y);
+        BOF4_CUDA_TRY(cudaGetLastError());
+    }
+    if (opq && capacity > 0) {
+        const uint16_t* val = static_cast<const uint16_t*>(d_out_val);
+        const uint16_t* xb = static_cast<const uint16_t*>(d_x);
+        if (scale_dtype == BOF4_F32)
+            gemm_tc_outlier_kernel<F32><<<kSMs * 4, 256, 0, st>>>(d_codes, d_scales, rows, cols, block_shift, d_codebook, xb,
+                                                                  n_rhs, d_out_idx, val, d_n_out, capacity, d_y);
+        else
+            gemm_tc_outlier_kernel<BF16><<<kSMs * 4, 256, 0, st>>>(d_codes, d_scales, rows, cols, block_shift, d_codebook, xb,
+                                                                   n_rhs, d_out_idx, val, d_n_out, capacity, d_y);
         BOF4_CUDA_TRY(cudaGetLastError());
     }
     return BOF4_OK;

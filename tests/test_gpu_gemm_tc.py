@@ -71,6 +71,33 @@ def test_quantised_matrix_times_batch(bof4, rows, cols, n_rhs, norm):
     assert np.all(np.abs(yt - ref) <= 1e-12 * mag)
 
 
+@pytest.mark.parametrize("rows,cols,n_rhs", [(256, 4096, 16), (384, 8192, 64)])
+def test_with_outlier_list(bof4, rows, cols, n_rhs):
+    """OPQ quantisation, then the batched product with the outlier list: the stored values replace
+    the decoded weights (Sec. 3.3).  Also a list that is cut off by its capacity."""
+    I = 64
+    lv = np.array(workloads.BOF4S_MSE_I64, np.float32)
+    w = workloads.inject_outliers(workloads.gaussian(rows * cols, 0.02, 9, torch.bfloat16), 0.02, 3e-4, 10.0, 40.0, 10)
+    tau = float(np.float32(bof4.bof4_opq_threshold(0.95, I)))
+    cap = rows * cols // 64
+    codes, scales, idx, val, cnt = bof4.bof4_quantize_opq(w.cuda(), I, 1, lv, tau, cap)
+    k = bof4.bof4_outlier_count(cnt, cap)
+    assert k > rows
+    x = workloads.gaussian(n_rhs * cols, 1.0, 11, torch.bfloat16).reshape(n_rhs, cols)
+    idx_h = idx[:k].cpu().numpy().astype(np.int64)
+    val_h = val[:k].view(torch.int16).cpu().numpy().view(np.uint16)
+    for use in (k, k // 2):
+        y, status = bof4.bof4_gemm_tc(codes, scales, rows, cols, I, lv, x.cuda(), outliers=(idx[:use], val[:use], cnt))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref, mag = oracle.gemm_bf16(codes.cpu().numpy(), scales.float().cpu().numpy(), rows, cols, I, lv,
+                                    x.float().numpy(), idx_h[:use], val_h[:use])
+        err = np.abs(y.cpu().numpy().astype(np.float64) - ref)
+        assert np.all(err <= 2.0 ** -14 * mag + 1e-30), float((err / mag).max())
+    plain, _ = bof4.bof4_gemm_tc(codes, scales, rows, cols, I, lv, x.cuda())
+    assert not torch.equal(plain, y)
+
+
 def test_gemm_tc_argument_errors(bof4):
     lv = np.array(workloads.BOF4S_MSE_I64, np.float32)
     codes = torch.zeros(128 * 64 // 2, dtype=torch.uint8, device="cuda")

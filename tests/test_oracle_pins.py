@@ -875,6 +875,11 @@ def test_batched_product_with_bf16_weights_by_hand_and_against_gemv():
     for b in range(3):                                                    # (ii)
         y, m = oracle.gemv(codes, scales, rows, cols, I, lv, X[b])
         assert np.array_equal(Y[:, b], y) and np.array_equal(mag[:, b], m)
+    # an outlier replaces exactly one weight: Y moves by (val - W[r, c]) * X[:, c] in its row only
+    val = oracle.f32_to_bf16_bits(np.array([3.5], np.float32))
+    Yo, _ = oracle.gemm_bf16(codes, scales, rows, cols, I, lv, X, np.array([cols + 5]), val)
+    assert np.array_equal(Yo[0], Y[0])
+    assert np.array_equal(Yo[1] - Y[1], (3.5 - W[1, 5]) * X[:, 5].astype(np.float64))
     lv2 = TAB6[:, 4].astype(np.float32)                                   # (iii)
     scales2 = np.array([0.0131, -0.0207, 0.0179, 0.0093], np.float32)
     Y2, mag2 = oracle.gemm_bf16(codes, scales2, rows, cols, I, lv2, X)
