@@ -19,6 +19,8 @@
 // the status word, the issuing thread still commits and waits (bounded) for what it has issued,
 // and the kernel frees its tensor memory and returns.  The epilogue reads the accumulator with
 // tcgen05.ld (one row per thread) and writes fp32.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace bof4 {
@@ -92,8 +94,8 @@ __device__ __forceinline__ float tc_scale<BF16>(const void* scales, int64_t b)
 template <class ST>
 __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm)
 gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales, int64_t cols, int block_shift,
-               const float* __restrict__ levels, const uint16_t* __restrict__ x, int n_rhs, float* __restrict__ y,
-               int kb_per_split, int* __restrict__ status)
+               const float* __restrict__ levels, const __grid_constant__ CUtensorMap x_map, int n_rhs,
+               float* __restrict__ y, int kb_per_split, int* __restrict__ status)
 {
     extern __shared__ unsigned char s_dyn[];
     // full[s]: the producers have filled stage s (one arrival per producer warp); empty[s]: the tensor
@@ -120,7 +122,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     if (tid == 0) {
         s_fail = 0;
         for (int s = 0; s < kTcStages; ++s) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_full[s])), "r"(kTcProducerWarps) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_full[s])), "r"(kTcProducerWarps + 1) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_empty[s])), "r"(1) : "memory");
         }
         asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_done)), "r"(1) : "memory");
@@ -176,7 +178,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
         }
     } else {
         // ---- producer warps: thread t decodes half a row (32 weights = 16 code bytes = four 16-byte
-        // chunks) of the 128 x 64 tile and copies up to two 16-byte chunks of the X tile
+        // chunks) of the 128 x 64 tile; the first of them also requests the X tile
         const int t = tid - 32;
         const int a_row = t >> 1, a_half = t & 1;
         const uint8_t* a_codes = codes + ((row0 + a_row) * cols) / 2 + a_half * 16;
@@ -185,7 +187,6 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
         struct Fetched {
             uint4 cc;
             float m;
-            uint4 xq[2];
         };
         auto fetch = [&](int kb) {  // what the thread reads from global memory for one k-block
             Fetched f;
@@ -196,13 +197,6 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
                          : "=r"(f.cc.x), "=r"(f.cc.y), "=r"(f.cc.z), "=r"(f.cc.w)
                          : "l"(a_codes + (int64_t)kb * (kTcK / 2)));
             f.m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) >> block_shift);
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int q = t + u * kTcProducers, n = q >> 3, ch = q & 7;
-                f.xq[u] = (q < n_rhs * 8)
-                              ? __ldg(reinterpret_cast<const uint4*>(x + (int64_t)n * cols + (int64_t)kb * kTcK + ch * 8))
-                              : make_uint4(0u, 0u, 0u, 0u);
-            }
             return f;
         };
         Fetched cur = fetch(0);
@@ -220,6 +214,18 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
                     break;
                 }
             }
+            if (t == 0) {
+                // the X tile (n_rhs rows of 64 values) comes by TMA straight into the swizzled layout; its
+                // bytes count towards the stage's "full" barrier together with the producer warps' arrivals
+                const uint32_t bar = smem_u32(&s_full[s]);
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)n_rhs * 128u)
+                             : "memory");
+                asm volatile(
+                    "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                    :
+                    : "r"(smem_u32(sb)), "l"(reinterpret_cast<uint64_t>(&x_map)), "r"(bar), "r"((kb0 + kb) * kTcK), "r"(0)
+                    : "memory");
+            }
             const float2 mm = make_float2(cur.m, cur.m);
             const uint32_t word[4] = {cur.cc.x, cur.cc.y, cur.cc.z, cur.cc.w};
 #pragma unroll
@@ -236,12 +242,6 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
                 }
                 const int chunk = a_half * 4 + j;
                 *reinterpret_cast<uint4*>(sa + a_off + ((chunk ^ (a_row & 7)) * 16)) = make_uint4(p[0], p[1], p[2], p[3]);
-            }
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {  // the X tile, same layout
-                const int q = t + u * kTcProducers, n = q >> 3, ch = q & 7;
-                if (q < n_rhs * 8)
-                    *reinterpret_cast<uint4*>(sb + (n >> 3) * 1024 + (n & 7) * 128 + ((ch ^ (n & 7)) * 16)) = cur.xq[u];
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
             __syncwarp();
@@ -268,7 +268,12 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
             for (int c = 0; c < 8; ++c) yrow[c0 + c] = __uint_as_float(v[c]);
         }
     }
-    if (failed && tid == 0) atomicExch(status, 1);
+    if (failed) {
+        // a TMA copy requested before the time-out may still be writing this CTA's shared memory: it
+        // takes microseconds; give it a bounded 100 before the CTA goes away
+        if (tid == 0) atomicExch(status, 1);
+        for (int i = 0; i < 100; ++i) __nanosleep(1000);
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0)
@@ -334,6 +339,43 @@ __global__ void gemm_tc_reduce_kernel(const float* __restrict__ part, int splits
 
 using namespace bof4;
 
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map of X (bf16 [n_rhs][cols]) with a box of 64 columns x n_rhs rows and the 128-byte swizzle:
+// one TMA load per k-block lands in the layout the tcgen05 descriptor of the B operand names.
+int make_x_map(const void* d_x, int64_t cols, int n_rhs, CUtensorMap* map)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        BOF4_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q));
+        if (!p || q != cudaDriverEntryPointSuccess) {
+            set_error("bof4_gemm_tc: the driver does not provide cuTensorMapEncodeTiled");
+            return BOF4_ERR_CUDA;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)n_rhs};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcK, (cuuint32_t)n_rhs};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d_x), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("bof4_gemm_tc: cuTensorMapEncodeTiled failed with code %d", (int)r);
+        return BOF4_ERR_CUDA;
+    }
+    return BOF4_OK;
+}
+
+}  // namespace
+
 extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int scale_dtype, int64_t rows, int64_t cols,
                             int block_size, const float* d_codebook, const void* d_x, int n_rhs,
                             const int32_t* d_out_idx, const void* d_out_val, const int64_t* d_n_out, int64_t capacity,
@@ -397,16 +439,18 @@ extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int sc
     const int per = kblocks / splits;
     int rc, block_shift = 0;
     while ((1 << block_shift) < block_size) ++block_shift;
+    CUtensorMap x_map;
+    if ((rc = make_x_map(d_x, cols, n_rhs, &x_map))) return rc;
     if (scale_dtype == BOF4_F32) {
         constexpr auto kern = gemm_tc_kernel<F32>;
         if ((rc = ensure_dynamic_smem<kern>(kTcSmem))) return rc;
-        kern<<<g, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_shift, d_codebook,
-                                             static_cast<const uint16_t*>(d_x), n_rhs, out, per, d_status);
+        kern<<<g, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_shift, d_codebook, x_map, n_rhs, out, per,
+                                             d_status);
     } else {
         constexpr auto kern = gemm_tc_kernel<BF16>;
         if ((rc = ensure_dynamic_smem<kern>(kTcSmem))) return rc;
-        kern<<<g, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_shift, d_codebook,
-                                             static_cast<const uint16_t*>(d_x), n_rhs, out, per, d_status);
+        kern<<<g, kTcThreads, kTcSmem, st>>>(d_codes, d_scales, cols, block_shift, d_codebook, x_map, n_rhs, out, per,
+                                             d_status);
     }
     BOF4_CUDA_TRY(cudaGetLastError());
     if (splits > 1) {
