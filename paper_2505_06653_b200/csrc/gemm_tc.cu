@@ -116,8 +116,11 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     // lanes L and L + 16: an 8-byte read is served half a warp at a time, so the 16 lanes of a half
     // never share a bank whatever their code bytes are.
     unsigned char* tab_ptr = tiles_ptr + kTcStages * (kTcABytes + kTcBBytes);
+    __shared__ float s_lv[kLevels];
+    if (tid < kLevels) s_lv[tid] = levels[tid];
+    __syncthreads();  // the table is filled from shared memory: no global read per entry
     for (int e = tid; e < 256 * 16; e += kTcThreads)
-        reinterpret_cast<float2*>(tab_ptr)[e] = make_float2(levels[e >> 8], levels[(e >> 4) & 15]);
+        reinterpret_cast<float2*>(tab_ptr)[e] = make_float2(s_lv[e >> 8], s_lv[(e >> 4) & 15]);
     const uint32_t tab = smem_u32(tab_ptr) + (uint32_t)(lane & 15) * 8u;
     if (tid == 0) {
         s_fail = 0;
@@ -199,19 +202,18 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
             f.m = tc_scale<ST>(scales, (a_first + (int64_t)kb * kTcK) >> block_shift);
             return f;
         };
-        Fetched cur = fetch(0);
-        for (int kb = 0; kb < kblocks; ++kb) {
+        // One k-block: wait for the stage, request X, decode, publish.  false: a wait ran out.
+        auto step = [&](int kb, const Fetched& cur) -> bool {
             const int s = kb % kTcStages;
             unsigned char* sa = tiles_ptr + s * (kTcABytes + kTcBBytes);
             unsigned char* sb = sa + kTcABytes;
-            const Fetched next = (kb + 1 < kblocks) ? fetch(kb + 1) : cur;  // on its way while this one is decoded
             if (kb >= kTcStages) {  // the tensor cores must have read what the stage held (k-block kb - stages)
                 int ok = 1;
                 if (lane == 0) ok = tc_wait(smem_u32(&s_empty[s]), (uint32_t)(((kb / kTcStages) - 1) & 1)) ? 1 : 0;
                 ok = __shfl_sync(kFull, ok, 0);
                 if (!ok) {
                     if (lane == 0) s_fail = 1;
-                    break;
+                    return false;
                 }
             }
             if (t == 0) {
@@ -247,7 +249,21 @@ gemm_tc_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
             __syncwarp();
             if (lane == 0)
                 asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&s_full[s])) : "memory");
-            cur = next;
+            return true;
+        };
+        // two fetch buffers used in turn (no register copies): the loads of k-block kb + 1 are in flight
+        // while k-block kb is decoded
+        {
+            Fetched fa = fetch(0), fb = fa;
+            int kb = 0;
+            while (kb < kblocks) {
+                if (kb + 1 < kblocks) fb = fetch(kb + 1);
+                if (!step(kb, fa)) break;
+                if (++kb >= kblocks) break;
+                if (kb + 1 < kblocks) fa = fetch(kb + 1);
+                if (!step(kb, fb)) break;
+                ++kb;
+            }
         }
     }
     // Every loop above is bounded, so every warp gets here.  After a time-out the issuing thread has
@@ -424,14 +440,15 @@ extern "C" int bof4_gemm_tc(const uint8_t* d_codes, const void* d_scales, int sc
         return BOF4_OK;
     }
     const int grid = (int)(rows / kTcM);
-    // K split: enough CTAs for four per SM, a divisor of the number of k-blocks, partial products in
-    // the workspace (none: no split)
+    // K split: enough CTAs to fill the SMs (kTcCtasPerSm each), a divisor of the number of k-blocks,
+    // partial products in the workspace (none: no split).  Measured: more and shorter CTAs than
+    // that cost more (table set-up, pipeline fill and drain, epilogue) than the fuller last wave gains.
     const int kblocks = (int)(cols / kTcK);
     int splits = 1;
     const size_t slab = (size_t)rows * n_rhs * sizeof(float);
     if (d_ws && !((uintptr_t)d_ws & 15u)) {
         for (int cand = 2; cand <= 8; ++cand)
-            if (kblocks % cand == 0 && (size_t)cand * slab <= ws_bytes && (int64_t)grid * (cand - 1) < kSMs * kTcCtasPerSm)
+            if (kblocks % cand == 0 && (size_t)cand * slab <= ws_bytes && (int64_t)grid * (cand - 1) < kSMs * 4)
                 splits = cand;
     }
     float* out = splits > 1 ? static_cast<float*>(d_ws) : d_y;
