@@ -51,6 +51,26 @@ def test_integer_valued_products_are_exact(bof4, rows, cols, n_rhs, I, scale_dty
     assert int(status1.item()) == 0 and torch.equal(y, y1)
 
 
+def test_random_shapes_are_exact(bof4):
+    """Seeded random shapes (row tiles, k-blocks that do and do not divide by the split factors,
+    every batch size and block size the entry point takes), integer-valued: bit for bit."""
+    rng = np.random.default_rng(2026)
+    for trial in range(24):
+        rows = 128 * int(rng.integers(1, 9))
+        I = int(rng.choice([32, 64, 128, 256, 1024]))
+        cols = max(I, 64) * int(rng.integers(1, 40))
+        n_rhs = int(rng.choice([16, 32, 48, 64]))
+        lv, codes, scales, X = _exact_case(rows, cols, n_rhs, I, 1000 + trial)
+        sd = torch.bfloat16 if trial % 2 else torch.float32
+        y, status = bof4.bof4_gemm_tc(torch.from_numpy(codes).cuda(), torch.from_numpy(scales).to(sd).cuda(),
+                                      rows, cols, I, lv, torch.from_numpy(X).to(torch.bfloat16).cuda(),
+                                      split=bool(trial % 3))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref, _ = oracle.gemm_bf16(codes, scales, rows, cols, I, lv, X)
+        assert np.array_equal(y.cpu().numpy().astype(np.float64), ref), (rows, cols, n_rhs, I)
+
+
 @pytest.mark.parametrize("rows,cols,n_rhs", [(256, 4096, 16), (512, 8192, 64), (128, 14336, 32)])
 @pytest.mark.parametrize("norm", [0, 1])
 def test_quantised_matrix_times_batch(bof4, rows, cols, n_rhs, norm):
